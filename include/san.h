@@ -1,0 +1,178 @@
+/*
+ * san.h -- C ABI of the shared-attention (SAN) decode library for NVIDIA B200 (sm_100a).
+ *
+ * The library implements the cached attention of auto-regressive Transformer decoding
+ * when attention weights are shared inside blocks of adjacent decoder layers
+ * ("Sharing Attention Weights for Fast Transformer", arXiv 1906.11024).
+ *
+ * Notation follows the paper: S = Softmax(Q.K^T / sqrt(d_k)) are the attention WEIGHTS
+ * (Eq. 1) and the attention OUTPUT is S.V (Eq. 2; the paper calls it A, this header calls
+ * it O).  In a block of pi adjacent layers only the lowest layer m computes S^m from its
+ * own queries and keys; layers m+1 .. m+pi-1 reuse S^m and apply it to their own values
+ * (Eq. 3-4).  Hence only block-first layers keep a key cache (Section 3.2, memory note).
+ *
+ * General rules
+ *  - Every function returns a status (SAN_OK = 0).  Nothing throws, traps or waits.
+ *  - All `d_` pointers are DEVICE pointers owned by the caller; all others are HOST
+ *    pointers.  The library allocates no device memory: the cache arena and the
+ *    workspace are caller buffers handed to san_create.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  No hot call
+ *    synchronises the host.  Calls on one context must be ordered on the device (same
+ *    stream, or events between streams): they share the context's workspace.
+ *  - Host-checkable mistakes (null pointers, shapes, an invalid policy, a layer outside
+ *    the block, capacity) are reported before anything is launched.  Mistakes visible
+ *    only on the device (an id out of range, a length < 1 or beyond capacity) make the
+ *    kernel skip that item and record the first such error in a device word, read back
+ *    with san_device_status.
+ *  - Element type is SAN_F32 or SAN_BF16 for q/k/v/x/outputs; S is always float32;
+ *    products, sums and the softmax are float32.  d_head must be 64.
+ *  - Sequences are numbered 0 .. max_sent*beam-1; sequence s belongs to sentence
+ *    s / beam (the beams of a sentence read the same encoder memory, Section 2).
+ *
+ * Cache layout inside the arena (head-major; every (id, head) panel is contiguous and
+ * each row is 64 elements = 128 B bf16 / 256 B f32, 16-byte aligned):
+ *    self K   [self block ][sequence][head][max_tgt_len][64]   (block-first layers only)
+ *    self V   [layer      ][sequence][head][max_tgt_len][64]
+ *    memory K [encdec block][sentence][head][max_src_len][64]
+ *    memory V [layer       ][sentence][head][max_src_len][64]  (one plane per BLOCK when
+ *                                                               encdec_shared_context)
+ *    AAN sum  [layer][sequence][n_heads*64] float32             (only when self_is_aan)
+ */
+#ifndef SAN_H_
+#define SAN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct san_ctx san_ctx; /* opaque; lives in host memory */
+
+enum {
+    SAN_OK = 0,
+    SAN_ERR_NULL = 1,         /* a required pointer is NULL */
+    SAN_ERR_SHAPE = 2,        /* a size or count is out of range */
+    SAN_ERR_POLICY = 3,       /* block sizes / block map do not describe a valid policy */
+    SAN_ERR_CAPACITY = 4,     /* a caller buffer is too small, or more blocks than key planes */
+    SAN_ERR_DTYPE = 5,
+    SAN_ERR_RANGE = 6,        /* layer/block/position outside what the policy or config allows */
+    SAN_ERR_CUDA = 7,         /* a CUDA runtime call failed (launch configuration, bad stream...) */
+    SAN_ERR_DEVICE_CHECK = 8, /* a kernel met an invalid id/length/position and skipped the item */
+    SAN_ERR_TIMEOUT = 9,      /* reserved for bounded device waits (the library has none) */
+    SAN_ERR_UNSUPPORTED = 10
+};
+enum { SAN_F32 = 0, SAN_BF16 = 1 };
+enum { SAN_SELF = 0, SAN_ENCDEC = 1 };
+
+#define SAN_MAX_LAYERS 64
+#define SAN_MAX_BEAM 8
+
+typedef struct {
+    int32_t n_layers;    /* M, 1..SAN_MAX_LAYERS */
+    int32_t n_heads;     /* H */
+    int32_t d_head;      /* must be 64 */
+    int32_t max_sent;    /* sentences the caches have room for */
+    int32_t beam;        /* sequences per sentence, 1..SAN_MAX_BEAM */
+    int32_t max_tgt_len; /* self-attention cache rows per sequence */
+    int32_t max_src_len; /* encoder-memory rows per sentence */
+    int32_t dtype;       /* SAN_F32 or SAN_BF16 */
+    int32_t self_is_aan; /* 1: decoder self-attention is the cumulative average (san_aan_step) */
+    int32_t encdec_shared_context; /* 1: Eq. 5, one O (and one V plane) per enc-dec block */
+} san_config;
+
+/* Bytes the caller must provide for a configuration whose self / enc-dec policies have
+ * n_self_blocks / n_encdec_blocks blocks (the key-cache planes; Section 3.2: layers that
+ * take their weights from another layer keep no keys).  Either output may be NULL. */
+int32_t san_query_bytes(const san_config* cfg, int32_t n_self_blocks, int32_t n_encdec_blocks,
+                        size_t* cache_bytes, size_t* workspace_bytes);
+
+/* Creates a context over caller-owned device buffers (256-byte aligned).  The sharing
+ * policies are given as block sizes {pi_1..pi_N} bottom-up (Section 3.3); their block
+ * counts fix the number of key planes carved out of the arena.  Zeroes the workspace
+ * header on the default stream and waits for it (the one synchronising call besides
+ * san_device_status).  The arena is not cleared. */
+int32_t san_create(const san_config* cfg, const int32_t* self_sizes, int32_t n_self,
+                   const int32_t* encdec_sizes, int32_t n_encdec, void* d_cache, size_t cache_bytes,
+                   void* d_workspace, size_t workspace_bytes, san_ctx** out);
+int32_t san_destroy(san_ctx* ctx);
+
+/* Sharing policy (Section 3.3): block sizes bottom-up with sum = n_layers and every size
+ * >= 1, or the same thing as a per-layer block id (starts at 0; each next layer keeps the
+ * id or raises it by one).  A policy with more blocks than the context has key planes is
+ * refused with SAN_ERR_CAPACITY.  Changing the policy does not move cached rows. */
+int32_t san_policy_set_sizes(san_ctx* ctx, int32_t kind, const int32_t* sizes, int32_t n_blocks);
+int32_t san_policy_set_map(san_ctx* ctx, int32_t kind, const int32_t* block_of_layer, int32_t n_layers);
+/* Any output may be NULL.  block_of_layer[n_layers], first_layer_of_block[n_blocks]. */
+int32_t san_policy_get_map(const san_ctx* ctx, int32_t kind, int32_t* block_of_layer,
+                           int32_t* first_layer_of_block, int32_t* n_blocks);
+
+/* Attention cache (Section 4.1 uses one; Section 2: enc-dec keys/values come from the
+ * encoder output).  Copies new rows into the caches of layers [layer_begin, layer_end):
+ *   kind = SAN_SELF   d_ids = sequence ids, rows go to the self-attention K/V caches;
+ *   kind = SAN_ENCDEC d_ids = sentence ids, rows go to the encoder-memory K/V.
+ * Item i writes d_nrows[i] rows (1 if d_nrows is NULL) starting at row d_pos[i] (0 if
+ * d_pos is NULL).  Source layout, `rows_per_item` = row capacity of one item (>= every
+ * d_nrows[i]; 1 for a decode step):
+ *   d_v_new [layers in range          ][n_items][rows_per_item][H][64]
+ *   d_k_new [block-first layers in range][n_items][rows_per_item][H][64]   (in layer order)
+ * d_k_new must be NULL iff the range holds no block-first layer.  With
+ * encdec_shared_context only block-first layers may be in an ENCDEC range.
+ * Not allowed for SAN_SELF when self_is_aan.  Payload is copied bit for bit. */
+int32_t san_cache_append(san_ctx* ctx, int32_t kind, int32_t layer_begin, int32_t layer_end,
+                         const void* d_k_new, const void* d_v_new, const int32_t* d_ids,
+                         const int32_t* d_pos, const int32_t* d_nrows, int32_t n_items,
+                         int32_t rows_per_item, void* stream);
+
+/* Eq. 1 for one decode step, at the lowest layer of `block` (Eq. 3):
+ *   S[j] = exp(z_j - max z) / sum_j exp(z_j - max z),  z_j = (q . K_j) / sqrt(64),
+ * over cached rows j in [0, d_lens[i]).
+ *   kind = SAN_SELF    d_ids sequence ids; d_q [n_items][H][64]; d_S [n_items][H][ld_s]
+ *   kind = SAN_ENCDEC  d_ids sentence ids; d_q [n_items][beam][H][64];
+ *                      d_S [n_items][beam][H][ld_s]; d_lens[i] = source length; every
+ *                      key tile is read once for all beams of the sentence.
+ * max_len is a host-side upper bound on d_lens (1..capacity; 0 = capacity) used to size
+ * the launch; a longer length is a device-check error.  ld_s >= max_len.  Entries of a
+ * row beyond its length are left untouched.  Long rows are split over several warps
+ * (partial max/sum in the workspace, combined by the last warp to finish; nothing waits). */
+int32_t san_attn_weights(san_ctx* ctx, int32_t kind, int32_t block, const void* d_q,
+                         const int32_t* d_ids, const int32_t* d_lens, int32_t n_items,
+                         int32_t max_len, float* d_S, int64_t ld_s, void* stream);
+
+/* Eq. 2 with Eq. 4: for every layer l in [layer_begin, layer_end), all inside `block`,
+ *   O_l = sum_{j in [p0, p1)} S[j] * V_l[j]
+ * with the block's weights S (layout as written by san_attn_weights) and each layer's own
+ * cached values, in one launch; S is staged on chip once per work item and reused for
+ * every layer.  p0 = d_pos_begin[i] (0 if NULL), p1 = d_pos_end[i].
+ *   d_out [layer_end-layer_begin][n_items]([beam])[H][64], element type = cfg.dtype
+ *         (rounded to nearest even from float32 for bf16).
+ * accumulate != 0 adds to what d_out holds (for finishing a layer whose newest value row
+ * arrived after the block's history was applied).  With encdec_shared_context (Eq. 5) an
+ * ENCDEC call must name exactly the block's first layer; the one output serves the block.
+ * max_len bounds d_pos_end as in san_attn_weights. */
+int32_t san_attn_apply(san_ctx* ctx, int32_t kind, int32_t block, int32_t layer_begin,
+                       int32_t layer_end, const float* d_S, int64_t ld_s, const int32_t* d_ids,
+                       const int32_t* d_pos_begin, const int32_t* d_pos_end, int32_t n_items,
+                       int32_t max_len, void* d_out, int32_t accumulate, void* stream);
+
+/* Average attention in place of decoder self-attention (the AAN model the paper combines
+ * with SAN in Table 6): for layers [layer_begin, layer_end) and item i with sequence
+ * d_ids[i] at 1-based target position d_t[i]:
+ *   sum_l[seq] += x_l[i];  out_l[i] = sum_l[seq] / d_t[i]      (mean of positions 1..t)
+ * d_t[i] == 1 restarts the sum from x.  d_x, d_out: [layers in range][n_items][H*64]. */
+int32_t san_aan_step(san_ctx* ctx, int32_t layer_begin, int32_t layer_end, const void* d_x,
+                     const int32_t* d_ids, const int32_t* d_t, int32_t n_items, void* d_out,
+                     void* stream);
+
+/* Reads (and clears) the device error word: *first_error = SAN_OK or the first
+ * device-check error since the last read; detail[0..3] (optional) = kernel tag, item,
+ * offending value, limit.  Synchronises `stream`. */
+int32_t san_device_status(san_ctx* ctx, int32_t* first_error, int32_t* detail, void* stream);
+
+const char* san_status_string(int32_t status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SAN_H_ */

@@ -1,0 +1,180 @@
+"""ctypes binding of include/san.h: same names, argument marshalling only.
+
+Device arguments may be torch CUDA tensors (their ``data_ptr()`` is passed) or raw
+integer addresses; ``stream`` may be a ``torch.cuda.Stream``, an integer handle or
+None (torch's current stream).  Every function returns the library's status code;
+``check`` turns a non-zero status into ``SanError``.
+
+There is no CPU fallback: if the CUDA library has not been built, ``lib()`` raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libsan_b200.so")
+
+SAN_OK = 0
+SAN_ERR_NULL, SAN_ERR_SHAPE, SAN_ERR_POLICY, SAN_ERR_CAPACITY, SAN_ERR_DTYPE = 1, 2, 3, 4, 5
+SAN_ERR_RANGE, SAN_ERR_CUDA, SAN_ERR_DEVICE_CHECK, SAN_ERR_TIMEOUT, SAN_ERR_UNSUPPORTED = 6, 7, 8, 9, 10
+SAN_F32, SAN_BF16 = 0, 1
+SAN_SELF, SAN_ENCDEC = 0, 1
+SAN_MAX_LAYERS, SAN_MAX_BEAM = 64, 8
+
+# every symbol include/san.h declares
+EXPORTS = (
+    "san_query_bytes", "san_create", "san_destroy",
+    "san_policy_set_sizes", "san_policy_set_map", "san_policy_get_map",
+    "san_cache_append", "san_attn_weights", "san_attn_apply", "san_aan_step",
+    "san_device_status", "san_status_string",
+)
+
+
+class san_config(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in (
+        "n_layers", "n_heads", "d_head", "max_sent", "beam", "max_tgt_len", "max_src_len",
+        "dtype", "self_is_aan", "encdec_shared_context")]
+
+
+class SanError(RuntimeError):
+    def __init__(self, status: int, where: str = ""):
+        self.status = status
+        super().__init__(f"{where}: status {status} ({san_status_string(status)})")
+
+
+_lib = None
+_I32P = C.POINTER(C.c_int32)
+
+
+def lib():
+    """Load libsan_b200.so (built by ``paper_1906_11024_b200.build``); raises if it is missing."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: run `python -m paper_1906_11024_b200.build` "
+                          "(there is no CPU fallback)")
+    L = C.CDLL(LIB_PATH)
+    vp, i32, i64, sz = C.c_void_p, C.c_int32, C.c_int64, C.c_size_t
+    L.san_query_bytes.argtypes = [C.POINTER(san_config), i32, i32, C.POINTER(sz), C.POINTER(sz)]
+    L.san_create.argtypes = [C.POINTER(san_config), _I32P, i32, _I32P, i32, vp, sz, vp, sz, C.POINTER(vp)]
+    L.san_destroy.argtypes = [vp]
+    L.san_policy_set_sizes.argtypes = [vp, i32, _I32P, i32]
+    L.san_policy_set_map.argtypes = [vp, i32, _I32P, i32]
+    L.san_policy_get_map.argtypes = [vp, i32, _I32P, _I32P, _I32P]
+    L.san_cache_append.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, i32, i32, vp]
+    L.san_attn_weights.argtypes = [vp, i32, i32, vp, vp, vp, i32, i32, vp, i64, vp]
+    L.san_attn_apply.argtypes = [vp, i32, i32, i32, i32, vp, i64, vp, vp, vp, i32, i32, vp, i32, vp]
+    L.san_aan_step.argtypes = [vp, i32, i32, vp, vp, vp, i32, vp, vp]
+    L.san_device_status.argtypes = [vp, _I32P, _I32P, vp]
+    L.san_status_string.argtypes = [i32]
+    L.san_status_string.restype = C.c_char_p
+    for name in EXPORTS:
+        if name != "san_status_string":
+            getattr(L, name).restype = i32
+    _lib = L
+    return L
+
+
+def _ptr(x) -> Optional[int]:
+    if x is None:
+        return None
+    if isinstance(x, int):
+        return x
+    return x.data_ptr()          # torch tensor
+
+
+def _stream(s) -> Optional[int]:
+    if s is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(s, int):
+        return s
+    return s.cuda_stream
+
+
+def _i32_array(v: Sequence[int]):
+    return (C.c_int32 * len(v))(*[int(x) for x in v])
+
+
+def check(status: int, where: str = "san") -> None:
+    if status != SAN_OK:
+        raise SanError(status, where)
+
+
+def san_status_string(status: int) -> str:
+    return lib().san_status_string(int(status)).decode()
+
+
+def san_query_bytes(cfg: san_config, n_self_blocks: int, n_encdec_blocks: int):
+    """Returns (status, cache_bytes, workspace_bytes)."""
+    cb, wb = C.c_size_t(0), C.c_size_t(0)
+    rc = lib().san_query_bytes(C.byref(cfg), n_self_blocks, n_encdec_blocks, C.byref(cb), C.byref(wb))
+    return rc, cb.value, wb.value
+
+
+def san_create(cfg: san_config, self_sizes, encdec_sizes, d_cache, cache_bytes, d_workspace, workspace_bytes):
+    """Returns (status, ctx handle)."""
+    h = C.c_void_p(None)
+    ss = _i32_array(self_sizes) if self_sizes is not None else None
+    es = _i32_array(encdec_sizes) if encdec_sizes is not None else None
+    rc = lib().san_create(C.byref(cfg), ss, len(self_sizes) if self_sizes is not None else 0,
+                          es, len(encdec_sizes) if encdec_sizes is not None else 0,
+                          _ptr(d_cache), cache_bytes, _ptr(d_workspace), workspace_bytes, C.byref(h))
+    return rc, h.value
+
+
+def san_destroy(ctx) -> int:
+    return lib().san_destroy(ctx)
+
+
+def san_policy_set_sizes(ctx, kind: int, sizes) -> int:
+    return lib().san_policy_set_sizes(ctx, kind, _i32_array(sizes), len(sizes))
+
+
+def san_policy_set_map(ctx, kind: int, block_of_layer) -> int:
+    return lib().san_policy_set_map(ctx, kind, _i32_array(block_of_layer), len(block_of_layer))
+
+
+def san_policy_get_map(ctx, kind: int):
+    """Returns (status, block_of_layer list, first_layer_of_block list)."""
+    bol = (C.c_int32 * SAN_MAX_LAYERS)(*([-1] * SAN_MAX_LAYERS))   # the library fills n_layers entries
+    first = (C.c_int32 * SAN_MAX_LAYERS)()
+    nb = C.c_int32(0)
+    rc = lib().san_policy_get_map(ctx, kind, bol, first, C.byref(nb))
+    if rc != SAN_OK:
+        return rc, [], []
+    return rc, [b for b in bol if b >= 0], list(first[:nb.value])
+
+
+def san_cache_append(ctx, kind, layer_begin, layer_end, d_k_new, d_v_new, d_ids, d_pos, d_nrows,
+                     n_items, rows_per_item=1, stream=None) -> int:
+    return lib().san_cache_append(ctx, kind, layer_begin, layer_end, _ptr(d_k_new), _ptr(d_v_new), _ptr(d_ids),
+                                  _ptr(d_pos), _ptr(d_nrows), n_items, rows_per_item, _stream(stream))
+
+
+def san_attn_weights(ctx, kind, block, d_q, d_ids, d_lens, n_items, max_len, d_S, ld_s, stream=None) -> int:
+    return lib().san_attn_weights(ctx, kind, block, _ptr(d_q), _ptr(d_ids), _ptr(d_lens), n_items, max_len,
+                                  _ptr(d_S), ld_s, _stream(stream))
+
+
+def san_attn_apply(ctx, kind, block, layer_begin, layer_end, d_S, ld_s, d_ids, d_pos_begin, d_pos_end,
+                   n_items, max_len, d_out, accumulate=0, stream=None) -> int:
+    return lib().san_attn_apply(ctx, kind, block, layer_begin, layer_end, _ptr(d_S), ld_s, _ptr(d_ids),
+                                _ptr(d_pos_begin), _ptr(d_pos_end), n_items, max_len, _ptr(d_out),
+                                int(accumulate), _stream(stream))
+
+
+def san_aan_step(ctx, layer_begin, layer_end, d_x, d_ids, d_t, n_items, d_out, stream=None) -> int:
+    return lib().san_aan_step(ctx, layer_begin, layer_end, _ptr(d_x), _ptr(d_ids), _ptr(d_t), n_items,
+                              _ptr(d_out), _stream(stream))
+
+
+def san_device_status(ctx, stream=None):
+    """Returns (status, first_error, detail[4]).  Synchronises the stream."""
+    fe = C.c_int32(0)
+    det = (C.c_int32 * 4)()
+    rc = lib().san_device_status(ctx, C.byref(fe), det, _stream(stream))
+    return rc, fe.value, list(det)

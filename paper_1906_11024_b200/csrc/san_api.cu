@@ -1,0 +1,401 @@
+// Host side of the C ABI declared in include/san.h: argument checks, the arena and
+// workspace layout, launch geometry.  Every step of the path runs in the kernels of
+// san_kernels.cuh; nothing here computes attention.
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <new>
+
+#include "san_ctx.h"
+#include "san_kernels.cuh"
+
+using namespace san;
+
+namespace {
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+int32_t check_config(const san_config* c) {
+    if (!c) return SAN_ERR_NULL;
+    if (c->n_layers < 1 || c->n_layers > SAN_MAX_LAYERS) return SAN_ERR_SHAPE;
+    if (c->n_heads < 1 || c->n_heads > 1024) return SAN_ERR_SHAPE;
+    if (c->d_head != kDh) return SAN_ERR_UNSUPPORTED;
+    if (c->max_sent < 1 || c->beam < 1 || c->beam > SAN_MAX_BEAM) return SAN_ERR_SHAPE;
+    if (c->max_tgt_len < 1 || c->max_src_len < 1) return SAN_ERR_SHAPE;
+    if (c->max_tgt_len > (1 << 20) || c->max_src_len > (1 << 20)) return SAN_ERR_SHAPE;
+    if ((int64_t)c->max_sent * c->beam > (1 << 24)) return SAN_ERR_SHAPE;
+    if (c->dtype != SAN_F32 && c->dtype != SAN_BF16) return SAN_ERR_DTYPE;
+    return SAN_OK;
+}
+
+// Arena and workspace layout; the one place that knows it.
+void layout(const san_config& c, int n_self_planes, int n_enc_planes, san_ctx* L) {
+    const size_t e = c.dtype == SAN_F32 ? 4 : 2;
+    const size_t n_seqs = (size_t)c.max_sent * c.beam;
+    L->elem_bytes = (int)e;
+    L->n_seqs = (int)n_seqs;
+    L->self_plane_bytes = align_up(n_seqs * c.n_heads * c.max_tgt_len * kDh * e, 256);
+    L->mem_plane_bytes = align_up((size_t)c.max_sent * c.n_heads * c.max_src_len * kDh * e, 256);
+    L->aan_plane_bytes = align_up(n_seqs * c.n_heads * kDh * sizeof(float), 256);
+    L->n_self_k_planes = c.self_is_aan ? 0 : n_self_planes;
+    L->n_self_v_planes = c.self_is_aan ? 0 : c.n_layers;
+    L->n_enc_k_planes = n_enc_planes;
+    L->n_enc_v_planes = c.encdec_shared_context ? n_enc_planes : c.n_layers;
+    size_t off = 0;
+    L->off_self_k = off; off += L->self_plane_bytes * L->n_self_k_planes;
+    L->off_self_v = off; off += L->self_plane_bytes * L->n_self_v_planes;
+    L->off_mem_k = off;  off += L->mem_plane_bytes * L->n_enc_k_planes;
+    L->off_mem_v = off;  off += L->mem_plane_bytes * L->n_enc_v_planes;
+    L->off_aan = off;    off += c.self_is_aan ? L->aan_plane_bytes * c.n_layers : 0;
+    L->cache_bytes_needed = std::max<size_t>(off, 256);
+
+    // workspace: error words | tickets [layer][row] | partial sums of split rows
+    const size_t rows = n_seqs * c.n_heads;
+    L->n_tickets = (size_t)c.n_layers * rows;
+    const size_t worst = L->n_tickets * 4 * kDh;   // four spans per (layer, row), one query row each
+    L->part_floats = std::min<size_t>(std::max<size_t>(worst, (size_t)1 << 18), (size_t)1 << 24);
+    L->ws_off_tickets = 256;
+    L->ws_off_part = align_up(256 + L->n_tickets * sizeof(int), 256);
+    L->ws_bytes_needed = L->ws_off_part + L->part_floats * sizeof(float);
+}
+
+inline int32_t cuda_status(cudaError_t e) { return e == cudaSuccess ? SAN_OK : SAN_ERR_CUDA; }
+
+int pick_nq_template(int nq) { return nq <= 1 ? 1 : nq <= 2 ? 2 : nq <= 4 ? 4 : 8; }
+
+// Positions per warp item.  Start with one span per row; halve it while the launch would
+// leave SMs idle; grow it back if the partial sums would not fit the workspace.
+void pick_spans(const san_ctx* ctx, long long units, int max_len, long long part_per_span_floats,
+                int* span_len, int* n_spans) {
+    const long long target = (long long)ctx->sm_count * 16;
+    int sl = (int)align_up((size_t)max_len, 32), ns = 1;
+    while (units * ns < target && sl > 32) {
+        sl = (int)align_up((size_t)ceil_div(sl, 2), 32);
+        ns = ceil_div(max_len, sl);
+    }
+    while (ns > 1 && part_per_span_floats * ns > (long long)ctx->part_floats) {
+        sl = (int)align_up((size_t)sl * 2, 32);
+        ns = ceil_div(max_len, sl);
+    }
+    *span_len = sl;
+    *n_spans = ns;
+}
+
+template <typename T>
+cudaError_t launch_weights(const WeightsParams& p, int nq_t, unsigned grid, cudaStream_t st) {
+    const unsigned block = kWarpsPerCta * 32;
+    switch (nq_t) {
+        case 1: weights_kernel<T, 1><<<grid, block, 0, st>>>(p); break;
+        case 2: weights_kernel<T, 2><<<grid, block, 0, st>>>(p); break;
+        case 4: weights_kernel<T, 4><<<grid, block, 0, st>>>(p); break;
+        default: weights_kernel<T, 8><<<grid, block, 0, st>>>(p); break;
+    }
+    return cudaGetLastError();
+}
+
+template <typename T>
+cudaError_t launch_apply(const ApplyParams& p, int nq_t, unsigned grid, cudaStream_t st) {
+    const unsigned block = kWarpsPerCta * 32;
+    switch (nq_t) {
+        case 1: apply_kernel<T, 1><<<grid, block, 0, st>>>(p); break;
+        case 2: apply_kernel<T, 2><<<grid, block, 0, st>>>(p); break;
+        case 4: apply_kernel<T, 4><<<grid, block, 0, st>>>(p); break;
+        default: apply_kernel<T, 8><<<grid, block, 0, st>>>(p); break;
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+extern "C" {
+
+int32_t san_query_bytes(const san_config* cfg, int32_t n_self_blocks, int32_t n_encdec_blocks,
+                        size_t* cache_bytes, size_t* workspace_bytes) {
+    int32_t rc = check_config(cfg);
+    if (rc != SAN_OK) return rc;
+    if (n_self_blocks < 1 || n_self_blocks > cfg->n_layers) return SAN_ERR_POLICY;
+    if (n_encdec_blocks < 1 || n_encdec_blocks > cfg->n_layers) return SAN_ERR_POLICY;
+    san_ctx tmp;
+    layout(*cfg, n_self_blocks, n_encdec_blocks, &tmp);
+    if (cache_bytes) *cache_bytes = tmp.cache_bytes_needed;
+    if (workspace_bytes) *workspace_bytes = tmp.ws_bytes_needed;
+    return SAN_OK;
+}
+
+int32_t san_create(const san_config* cfg, const int32_t* self_sizes, int32_t n_self,
+                   const int32_t* encdec_sizes, int32_t n_encdec, void* d_cache, size_t cache_bytes,
+                   void* d_workspace, size_t workspace_bytes, san_ctx** out) {
+    if (!out) return SAN_ERR_NULL;
+    *out = nullptr;
+    int32_t rc = check_config(cfg);
+    if (rc != SAN_OK) return rc;
+    if (!self_sizes || !encdec_sizes || !d_cache || !d_workspace) return SAN_ERR_NULL;
+    Policy ps, pe;
+    if ((rc = policy_from_sizes(self_sizes, n_self, cfg->n_layers, &ps)) != SAN_OK) return rc;
+    if ((rc = policy_from_sizes(encdec_sizes, n_encdec, cfg->n_layers, &pe)) != SAN_OK) return rc;
+    if (((uintptr_t)d_cache & 255) || ((uintptr_t)d_workspace & 255)) return SAN_ERR_SHAPE;
+    san_ctx* ctx = new (std::nothrow) san_ctx;
+    if (!ctx) return SAN_ERR_CAPACITY;
+    ctx->cfg = *cfg;
+    ctx->self_pol = ps;
+    ctx->enc_pol = pe;
+    layout(*cfg, n_self, n_encdec, ctx);
+    if (cache_bytes < ctx->cache_bytes_needed || workspace_bytes < ctx->ws_bytes_needed) {
+        delete ctx;
+        return SAN_ERR_CAPACITY;
+    }
+    ctx->cache = static_cast<char*>(d_cache);
+    ctx->ws = static_cast<char*>(d_workspace);
+    ctx->err = reinterpret_cast<int*>(ctx->ws);
+    ctx->tickets = reinterpret_cast<int*>(ctx->ws + ctx->ws_off_tickets);
+    ctx->part = reinterpret_cast<float*>(ctx->ws + ctx->ws_off_part);
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, dev);
+    // error words and tickets start at zero; tickets return to zero after every launch
+    if (e == cudaSuccess) e = cudaMemset(ctx->ws, 0, ctx->ws_off_part);
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) {
+        delete ctx;
+        return SAN_ERR_CUDA;
+    }
+    *out = ctx;
+    return SAN_OK;
+}
+
+int32_t san_destroy(san_ctx* ctx) {
+    if (!ctx) return SAN_ERR_NULL;
+    delete ctx;
+    return SAN_OK;
+}
+
+int32_t san_policy_set_sizes(san_ctx* ctx, int32_t kind, const int32_t* sizes, int32_t n_blocks) {
+    if (!ctx || !sizes) return SAN_ERR_NULL;
+    if (kind != SAN_SELF && kind != SAN_ENCDEC) return SAN_ERR_RANGE;
+    Policy p;
+    int32_t rc = policy_from_sizes(sizes, n_blocks, ctx->cfg.n_layers, &p);
+    if (rc != SAN_OK) return rc;
+    const int planes = kind == SAN_SELF ? (ctx->cfg.self_is_aan ? ctx->cfg.n_layers : ctx->n_self_k_planes)
+                                        : ctx->n_enc_k_planes;
+    if (p.n_blocks > planes) return SAN_ERR_CAPACITY;
+    (kind == SAN_SELF ? ctx->self_pol : ctx->enc_pol) = p;
+    return SAN_OK;
+}
+
+int32_t san_policy_set_map(san_ctx* ctx, int32_t kind, const int32_t* block_of_layer, int32_t n_layers) {
+    if (!ctx || !block_of_layer) return SAN_ERR_NULL;
+    if (kind != SAN_SELF && kind != SAN_ENCDEC) return SAN_ERR_RANGE;
+    if (n_layers != ctx->cfg.n_layers) return SAN_ERR_SHAPE;
+    Policy p;
+    int32_t rc = policy_from_map(block_of_layer, n_layers, &p);
+    if (rc != SAN_OK) return rc;
+    return san_policy_set_sizes(ctx, kind, p.size_of_block, p.n_blocks);
+}
+
+int32_t san_policy_get_map(const san_ctx* ctx, int32_t kind, int32_t* block_of_layer,
+                           int32_t* first_layer_of_block, int32_t* n_blocks) {
+    if (!ctx) return SAN_ERR_NULL;
+    if (kind != SAN_SELF && kind != SAN_ENCDEC) return SAN_ERR_RANGE;
+    const Policy& p = kind == SAN_SELF ? ctx->self_pol : ctx->enc_pol;
+    if (block_of_layer) std::memcpy(block_of_layer, p.block_of_layer, sizeof(int32_t) * p.n_layers);
+    if (first_layer_of_block) std::memcpy(first_layer_of_block, p.first_layer_of_block, sizeof(int32_t) * p.n_blocks);
+    if (n_blocks) *n_blocks = p.n_blocks;
+    return SAN_OK;
+}
+
+int32_t san_cache_append(san_ctx* ctx, int32_t kind, int32_t layer_begin, int32_t layer_end,
+                         const void* d_k_new, const void* d_v_new, const int32_t* d_ids,
+                         const int32_t* d_pos, const int32_t* d_nrows, int32_t n_items,
+                         int32_t rows_per_item, void* stream) {
+    if (!ctx || !d_v_new || !d_ids) return SAN_ERR_NULL;
+    if (kind != SAN_SELF && kind != SAN_ENCDEC) return SAN_ERR_RANGE;
+    const san_config& c = ctx->cfg;
+    if (kind == SAN_SELF && c.self_is_aan) return SAN_ERR_UNSUPPORTED;
+    if (layer_begin < 0 || layer_end > c.n_layers || layer_begin >= layer_end) return SAN_ERR_RANGE;
+    const int cap = kind == SAN_SELF ? c.max_tgt_len : c.max_src_len;
+    const int max_ids = kind == SAN_SELF ? ctx->n_seqs : c.max_sent;
+    if (n_items < 0 || n_items > max_ids) return SAN_ERR_SHAPE;
+    if (rows_per_item < 1 || rows_per_item > cap) return SAN_ERR_SHAPE;
+    const Policy& pol = kind == SAN_SELF ? ctx->self_pol : ctx->enc_pol;
+    const bool v_by_block = (kind == SAN_ENCDEC && c.encdec_shared_context);
+
+    AppendParams p;
+    int n_first = 0;
+    for (int l = layer_begin; l < layer_end; ++l) {
+        const int lr = l - layer_begin;
+        const bool first = pol.is_first(l);
+        if (v_by_block && !first) return SAN_ERR_RANGE;   // Eq. 5: upper layers of a block keep no memory
+        p.v_plane[lr] = (short)(v_by_block ? pol.block_of_layer[l] : l);
+        p.k_plane[lr] = (short)(first ? pol.block_of_layer[l] : -1);
+        p.k_src[lr] = (short)(first ? n_first : 0);
+        n_first += first ? 1 : 0;
+    }
+    if (n_first > 0 && !d_k_new) return SAN_ERR_NULL;     // a block-first layer needs its keys
+    if (n_first == 0 && d_k_new) return SAN_ERR_RANGE;    // keys offered to layers that keep none
+    if (n_items == 0) return SAN_OK;
+
+    const size_t plane = kind == SAN_SELF ? ctx->self_plane_bytes : ctx->mem_plane_bytes;
+    p.k_new = static_cast<const char*>(d_k_new);
+    p.v_new = static_cast<const char*>(d_v_new);
+    p.K = ctx->cache + (kind == SAN_SELF ? ctx->off_self_k : ctx->off_mem_k);
+    p.V = ctx->cache + (kind == SAN_SELF ? ctx->off_self_v : ctx->off_mem_v);
+    p.k_plane_bytes = (long long)plane;
+    p.v_plane_bytes = (long long)plane;
+    p.ids = d_ids; p.pos = d_pos; p.nrows = d_nrows;
+    p.n_items = n_items; p.rows_per_item = rows_per_item; p.H = c.n_heads; p.cap_len = cap;
+    p.max_ids = max_ids; p.n_layers = layer_end - layer_begin; p.row_bytes = kDh * ctx->elem_bytes;
+    p.err = ctx->err;
+    const long long units = 2LL * p.n_layers * n_items * rows_per_item * c.n_heads * (p.row_bytes / 16);
+    const long long grid = (units + 255) / 256;
+    if (grid > 0x7fffffffLL) return SAN_ERR_SHAPE;
+    append_kernel<<<(unsigned)grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(p);
+    return cuda_status(cudaGetLastError());
+}
+
+int32_t san_attn_weights(san_ctx* ctx, int32_t kind, int32_t block, const void* d_q,
+                         const int32_t* d_ids, const int32_t* d_lens, int32_t n_items,
+                         int32_t max_len, float* d_S, int64_t ld_s, void* stream) {
+    if (!ctx || !d_q || !d_ids || !d_lens || !d_S) return SAN_ERR_NULL;
+    if (kind != SAN_SELF && kind != SAN_ENCDEC) return SAN_ERR_RANGE;
+    const san_config& c = ctx->cfg;
+    if (kind == SAN_SELF && c.self_is_aan) return SAN_ERR_UNSUPPORTED;
+    const Policy& pol = kind == SAN_SELF ? ctx->self_pol : ctx->enc_pol;
+    if (block < 0 || block >= pol.n_blocks) return SAN_ERR_RANGE;
+    const int cap = kind == SAN_SELF ? c.max_tgt_len : c.max_src_len;
+    const int max_ids = kind == SAN_SELF ? ctx->n_seqs : c.max_sent;
+    if (n_items < 0 || n_items > max_ids) return SAN_ERR_SHAPE;
+    if (max_len == 0) max_len = cap;
+    if (max_len < 1 || max_len > cap) return SAN_ERR_SHAPE;
+    if (ld_s < max_len) return SAN_ERR_SHAPE;
+    if (n_items == 0) return SAN_OK;
+
+    WeightsParams p;
+    const size_t plane = kind == SAN_SELF ? ctx->self_plane_bytes : ctx->mem_plane_bytes;
+    p.q = d_q;
+    p.K = ctx->cache + (kind == SAN_SELF ? ctx->off_self_k : ctx->off_mem_k) + plane * block;
+    p.ids = d_ids; p.lens = d_lens; p.S = d_S; p.ld_s = ld_s;
+    p.n_items = n_items; p.H = c.n_heads; p.nq = kind == SAN_SELF ? 1 : c.beam;
+    p.cap_len = cap; p.max_ids = max_ids; p.max_len = max_len;
+    const long long rows = (long long)n_items * c.n_heads;
+    pick_spans(ctx, rows, max_len, rows * p.nq * 2, &p.span_len, &p.n_spans_max);
+    p.part = ctx->part; p.tickets = ctx->tickets; p.err = ctx->err;
+    p.scale_log2e = (float)(1.4426950408889634 / std::sqrt((double)kDh));
+    const long long warps = rows * p.n_spans_max;
+    const long long grid = (warps + kWarpsPerCta - 1) / kWarpsPerCta;
+    if (grid > 0x7fffffffLL) return SAN_ERR_SHAPE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int nq_t = pick_nq_template(p.nq);
+    cudaError_t e = c.dtype == SAN_BF16 ? launch_weights<__nv_bfloat16>(p, nq_t, (unsigned)grid, st)
+                                        : launch_weights<float>(p, nq_t, (unsigned)grid, st);
+    return cuda_status(e);
+}
+
+int32_t san_attn_apply(san_ctx* ctx, int32_t kind, int32_t block, int32_t layer_begin,
+                       int32_t layer_end, const float* d_S, int64_t ld_s, const int32_t* d_ids,
+                       const int32_t* d_pos_begin, const int32_t* d_pos_end, int32_t n_items,
+                       int32_t max_len, void* d_out, int32_t accumulate, void* stream) {
+    if (!ctx || !d_S || !d_ids || !d_pos_end || !d_out) return SAN_ERR_NULL;
+    if (kind != SAN_SELF && kind != SAN_ENCDEC) return SAN_ERR_RANGE;
+    const san_config& c = ctx->cfg;
+    if (kind == SAN_SELF && c.self_is_aan) return SAN_ERR_UNSUPPORTED;
+    const Policy& pol = kind == SAN_SELF ? ctx->self_pol : ctx->enc_pol;
+    if (block < 0 || block >= pol.n_blocks) return SAN_ERR_RANGE;
+    const int first = pol.first_layer_of_block[block], size = pol.size_of_block[block];
+    if (layer_begin < first || layer_end > first + size || layer_begin >= layer_end) return SAN_ERR_RANGE;
+    const bool v_by_block = (kind == SAN_ENCDEC && c.encdec_shared_context);
+    if (v_by_block && (layer_begin != first || layer_end != first + 1)) return SAN_ERR_RANGE;
+    const int cap = kind == SAN_SELF ? c.max_tgt_len : c.max_src_len;
+    const int max_ids = kind == SAN_SELF ? ctx->n_seqs : c.max_sent;
+    if (n_items < 0 || n_items > max_ids) return SAN_ERR_SHAPE;
+    if (max_len == 0) max_len = cap;
+    if (max_len < 1 || max_len > cap) return SAN_ERR_SHAPE;
+    if (ld_s < max_len) return SAN_ERR_SHAPE;
+    if (n_items == 0) return SAN_OK;
+
+    ApplyParams p;
+    const size_t plane = kind == SAN_SELF ? ctx->self_plane_bytes : ctx->mem_plane_bytes;
+    const int v_plane0 = v_by_block ? block : layer_begin;
+    p.S = d_S; p.ld_s = ld_s;
+    p.V = ctx->cache + (kind == SAN_SELF ? ctx->off_self_v : ctx->off_mem_v) + plane * v_plane0;
+    p.plane_elems = (long long)(plane / ctx->elem_bytes);
+    p.ids = d_ids; p.pos_begin = d_pos_begin; p.pos_end = d_pos_end; p.out = d_out;
+    p.n_items = n_items; p.H = c.n_heads; p.nq = kind == SAN_SELF ? 1 : c.beam;
+    p.cap_len = cap; p.max_ids = max_ids; p.max_len = max_len;
+    p.n_layers = layer_end - layer_begin;
+    p.accumulate = accumulate ? 1 : 0;
+    const long long rows = (long long)n_items * c.n_heads;
+    // enough rows to fill the GPU: one warp keeps S on chip for every layer of the call;
+    // otherwise give each layer its own warp, then split the positions as well
+    p.layers_per_warp = (rows >= (long long)ctx->sm_count * 16) ? p.n_layers : 1;
+    const int n_lgroups = ceil_div(p.n_layers, p.layers_per_warp);
+    pick_spans(ctx, rows * n_lgroups, max_len, rows * p.n_layers * p.nq * kDh, &p.span_len, &p.n_spans_max);
+    p.part = ctx->part; p.tickets = ctx->tickets; p.err = ctx->err;
+    const long long warps = rows * n_lgroups * p.n_spans_max;
+    const long long grid = (warps + kWarpsPerCta - 1) / kWarpsPerCta;
+    if (grid > 0x7fffffffLL) return SAN_ERR_SHAPE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int nq_t = pick_nq_template(p.nq);
+    cudaError_t e = c.dtype == SAN_BF16 ? launch_apply<__nv_bfloat16>(p, nq_t, (unsigned)grid, st)
+                                        : launch_apply<float>(p, nq_t, (unsigned)grid, st);
+    return cuda_status(e);
+}
+
+int32_t san_aan_step(san_ctx* ctx, int32_t layer_begin, int32_t layer_end, const void* d_x,
+                     const int32_t* d_ids, const int32_t* d_t, int32_t n_items, void* d_out,
+                     void* stream) {
+    if (!ctx || !d_x || !d_ids || !d_t || !d_out) return SAN_ERR_NULL;
+    const san_config& c = ctx->cfg;
+    if (!c.self_is_aan) return SAN_ERR_UNSUPPORTED;
+    if (layer_begin < 0 || layer_end > c.n_layers || layer_begin >= layer_end) return SAN_ERR_RANGE;
+    if (n_items < 0 || n_items > ctx->n_seqs) return SAN_ERR_SHAPE;
+    if (n_items == 0) return SAN_OK;
+    AanParams p;
+    p.x = d_x; p.out = d_out;
+    p.sum = reinterpret_cast<float*>(ctx->cache + ctx->off_aan);
+    p.ids = d_ids; p.t = d_t; p.n_items = n_items; p.d = c.n_heads * kDh;
+    p.max_ids = ctx->n_seqs; p.max_t = c.max_tgt_len;
+    p.n_layers = layer_end - layer_begin; p.layer_begin = layer_begin; p.err = ctx->err;
+    const long long units = (long long)p.n_layers * n_items * (p.d / 4);
+    const long long grid = (units + 255) / 256;
+    if (grid > 0x7fffffffLL) return SAN_ERR_SHAPE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (c.dtype == SAN_BF16) aan_kernel<__nv_bfloat16><<<(unsigned)grid, 256, 0, st>>>(p);
+    else aan_kernel<float><<<(unsigned)grid, 256, 0, st>>>(p);
+    return cuda_status(cudaGetLastError());
+}
+
+int32_t san_device_status(san_ctx* ctx, int32_t* first_error, int32_t* detail, void* stream) {
+    if (!ctx || !first_error) return SAN_ERR_NULL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int words[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    cudaError_t e = cudaMemcpyAsync(words, ctx->err, sizeof(words), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e == cudaSuccess && words[0] != 0) {
+        e = cudaMemsetAsync(ctx->err, 0, sizeof(words), st);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    }
+    if (e != cudaSuccess) return SAN_ERR_CUDA;
+    *first_error = words[0];
+    if (detail) for (int i = 0; i < 4; ++i) detail[i] = words[1 + i];
+    return SAN_OK;
+}
+
+const char* san_status_string(int32_t status) {
+    switch (status) {
+        case SAN_OK: return "ok";
+        case SAN_ERR_NULL: return "a required pointer is NULL";
+        case SAN_ERR_SHAPE: return "a size or count is out of range";
+        case SAN_ERR_POLICY: return "invalid sharing policy";
+        case SAN_ERR_CAPACITY: return "a buffer is too small or the policy has more blocks than key planes";
+        case SAN_ERR_DTYPE: return "unknown element type";
+        case SAN_ERR_RANGE: return "layer, block or position outside the allowed range";
+        case SAN_ERR_CUDA: return "a CUDA runtime call failed";
+        case SAN_ERR_DEVICE_CHECK: return "a kernel skipped an item with an invalid id, length or position";
+        case SAN_ERR_TIMEOUT: return "a bounded device wait ran out";
+        case SAN_ERR_UNSUPPORTED: return "not supported by this configuration";
+        default: return "unknown status";
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,30 @@
+// The context behind the opaque san_ctx handle: host-side tables plus pointers into the
+// caller's device buffers.  Nothing here owns device memory.
+#pragma once
+
+#include <stddef.h>
+#include <stdint.h>
+
+#include "../../include/san.h"
+#include "san_policy.h"
+
+struct san_ctx {
+    san_config cfg;
+    san::Policy self_pol, enc_pol;
+    int elem_bytes = 0, n_seqs = 0, sm_count = 0;
+
+    // cache arena (caller-owned)
+    char* cache = nullptr;
+    size_t cache_bytes_needed = 0;
+    size_t self_plane_bytes = 0, mem_plane_bytes = 0, aan_plane_bytes = 0;
+    int n_self_k_planes = 0, n_self_v_planes = 0, n_enc_k_planes = 0, n_enc_v_planes = 0;
+    size_t off_self_k = 0, off_self_v = 0, off_mem_k = 0, off_mem_v = 0, off_aan = 0;
+
+    // workspace (caller-owned): error words, tickets of split rows, their partial sums
+    char* ws = nullptr;
+    size_t ws_bytes_needed = 0, ws_off_tickets = 0, ws_off_part = 0;
+    size_t n_tickets = 0, part_floats = 0;
+    int* err = nullptr;
+    int* tickets = nullptr;
+    float* part = nullptr;
+};

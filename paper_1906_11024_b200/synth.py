@@ -187,3 +187,13 @@ def beam_parents(w: Workload, step: int) -> np.ndarray:
     """A random parent beam (0..beam-1) for every sequence, as beam search would pick."""
     rng = np.random.default_rng([int(w.seed), TAG_PARENT, int(step)])
     return rng.integers(0, w.beam, size=w.n_seqs, dtype=np.int64).astype(np.int32)
+
+
+def self_prefill(w: Workload, layer: int):
+    """Keys and values already cached before the first checked step: ``[n_seqs, max_tgt, H, d_h]``.
+
+    Rows at or beyond a sequence's prefix length are drawn but never used.
+    """
+    shp = (w.n_seqs, w.max_tgt_len(), w.n_heads, w.d_head)
+    return (normal(w.seed, TAG_PREFIX, 1, layer, shp, w.dtype),
+            normal(w.seed, TAG_PREFIX, 2, layer, shp, w.dtype))

@@ -1,0 +1,256 @@
+"""Edge cases of the CUDA path: bit-exact cache contents, device-side checks that skip
+(never fault), position ranges with accumulate, runtime policy changes, empty inputs."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import san_oracle as so
+from paper_1906_11024_b200 import binding as B
+from paper_1906_11024_b200 import build as san_build
+from paper_1906_11024_b200 import synth
+from paper_1906_11024_b200.driver import Decoder, to_device, to_host_f32
+from tests.helpers import TOL, normwise_err, weights_err
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    san_build.build()
+    B.lib()
+
+
+def _small(dtype=synth.BF16, **kw):
+    base = dict(name="edge", dtype=dtype, n_layers=4, n_heads=2, d_head=64, n_sent=3, beam=2,
+                self_blocks=(1, 3), encdec_blocks=(2, 2), src_lo=5, src_hi=9, tgt_rule="fixed", tgt_fixed=12,
+                ragged_prefix=False, self_is_aan=False, seed=77)
+    base.update(kw)
+    return synth.Workload(**base)
+
+
+def _i32(x, dev):
+    return torch.tensor(x, dtype=torch.int32, device=dev)
+
+
+@pytest.mark.parametrize("dtype", [synth.BF16, synth.F32])
+def test_cache_contents_bit_exact_after_scripted_appends(dtype):
+    """The arena layout is [self K planes][self V planes][memory K][memory V], each plane
+    [id][head][row][64]; after a scripted series of appends it equals a host-side scatter."""
+    w = _small(dtype)
+    dec = Decoder(w)
+    dev = dec.device
+    M, H, dh, n, T = w.n_layers, w.n_heads, w.d_head, w.n_seqs, w.max_tgt_len()
+    e = w.elem_bytes
+    udt = np.uint16 if dtype == synth.BF16 else np.uint32
+    Ns = len(w.self_blocks)
+    dec.cache.zero_()
+    expK = np.zeros((Ns, n, H, T, dh), udt)
+    expV = np.zeros((M, n, H, T, dh), udt)
+    bits = (lambda a: synth.bf16_bits(a)) if dtype == synth.BF16 else (lambda a: a.view(np.uint32))
+    script = [([0, 1, 2, 3, 4, 5], [0, 0, 0, 0, 0, 0]), ([5, 2], [1, 1]), ([3], [11]), ([0, 1, 2, 3, 4, 5], [4, 3, 2, 1, 7, 2])]
+    for step, (ids, pos) in enumerate(script):
+        qs, ks, vs = zip(*[synth.self_qkv(w, step, l) for l in range(M)])
+        k_new = np.stack([ks[l][ids] for l in dec.self_first])
+        v_new = np.stack([vs[l][ids] for l in range(M)])
+        rc = B.san_cache_append(dec.ctx, B.SAN_SELF, 0, M, to_device(k_new, dtype, dev), to_device(v_new, dtype, dev),
+                                _i32(ids, dev), _i32(pos, dev), None, len(ids), 1)
+        assert rc == B.SAN_OK
+        for i, (s, p) in enumerate(zip(ids, pos)):
+            expK[:, s, :, p, :] = bits(k_new[:, i])
+            expV[:, s, :, p, :] = bits(v_new[:, i])
+    torch.cuda.synchronize()
+    assert dec.device_status()[0] == 0
+    raw = dec.cache.cpu().numpy()
+    plane = n * H * T * dh * e
+    gotK = raw[:Ns * plane].view(udt).reshape(Ns, n, H, T, dh)
+    gotV = raw[Ns * plane:(Ns + M) * plane].view(udt).reshape(M, n, H, T, dh)
+    assert np.array_equal(gotK, expK)
+    assert np.array_equal(gotV, expV)
+    # encoder memory: bulk rows, ragged per sentence; rows beyond a sentence's length stay untouched
+    src = dec.load_encoder_memory()
+    raw = dec.cache.cpu().numpy()
+    Ls = w.max_src_len()
+    mplane = w.n_sent * H * Ls * dh * e
+    off = (Ns + M) * plane
+    Ne = len(w.encdec_blocks)
+    gotKm = raw[off:off + Ne * mplane].view(udt).reshape(Ne, w.n_sent, H, Ls, dh)
+    gotVm = raw[off + Ne * mplane: off + (Ne + M) * mplane].view(udt).reshape(M, w.n_sent, H, Ls, dh)
+    for l in range(M):
+        Km, Vm = synth.encoder_memory(w, l)
+        for g in range(w.n_sent):
+            L = src[g]
+            assert np.array_equal(gotVm[l, g, :, :L], bits(Vm[g, :L]).transpose(1, 0, 2))
+            assert not gotVm[l, g, :, L:].any()
+            if l in dec.enc_first:
+                c = dec.enc_first.index(l)
+                assert np.array_equal(gotKm[c, g, :, :L], bits(Km[g, :L]).transpose(1, 0, 2))
+                assert not gotKm[c, g, :, L:].any()
+    dec.close()
+
+
+def test_device_checks_skip_bad_items_and_report():
+    w = _small()
+    dec = Decoder(w)
+    dev = dec.device
+    M, n = w.n_layers, w.n_seqs
+    sb = dec.new_step_buffers()
+    host = dec.fill_step_inputs(sb, 0, np.arange(n), np.zeros(n, np.int32))
+    dec.load_encoder_memory()
+    dec.step(sb)
+    assert dec.device_status()[0] == 0
+    good = to_host_f32(sb.O_self).copy()
+    # (a) a sequence id out of range in append: that item is skipped, the rest is written
+    sb.ids.copy_(_i32([0, 1, 99, 3, 4, 5], dev))
+    rc = B.san_cache_append(dec.ctx, B.SAN_SELF, 0, M, sb.k_new, sb.v_new, sb.ids, sb.pos, None, n, 1)
+    assert rc == B.SAN_OK
+    err, detail = dec.device_status()
+    assert err == B.SAN_ERR_DEVICE_CHECK and detail[1] == 2 and detail[2] == 99
+    assert dec.device_status()[0] == 0            # reading clears the word
+    # (b) a position beyond capacity
+    sb.ids.copy_(_i32(list(range(n)), dev))
+    sb.pos.copy_(_i32([0, 0, 0, w.max_tgt_len(), 0, 0], dev))
+    B.san_cache_append(dec.ctx, B.SAN_SELF, 0, M, sb.k_new, sb.v_new, sb.ids, sb.pos, None, n, 1)
+    err, detail = dec.device_status()
+    assert err == B.SAN_ERR_DEVICE_CHECK and detail[1] == 3
+    # (c) weights with a zero length and a length beyond the host bound: rows skipped, others fine
+    sb.pos.zero_()
+    S = torch.full_like(sb.S_self[0], -7.0)
+    sb.lens.copy_(_i32([1, 0, 1, 1, 5, 1], dev))
+    rc = B.san_attn_weights(dec.ctx, B.SAN_SELF, 0, sb.q_self[0], sb.ids, sb.lens, n, 4, S, dec.ld_t)
+    assert rc == B.SAN_OK
+    err, detail = dec.device_status()
+    assert err == B.SAN_ERR_DEVICE_CHECK
+    Sh = S.cpu().numpy()
+    assert np.all(Sh[[0, 2, 3, 5], :, 0] == 1.0)           # a cache of one position
+    assert np.all(Sh[[1, 4]] == -7.0)                      # skipped rows untouched
+    # (d) apply with an end before the begin
+    pb, pe = _i32([0, 2, 0, 0, 0, 0], dev), _i32([1, 1, 1, 1, 1, 1], dev)
+    out = torch.zeros_like(sb.O_self[:1])
+    B.san_attn_apply(dec.ctx, B.SAN_SELF, 0, 0, 1, sb.S_self[0], dec.ld_t, sb.ids, pb, pe, n, 0, out, 0)
+    assert dec.device_status()[0] == B.SAN_ERR_DEVICE_CHECK
+    # the context is still usable and gives the same answer as before
+    sb2 = dec.new_step_buffers()
+    dec.fill_step_inputs(sb2, 0, np.arange(n), np.zeros(n, np.int32))
+    dec.step(sb2)
+    assert dec.device_status()[0] == 0
+    assert np.array_equal(to_host_f32(sb2.O_self), good)
+    dec.close()
+
+
+def test_host_checks_on_a_live_context():
+    w = _small()
+    dec = Decoder(w)
+    sb = dec.new_step_buffers()
+    n, M, ctx = w.n_seqs, w.n_layers, dec.ctx
+    # keys for a range without a block-first layer / missing keys for one that has it
+    assert B.san_cache_append(ctx, B.SAN_SELF, 2, 4, sb.k_new, sb.v_new, sb.ids, sb.pos, None, n, 1) == B.SAN_ERR_RANGE
+    assert B.san_cache_append(ctx, B.SAN_SELF, 0, 2, None, sb.v_new, sb.ids, sb.pos, None, n, 1) == B.SAN_ERR_NULL
+    assert B.san_cache_append(ctx, B.SAN_SELF, 0, 5, sb.k_new, sb.v_new, sb.ids, sb.pos, None, n, 1) == B.SAN_ERR_RANGE
+    assert B.san_cache_append(ctx, B.SAN_SELF, 0, 4, sb.k_new, sb.v_new, sb.ids, sb.pos, None, n + 1, 1) == B.SAN_ERR_SHAPE
+    assert B.san_cache_append(ctx, 2, 0, 4, sb.k_new, sb.v_new, sb.ids, sb.pos, None, n, 1) == B.SAN_ERR_RANGE
+    assert B.san_attn_weights(ctx, B.SAN_SELF, 2, sb.q_self[0], sb.ids, sb.lens, n, 0, sb.S_self[0], dec.ld_t) == B.SAN_ERR_RANGE
+    assert B.san_attn_weights(ctx, B.SAN_SELF, 0, sb.q_self[0], sb.ids, sb.lens, n, 13, sb.S_self[0], dec.ld_t) == B.SAN_ERR_SHAPE
+    assert B.san_attn_weights(ctx, B.SAN_SELF, 0, sb.q_self[0], sb.ids, sb.lens, n, 12, sb.S_self[0], 8) == B.SAN_ERR_SHAPE
+    # a layer outside the block
+    assert B.san_attn_apply(ctx, B.SAN_SELF, 1, 0, 2, sb.S_self[1], dec.ld_t, sb.ids, None, sb.lens, n, 0, sb.O_self, 0) == B.SAN_ERR_RANGE
+    assert B.san_attn_apply(ctx, B.SAN_SELF, 0, 0, 2, sb.S_self[0], dec.ld_t, sb.ids, None, sb.lens, n, 0, sb.O_self, 0) == B.SAN_ERR_RANGE
+    assert B.san_aan_step(ctx, 0, M, sb.v_new, sb.ids, sb.lens, n, sb.O_self) == B.SAN_ERR_UNSUPPORTED
+    # zero items is a no-op
+    assert B.san_attn_weights(ctx, B.SAN_SELF, 0, sb.q_self[0], sb.ids, sb.lens, 0, 0, sb.S_self[0], dec.ld_t) == B.SAN_OK
+    assert B.san_cache_append(ctx, B.SAN_SELF, 0, 4, sb.k_new, sb.v_new, sb.ids, sb.pos, None, 0, 1) == B.SAN_OK
+    dec.close()
+
+
+def test_policy_tables_and_runtime_change():
+    """Integer tables are bit-exact; a policy with more blocks than key planes is refused."""
+    w = _small(self_blocks=(2, 2), encdec_blocks=(4,))
+    dec = Decoder(w)
+    ctx = dec.ctx
+    assert B.san_policy_get_map(ctx, B.SAN_SELF) == (0, [0, 0, 1, 1], [0, 2])
+    assert B.san_policy_get_map(ctx, B.SAN_ENCDEC) == (0, [0, 0, 0, 0], [0])
+    assert B.san_policy_set_sizes(ctx, B.SAN_SELF, [1, 3]) == B.SAN_OK
+    assert B.san_policy_get_map(ctx, B.SAN_SELF) == (0, [0, 1, 1, 1], [0, 1])
+    assert B.san_policy_set_map(ctx, B.SAN_SELF, [0, 0, 0, 0]) == B.SAN_OK
+    assert B.san_policy_get_map(ctx, B.SAN_SELF) == (0, [0, 0, 0, 0], [0])
+    assert B.san_policy_set_sizes(ctx, B.SAN_SELF, [1, 1, 2]) == B.SAN_ERR_CAPACITY       # 3 blocks, 2 key planes
+    assert B.san_policy_set_sizes(ctx, B.SAN_ENCDEC, [2, 2]) == B.SAN_ERR_CAPACITY
+    assert B.san_policy_set_sizes(ctx, B.SAN_SELF, [2, 3]) == B.SAN_ERR_POLICY
+    assert B.san_policy_set_map(ctx, B.SAN_SELF, [0, 2, 2, 2]) == B.SAN_ERR_POLICY
+    assert B.san_policy_set_map(ctx, B.SAN_SELF, [0, 0, 1]) == B.SAN_ERR_SHAPE
+    assert B.san_policy_get_map(ctx, B.SAN_SELF) == (0, [0, 0, 0, 0], [0])                  # unchanged by failures
+    dec.close()
+
+
+@pytest.mark.parametrize("dtype", [synth.BF16, synth.F32])
+def test_history_then_newest_row_with_accumulate(dtype):
+    """A layer whose newest value row arrives late: apply the block's weights to the history
+    [0,t) for all layers in one launch, then add S_t * v_t per layer with accumulate."""
+    w = _small(dtype, self_blocks=(4,), tgt_fixed=40)
+    dec = Decoder(w)
+    dev = dec.device
+    M, n, H, dh = w.n_layers, w.n_seqs, w.n_heads, w.d_head
+    T = 37
+    ids = np.arange(n, dtype=np.int32)
+    o = so.Oracle(M, H, dh, w.n_sent, w.beam, w.max_tgt_len(), w.max_src_len(), w.self_blocks, w.encdec_blocks)
+    for l in range(M):
+        K, V = synth.self_prefill(w, l)
+        k_dev = to_device(K, dtype, dev) if l == 0 else None
+        rows = _i32([T] * n, dev)
+        assert B.san_cache_append(dec.ctx, B.SAN_SELF, l, l + 1, k_dev, to_device(V, dtype, dev), _i32(ids, dev), None,
+                                  rows, n, w.max_tgt_len()) == B.SAN_OK
+        for p in range(T):
+            o.self_append(l, ids, np.full(n, p), K[:, p] if l == 0 else None, V[:, p])
+    q = synth.self_qkv(w, 0, 0)[0]
+    lens = _i32([T] * n, dev)
+    S = torch.zeros(n, H, dec.ld_t, device=dev)
+    assert B.san_attn_weights(dec.ctx, B.SAN_SELF, 0, to_device(q, dtype, dev), _i32(ids, dev), lens, n, T, S, dec.ld_t) == 0
+    out = torch.zeros(M, n, H, dh, dtype=dec.tdtype, device=dev)
+    hist_end = _i32([T - 1] * n, dev)
+    assert B.san_attn_apply(dec.ctx, B.SAN_SELF, 0, 0, M, S, dec.ld_t, _i32(ids, dev), None, hist_end, n, T, out, 0) == 0
+    for l in range(M):   # the newest row of each layer, one layer at a time
+        assert B.san_attn_apply(dec.ctx, B.SAN_SELF, 0, l, l + 1, S, dec.ld_t, _i32(ids, dev), hist_end, lens, n, T,
+                                out[l], 1) == 0
+    assert dec.device_status()[0] == 0
+    got = to_host_f32(out)
+    for l in range(M):
+        Sref, Oref = o.self_attend(l, ids, np.full(n, T), q if l == 0 else None)
+        # bf16 output is rounded twice on this route (history, then history + newest row)
+        assert normwise_err(got[l], Oref) <= TOL[dtype]
+        if l == 0:
+            assert weights_err(S.cpu().numpy()[:, :, :T], Sref[:, :, :T]) <= 1e-5
+    # an empty range writes zeros (or leaves the output alone with accumulate)
+    z = torch.ones(1, n, H, dh, dtype=dec.tdtype, device=dev)
+    zero = _i32([0] * n, dev)
+    assert B.san_attn_apply(dec.ctx, B.SAN_SELF, 0, 0, 1, S, dec.ld_t, _i32(ids, dev), None, zero, n, T, z, 0) == 0
+    assert not to_host_f32(z).any()
+    dec.close()
+
+
+def test_results_do_not_depend_on_item_order_or_subset():
+    w = _small()
+    dec = Decoder(w)
+    dec.load_encoder_memory()
+    n = w.n_seqs
+    pos = np.array([3, 0, 5, 1, 2, 4], np.int32)
+    # fill some history first
+    for l in range(w.n_layers):
+        K, V = synth.self_prefill(w, l)
+        dev = dec.device
+        B.check(B.san_cache_append(dec.ctx, B.SAN_SELF, l, l + 1, to_device(K, w.dtype, dev) if l in dec.self_first else None,
+                                   to_device(V, w.dtype, dev), _i32(list(range(n)), dev), None, _i32(pos.tolist(), dev), n,
+                                   w.max_tgt_len()))
+    sb = dec.new_step_buffers()
+    dec.fill_step_inputs(sb, 3, np.arange(n), pos)
+    dec.step(sb)
+    full = to_host_f32(sb.O_self).copy()
+    fullS = sb.S_self.cpu().numpy().copy()
+    pick = np.array([4, 5, 0, 1], np.int32)         # whole sentences 2 and 0, reordered
+    sb2 = dec.new_step_buffers(len(pick), 2)
+    dec.fill_step_inputs(sb2, 3, pick, pos[pick], np.array([2, 0], np.int32))
+    dec.step(sb2)
+    assert dec.device_status()[0] == 0
+    assert np.array_equal(to_host_f32(sb2.O_self), full[:, pick])
+    for i, s in enumerate(pick):
+        L = pos[s] + 1
+        assert np.array_equal(sb2.S_self.cpu().numpy()[:, i, :, :L], fullS[:, s, :, :L])
+    dec.close()

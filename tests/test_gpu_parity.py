@@ -1,0 +1,166 @@
+"""Parity of the CUDA path (through the C ABI) against the CPU oracle, element by element.
+
+Tolerances: outputs O within 1e-5 (float32) / 1e-2 (bf16 inputs, float32 accumulation),
+measured per output vector as ||x - ref||_inf / ||ref||_inf; weights S within 1e-5
+element-wise (relative, floor 1e-7) with rows summing to one; cache contents bit-exact.
+"""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from paper_1906_11024_b200 import binding as B
+from paper_1906_11024_b200 import build as san_build
+from paper_1906_11024_b200 import synth
+from paper_1906_11024_b200.driver import Decoder, to_device, to_host_f32
+from tests.helpers import TOL, TOL_S, OracleRun, normwise_err, weights_err
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    san_build.build()
+    B.lib()
+
+
+def _compare(w, dec, sb, ref, n, lens, src_lens_per_seq, tag):
+    tol = TOL[w.dtype]
+    first_error, detail = dec.device_status()
+    assert first_error == 0, (tag, first_error, detail)
+    if not w.self_is_aan:
+        S = to_host_f32(sb.S_self)
+        for b in range(S.shape[0]):
+            for i in range(n):
+                L = int(lens[i])
+                err = weights_err(S[b, i, :, :L], ref["S_self"][b, i, :, :L])
+                assert err <= TOL_S, (tag, "S_self", b, i, err)
+                assert np.abs(S[b, i, :, :L].astype(np.float64).sum(-1) - 1.0).max() <= 1e-5
+    O = to_host_f32(sb.O_self)
+    err = normwise_err(O, ref["O_self"])
+    assert err <= tol, (tag, "O_self", err)
+    S = to_host_f32(sb.S_enc)
+    for c in range(S.shape[0]):
+        for i in range(S.shape[1]):
+            L = int(src_lens_per_seq[i])
+            e2 = weights_err(S[c, i, :, :L], ref["S_enc"][c, i, :, :L])
+            assert e2 <= TOL_S, (tag, "S_enc", c, i, e2)
+    O = to_host_f32(sb.O_enc)
+    err = normwise_err(O, ref["O_enc"])
+    assert err <= tol, (tag, "O_enc", err)
+
+
+def _run(w, check_steps=None, max_steps=None, shared_context=False, jumps=None):
+    """Decode the workload on both sides.  Sequences start at their prefix length, advance in
+    lock-step and drop out when their sentence is done.  ``jumps`` = list of (start_pos, n_steps)
+    segments for long runs: the caches are re-prefilled to start_pos before each segment."""
+    dec = Decoder(w, encdec_shared_context=shared_context)
+    orc = OracleRun(w, shared_context)
+    dec.load_encoder_memory()
+    T = np.repeat(w.tgt_lens(), w.beam)
+    src_seq = np.repeat(w.src_lens(), w.beam)
+    all_ids = np.arange(w.n_seqs, dtype=np.int32)
+    segments = jumps if jumps else [(None, max_steps if max_steps else int(T.max()))]
+    checked = 0
+    for start, n_steps in segments:
+        pos = w.prefix_lens().astype(np.int32) if start is None else np.full(w.n_seqs, start, np.int32)
+        if not w.self_is_aan and pos.max() > 0:
+            _prefill(dec, orc, w, all_ids, pos)
+        for g in range(n_steps):
+            active = all_ids[pos < T]
+            if len(active) == 0:
+                break
+            # whole sentences stay active together (all beams of a sentence share T)
+            sent = np.unique(active // w.beam).astype(np.int32)
+            sb = dec.new_step_buffers(len(active), len(sent))
+            step_id = g if start is None else 100000 + start + g
+            host = dec.fill_step_inputs(sb, step_id, active, pos[active], sent)
+            dec.step(sb)
+            do_check = check_steps is None or g in check_steps
+            ref = orc.step(host, active, pos[active], want_S=do_check)
+            if do_check:
+                _compare(w, dec, sb, ref, len(active), pos[active] + 1, src_seq[host["beams"]], (w.name, start, g))
+                checked += 1
+            pos[active] += 1
+    assert checked > 0
+    dec.close()
+
+
+def _prefill(dec, orc, w, ids, n_rows):
+    orc.prefill(ids, n_rows)
+    dev = dec.device
+    t_ids = torch.from_numpy(ids).to(dev)
+    t_rows = torch.from_numpy(n_rows.astype(np.int32)).to(dev)
+    for l in range(w.n_layers):
+        K, V = synth.self_prefill(w, l)
+        k_dev = to_device(K, w.dtype, dev) if l in dec.self_first else None
+        v_dev = to_device(V, w.dtype, dev)
+        B.check(B.san_cache_append(dec.ctx, B.SAN_SELF, l, l + 1, k_dev, v_dev, t_ids, None, t_rows,
+                                   len(ids), w.max_tgt_len()), "prefill")
+    torch.cuda.synchronize(dev)
+
+
+def test_tiny_fp32_every_step():
+    """First configuration in full: float32, blocks {2,2,2} / {3,3}, 16 steps, tolerance 1e-5."""
+    _run(synth.WORKLOADS["tiny"])
+
+
+def test_tiny_fp32_unshared_equals_standard_attention():
+    _run(synth.unshared(synth.WORKLOADS["tiny"]))
+
+
+def test_base_bf16_scaled_every_step():
+    _run(synth.scaled(synth.WORKLOADS["base"], 8))
+
+
+def test_base_bf16_full_size_sampled_steps():
+    w = synth.WORKLOADS["base"]
+    last = int(w.tgt_lens().max()) - 1
+    _run(w, check_steps={0, 1, 17, 33, last})
+
+
+def test_big_bf16_ragged_scaled_every_step():
+    _run(synth.scaled(synth.WORKLOADS["big"], 6))
+
+
+def test_big_bf16_full_size_sampled_steps():
+    _run(synth.WORKLOADS["big"], check_steps={0, 5, 40}, max_steps=41)
+
+
+def test_long_bf16_split_rows_scaled():
+    """Few rows and long caches: rows are split over several warps (ticket combine)."""
+    w = synth.scaled(synth.WORKLOADS["long"], 2)
+    _run(w, jumps=[(0, 3), (30, 4), (62, 4), (126, 4), (254, 4), (508, 4)])
+
+
+def test_long_bf16_full_size_sampled_steps():
+    _run(synth.WORKLOADS["long"], jumps=[(0, 2), (63, 3), (255, 3), (510, 2)])
+
+
+def test_aan_bf16_scaled_every_step():
+    _run(synth.scaled(synth.WORKLOADS["aan"], 8), max_steps=80)
+
+
+def test_aan_bf16_full_size_sampled_steps():
+    _run(synth.WORKLOADS["aan"], check_steps={0, 1, 40, 79})
+
+
+def test_encdec_shared_context_eq5():
+    """Eq. 5: one output per enc-dec block; upper layers of the block reuse it."""
+    _run(synth.scaled(synth.WORKLOADS["base"], 4), max_steps=6, shared_context=True)
+    _run(dataclasses.replace(synth.scaled(synth.WORKLOADS["tiny"], 2), encdec_blocks=(3, 3)), max_steps=4,
+         shared_context=True)
+
+
+@pytest.mark.parametrize("beam", [1, 2, 3, 5, 8])
+def test_other_beam_sizes(beam):
+    """The paper sweeps beam sizes (Figure 5); key tiles are scored once for all beams."""
+    w = dataclasses.replace(synth.scaled(synth.WORKLOADS["base"], 3), beam=beam, name=f"beam{beam}")
+    _run(w, max_steps=5)
+
+
+def test_fp32_long_rows_and_splits():
+    w = dataclasses.replace(synth.WORKLOADS["tiny"], name="tiny-long", src_lo=300, src_hi=300,
+                            tgt_rule="fixed", tgt_fixed=300)
+    _run(w, jumps=[(0, 2), (127, 3), (255, 3), (297, 3)])
