@@ -1,0 +1,494 @@
+#!/usr/bin/env python
+"""Benchmark of the shared-attention decode step.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload base|big|long|aan|tiny]
+    python bench.py --impl reference ...          # the CPU oracle as the reference arm
+
+A step is one decode step of the whole attention path (cache append, weights, apply for
+self and encoder-decoder attention of every layer, or AAN + enc-dec) for every sequence of
+the workload, at the decode run's average state (each sequence at the middle of its own
+target length; the ragged configuration at its seeded prefix lengths).  Steps rotate over
+several independent replicas of the device state so that consecutive steps touch disjoint
+memory far larger than L2.  Prints ONE JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "decode-step attention tokens/sec"
+UNIT = "tokens/s"
+L2_BYTES = 126e6
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+# ------------------------------------------------------------------------------- workload state
+def state_positions(w):
+    """Row each sequence writes in the benchmarked step (its cache length is this + 1)."""
+    T = np.repeat(w.tgt_lens(), w.beam).astype(np.int32)
+    if w.ragged_prefix:
+        return w.prefix_lens().astype(np.int32)
+    return ((T + 1) // 2 - 1).astype(np.int32)               # middle of the run: length ceil(T/2)
+
+
+def algorithmic_bytes(w, pos):
+    """Bytes the method itself must move per step (K/V reads are the roofline count)."""
+    M, H, d, e = w.n_layers, w.n_heads, w.d_model, w.elem_bytes
+    n = w.n_seqs
+    src = w.src_lens().astype(np.int64)
+    Ns, Ne = len(w.self_blocks), len(w.encdec_blocks)
+    L = pos.astype(np.int64) + 1
+    out = {}
+    if w.self_is_aan:
+        out["self_kv"] = 0
+        out["aan"] = M * n * d * (2 * e + 8)
+        s_self = 0
+        small_self = 0
+    else:
+        out["self_kv"] = int((Ns + M) * L.sum() * d * e)
+        out["aan"] = 0
+        s_self = 8 * H * Ns * int(L.sum())
+        small_self = Ns * n * d * e + M * n * d * e + (Ns + M) * n * d * e       # q, O, appended rows
+    out["encdec_kv"] = int((Ne + M) * src.sum() * d * e)                          # once per sentence
+    s_enc = 8 * H * Ne * int(np.repeat(src, w.beam).sum())
+    small_enc = Ne * n * d * e + M * n * d * e
+    out["S"] = s_self + s_enc
+    out["small"] = small_self + small_enc
+    out["kv"] = out["self_kv"] + out["encdec_kv"] + out["aan"]
+    out["total"] = out["kv"] + out["S"] + out["small"]
+    return out
+
+
+def measured_peak_gbs():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# ------------------------------------------------------------------------------------ clocks
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), [c.strip() for c in line.split(",")]))
+
+    def stop(self, t0, t1):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        rows = [r for (t, r) in self.rows if t0 - 0.05 <= t <= t1 + 0.15] or [r for _, r in self.rows]
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except Exception:
+                continue
+            for nm, val in zip(names, r[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------- the GPU arm
+def build_replicas(w, n_rep, device):
+    import torch
+    from paper_1906_11024_b200.driver import Decoder
+    pos = state_positions(w)
+    ids = np.arange(w.n_seqs, dtype=np.int32)
+    decs, sbs = [], []
+    for r in range(n_rep):
+        dec = Decoder(w, device)
+        gen = torch.Generator(device=device)
+        gen.manual_seed(1000 + r)
+        # cache contents: seeded N(0,1) in the storage dtype (the AAN running sums are float32)
+        if w.self_is_aan:
+            dec.cache.view(torch.float32).normal_(generator=gen)
+            dec.load_encoder_memory()
+        else:
+            dec.cache.view(dec.tdtype).normal_(generator=gen)
+        sb = dec.new_step_buffers()
+        dec.fill_step_inputs(sb, r, ids, pos)
+        sb.max_len = int(pos.max()) + 1
+        sb.max_src = int(w.src_lens().max())
+        decs.append(dec)
+        sbs.append(sb)
+    torch.cuda.synchronize(device)
+    return decs, sbs, pos
+
+
+def capture(fn, device):
+    """Capture the launches fn() issues on torch's current stream into a CUDA graph."""
+    import torch
+    g = torch.cuda.CUDAGraph()
+    s = torch.cuda.Stream(device)
+    s.wait_stream(torch.cuda.current_stream(device))
+    with torch.cuda.stream(s):
+        fn()                                   # warm-up outside capture (module load, first launch)
+    torch.cuda.current_stream(device).wait_stream(s)
+    torch.cuda.synchronize(device)
+    with torch.cuda.graph(g):
+        fn()
+    return g
+
+
+def time_steps(decs, sbs, steps, warmup, device, barrier):
+    """W untimed + exactly K timed steps; steps rotate over the replicas.  Returns seconds."""
+    import torch
+    R = len(decs)
+    launches = [0]
+
+    def one(r):
+        launches[0] = decs[r].step(sbs[r])
+
+    cycle = capture(lambda: [one(r) for r in range(R)], device)
+    singles = [capture(lambda r=r: one(r), device) for r in range(max(steps % R, max(warmup, 3) % R))]
+
+    def run(k):
+        for _ in range(k // R):
+            cycle.replay()
+        for r in range(k % R):
+            singles[r].replay()
+
+    run(max(warmup, 3))
+    barrier()
+    torch.cuda.synchronize(device)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.time()
+    e0.record()
+    run(steps)
+    e1.record()
+    torch.cuda.synchronize(device)
+    t1 = time.time()
+    barrier()
+    return e0.elapsed_time(e1) * 1e-3, launches[0], (t0, t1)
+
+
+def time_dominant_kernel(w, decs, sbs, device, reps=20):
+    """Average duration of one san_attn_apply launch over the self-attention caches (the
+    kernel that moves most bytes), launches rotating over replicas and blocks."""
+    import torch
+    from paper_1906_11024_b200 import binding as B
+    R = len(decs)
+    if w.self_is_aan:
+        kind, firsts, sizes = B.SAN_ENCDEC, decs[0].enc_first, decs[0].enc_sizes
+    else:
+        kind, firsts, sizes = B.SAN_SELF, decs[0].self_first, decs[0].self_sizes
+
+    def launch_all():
+        n = 0
+        for r in range(R):
+            d, sb = decs[r], sbs[r]
+            for b, (first, size) in enumerate(zip(firsts, sizes)):
+                if kind == B.SAN_SELF:
+                    B.check(B.san_attn_apply(d.ctx, kind, b, first, first + size, sb.S_self[b], d.ld_t, sb.ids, None,
+                                             sb.lens, sb.ids.shape[0], sb.max_len, sb.O_self[first], 0))
+                else:
+                    B.check(B.san_attn_apply(d.ctx, kind, b, first, first + size, sb.S_enc[b], d.ld_s, sb.sent_ids, None,
+                                             sb.src_lens, sb.sent_ids.shape[0], sb.max_src, sb.O_enc[first], 0))
+                n += 1
+        return n
+
+    count = [0]
+    g = capture(lambda: count.__setitem__(0, launch_all()), device)
+    for _ in range(3):
+        g.replay()
+    torch.cuda.synchronize(device)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        g.replay()
+    e1.record()
+    torch.cuda.synchronize(device)
+    return e0.elapsed_time(e1) * 1e-3 / (reps * count[0]), count[0] // R
+
+
+def dominant_kernel_bytes(w, pos):
+    """Algorithmic bytes of one san_attn_apply launch (mean over the blocks of the kind)."""
+    H, d, e = w.n_heads, w.d_model, w.elem_bytes
+    if w.self_is_aan:
+        sizes = w.encdec_blocks
+        rows = int(w.src_lens().astype(np.int64).sum())
+        s_rows = int(np.repeat(w.src_lens(), w.beam).astype(np.int64).sum())
+    else:
+        sizes = w.self_blocks
+        rows = int((pos.astype(np.int64) + 1).sum())
+        s_rows = rows
+    per = [pi * rows * d * e + 4 * H * s_rows + pi * w.n_seqs * d * e for pi in sizes]
+    return float(np.mean(per))
+
+
+def time_e2e(w, dec, sb, steps, device):
+    """The same step with HOST buffers: every step copies its inputs from pinned host memory
+    to the device, runs the library calls, and reads the outputs back."""
+    import torch
+    names_in = ["x_aan", "t_aan"] if w.self_is_aan else ["q_self", "k_new", "v_new"]
+    names_in += ["q_enc", "ids", "pos", "lens", "sent_ids", "src_lens"]
+    names_out = ["O_self", "O_enc"]
+    host_in = {k: getattr(sb, k).cpu().pin_memory() for k in names_in}
+    host_out = {k: torch.empty_like(getattr(sb, k), device="cpu").pin_memory() for k in names_out}
+    h2d = sum(t.numel() * t.element_size() for t in host_in.values())
+    d2h = sum(t.numel() * t.element_size() for t in host_out.values())
+
+    def one():
+        for k, t in host_in.items():
+            getattr(sb, k).copy_(t, non_blocking=True)
+        dec.step(sb)
+        for k, t in host_out.items():
+            t.copy_(getattr(sb, k), non_blocking=True)
+
+    for _ in range(3):
+        one()
+    torch.cuda.synchronize(device)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        one()
+    e1.record()
+    torch.cuda.synchronize(device)
+    return e0.elapsed_time(e1) * 1e-3, h2d, d2h
+
+
+# ------------------------------------------------------------------------- the CPU oracle arm
+def oracle_sample(w, n_sent_sample):
+    """Oracle state for the first sentences of the workload at the benchmarked positions."""
+    from paper_1906_11024_b200 import synth
+    from tests.helpers import OracleRun
+    ws = synth.scaled(w, min(n_sent_sample, w.n_sent), w.name + "-sample")
+    orc = OracleRun(ws)
+    pos = state_positions(ws)
+    ids = np.arange(ws.n_seqs, dtype=np.int32)
+    if not ws.self_is_aan and pos.max() > 0:
+        orc.prefill(ids, pos)
+    # host inputs of one step, produced the same way the driver does it (no device involved)
+    host = {}
+    first_s = list(np.cumsum((0,) + tuple(ws.self_blocks))[:-1])
+    first_e = list(np.cumsum((0,) + tuple(ws.encdec_blocks))[:-1])
+    if ws.self_is_aan:
+        host["x"] = np.stack([synth.aan_x(ws, 0, l) for l in range(ws.n_layers)])
+        for t in range(int(pos.max())):          # history of the running average
+            for l in range(ws.n_layers):
+                orc.o.aan_step(l, ids, np.full(ws.n_seqs, t + 1), synth.aan_x(ws, 1000 + t, l))
+    else:
+        qkv = [synth.self_qkv(ws, 0, l) for l in range(ws.n_layers)]
+        host["q"] = np.stack([qkv[l][0] for l in first_s])
+        host["k"] = np.stack([qkv[l][1] for l in first_s])
+        host["v"] = np.stack([qkv[l][2] for l in range(ws.n_layers)])
+    host["q_enc"] = np.stack([synth.encdec_q(ws, 0, l) for l in first_e])
+    host["beams"] = ids
+    return ws, orc, host, ids, pos
+
+
+def time_oracle(w, budget_s=12.0, n_sent_sample=8, max_steps=50, exact_steps=None, warmup=1):
+    """Times the oracle as it stands.  Without exact_steps: as many steps as fit the budget."""
+    ws, orc, host, ids, pos = oracle_sample(w, n_sent_sample)
+    for _ in range(max(warmup, 1)):
+        orc.step(host, ids, pos, want_S=False)           # touches every page once
+    t0 = time.perf_counter()
+    steps = 0
+    if exact_steps is not None:
+        for _ in range(exact_steps):
+            orc.step(host, ids, pos, want_S=False)
+        steps = exact_steps
+    else:
+        while steps < max_steps and (steps == 0 or time.perf_counter() - t0 < budget_s):
+            orc.step(host, ids, pos, want_S=False)
+            steps += 1
+    dt = time.perf_counter() - t0
+    cores = len(os.sched_getaffinity(0))
+    threads = int(os.environ.get("OMP_NUM_THREADS", cores))
+    return {"value": ws.n_seqs * steps / dt, "unit": UNIT, "cores": min(cores, threads), "kind": "oracle",
+            "sample": f"{steps} steps of the first {ws.n_sent} sentences x beam {ws.beam} "
+                      f"({ws.n_seqs} sequences) of '{w.name}' at the benchmarked cache lengths",
+            "ms_per_step": dt / steps * 1e3, "steps": steps}
+
+
+# ---------------------------------------------------------------------------------------- main
+def config_dict(w, extra=None):
+    c = {"workload": f"{w.name}: {w.n_layers} layers, d_model {w.d_model}, {w.n_heads} heads, "
+                     f"{w.n_sent} sentences x beam {w.beam}, source lengths U[{w.src_lo},{w.src_hi}]",
+         "self_blocks": list(w.self_blocks) if not w.self_is_aan else "AAN",
+         "encdec_blocks": list(w.encdec_blocks), "storage": w.dtype, "accumulate": "f32"}
+    if extra:
+        c.update(extra)
+    return c
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    res = time_oracle(w, n_sent_sample=2, exact_steps=max(args.steps, 1), warmup=args.warmup)
+    line = {"impl": "reference", "metric": METRIC, "value": res["value"], "unit": UNIT, "n_gpus": args.gpus,
+            "steps": res["steps"], "warmup": max(args.warmup, 1), "ms_per_step": res["ms_per_step"], "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": config_dict(w, {"note": "CPU oracle on a bounded sample of the workload"}),
+            "cpu_baseline": {k: res[k] for k in ("value", "unit", "cores", "kind", "sample")},
+            "e2e": {"value": res["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20000)
+    ap.add_argument("--warmup", type=int, default=200)
+    ap.add_argument("--impl", default="san", choices=["san", "reference"])
+    ap.add_argument("--workload", default="base", choices=["tiny", "base", "big", "long", "aan"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-unshared", action="store_true")
+    args = ap.parse_args()
+
+    from paper_1906_11024_b200 import synth
+    w = synth.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    import torch
+    from paper_1906_11024_b200 import build as san_build
+    from paper_1906_11024_b200 import binding
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the attention path has no CPU fallback")
+    san_build.build()
+    binding.lib()
+    device = torch.device(f"cuda:{local_rank}")
+    torch.cuda.set_device(device)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=device)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+
+    peak, peak_kind = measured_peak_gbs()
+    pos = state_positions(w)
+    ab = algorithmic_bytes(w, pos)
+    n_rep = int(min(16, max(2, math.ceil(3 * L2_BYTES / max(ab["total"], 1)))))
+    decs, sbs, pos = build_replicas(w, n_rep, device)
+
+    phys = local_rank
+    cvd = os.environ.get("CUDA_VISIBLE_DEVICES", "")
+    if cvd:
+        parts = [x.strip() for x in cvd.split(",")]
+        if local_rank < len(parts) and parts[local_rank].isdigit():
+            phys = int(parts[local_rank])
+    sampler = ClockSampler(phys)
+    sampler.start()
+    secs, launches_per_step, (t0, t1) = time_steps(decs, sbs, args.steps, args.warmup, device, barrier)
+    clocks = sampler.stop(t0, t1)
+    err = [d.device_status()[0] for d in decs]
+    assert not any(err), f"device check failed during the timed region: {err}"
+
+    t = torch.tensor([secs], dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)      # max over ranks; every rank ran the same workload
+    secs_max = float(t.item())
+    tokens = w.n_seqs * args.steps * world
+    value = tokens / secs_max
+
+    dom_s, dom_per_step = time_dominant_kernel(w, decs, sbs, device)
+    dom_bytes = dominant_kernel_bytes(w, pos)
+    e2e_s, h2d, d2h = time_e2e(w, decs[0], sbs[0], min(args.steps, 100), device)
+    e2e_steps = min(args.steps, 100)
+
+    unshared = None
+    if not args.no_unshared and rank == 0:
+        for d in decs:
+            d.close()
+        del decs, sbs
+        torch.cuda.empty_cache()
+        wu = synth.unshared(w)
+        abu = algorithmic_bytes(wu, pos)
+        decs_u, sbs_u, _ = build_replicas(wu, n_rep, device)
+        su, lu, _ = time_steps(decs_u, sbs_u, args.steps, args.warmup, device, lambda: None)
+        unshared = {"value": wu.n_seqs * args.steps / su, "unit": UNIT, "ms_per_step": su / args.steps * 1e3,
+                    "kv_bytes_per_step": abu["kv"], "bytes_per_step": abu["total"],
+                    "hbm_gbs": abu["total"] / (su / args.steps) / 1e9, "gpu_launches_per_step": lu}
+        for d in decs_u:
+            d.close()
+        del decs_u, sbs_u
+        torch.cuda.empty_cache()
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    ms = secs_max / args.steps * 1e3
+    step_gbs = ab["total"] / (secs_max / args.steps) / 1e9
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32" if w.dtype == "f32" else "bf16", "data": "synthetic",
+        "config": config_dict(w, {"l2": f"steps rotate over {n_rep} independent replicas of the device state "
+                                        f"({ab['total'] * n_rep / 1e6:.0f} MB touched per cycle, L2 is 126 MB)",
+                                  "state": "each sequence at the middle of its target length"
+                                           if not w.ragged_prefix else "seeded ragged prefix lengths",
+                                  "mean_cache_len": float((pos + 1).mean()), "mean_src_len": float(w.src_lens().mean()),
+                                  "multi_gpu": "replicas only: no sharding, no collective"}),
+        "gpu_launches": launches_per_step * args.steps, "gpu_launches_per_step": launches_per_step,
+        "hbm": {"kv_bytes_per_step": ab["kv"], "bytes_per_step": ab["total"], "achieved_gbs": step_gbs,
+                "frac_of_measured": step_gbs / peak, "frac_of_nominal_8tbs": step_gbs / NOMINAL_HBM_GBS,
+                "peak_kind": peak_kind},
+        "roofline": {"bound": "hbm", "kernel": "san_attn_apply (apply_kernel)", "achieved": dom_bytes / dom_s / 1e9,
+                     "peak": peak, "unit": "GB/s", "frac": dom_bytes / dom_s / 1e9 / peak, "peak_kind": peak_kind,
+                     "bytes_per_launch": dom_bytes, "us_per_launch": dom_s * 1e6, "launches_per_step": dom_per_step,
+                     "traffic": None},
+        "e2e": {"value": w.n_seqs * e2e_steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "ms_per_step": e2e_s / e2e_steps * 1e3},
+        "clocks": clocks,
+    }
+    if unshared is not None:
+        unshared["speedup_from_sharing"] = value / world / unshared["value"]
+        unshared["kv_bytes_ratio_shared_over_unshared"] = ab["kv"] / unshared["kv_bytes_per_step"]
+        line["unshared"] = unshared
+    if world == 1 and not args.no_cpu_baseline:
+        cb = time_oracle(w)
+        line["cpu_baseline"] = {k: cb[k] for k in ("value", "unit", "cores", "kind", "sample")}
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
