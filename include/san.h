@@ -170,6 +170,41 @@ int32_t san_aan_step(san_ctx* ctx, int32_t layer_begin, int32_t layer_end, const
  * offending value, limit.  Synchronises `stream`. */
 int32_t san_device_status(san_ctx* ctx, int32_t* first_error, int32_t* detail, void* stream);
 
+/* The weights step of san_attn_weights for callers that cannot allocate device memory.
+ * (The paper has no counterpart: this entry point exists for deployment reasons only.)
+ *
+ * A decode loop inside a serving process often may not call cudaMalloc: the server's
+ * cache manager has reserved all of HBM, a plug-in contract forbids allocation while
+ * serving, or the stall that cudaMalloc/cudaFree impose on every stream of the device is
+ * not acceptable.  Such a caller cannot create a san_ctx, which needs a workspace buffer.
+ * This call needs neither: it takes the key panel directly and keeps the scratch of
+ * split rows (tickets, partial max/sum) in a fixed 1 MiB array inside the library image,
+ * present on every GPU that loads the library until the process exits.  It calls no
+ * cudaMalloc, cudaFree or other allocating routine.
+ *
+ *   dtype      SAN_F32 or SAN_BF16 (element type of d_q and d_K)
+ *   n_queries  query rows sharing each key panel: 1 for self-attention, the beam size for
+ *              encoder memory (1..SAN_MAX_BEAM)
+ *   d_q        [n_items][n_queries][n_heads][64]
+ *   d_K        key plane [max_ids][n_heads][cap_len][64], the layout of the context's planes
+ *   d_ids, d_lens, n_items, max_len, d_S, ld_s   as in san_attn_weights;
+ *              d_S is [n_items][n_queries][n_heads][ld_s]
+ *   d_status   optional device int32[8]: cleared, then [0] = SAN_ERR_DEVICE_CHECK and
+ *              [1..4] = kernel tag, item, value, limit if an item was skipped
+ *
+ * Limits: n_items * n_heads <= 65536 rows, else SAN_ERR_CAPACITY (use a context instead).
+ * The first call on each device looks up the array's device address (with that device
+ * current); make that first call before any stream capture begins.  Every call on a
+ * device uses the same array and finds what the previous call left there; the call clears
+ * the tickets and status words it needs on `stream` before launching.  Two calls whose
+ * kernels may overlap on one GPU (different streams without an event between them, or
+ * different host threads doing so) race on the array: order them. */
+int32_t san_attn_weights_static(int32_t dtype, int32_t n_heads, int32_t n_queries, const void* d_q,
+                                const void* d_K, int32_t max_ids, int32_t cap_len,
+                                const int32_t* d_ids, const int32_t* d_lens, int32_t n_items,
+                                int32_t max_len, float* d_S, int64_t ld_s, int32_t* d_status,
+                                void* stream);
+
 const char* san_status_string(int32_t status);
 
 #ifdef __cplusplus

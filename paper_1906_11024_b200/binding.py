@@ -28,7 +28,7 @@ EXPORTS = (
     "san_query_bytes", "san_create", "san_destroy",
     "san_policy_set_sizes", "san_policy_set_map", "san_policy_get_map",
     "san_cache_append", "san_attn_weights", "san_attn_apply", "san_aan_step",
-    "san_device_status", "san_status_string",
+    "san_device_status", "san_status_string", "san_attn_weights_static",
 )
 
 
@@ -69,6 +69,7 @@ def lib():
     L.san_attn_apply.argtypes = [vp, i32, i32, i32, i32, vp, i64, vp, vp, vp, i32, i32, vp, i32, vp]
     L.san_aan_step.argtypes = [vp, i32, i32, vp, vp, vp, i32, vp, vp]
     L.san_device_status.argtypes = [vp, _I32P, _I32P, vp]
+    L.san_attn_weights_static.argtypes = [i32, i32, i32, vp, vp, i32, i32, vp, vp, i32, i32, vp, i64, vp, vp]
     L.san_status_string.argtypes = [i32]
     L.san_status_string.restype = C.c_char_p
     for name in EXPORTS:
@@ -178,3 +179,12 @@ def san_device_status(ctx, stream=None):
     det = (C.c_int32 * 4)()
     rc = lib().san_device_status(ctx, C.byref(fe), det, _stream(stream))
     return rc, fe.value, list(det)
+
+
+def san_attn_weights_static(dtype, n_heads, n_queries, d_q, d_K, max_ids, cap_len, d_ids, d_lens, n_items,
+                            max_len, d_S, ld_s, d_status=None, stream=None) -> int:
+    """The weights step without a context or workspace, for callers that cannot allocate
+    device memory (see include/san.h).  ``d_K`` is the device address of a key plane."""
+    return lib().san_attn_weights_static(dtype, n_heads, n_queries, _ptr(d_q), _ptr(d_K), max_ids, cap_len,
+                                         _ptr(d_ids), _ptr(d_lens), n_items, max_len, _ptr(d_S), ld_s,
+                                         _ptr(d_status), _stream(stream))

@@ -104,7 +104,7 @@ struct AppendParams {
 
 // One thread moves 16 bytes.  Unit order (fastest first): 16-byte piece, head, row, item,
 // layer, {V,K}; so a warp writes whole rows.
-__global__ void __launch_bounds__(256) append_kernel(const AppendParams p) {
+static __global__ void __launch_bounds__(256) append_kernel(const AppendParams p) {
     const int pieces = p.row_bytes >> 4;
     const long long per_kind = (long long)p.n_layers * p.n_items * p.rows_per_item * p.H * pieces;
     long long u = (long long)blockIdx.x * blockDim.x + threadIdx.x;
