@@ -44,8 +44,9 @@ def state_positions(w):
     return ((T + 1) // 2 - 1).astype(np.int32)               # middle of the run: length ceil(T/2)
 
 
-def algorithmic_bytes(w, pos):
-    """Bytes the method itself must move per step (K/V reads are the roofline count)."""
+def algorithmic_bytes(w, pos, fused=False):
+    """Bytes the method itself must move per step (K/V reads are the roofline count).
+    In the one-launch step S is written for the caller but never read back."""
     M, H, d, e = w.n_layers, w.n_heads, w.d_model, w.elem_bytes
     n = w.n_seqs
     src = w.src_lens().astype(np.int64)
@@ -65,7 +66,7 @@ def algorithmic_bytes(w, pos):
     out["encdec_kv"] = int((Ne + M) * src.sum() * d * e)                          # once per sentence
     s_enc = 8 * H * Ne * int(np.repeat(src, w.beam).sum())
     small_enc = Ne * n * d * e + M * n * d * e
-    out["S"] = s_self + s_enc
+    out["S"] = (s_self + s_enc) // (2 if fused else 1)
     out["small"] = small_self + small_enc
     out["kv"] = out["self_kv"] + out["encdec_kv"] + out["aan"]
     out["total"] = out["kv"] + out["S"] + out["small"]
@@ -165,14 +166,14 @@ def capture(fn, device):
     return g
 
 
-def time_steps(decs, sbs, steps, warmup, device, barrier):
+def time_steps(decs, sbs, steps, warmup, device, barrier, fused=True):
     """W untimed + exactly K timed steps; steps rotate over the replicas.  Returns seconds."""
     import torch
     R = len(decs)
     launches = [0]
 
     def one(r):
-        launches[0] = decs[r].step(sbs[r])
+        launches[0] = decs[r].step_fused(sbs[r]) if fused else decs[r].step(sbs[r])
 
     cycle = capture(lambda: [one(r) for r in range(R)], device)
     singles = [capture(lambda r=r: one(r), device) for r in range(max(steps % R, max(warmup, 3) % R))]
@@ -251,7 +252,7 @@ def dominant_kernel_bytes(w, pos):
     return float(np.mean(per))
 
 
-def time_e2e(w, dec, sb, steps, device):
+def time_e2e(w, dec, sb, steps, device, fused=True):
     """The same step with HOST buffers: every step copies its inputs from pinned host memory
     to the device, runs the library calls, and reads the outputs back."""
     import torch
@@ -266,7 +267,7 @@ def time_e2e(w, dec, sb, steps, device):
     def one():
         for k, t in host_in.items():
             getattr(sb, k).copy_(t, non_blocking=True)
-        dec.step(sb)
+        dec.step_fused(sb) if fused else dec.step(sb)
         for k, t in host_out.items():
             t.copy_(getattr(sb, k), non_blocking=True)
 
@@ -368,6 +369,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=200)
     ap.add_argument("--impl", default="san", choices=["san", "reference"])
     ap.add_argument("--workload", default="base", choices=["tiny", "base", "big", "long", "aan"])
+    ap.add_argument("--path", default="fused", choices=["fused", "calls"],
+                    help="fused: san_decode_step, one launch per step; calls: append/weights/apply launches")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-unshared", action="store_true")
     args = ap.parse_args()
@@ -402,7 +405,8 @@ def main():
 
     peak, peak_kind = measured_peak_gbs()
     pos = state_positions(w)
-    ab = algorithmic_bytes(w, pos)
+    fused = args.path == "fused"
+    ab = algorithmic_bytes(w, pos, fused)
     n_rep = int(min(16, max(2, math.ceil(3 * L2_BYTES / max(ab["total"], 1)))))
     decs, sbs, pos = build_replicas(w, n_rep, device)
 
@@ -414,7 +418,7 @@ def main():
             phys = int(parts[local_rank])
     sampler = ClockSampler(phys)
     sampler.start()
-    secs, launches_per_step, (t0, t1) = time_steps(decs, sbs, args.steps, args.warmup, device, barrier)
+    secs, launches_per_step, (t0, t1) = time_steps(decs, sbs, args.steps, args.warmup, device, barrier, fused)
     clocks = sampler.stop(t0, t1)
     err = [d.device_status()[0] for d in decs]
     assert not any(err), f"device check failed during the timed region: {err}"
@@ -426,9 +430,12 @@ def main():
     tokens = w.n_seqs * args.steps * world
     value = tokens / secs_max
 
-    dom_s, dom_per_step = time_dominant_kernel(w, decs, sbs, device)
-    dom_bytes = dominant_kernel_bytes(w, pos)
-    e2e_s, h2d, d2h = time_e2e(w, decs[0], sbs[0], min(args.steps, 100), device)
+    if fused:      # one kernel per step: its launch duration is the step time of the timed region
+        dom_s, dom_per_step, dom_bytes, dom_name = secs / args.steps, 1, float(ab["total"]), "san_decode_step (decode_step_kernel)"
+    else:
+        dom_s, dom_per_step = time_dominant_kernel(w, decs, sbs, device)
+        dom_bytes, dom_name = dominant_kernel_bytes(w, pos), "san_attn_apply (apply_kernel)"
+    e2e_s, h2d, d2h = time_e2e(w, decs[0], sbs[0], min(args.steps, 100), device, fused)
     e2e_steps = min(args.steps, 100)
 
     unshared = None
@@ -438,9 +445,9 @@ def main():
         del decs, sbs
         torch.cuda.empty_cache()
         wu = synth.unshared(w)
-        abu = algorithmic_bytes(wu, pos)
+        abu = algorithmic_bytes(wu, pos, fused)
         decs_u, sbs_u, _ = build_replicas(wu, n_rep, device)
-        su, lu, _ = time_steps(decs_u, sbs_u, args.steps, args.warmup, device, lambda: None)
+        su, lu, _ = time_steps(decs_u, sbs_u, args.steps, args.warmup, device, lambda: None, fused)
         unshared = {"value": wu.n_seqs * args.steps / su, "unit": UNIT, "ms_per_step": su / args.steps * 1e3,
                     "kv_bytes_per_step": abu["kv"], "bytes_per_step": abu["total"],
                     "hbm_gbs": abu["total"] / (su / args.steps) / 1e9, "gpu_launches_per_step": lu}
@@ -465,12 +472,14 @@ def main():
                                   "state": "each sequence at the middle of its target length"
                                            if not w.ragged_prefix else "seeded ragged prefix lengths",
                                   "mean_cache_len": float((pos + 1).mean()), "mean_src_len": float(w.src_lens().mean()),
+                                  "path": "san_decode_step, one launch per step" if fused
+                                          else "san_cache_append + san_attn_weights/apply per block",
                                   "multi_gpu": "replicas only: no sharding, no collective"}),
         "gpu_launches": launches_per_step * args.steps, "gpu_launches_per_step": launches_per_step,
         "hbm": {"kv_bytes_per_step": ab["kv"], "bytes_per_step": ab["total"], "achieved_gbs": step_gbs,
                 "frac_of_measured": step_gbs / peak, "frac_of_nominal_8tbs": step_gbs / NOMINAL_HBM_GBS,
                 "peak_kind": peak_kind},
-        "roofline": {"bound": "hbm", "kernel": "san_attn_apply (apply_kernel)", "achieved": dom_bytes / dom_s / 1e9,
+        "roofline": {"bound": "hbm", "kernel": dom_name, "achieved": dom_bytes / dom_s / 1e9,
                      "peak": peak, "unit": "GB/s", "frac": dom_bytes / dom_s / 1e9 / peak, "peak_kind": peak_kind,
                      "bytes_per_launch": dom_bytes, "us_per_launch": dom_s * 1e6, "launches_per_step": dom_per_step,
                      "traffic": None},

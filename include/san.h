@@ -165,6 +165,40 @@ int32_t san_aan_step(san_ctx* ctx, int32_t layer_begin, int32_t layer_end, const
                      const int32_t* d_ids, const int32_t* d_t, int32_t n_items, void* d_out,
                      void* stream);
 
+/* One whole decode step in ONE launch: for every block of both attention kinds, append
+ * this step's rows (Section 4.1 cache), compute the block's weights at its lowest layer
+ * (Eq. 1, Eq. 3) and apply them to the values of every layer of the block (Eq. 2, Eq. 4;
+ * Eq. 5 with encdec_shared_context); with self_is_aan the cumulative average replaces
+ * the self-attention part.  Same arithmetic and outputs as the sequence
+ *     san_cache_append(SELF, 0..M) ; per block san_attn_weights + san_attn_apply
+ * for inputs laid out for all layers at once (a caller that has every layer's q/k/v of
+ * the step up front, e.g. a benchmark or a speculative/batched front end):
+ *   d_q_self, d_k_new [n_self_blocks][n_seqs][H][64]   rows of the block-first layers
+ *   d_v_new           [n_layers][n_seqs][H][64]
+ *   d_seq_ids, d_pos  sequence ids and the row each writes this step (length = pos + 1)
+ *   d_S_self          [n_self_blocks][n_seqs][H][ld_t] float32, or NULL if not wanted
+ *   d_O_self          [n_layers][n_seqs][H][64]
+ *   d_q_enc           [n_encdec_blocks][n_sent][beam][H][64]
+ *   d_sent_ids, d_src_lens   sentence ids and their source lengths
+ *   d_S_enc           [n_encdec_blocks][n_sent*beam][H][ld_s] float32, or NULL
+ *   d_O_enc           [n_layers (or n_encdec_blocks with Eq. 5)][n_sent*beam][H][64]
+ *   d_x_aan, d_t      [n_layers][n_seqs][H*64] and 1-based positions (self_is_aan only;
+ *                     the averages go to d_O_self)
+ * n_seqs == 0 skips the self/AAN part, n_sent == 0 the enc-dec part.  max_len / max_src
+ * are host bounds on pos+1 / source lengths (0 = capacity).  Rows longer than the on-chip
+ * score buffer are split into at most 32 spans; a bound that would need more returns
+ * SAN_ERR_UNSUPPORTED (use the separate calls).  The kernel's waits on its own copies are
+ * bounded: if one runs out the step reports SAN_ERR_TIMEOUT through san_device_status. */
+typedef struct {
+    const void* d_q_self; const void* d_k_new; const void* d_v_new;
+    const int32_t* d_seq_ids; const int32_t* d_pos; int32_t n_seqs; int32_t max_len;
+    float* d_S_self; int64_t ld_t; void* d_O_self;
+    const void* d_q_enc; const int32_t* d_sent_ids; const int32_t* d_src_lens; int32_t n_sent; int32_t max_src;
+    float* d_S_enc; int64_t ld_s; void* d_O_enc;
+    const void* d_x_aan; const int32_t* d_t;
+} san_step_args;
+int32_t san_decode_step(san_ctx* ctx, const san_step_args* args, void* stream);
+
 /* Reads (and clears) the device error word: *first_error = SAN_OK or the first
  * device-check error since the last read; detail[0..3] (optional) = kernel tag, item,
  * offending value, limit.  Synchronises `stream`. */

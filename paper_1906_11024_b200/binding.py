@@ -28,7 +28,7 @@ EXPORTS = (
     "san_query_bytes", "san_create", "san_destroy",
     "san_policy_set_sizes", "san_policy_set_map", "san_policy_get_map",
     "san_cache_append", "san_attn_weights", "san_attn_apply", "san_aan_step",
-    "san_device_status", "san_status_string", "san_attn_weights_static",
+    "san_device_status", "san_status_string", "san_attn_weights_static", "san_decode_step",
 )
 
 
@@ -36,6 +36,18 @@ class san_config(C.Structure):
     _fields_ = [(n, C.c_int32) for n in (
         "n_layers", "n_heads", "d_head", "max_sent", "beam", "max_tgt_len", "max_src_len",
         "dtype", "self_is_aan", "encdec_shared_context")]
+
+
+class san_step_args(C.Structure):
+    _fields_ = [
+        ("d_q_self", C.c_void_p), ("d_k_new", C.c_void_p), ("d_v_new", C.c_void_p),
+        ("d_seq_ids", C.c_void_p), ("d_pos", C.c_void_p), ("n_seqs", C.c_int32), ("max_len", C.c_int32),
+        ("d_S_self", C.c_void_p), ("ld_t", C.c_int64), ("d_O_self", C.c_void_p),
+        ("d_q_enc", C.c_void_p), ("d_sent_ids", C.c_void_p), ("d_src_lens", C.c_void_p),
+        ("n_sent", C.c_int32), ("max_src", C.c_int32),
+        ("d_S_enc", C.c_void_p), ("ld_s", C.c_int64), ("d_O_enc", C.c_void_p),
+        ("d_x_aan", C.c_void_p), ("d_t", C.c_void_p),
+    ]
 
 
 class SanError(RuntimeError):
@@ -70,6 +82,7 @@ def lib():
     L.san_aan_step.argtypes = [vp, i32, i32, vp, vp, vp, i32, vp, vp]
     L.san_device_status.argtypes = [vp, _I32P, _I32P, vp]
     L.san_attn_weights_static.argtypes = [i32, i32, i32, vp, vp, i32, i32, vp, vp, i32, i32, vp, i64, vp, vp]
+    L.san_decode_step.argtypes = [vp, C.POINTER(san_step_args), vp]
     L.san_status_string.argtypes = [i32]
     L.san_status_string.restype = C.c_char_p
     for name in EXPORTS:
@@ -188,3 +201,14 @@ def san_attn_weights_static(dtype, n_heads, n_queries, d_q, d_K, max_ids, cap_le
     return lib().san_attn_weights_static(dtype, n_heads, n_queries, _ptr(d_q), _ptr(d_K), max_ids, cap_len,
                                          _ptr(d_ids), _ptr(d_lens), n_items, max_len, _ptr(d_S), ld_s,
                                          _ptr(d_status), _stream(stream))
+
+
+def san_decode_step(ctx, *, d_q_self=None, d_k_new=None, d_v_new=None, d_seq_ids=None, d_pos=None, n_seqs=0,
+                    max_len=0, d_S_self=None, ld_t=0, d_O_self=None, d_q_enc=None, d_sent_ids=None,
+                    d_src_lens=None, n_sent=0, max_src=0, d_S_enc=None, ld_s=0, d_O_enc=None, d_x_aan=None,
+                    d_t=None, stream=None) -> int:
+    """One whole decode step in one launch (see include/san.h)."""
+    a = san_step_args(_ptr(d_q_self), _ptr(d_k_new), _ptr(d_v_new), _ptr(d_seq_ids), _ptr(d_pos), n_seqs, max_len,
+                      _ptr(d_S_self), ld_t, _ptr(d_O_self), _ptr(d_q_enc), _ptr(d_sent_ids), _ptr(d_src_lens),
+                      n_sent, max_src, _ptr(d_S_enc), ld_s, _ptr(d_O_enc), _ptr(d_x_aan), _ptr(d_t))
+    return lib().san_decode_step(ctx, C.byref(a), _stream(stream))

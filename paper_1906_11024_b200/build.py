@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsan_b200.so")
 SOURCES = ["san_api.cu", "san_static.cu", "san_policy.cpp"]
-HEADERS = ["san_kernels.cuh", "san_ctx.h", "san_policy.h", os.path.join("..", "..", "include", "san.h")]
+HEADERS = ["san_kernels.cuh", "san_fused.cuh", "san_ctx.h", "san_policy.h", os.path.join("..", "..", "include", "san.h")]
 
 
 def _stale() -> bool:

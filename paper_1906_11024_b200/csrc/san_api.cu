@@ -8,6 +8,7 @@
 
 #include "san_ctx.h"
 #include "san_kernels.cuh"
+#include "san_fused.cuh"
 
 using namespace san;
 
@@ -52,9 +53,9 @@ void layout(const san_config& c, int n_self_planes, int n_enc_planes, san_ctx* L
 
     // workspace: error words | tickets [layer][row] | partial sums of split rows
     const size_t rows = n_seqs * c.n_heads;
-    L->n_tickets = (size_t)c.n_layers * rows;
-    const size_t worst = L->n_tickets * 4 * kDh;   // four spans per (layer, row), one query row each
-    L->part_floats = std::min<size_t>(std::max<size_t>(worst, (size_t)1 << 18), (size_t)1 << 24);
+    L->n_tickets = (size_t)2 * c.n_layers * rows;   // self rows and enc-dec rows of one fused step
+    const size_t worst = L->n_tickets * 8 * kDh;   // eight spans per (layer, row), one query row each
+    L->part_floats = std::min<size_t>(std::max<size_t>(worst, (size_t)1 << 18), (size_t)1 << 26);
     L->ws_off_tickets = 256;
     L->ws_off_part = align_up(256 + L->n_tickets * sizeof(int), 256);
     L->ws_bytes_needed = L->ws_off_part + L->part_floats * sizeof(float);
@@ -363,6 +364,127 @@ int32_t san_aan_step(san_ctx* ctx, int32_t layer_begin, int32_t layer_end, const
     if (c.dtype == SAN_BF16) aan_kernel<__nv_bfloat16><<<(unsigned)grid, 256, 0, st>>>(p);
     else aan_kernel<float><<<(unsigned)grid, 256, 0, st>>>(p);
     return cuda_status(cudaGetLastError());
+}
+
+int32_t san_decode_step(san_ctx* ctx, const san_step_args* a, void* stream) {
+    if (!ctx || !a) return SAN_ERR_NULL;
+    const san_config& c = ctx->cfg;
+    const bool aan = c.self_is_aan != 0;
+    const int n_seqs = a->n_seqs, n_sent = a->n_sent;
+    if (n_seqs < 0 || n_seqs > ctx->n_seqs || n_sent < 0 || n_sent > c.max_sent) return SAN_ERR_SHAPE;
+    if (n_seqs > 0) {
+        if (!a->d_seq_ids || !a->d_O_self) return SAN_ERR_NULL;
+        if (aan ? (!a->d_x_aan || !a->d_t) : (!a->d_q_self || !a->d_k_new || !a->d_v_new || !a->d_pos)) return SAN_ERR_NULL;
+    }
+    if (n_sent > 0 && (!a->d_q_enc || !a->d_sent_ids || !a->d_src_lens || !a->d_O_enc)) return SAN_ERR_NULL;
+    int max_len = a->max_len == 0 ? c.max_tgt_len : a->max_len;
+    int max_src = a->max_src == 0 ? c.max_src_len : a->max_src;
+    if (max_len < 1 || max_len > c.max_tgt_len || max_src < 1 || max_src > c.max_src_len) return SAN_ERR_SHAPE;
+    if (n_seqs > 0 && !aan && a->d_S_self && a->ld_t < max_len) return SAN_ERR_SHAPE;
+    if (n_sent > 0 && a->d_S_enc && a->ld_s < max_src) return SAN_ERR_SHAPE;
+    if (n_seqs == 0 && n_sent == 0) return SAN_OK;
+
+    const bool bf16 = c.dtype == SAN_BF16;
+    const int row_bytes = kDh * ctx->elem_bytes;
+    const int TR = kStageBytes / row_bytes;
+    const int nqe = pick_nq_template(c.beam);
+    const bool do_self = n_seqs > 0 && !aan;
+    const bool do_enc = n_sent > 0;
+    int pi_self = 1, pi_enc = 1;
+    for (int b = 0; b < ctx->self_pol.n_blocks; ++b) pi_self = std::max(pi_self, ctx->self_pol.size_of_block[b]);
+    for (int b = 0; b < ctx->enc_pol.n_blocks; ++b) pi_enc = std::max(pi_enc, ctx->enc_pol.size_of_block[b]);
+    if (c.encdec_shared_context) pi_enc = 1;
+    const long long rows_self = do_self ? (long long)ctx->self_pol.n_blocks * n_seqs * c.n_heads : 0;
+    const long long rows_enc = do_enc ? (long long)ctx->enc_pol.n_blocks * n_sent * c.n_heads : 0;
+    if ((size_t)(rows_self + rows_enc) > ctx->n_tickets) return SAN_ERR_CAPACITY;
+
+    // positions per item: what the on-chip score buffer holds, then smaller while items are
+    // fat (long tails) or too few to fill the persistent warps
+    auto first_span = [&](int bound, int cap_z, int pi) {
+        int sp = std::min(cap_z, (int)align_up((size_t)bound, (size_t)TR));
+        while (sp > 32 && (long long)sp * (1 + pi) * row_bytes > (128 << 10)) sp = std::max(32, (int)align_up((size_t)ceil_div(sp, 2), TR));
+        return sp;
+    };
+    int span_self = first_span(max_len, kZFloats, pi_self);
+    int span_enc = first_span(max_src, kZFloats / nqe, pi_enc);
+    const long long warps = (long long)ctx->sm_count * kFusedWarps;
+    auto items = [&]() {
+        return rows_self * ceil_div(max_len, span_self) + rows_enc * ceil_div(max_src, span_enc);
+    };
+    while (items() < 3 * warps) {
+        const long long bs = do_self ? (long long)span_self * (1 + pi_self) : 0;
+        const long long be = do_enc ? (long long)span_enc * (1 + pi_enc) : 0;
+        if (bs >= be && span_self > 32 && ceil_div(max_len, span_self) < ceil_div(max_len, 32)) span_self = std::max(32, (int)align_up((size_t)ceil_div(span_self, 2), TR));
+        else if (be > 0 && span_enc > 32 && ceil_div(max_src, span_enc) < ceil_div(max_src, 32)) span_enc = std::max(32, (int)align_up((size_t)ceil_div(span_enc, 2), TR));
+        else if (bs > 0 && span_self > 32 && ceil_div(max_len, span_self) < ceil_div(max_len, 32)) span_self = std::max(32, (int)align_up((size_t)ceil_div(span_self, 2), TR));
+        else break;
+    }
+    const int stride_self = 2 + pi_self * kDh, stride_enc = 2 * nqe + pi_enc * nqe * kDh;
+    auto part_need = [&]() {
+        const int ns = ceil_div(max_len, span_self), ne = ceil_div(max_src, span_enc);
+        return (ns > 1 ? rows_self * ns * stride_self : 0) + (ne > 1 ? rows_enc * ne * stride_enc : 0);
+    };
+    while (part_need() > (long long)ctx->part_floats) {   // fewer, longer spans until the partial sums fit
+        if (span_self < kZFloats && ceil_div(max_len, span_self) > 1 &&
+            (long long)rows_self * stride_self * ceil_div(max_len, span_self) >= (long long)rows_enc * stride_enc * ceil_div(max_src, span_enc))
+            span_self = std::min(kZFloats, span_self * 2);
+        else if (span_enc < kZFloats / nqe && ceil_div(max_src, span_enc) > 1) span_enc = std::min(kZFloats / nqe, span_enc * 2);
+        else if (span_self < kZFloats && ceil_div(max_len, span_self) > 1) span_self = std::min(kZFloats, span_self * 2);
+        else return SAN_ERR_UNSUPPORTED;
+    }
+    const int ns_self = do_self ? ceil_div(max_len, span_self) : 1, ns_enc = do_enc ? ceil_div(max_src, span_enc) : 1;
+    if (ns_self > kMaxSpans || ns_enc > kMaxSpans) return SAN_ERR_UNSUPPORTED;
+
+    StepParams p;
+    std::memset(&p, 0, sizeof(p));
+    p.q_self = static_cast<const char*>(a->d_q_self); p.k_new = static_cast<const char*>(a->d_k_new);
+    p.v_new = static_cast<const char*>(a->d_v_new);
+    p.seq_ids = a->d_seq_ids; p.pos = a->d_pos; p.S_self = a->d_S_self; p.ld_t = a->ld_t;
+    p.O_self = static_cast<char*>(a->d_O_self); p.n_seqs = n_seqs; p.max_len = max_len;
+    p.q_enc = static_cast<const char*>(a->d_q_enc); p.sent_ids = a->d_sent_ids; p.src_lens = a->d_src_lens;
+    p.S_enc = a->d_S_enc; p.ld_s = a->ld_s; p.O_enc = static_cast<char*>(a->d_O_enc); p.n_sent = n_sent; p.max_src = max_src;
+    if (aan && n_seqs > 0) {
+        p.x_aan = static_cast<const char*>(a->d_x_aan); p.t_aan = a->d_t;
+        p.aan_sum = reinterpret_cast<float*>(ctx->cache + ctx->off_aan); p.n_aan_layers = c.n_layers;
+    }
+    p.H = c.n_heads; p.beam = c.beam;
+    p.n_self_blocks = do_self ? ctx->self_pol.n_blocks : 0; p.n_enc_blocks = do_enc ? ctx->enc_pol.n_blocks : 0;
+    p.cap_tgt = c.max_tgt_len; p.cap_src = c.max_src_len; p.max_seqs = ctx->n_seqs; p.max_sent = c.max_sent;
+    p.enc_v_by_block = c.encdec_shared_context ? 1 : 0;
+    p.selfK = ctx->cache + ctx->off_self_k; p.selfV = ctx->cache + ctx->off_self_v;
+    p.memK = ctx->cache + ctx->off_mem_k; p.memV = ctx->cache + ctx->off_mem_v;
+    p.self_plane_bytes = (long long)ctx->self_plane_bytes; p.mem_plane_bytes = (long long)ctx->mem_plane_bytes;
+    p.self_span = span_self; p.self_nspans = ns_self; p.enc_span = span_enc; p.enc_nspans = ns_enc;
+    p.n_enc_items = rows_enc * ns_enc; p.n_items = p.n_enc_items + rows_self * ns_self;
+    p.enc_part_stride = stride_enc; p.self_part_stride = stride_self;
+    p.self_part_base = ns_enc > 1 ? rows_enc * ns_enc * stride_enc : 0;
+    p.part = ctx->part; p.tickets = ctx->tickets; p.err = ctx->err;
+    p.scale_log2e = (float)(1.4426950408889634 / std::sqrt((double)kDh));
+    for (int b = 0; b < ctx->self_pol.n_blocks; ++b) {
+        p.self_first[b] = (unsigned char)ctx->self_pol.first_layer_of_block[b];
+        p.self_size[b] = (unsigned char)ctx->self_pol.size_of_block[b];
+    }
+    for (int b = 0; b < ctx->enc_pol.n_blocks; ++b) {
+        p.enc_first[b] = (unsigned char)ctx->enc_pol.first_layer_of_block[b];
+        p.enc_size[b] = (unsigned char)ctx->enc_pol.size_of_block[b];
+    }
+
+    const void* fn = nullptr;
+    if (bf16) fn = nqe == 1 ? (const void*)decode_step_kernel<__nv_bfloat16, 1> : nqe == 2 ? (const void*)decode_step_kernel<__nv_bfloat16, 2>
+                   : nqe == 4 ? (const void*)decode_step_kernel<__nv_bfloat16, 4> : (const void*)decode_step_kernel<__nv_bfloat16, 8>;
+    else fn = nqe == 1 ? (const void*)decode_step_kernel<float, 1> : nqe == 2 ? (const void*)decode_step_kernel<float, 2>
+              : nqe == 4 ? (const void*)decode_step_kernel<float, 4> : (const void*)decode_step_kernel<float, 8>;
+    const size_t smem = fused_smem_bytes();
+    if (!ctx->fused_attr_set) {
+        if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return SAN_ERR_CUDA;
+        ctx->fused_attr_set = true;
+    }
+    long long ctas = std::min<long long>(ctx->sm_count, (p.n_items + kFusedWarps - 1) / kFusedWarps);
+    if (p.x_aan) ctas = ctx->sm_count;     // the running average is spread over every thread of the grid
+    if (ctas < 1) ctas = 1;
+    void* args[] = {&p};
+    cudaError_t e = cudaLaunchKernel(fn, dim3((unsigned)ctas), dim3(kFusedWarps * 32), args, smem, static_cast<cudaStream_t>(stream));
+    return cuda_status(e);
 }
 
 int32_t san_device_status(san_ctx* ctx, int32_t* first_error, int32_t* detail, void* stream) {

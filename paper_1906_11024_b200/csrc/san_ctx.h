@@ -27,4 +27,5 @@ struct san_ctx {
     int* err = nullptr;
     int* tickets = nullptr;
     float* part = nullptr;
+    bool fused_attr_set = false;   // shared-memory opt-in of the one-launch step kernel done
 };

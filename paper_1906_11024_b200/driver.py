@@ -194,6 +194,21 @@ class Decoder:
             launches += 2
         return launches
 
+    def step_fused(self, sb: StepBuffers, stream=None) -> int:
+        """The same decode step as ``step`` in one launch (san_decode_step)."""
+        w = self.w
+        n, n_sent = sb.ids.shape[0], sb.sent_ids.shape[0]
+        kw = dict(d_seq_ids=sb.ids, n_seqs=n, max_len=sb.max_len, d_O_self=sb.O_self,
+                  d_q_enc=sb.q_enc, d_sent_ids=sb.sent_ids, d_src_lens=sb.src_lens, n_sent=n_sent, max_src=sb.max_src,
+                  d_S_enc=sb.S_enc, ld_s=self.ld_s, d_O_enc=sb.O_enc, stream=stream)
+        if w.self_is_aan:
+            kw.update(d_x_aan=sb.x_aan, d_t=sb.t_aan)
+        else:
+            kw.update(d_q_self=sb.q_self, d_k_new=sb.k_new, d_v_new=sb.v_new, d_pos=sb.pos, d_S_self=sb.S_self,
+                      ld_t=self.ld_t)
+        B.check(B.san_decode_step(self.ctx, **kw), "san_decode_step")
+        return 1
+
     def device_status(self, stream=None):
         rc, first_error, detail = B.san_device_status(self.ctx, stream)
         B.check(rc, "san_device_status")

@@ -51,7 +51,7 @@ def _compare(w, dec, sb, ref, n, lens, src_lens_per_seq, tag):
     assert err <= tol, (tag, "O_enc", err)
 
 
-def _run(w, check_steps=None, max_steps=None, shared_context=False, jumps=None):
+def _run(w, check_steps=None, max_steps=None, shared_context=False, jumps=None, fused=False):
     """Decode the workload on both sides.  Sequences start at their prefix length, advance in
     lock-step and drop out when their sentence is done.  ``jumps`` = list of (start_pos, n_steps)
     segments for long runs: the caches are re-prefilled to start_pos before each segment."""
@@ -76,7 +76,7 @@ def _run(w, check_steps=None, max_steps=None, shared_context=False, jumps=None):
             sb = dec.new_step_buffers(len(active), len(sent))
             step_id = g if start is None else 100000 + start + g
             host = dec.fill_step_inputs(sb, step_id, active, pos[active], sent)
-            dec.step(sb)
+            (dec.step_fused if fused else dec.step)(sb)
             do_check = check_steps is None or g in check_steps
             ref = orc.step(host, active, pos[active], want_S=do_check)
             if do_check:
@@ -164,3 +164,56 @@ def test_fp32_long_rows_and_splits():
     w = dataclasses.replace(synth.WORKLOADS["tiny"], name="tiny-long", src_lo=300, src_hi=300,
                             tgt_rule="fixed", tgt_fixed=300)
     _run(w, jumps=[(0, 2), (127, 3), (255, 3), (297, 3)])
+
+
+# ------------------------------------------------------------------ the one-launch decode step
+FUSED_CASES = {
+    "tiny": lambda: _run(synth.WORKLOADS["tiny"], fused=True),
+    "tiny-unshared": lambda: _run(synth.unshared(synth.WORKLOADS["tiny"]), fused=True),
+    "base-scaled": lambda: _run(synth.scaled(synth.WORKLOADS["base"], 8), fused=True),
+    "base-full": lambda: _run(synth.WORKLOADS["base"], check_steps={0, 1, 17, 33, 65}, fused=True),
+    "big-scaled-ragged": lambda: _run(synth.scaled(synth.WORKLOADS["big"], 6), fused=True),
+    "big-full": lambda: _run(synth.WORKLOADS["big"], check_steps={0, 5, 40}, max_steps=41, fused=True),
+    "long-scaled-split": lambda: _run(synth.scaled(synth.WORKLOADS["long"], 2),
+                                      jumps=[(0, 3), (30, 4), (62, 4), (126, 4), (254, 4), (508, 4)], fused=True),
+    "long-full": lambda: _run(synth.WORKLOADS["long"], jumps=[(0, 2), (63, 3), (255, 3), (510, 2)], fused=True),
+    "aan-scaled": lambda: _run(synth.scaled(synth.WORKLOADS["aan"], 8), max_steps=80, fused=True),
+    "aan-full": lambda: _run(synth.WORKLOADS["aan"], check_steps={0, 1, 40, 79}, fused=True),
+    "eq5-shared-context": lambda: _run(synth.scaled(synth.WORKLOADS["base"], 4), max_steps=6, shared_context=True,
+                                       fused=True),
+    "fp32-long-rows": lambda: _run(dataclasses.replace(synth.WORKLOADS["tiny"], name="tiny-long", src_lo=300, src_hi=300,
+                                                       tgt_rule="fixed", tgt_fixed=300),
+                                   jumps=[(0, 2), (127, 3), (255, 3), (297, 3)], fused=True),
+}
+
+
+@pytest.mark.parametrize("case", sorted(FUSED_CASES))
+def test_one_launch_step_matches_oracle(case):
+    FUSED_CASES[case]()
+
+
+@pytest.mark.parametrize("beam", [1, 2, 3, 5, 8])
+def test_one_launch_step_other_beam_sizes(beam):
+    w = dataclasses.replace(synth.scaled(synth.WORKLOADS["base"], 3), beam=beam, name=f"beam{beam}")
+    _run(w, max_steps=5, fused=True)
+
+
+def test_one_launch_step_writes_the_cache_like_append():
+    """After a fused step the caches hold this step's rows bit for bit (same as san_cache_append)."""
+    w = synth.scaled(synth.WORKLOADS["base"], 3)
+    a, b = Decoder(w), Decoder(w)
+    for d in (a, b):
+        d.cache.zero_()
+        d.load_encoder_memory()
+    ids = np.arange(w.n_seqs, dtype=np.int32)
+    for step in range(4):
+        pos = np.full(w.n_seqs, step, np.int32)
+        sa, sb_ = a.new_step_buffers(), b.new_step_buffers()
+        a.fill_step_inputs(sa, step, ids, pos)
+        b.fill_step_inputs(sb_, step, ids, pos)
+        a.step(sa)
+        b.step_fused(sb_)
+    torch.cuda.synchronize()
+    assert a.device_status()[0] == 0 and b.device_status()[0] == 0
+    assert torch.equal(a.cache, b.cache)
+    a.close(); b.close()
