@@ -65,6 +65,18 @@ inline int32_t cuda_status(cudaError_t e) { return e == cudaSuccess ? SAN_OK : S
 
 int pick_nq_template(int nq) { return nq <= 1 ? 1 : nq <= 2 ? 2 : nq <= 4 ? 4 : 8; }
 
+// Multiplier and shift for FastDiv (exact for dividends below 2^31).
+FastDiv make_fastdiv(unsigned d) {
+    FastDiv f;
+    unsigned shift = 0;
+    while ((1ull << shift) < d) ++shift;
+    f.shift = shift;
+    f.mul = (unsigned)((((unsigned long long)1 << 32) * (((unsigned long long)1 << shift) - d)) / d + 1);
+    f.div = d;
+    return f;
+}
+inline int part_header_floats(int nq_t) { return (2 * nq_t + 3) / 4 * 4; }   // (max, sum) per query, 16-byte padded
+
 // Positions per warp item.  Start with one span per row; halve it while the launch would
 // leave SMs idle; grow it back if the partial sums would not fit the workspace.
 void pick_spans(const san_ctx* ctx, long long units, int max_len, long long part_per_span_floats,
@@ -419,7 +431,7 @@ int32_t san_decode_step(san_ctx* ctx, const san_step_args* a, void* stream) {
         else if (bs > 0 && span_self > 32 && ceil_div(max_len, span_self) < ceil_div(max_len, 32)) span_self = std::max(32, (int)align_up((size_t)ceil_div(span_self, 2), TR));
         else break;
     }
-    const int stride_self = 2 + pi_self * kDh, stride_enc = 2 * nqe + pi_enc * nqe * kDh;
+    const int stride_self = part_header_floats(1) + pi_self * kDh, stride_enc = part_header_floats(nqe) + pi_enc * nqe * kDh;
     auto part_need = [&]() {
         const int ns = ceil_div(max_len, span_self), ne = ceil_div(max_src, span_enc);
         return (ns > 1 ? rows_self * ns * stride_self : 0) + (ne > 1 ? rows_enc * ne * stride_enc : 0);
@@ -448,14 +460,19 @@ int32_t san_decode_step(san_ctx* ctx, const san_step_args* a, void* stream) {
         p.aan_sum = reinterpret_cast<float*>(ctx->cache + ctx->off_aan); p.n_aan_layers = c.n_layers;
     }
     p.H = c.n_heads; p.beam = c.beam;
-    p.n_self_blocks = do_self ? ctx->self_pol.n_blocks : 0; p.n_enc_blocks = do_enc ? ctx->enc_pol.n_blocks : 0;
     p.cap_tgt = c.max_tgt_len; p.cap_src = c.max_src_len; p.max_seqs = ctx->n_seqs; p.max_sent = c.max_sent;
     p.enc_v_by_block = c.encdec_shared_context ? 1 : 0;
     p.selfK = ctx->cache + ctx->off_self_k; p.selfV = ctx->cache + ctx->off_self_v;
     p.memK = ctx->cache + ctx->off_mem_k; p.memV = ctx->cache + ctx->off_mem_v;
     p.self_plane_bytes = (long long)ctx->self_plane_bytes; p.mem_plane_bytes = (long long)ctx->mem_plane_bytes;
     p.self_span = span_self; p.self_nspans = ns_self; p.enc_span = span_enc; p.enc_nspans = ns_enc;
-    p.n_enc_items = rows_enc * ns_enc; p.n_items = p.n_enc_items + rows_self * ns_self;
+    if (rows_enc * ns_enc + rows_self * ns_self > (1ll << 30)) return SAN_ERR_UNSUPPORTED;
+    p.n_enc_items = (unsigned)(rows_enc * ns_enc); p.n_items = p.n_enc_items + (unsigned)(rows_self * ns_self);
+    p.n_enc_rows = (unsigned)rows_enc;
+    p.enc_div_span = make_fastdiv((unsigned)ns_enc); p.enc_div_h = make_fastdiv((unsigned)c.n_heads);
+    p.enc_div_item = make_fastdiv((unsigned)std::max(n_sent, 1));
+    p.self_div_span = make_fastdiv((unsigned)ns_self); p.self_div_h = make_fastdiv((unsigned)c.n_heads);
+    p.self_div_item = make_fastdiv((unsigned)std::max(n_seqs, 1));
     p.enc_part_stride = stride_enc; p.self_part_stride = stride_self;
     p.self_part_base = ns_enc > 1 ? rows_enc * ns_enc * stride_enc : 0;
     p.part = ctx->part; p.tickets = ctx->tickets; p.err = ctx->err;

@@ -2,15 +2,18 @@
 // for every block of both attention kinds, plus the AAN running average.
 //
 // Every (kind, block, item, head[, span]) is independent, so the step is a flat list of
-// work items drained by persistent warps.  Each warp owns a ring of shared-memory stages
-// fed by bulk asynchronous copies (cp.async.bulk, completion on an mbarrier): the query
-// rows, then the key panel in tiles, then the value panel of every layer of the block in
-// tiles.  Copies are issued up to kFusedStages tiles ahead of their use and run on into
-// the next item, so the loads of an item never wait for the arithmetic of the one before.
-// For self-attention the newest position is not in the cache yet: its key/value rows are
+// work items (encoder-memory items, the big ones, first).  CTA b owns items b, b+G, b+2G,
+// ... (G = CTAs in the grid), so every CTA gets the same mix; its warps take the next one
+// from a counter in shared memory.  Each warp owns a ring of shared-memory stages fed by
+// bulk asynchronous copies (cp.async.bulk, completion on an mbarrier): the query rows,
+// then the key panel in tiles, then the value panel of every layer of the block in tiles.
+// Copies are issued several tiles ahead of their use and run on into the next item, so
+// the loads of an item never wait for the arithmetic of the one before.  For
+// self-attention the newest position is not in the cache yet: its key/value rows are
 // copied from the caller's k_new/v_new into the last tile beside the cached rows, and
 // written to the cache from there.  S never leaves the chip between weights and apply
-// (it is also written out for the caller).
+// (it is also written out for the caller).  Arithmetic is float32 (packed two-wide FMAs)
+// on the CUDA cores.
 #pragma once
 
 #include "san_kernels.cuh"
@@ -18,16 +21,26 @@
 namespace san {
 
 constexpr int kStageBytes = 4096;   // one tile: 32 bf16 rows or 16 float32 rows
-constexpr int kFusedWarps = 12;
-constexpr int kFusedStages = 4;
-constexpr int kZFloats = 512;       // scores a warp keeps on chip: span <= kZFloats / NQ
-constexpr int kDescSlots = 4;       // decoded items a warp may have in flight
+constexpr int kFusedWarps = 16;
+constexpr int kFusedStages = 3;
+constexpr int kZFloats = 256;       // scores a warp keeps on chip: span <= kZFloats / NQ
+constexpr int kDescSlots = 6;       // decoded items a warp keeps (in flight, being finished, being decoded)
 constexpr int kMaxSpans = 32;
 
 enum { TAG_STEP = 6 };
 
+// Exact division of n < 2^31 by a fixed divisor with one multiply-high (Granlund and
+// Montgomery's round-up method): q = (mulhi(n, mul) + n) >> shift.
+struct FastDiv {
+    unsigned mul, shift, div;
+    __device__ __forceinline__ void divmod(unsigned n, unsigned* q, unsigned* r) const {
+        *q = (unsigned)(((unsigned long long)__umulhi(n, mul) + n) >> shift);
+        *r = n - *q * div;
+    }
+};
+
 struct StepParams {
-    // decoder self-attention (absent when n_self_blocks == 0)
+    // decoder self-attention
     const char* q_self; const char* k_new; const char* v_new;   // [N_s][n][H][64], same, [M][n][H][64]
     const int* seq_ids; const int* pos;                         // row written this step; length = pos + 1
     float* S_self; long long ld_t; char* O_self;                // S may be null
@@ -40,13 +53,15 @@ struct StepParams {
     // AAN in place of self-attention (absent when x_aan == null)
     const char* x_aan; const int* t_aan; float* aan_sum; int n_aan_layers;
     // geometry
-    int H, beam, n_self_blocks, n_enc_blocks, cap_tgt, cap_src, max_seqs, max_sent, enc_v_by_block;
+    int H, beam, cap_tgt, cap_src, max_seqs, max_sent, enc_v_by_block;
     char* selfK; char* selfV; char* memK; char* memV;
     long long self_plane_bytes, mem_plane_bytes;
     int self_span, self_nspans, enc_span, enc_nspans;           // positions per item, spans per row at the bound
-    long long n_enc_items, n_items;                             // enc items come first in the list
+    unsigned n_enc_items, n_items;                              // enc items come first in the list
+    unsigned n_enc_rows;
     long long self_part_base;                                   // float offset of the self rows' partials
     int enc_part_stride, self_part_stride;                      // floats per (row, span)
+    FastDiv enc_div_span, enc_div_h, enc_div_item, self_div_span, self_div_h, self_div_item;
     float* part; int* tickets; int* err;
     float scale_log2e;
     unsigned char self_first[SAN_MAX_LAYERS], self_size[SAN_MAX_LAYERS];
@@ -61,9 +76,9 @@ struct ItemDesc {
     const char* knew; const char* vnew; long long vnew_stride;   // newest rows (self only)
     float* S; long long S_qstride;            // S row of query 0 (may be null)
     char* O; long long O_lstride, O_qstride;  // output of (first layer, query 0)
-    long long row_id;                         // ticket index of the row
     float* part;                              // partial sums of this (row, span)
-    int kind, nq, pi, len, j0, j1, n_spans, span, n_pos_tiles, n_tiles, has_new, part_stride;
+    unsigned row_id;                          // ticket index of the row
+    int kind, nq, pi, len, j0, j1, n_spans, span, has_new, part_stride;
 };
 
 // ------------------------------------------------------------------------------ PTX helpers
@@ -72,22 +87,21 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)_
 __device__ __forceinline__ void mbar_init(uint64_t* bar, int count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
 }
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
     asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
-                 : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
 // Bounded wait: gives up after about a second and reports it; never spins for ever.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
-    if (mbar_try_wait(bar, parity)) return true;
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity) {
     const long long t0 = clock64();
     while (!mbar_try_wait(bar, parity)) {
         if (clock64() - t0 > 2000000000LL) return false;
@@ -100,63 +114,114 @@ template <typename T> struct FusedGeom {
     static constexpr int TR = kStageBytes / ROW_BYTES;   // rows per tile
 };
 
-// ------------------------------------------------------------------------------ the kernel
+// 16 bytes of a row as packed float pairs
+template <typename T> struct Pairs;
+template <> struct Pairs<__nv_bfloat16> {
+    static constexpr int N = 4;
+    static __device__ __forceinline__ void load(const uint4& v, float2* f) {
+        f[0] = make_float2(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xffff0000u));
+        f[1] = make_float2(__uint_as_float(v.y << 16), __uint_as_float(v.y & 0xffff0000u));
+        f[2] = make_float2(__uint_as_float(v.z << 16), __uint_as_float(v.z & 0xffff0000u));
+        f[3] = make_float2(__uint_as_float(v.w << 16), __uint_as_float(v.w & 0xffff0000u));
+    }
+    static __device__ __forceinline__ uint4 store(const float2* f) {
+        uint4 v;
+        __nv_bfloat162 a = __floats2bfloat162_rn(f[0].x, f[0].y), b = __floats2bfloat162_rn(f[1].x, f[1].y);
+        __nv_bfloat162 c = __floats2bfloat162_rn(f[2].x, f[2].y), d = __floats2bfloat162_rn(f[3].x, f[3].y);
+        v.x = *reinterpret_cast<uint32_t*>(&a); v.y = *reinterpret_cast<uint32_t*>(&b);
+        v.z = *reinterpret_cast<uint32_t*>(&c); v.w = *reinterpret_cast<uint32_t*>(&d);
+        return v;
+    }
+};
+template <> struct Pairs<float> {
+    static constexpr int N = 2;
+    static __device__ __forceinline__ void load(const uint4& v, float2* f) {
+        f[0] = make_float2(__uint_as_float(v.x), __uint_as_float(v.y));
+        f[1] = make_float2(__uint_as_float(v.z), __uint_as_float(v.w));
+    }
+    static __device__ __forceinline__ uint4 store(const float2* f) {
+        return make_uint4(__float_as_uint(f[0].x), __float_as_uint(f[0].y), __float_as_uint(f[1].x), __float_as_uint(f[1].y));
+    }
+};
+
+// ------------------------------------------------------------------------------ the warp
 template <typename T>
 struct FusedWarp {
     using G = RowGeom<T>;
     using F = FusedGeom<T>;
+    using P = Pairs<T>;
     static constexpr int VEC = G::VEC, LPR = G::LPR, RPW = 32 / LPR, ROW_BYTES = F::ROW_BYTES, TR = F::TR;
+    static constexpr int NP = P::N;          // float pairs per 16 bytes
+    static constexpr int BLK = 8;            // rows per inner block
+    static constexpr int UN = BLK / RPW;     // loads per lane per block
 
     const StepParams& p;
-    char* ring;            // kFusedStages stages of this warp
-    uint64_t* bars;        // one per stage
-    float* zs;             // kZFloats scores
+    uint32_t ring, bars;   // shared-space addresses: stages and their barriers
+    const char* ring_g;    // the same stages through a generic pointer
+    float* zs;             // kZFloats floats
     ItemDesc* descs;       // kDescSlots
+    unsigned* cta_next;    // shared counter: next slot of this CTA's item sequence to hand out
     int lane, g, c;
-    long long stride;      // warps in the grid
-    // copy side
-    long long p_item; int p_tile; unsigned p_seq; unsigned p_n;   // next item / tile to issue; tiles issued; items decoded
-    int pre_id, pre_len;   // metadata of p_item, fetched ahead
+    // copy side: the item being issued, the next one (metadata on its way), the one after
+    bool p_active;
+    unsigned p_seq, p_n;
+    int p_which, p_s0, p_j0, p_j1, p_pi, p_q_done;
+    const char* p_panel;
+    unsigned nx_item; int nx_id, nx_len;      // next item and its prefetched id / length
+    unsigned nn_item;                         // the item after that
     // math side
     unsigned c_seq, c_n;
     bool dead;             // a wait ran out: stop issuing, drain, leave
 
     __device__ FusedWarp(const StepParams& pp) : p(pp) {}
 
-    // ---- item list: [enc items][self items]; within a kind: ((block, item, head), span)
-    __device__ void fetch_meta(long long it, int* id, int* len) const {
-        if (it >= p.n_items) { *id = 0; *len = 0; return; }
-        if (it < p.n_enc_items) {
-            const long long row = it / p.enc_nspans;
-            const int item = (int)((row / p.H) % p.n_sent);
-            *id = p.sent_ids[item]; *len = p.src_lens[item];
-        } else {
-            const long long row = (it - p.n_enc_items) / p.self_nspans;
-            const int item = (int)((row / p.H) % p.n_seqs);
-            *id = p.seq_ids[item]; *len = p.pos[item] + 1;
-        }
+    __device__ __forceinline__ unsigned item_of_slot(unsigned k) const {
+        const unsigned long long it = (unsigned long long)k * gridDim.x + blockIdx.x;
+        return it < p.n_items ? (unsigned)it : p.n_items;
+    }
+    __device__ __forceinline__ unsigned grab() {
+        unsigned k = 0;
+        if (lane == 0) k = atomicAdd(cta_next, 1u);
+        return item_of_slot(__shfl_sync(0xffffffffu, k, 0));
     }
 
-    // Decodes item `it` into *d; returns false if the item is to be skipped.
-    __device__ bool decode(long long it, int id, int len, ItemDesc* d) const {
-        const bool enc = it < p.n_enc_items;
-        const long long local = enc ? it : it - p.n_enc_items;
-        const int nspans_max = enc ? p.enc_nspans : p.self_nspans;
+    // ---- item list: [enc items][self items]; within a kind: (((block, item), head), span)
+    __device__ __forceinline__ void split(unsigned it, bool* enc, unsigned* block, unsigned* item, unsigned* h, unsigned* span,
+                                          unsigned* row) const {
+        *enc = it < p.n_enc_items;
+        unsigned bi;
+        if (*enc) {
+            p.enc_div_span.divmod(it, row, span);
+            p.enc_div_h.divmod(*row, &bi, h);
+            p.enc_div_item.divmod(bi, block, item);
+        } else {
+            p.self_div_span.divmod(it - p.n_enc_items, row, span);
+            p.self_div_h.divmod(*row, &bi, h);
+            p.self_div_item.divmod(bi, block, item);
+        }
+    }
+    __device__ __forceinline__ void fetch_meta(unsigned it, int* id, int* len) const {
+        *id = 0; *len = 0;
+        if (it >= p.n_items) return;
+        bool enc; unsigned block, item, h, span, row;
+        split(it, &enc, &block, &item, &h, &span, &row);
+        if (enc) { *id = p.sent_ids[item]; *len = p.src_lens[item]; }
+        else { *id = p.seq_ids[item]; *len = p.pos[item] + 1; }
+    }
+
+    // Decodes item `it` into *d (lane 0 writes it); returns false if the item is to be skipped.
+    __device__ bool decode(unsigned it, int id, int len, ItemDesc* d) const {
+        bool enc; unsigned block, item, h, span, row;
+        split(it, &enc, &block, &item, &h, &span, &row);
         const int span_len = enc ? p.enc_span : p.self_span;
-        const int span = (int)(local % nspans_max);
-        const long long row = local / nspans_max;
-        const int h = (int)(row % p.H);
-        const int n_it = enc ? p.n_sent : p.n_seqs;
-        const int item = (int)((row / p.H) % n_it);
-        const int block = (int)(row / ((long long)p.H * n_it));
         const int max_ids = enc ? p.max_sent : p.max_seqs;
         const int bound = enc ? p.max_src : p.max_len;
         const bool reporter = (lane == 0 && span == 0 && h == 0 && block == 0);
-        if (id < 0 || id >= max_ids) { if (reporter) record_error(p.err, TAG_STEP, item, id, max_ids); return false; }
-        if (len < 1 || len > bound) { if (reporter) record_error(p.err, TAG_STEP, item, len, bound); return false; }
-        const int j0 = span * span_len;
+        if (id < 0 || id >= max_ids) { if (reporter) record_error(p.err, TAG_STEP, (int)item, id, max_ids); return false; }
+        if (len < 1 || len > bound) { if (reporter) record_error(p.err, TAG_STEP, (int)item, len, bound); return false; }
+        const int j0 = (int)span * span_len;
         if (j0 >= len) return false;                      // a shorter row has fewer spans
-        if (lane != 0) return true;                       // one lane fills the descriptor
+        if (lane != 0) return true;
         const int j1 = min(len, j0 + span_len);
         const int nq = enc ? p.beam : 1;
         const int first = enc ? p.enc_first[block] : p.self_first[block];
@@ -164,23 +229,23 @@ struct FusedWarp {
         const int cap = enc ? p.cap_src : p.cap_tgt;
         const long long plane = enc ? p.mem_plane_bytes : p.self_plane_bytes;
         const long long panel = (((long long)id * p.H + h) * cap) * ROW_BYTES;
+        const int nspans_max = enc ? p.enc_nspans : p.self_nspans;
         d->kind = enc ? 1 : 0; d->nq = nq; d->pi = pi; d->len = len; d->j0 = j0; d->j1 = j1;
-        d->n_spans = (len + span_len - 1) / span_len; d->span = span;
-        d->n_pos_tiles = (j1 - j0 + TR - 1) / TR;
-        d->n_tiles = 1 + d->n_pos_tiles * (1 + pi);
+        d->n_spans = (len + span_len - 1) / span_len; d->span = (int)span;
         d->has_new = (!enc && j1 == len) ? 1 : 0;
-        d->row_id = enc ? row : (p.n_enc_items / p.enc_nspans) + row;
+        d->row_id = enc ? row : p.n_enc_rows + row;
         d->part_stride = enc ? p.enc_part_stride : p.self_part_stride;
-        d->part = p.part + (enc ? 0 : p.self_part_base) + (row * nspans_max + span) * (long long)d->part_stride;
+        d->part = p.part + (enc ? 0 : p.self_part_base) + ((long long)row * nspans_max + span) * (long long)d->part_stride;
+        d->v_plane = plane;
         if (enc) {
             d->q = p.q_enc + ((((long long)block * p.n_sent + item) * nq) * p.H + h) * ROW_BYTES;
             d->q_stride = (long long)p.H * ROW_BYTES;
             d->Kp = p.memK + block * plane + panel;
-            d->Vp = p.memV + (p.enc_v_by_block ? block : first) * plane + panel;
+            d->Vp = p.memV + (p.enc_v_by_block ? (int)block : first) * plane + panel;
             d->knew = nullptr; d->vnew = nullptr; d->vnew_stride = 0;
             d->S = p.S_enc ? p.S_enc + ((((long long)block * p.n_sent + item) * nq) * p.H + h) * p.ld_s : nullptr;
             d->S_qstride = (long long)p.H * p.ld_s;
-            const int o_first = p.enc_v_by_block ? block : first;
+            const int o_first = p.enc_v_by_block ? (int)block : first;
             d->O = p.O_enc + ((((long long)o_first * p.n_sent + item) * nq) * p.H + h) * ROW_BYTES;
             d->O_lstride = (long long)p.n_sent * nq * p.H * ROW_BYTES;
             d->O_qstride = (long long)p.H * ROW_BYTES;
@@ -197,152 +262,156 @@ struct FusedWarp {
             d->O = p.O_self + first * in_layer + in_row;
             d->O_lstride = in_layer; d->O_qstride = 0;
         }
-        d->v_plane = plane;
         return true;
     }
 
-    // Moves the copy side to the next item that is not skipped and decodes it.
+    // Makes the next item that is not skipped the one being issued.
     __device__ void next_item() {
-        while (p_item < p.n_items) {
+        p_active = false;
+        while (nx_item < p.n_items) {
             ItemDesc* d = &descs[p_n % kDescSlots];
-            const bool ok = decode(p_item, pre_id, pre_len, d);
+            const bool ok = decode(nx_item, nx_id, nx_len, d);
+            // shift the look-ahead: the item after becomes next (its metadata loads start now)
+            nx_item = nn_item;
+            fetch_meta(nx_item, &nx_id, &nx_len);
+            nn_item = (nx_item < p.n_items) ? grab() : nx_item;
             if (ok) {
                 __syncwarp();
-                p_n += 1; p_tile = 0;
-                fetch_meta(p_item + stride, &pre_id, &pre_len);   // used when this item's tiles are all issued
+                p_n += 1; p_active = true;
+                p_q_done = 0; p_which = 0; p_j0 = d->j0; p_j1 = d->j1; p_pi = d->pi; p_s0 = p_j0;
+                p_panel = d->Kp;
                 return;
             }
-            p_item += stride;
-            fetch_meta(p_item, &pre_id, &pre_len);
         }
     }
 
-    // Issues the copies of one tile of the item being produced, if any is left.
+    // Issues the copies of one tile of the item being issued, if any is left.
     __device__ void produce() {
-        if (dead || p_item >= p.n_items) return;
+        if (dead || !p_active) return;
+        const ItemDesc& d = descs[(p_n - 1) % kDescSlots];
+        const unsigned s = p_seq % kFusedStages;
         if (lane == 0) {
-            const ItemDesc& d = descs[(p_n - 1) % kDescSlots];
-            const unsigned s = p_seq % kFusedStages;
-            char* dst = ring + s * kStageBytes;
-            uint64_t* bar = bars + s;
-            if (p_tile == 0) {
+            const uint32_t dst = ring + s * kStageBytes;
+            const uint32_t bar = bars + s * 8;
+            if (!p_q_done) {
                 mbar_expect_tx(bar, (uint32_t)(d.nq * ROW_BYTES));
                 for (int qi = 0; qi < d.nq; ++qi) bulk_g2s(dst + qi * ROW_BYTES, d.q + qi * d.q_stride, ROW_BYTES, bar);
             } else {
-                const int u = p_tile - 1;
-                const int which = u / d.n_pos_tiles, ct = u % d.n_pos_tiles;
-                const int s0 = d.j0 + ct * TR;
-                const int r = min(TR, d.j1 - s0);
-                const bool with_new = d.has_new && (s0 + r == d.len);
+                const int r = min(TR, p_j1 - p_s0);
+                const bool with_new = d.has_new && (p_s0 + r == p_j1);
                 const int r_cache = with_new ? r - 1 : r;
-                const char* src = (which == 0 ? d.Kp : d.Vp + (long long)(which - 1) * d.v_plane) + (long long)s0 * ROW_BYTES;
                 mbar_expect_tx(bar, (uint32_t)(r * ROW_BYTES));
-                if (r_cache > 0) bulk_g2s(dst, src, (uint32_t)(r_cache * ROW_BYTES), bar);
+                if (r_cache > 0) bulk_g2s(dst, p_panel + (long long)p_s0 * ROW_BYTES, (uint32_t)(r_cache * ROW_BYTES), bar);
                 if (with_new) {
-                    const char* nsrc = which == 0 ? d.knew : d.vnew + (long long)(which - 1) * d.vnew_stride;
+                    const char* nsrc = p_which == 0 ? d.knew : d.vnew + (long long)(p_which - 1) * d.vnew_stride;
                     bulk_g2s(dst + r_cache * ROW_BYTES, nsrc, ROW_BYTES, bar);
                 }
             }
         }
-        p_seq += 1; p_tile += 1;
-        const int n_tiles = descs[(p_n - 1) % kDescSlots].n_tiles;
-        if (p_tile == n_tiles) { p_item += stride; next_item(); }
+        p_seq += 1;
+        if (!p_q_done) { p_q_done = 1; return; }
+        p_s0 += TR;
+        if (p_s0 >= p_j1) {
+            p_which += 1; p_s0 = p_j0;
+            if (p_which > p_pi) { next_item(); return; }
+            p_panel = d.Vp + (long long)(p_which - 1) * d.v_plane;
+        }
     }
 
     // Waits for the next tile in order; returns its stage or null after a timeout.
-    __device__ const char* acquire() {
+    __device__ __forceinline__ const char* acquire() {
         const unsigned s = c_seq % kFusedStages;
-        if (!mbar_wait(bars + s, (c_seq / kFusedStages) & 1)) {
-            if (lane == 0) { if (atomicCAS(&p.err[0], 0, (int)SAN_ERR_TIMEOUT) == 0) { p.err[1] = TAG_STEP; p.err[2] = (int)c_seq; } }
-            dead = true;
-            return nullptr;
+        const uint32_t bar = bars + s * 8, par = (c_seq / kFusedStages) & 1;
+        if (!mbar_try_wait(bar, par)) {
+            if (!mbar_wait_slow(bar, par)) {
+                if (lane == 0 && atomicCAS(&p.err[0], 0, (int)SAN_ERR_TIMEOUT) == 0) { p.err[1] = TAG_STEP; p.err[2] = (int)c_seq; }
+                dead = true;
+                return nullptr;
+            }
         }
-        return ring + s * kStageBytes;
+        return ring_g + s * kStageBytes;
     }
     // Every lane is done with the tile: hand the stage back to the copy side.
-    __device__ void release() {
+    __device__ __forceinline__ void release() {
         __syncwarp();
         c_seq += 1;
         produce();
     }
 
     template <int NQ> __device__ bool process(const ItemDesc& d);
-    __device__ void drain();
-};
+    template <int NQ> __device__ void combine(const ItemDesc& d);
 
-// After a timeout: the copies already issued may still land in this warp's stages, so give
-// each a last bounded chance to finish before the CTA's shared memory can go away.
-template <typename T>
-__device__ void FusedWarp<T>::drain() {
-    while (c_seq != p_seq) {
-        const unsigned s = c_seq % kFusedStages;
-        const uint32_t par = (c_seq / kFusedStages) & 1;
-        const long long t0 = clock64();
-        while (!mbar_try_wait(bars + s, par)) { if (clock64() - t0 > 200000000LL) break; }
-        c_seq += 1;
+    // After a timeout: copies already issued may still land in this warp's stages, so give
+    // each a last bounded chance to finish before the CTA's shared memory can go away.
+    __device__ void drain() {
+        while (c_seq != p_seq) {
+            const unsigned s = c_seq % kFusedStages;
+            const uint32_t par = (c_seq / kFusedStages) & 1;
+            const long long t0 = clock64();
+            while (!mbar_try_wait(bars + s * 8, par)) { if (clock64() - t0 > 200000000LL) break; }
+            c_seq += 1;
+        }
     }
-}
+};
 
 template <typename T>
 template <int NQ>
 __device__ bool FusedWarp<T>::process(const ItemDesc& d) {
-    constexpr int UNROLL = 4;
     constexpr int ZQ = kZFloats / NQ;          // score slots per query row
-    const int n = d.j1 - d.j0;
-    const int nq = d.nq;
+    constexpr int HDR = (2 * NQ + 3) / 4 * 4;  // (max, sum) per query ahead of a span's partial sums
+    const int j0 = d.j0, n = d.j1 - d.j0, nq = d.nq, has_new = d.has_new, pi = d.pi;
 
-    // ---- tile 0: the query rows
-    float qf[NQ][VEC];
+    // ---- tile 0: the query rows, scaled into the log2 domain
+    float2 q2[NQ][NP];
     {
         const char* st = acquire();
         if (!st) return false;
+        const float sc = p.scale_log2e;
 #pragma unroll
         for (int qi = 0; qi < NQ; ++qi) {
             if (qi < nq) {
-                unpack16<T>(*reinterpret_cast<const uint4*>(st + qi * ROW_BYTES + c * 16), qf[qi]);
+                P::load(*reinterpret_cast<const uint4*>(st + qi * ROW_BYTES + c * 16), q2[qi]);
 #pragma unroll
-                for (int e = 0; e < VEC; ++e) qf[qi][e] *= p.scale_log2e;
+                for (int e = 0; e < NP; ++e) { q2[qi][e].x *= sc; q2[qi][e].y *= sc; }
             } else {
 #pragma unroll
-                for (int e = 0; e < VEC; ++e) qf[qi][e] = 0.f;
+                for (int e = 0; e < NP; ++e) q2[qi][e] = make_float2(0.f, 0.f);
             }
         }
         release();
     }
 
     // ---- key tiles: scores into zs
-    for (int ct = 0; ct < d.n_pos_tiles; ++ct) {
+    for (int s0 = 0; s0 < n; s0 += TR) {
         const char* st = acquire();
         if (!st) return false;
-        const int r = min(TR, n - ct * TR);
-        const bool with_new = d.has_new && (ct == d.n_pos_tiles - 1);
+        const int r = min(TR, n - s0);
+        const bool with_new = has_new && (s0 + r == n);
+        for (int jb = 0; jb < r; jb += BLK) {
+            uint4 kv[UN];
 #pragma unroll
-        for (int jb = 0; jb < TR; jb += RPW * UNROLL) {
-            if (jb < r) {
-                uint4 kv[UNROLL];
+            for (int u = 0; u < UN; ++u) {
+                const int j = jb + u * RPW + g;
+                kv[u] = (j < r) ? *reinterpret_cast<const uint4*>(st + j * ROW_BYTES + c * 16) : make_uint4(0, 0, 0, 0);
+            }
 #pragma unroll
-                for (int u = 0; u < UNROLL; ++u) {
-                    const int j = jb + u * RPW + g;
-                    kv[u] = (j < r) ? *reinterpret_cast<const uint4*>(st + j * ROW_BYTES + c * 16) : make_uint4(0, 0, 0, 0);
+            for (int u = 0; u < UN; ++u) {
+                const int j = jb + u * RPW + g;
+                float2 k2[NP];
+                P::load(kv[u], k2);
+#pragma unroll
+                for (int qi = 0; qi < NQ; ++qi) {
+                    float2 a = make_float2(0.f, 0.f);
+#pragma unroll
+                    for (int e = 0; e < NP; ++e) a = __ffma2_rn(q2[qi][e], k2[e], a);
+                    float dot = a.x + a.y;
+#pragma unroll
+                    for (int o = LPR / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+                    if (c == 0 && j < r) zs[qi * ZQ + s0 + j] = dot;
                 }
-#pragma unroll
-                for (int u = 0; u < UNROLL; ++u) {
-                    const int j = jb + u * RPW + g;
-                    float kf[VEC];
-                    unpack16<T>(kv[u], kf);
-#pragma unroll
-                    for (int qi = 0; qi < NQ; ++qi) {
-                        float dot = 0.f;
-#pragma unroll
-                        for (int e = 0; e < VEC; ++e) dot = fmaf(qf[qi][e], kf[e], dot);
-#pragma unroll
-                        for (int o = LPR / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-                        if (c == 0 && j < r) zs[qi * ZQ + ct * TR + j] = dot;
-                    }
-                    // the newest key row goes into the cache from here
-                    if (with_new && j == r - 1)
-                        *reinterpret_cast<uint4*>(const_cast<char*>(d.Kp) + (long long)(d.len - 1) * ROW_BYTES + c * 16) = kv[u];
-                }
+                // the newest key row goes into the cache from here
+                if (with_new && j == r - 1)
+                    *reinterpret_cast<uint4*>(const_cast<char*>(d.Kp) + (long long)(d.len - 1) * ROW_BYTES + c * 16) = kv[u];
             }
         }
         release();
@@ -350,6 +419,7 @@ __device__ bool FusedWarp<T>::process(const ItemDesc& d) {
 
     // ---- softmax over the span (log2 domain)
     float part_m[NQ], part_l[NQ];
+    const int n_spans = d.n_spans;
 #pragma unroll
     for (int qi = 0; qi < NQ; ++qi) {
         part_m[qi] = 0.f; part_l[qi] = 1.f;
@@ -361,10 +431,11 @@ __device__ bool FusedWarp<T>::process(const ItemDesc& d) {
             for (int jj = lane; jj < n; jj += 32) { const float e = exp2f(zs[qi * ZQ + jj] - m); zs[qi * ZQ + jj] = e; s += e; }
             s = warp_sum(s);
             part_m[qi] = m; part_l[qi] = s;
-            float* Srow = d.S ? d.S + qi * d.S_qstride + d.j0 : nullptr;
-            if (d.n_spans == 1) {
+            float* Srow = d.S ? d.S + qi * d.S_qstride + j0 : nullptr;
+            if (n_spans == 1) {
+                const float inv = 1.0f / s;
                 for (int jj = lane; jj < n; jj += 32) {
-                    const float w = zs[qi * ZQ + jj] / s;
+                    const float w = zs[qi * ZQ + jj] * inv;
                     zs[qi * ZQ + jj] = w;
                     if (Srow) Srow[jj] = w;
                 }
@@ -375,44 +446,41 @@ __device__ bool FusedWarp<T>::process(const ItemDesc& d) {
     }
     __syncwarp();
 
-    // ---- value tiles, layer by layer
-    float* part = d.part;
-    for (int l = 0; l < d.pi; ++l) {
-        float acc[NQ][VEC];
+    // ---- value tiles, layer by layer (score rows of absent queries hold zeros)
+    for (int l = 0; l < pi; ++l) {
+        float2 acc[NQ][NP];
 #pragma unroll
         for (int qi = 0; qi < NQ; ++qi)
 #pragma unroll
-            for (int e = 0; e < VEC; ++e) acc[qi][e] = 0.f;
-        for (int ct = 0; ct < d.n_pos_tiles; ++ct) {
+            for (int e = 0; e < NP; ++e) acc[qi][e] = make_float2(0.f, 0.f);
+        for (int s0 = 0; s0 < n; s0 += TR) {
             const char* st = acquire();
             if (!st) return false;
-            const int r = min(TR, n - ct * TR);
-            const bool with_new = d.has_new && (ct == d.n_pos_tiles - 1);
+            const int r = min(TR, n - s0);
+            const bool with_new = has_new && (s0 + r == n);
+            for (int jb = 0; jb < r; jb += BLK) {
+                uint4 vv[UN];
 #pragma unroll
-            for (int jb = 0; jb < TR; jb += RPW * UNROLL) {
-                if (jb < r) {
-                    uint4 vv[UNROLL];
+                for (int u = 0; u < UN; ++u) {
+                    const int j = jb + u * RPW + g;
+                    vv[u] = (j < r) ? *reinterpret_cast<const uint4*>(st + j * ROW_BYTES + c * 16) : make_uint4(0, 0, 0, 0);
+                }
 #pragma unroll
-                    for (int u = 0; u < UNROLL; ++u) {
-                        const int j = jb + u * RPW + g;
-                        vv[u] = (j < r) ? *reinterpret_cast<const uint4*>(st + j * ROW_BYTES + c * 16) : make_uint4(0, 0, 0, 0);
-                    }
+                for (int u = 0; u < UN; ++u) {
+                    const int j = jb + u * RPW + g;
+                    if (j < r) {
+                        float2 v2[NP];
+                        P::load(vv[u], v2);
 #pragma unroll
-                    for (int u = 0; u < UNROLL; ++u) {
-                        const int j = jb + u * RPW + g;
-                        if (j < r) {
-                            float vf[VEC];
-                            unpack16<T>(vv[u], vf);
+                        for (int qi = 0; qi < NQ; ++qi) {
+                            const float s = zs[qi * ZQ + s0 + j];
+                            const float2 ss = make_float2(s, s);
 #pragma unroll
-                            for (int qi = 0; qi < NQ; ++qi) {
-                                const float s = (qi < nq) ? zs[qi * ZQ + ct * TR + j] : 0.f;
-#pragma unroll
-                                for (int e = 0; e < VEC; ++e) acc[qi][e] = fmaf(s, vf[e], acc[qi][e]);
-                            }
-                            if (with_new && j == r - 1)
-                                *reinterpret_cast<uint4*>(const_cast<char*>(d.Vp) + (long long)l * d.v_plane +
-                                                          (long long)(d.len - 1) * ROW_BYTES + c * 16) = vv[u];
+                            for (int e = 0; e < NP; ++e) acc[qi][e] = __ffma2_rn(ss, v2[e], acc[qi][e]);
                         }
+                        if (with_new && j == r - 1)
+                            *reinterpret_cast<uint4*>(const_cast<char*>(d.Vp) + (long long)l * d.v_plane +
+                                                      (long long)(d.len - 1) * ROW_BYTES + c * 16) = vv[u];
                     }
                 }
             }
@@ -421,71 +489,103 @@ __device__ bool FusedWarp<T>::process(const ItemDesc& d) {
 #pragma unroll
         for (int qi = 0; qi < NQ; ++qi)
 #pragma unroll
-            for (int e = 0; e < VEC; ++e)
+            for (int e = 0; e < NP; ++e)
 #pragma unroll
-                for (int o = LPR; o < 32; o <<= 1) acc[qi][e] += __shfl_xor_sync(0xffffffffu, acc[qi][e], o);
+                for (int o = LPR; o < 32; o <<= 1) {
+                    acc[qi][e].x += __shfl_xor_sync(0xffffffffu, acc[qi][e].x, o);
+                    acc[qi][e].y += __shfl_xor_sync(0xffffffffu, acc[qi][e].y, o);
+                }
         if (g == 0) {
 #pragma unroll
             for (int qi = 0; qi < NQ; ++qi) {
                 if (qi < nq) {
-                    if (d.n_spans == 1) {
-                        *reinterpret_cast<uint4*>(d.O + l * d.O_lstride + qi * d.O_qstride + c * 16) = pack16<T>(acc[qi]);
+                    if (n_spans == 1) {
+                        *reinterpret_cast<uint4*>(d.O + l * d.O_lstride + qi * d.O_qstride + c * 16) = P::store(acc[qi]);
                     } else {
-                        float* pp = part + 2 * NQ + ((long long)l * NQ + qi) * kDh + c * VEC;
+                        float2* pp = reinterpret_cast<float2*>(d.part + HDR + ((long long)l * NQ + qi) * kDh + c * VEC);
 #pragma unroll
-                        for (int e = 0; e < VEC; ++e) pp[e] = acc[qi][e];
+                        for (int e = 0; e < NP; ++e) pp[e] = acc[qi][e];
                     }
                 }
             }
         }
     }
-    if (d.n_spans == 1) return true;
+    if (n_spans == 1) return true;
 
     // ---- split row: park (max, sum); the last span to arrive combines all of them
     if (lane == 0) {
 #pragma unroll
-        for (int qi = 0; qi < NQ; ++qi) { part[qi] = part_m[qi]; part[NQ + qi] = part_l[qi]; }
+        for (int qi = 0; qi < NQ; ++qi) { d.part[qi] = part_m[qi]; d.part[NQ + qi] = part_l[qi]; }
     }
     __threadfence();
     __syncwarp();
     int t = 0;
     if (lane == 0) t = atomicAdd(p.tickets + d.row_id, 1);
     t = __shfl_sync(0xffffffffu, t, 0);
-    if (t != d.n_spans - 1) return true;
+    if (t == n_spans - 1) combine<NQ>(d);
+    return true;
+}
+
+// The last span of a split row: softmax weights across spans, then S and every layer's O.
+template <typename T>
+template <int NQ>
+__device__ void FusedWarp<T>::combine(const ItemDesc& d) {
+    constexpr int HDR = (2 * NQ + 3) / 4 * 4;
     __threadfence();
-    const float* row_part = part - (long long)d.span * d.part_stride;
+    const int n_spans = d.n_spans, nq = d.nq, stride = d.part_stride;
+    const float* row_part = d.part - (long long)d.span * stride;
     const int span_len = d.kind ? p.enc_span : p.self_span;
-    for (int qi = 0; qi < nq; ++qi) {
-        // lane sp holds span sp's weight exp2(m_sp - M) / total
+    // zs[sp * NQ + qi] = exp2(m_sp - M) / total  (zs is free: every layer of this span is done)
+    __syncwarp();
+    for (int qi = 0; qi < NQ; ++qi) {
         float m = -INFINITY, l = 0.f;
-        if (lane < d.n_spans) { m = __ldcg(row_part + (long long)lane * d.part_stride + qi); l = __ldcg(row_part + (long long)lane * d.part_stride + NQ + qi); }
+        if (lane < n_spans && qi < nq) { m = __ldcg(row_part + (long long)lane * stride + qi); l = __ldcg(row_part + (long long)lane * stride + NQ + qi); }
         const float M = warp_max(m);
-        const float wl = (lane < d.n_spans) ? l * exp2f(m - M) : 0.f;
+        const float wl = (lane < n_spans && qi < nq) ? l * exp2f(m - M) : 0.f;
         const float tot = warp_sum(wl);
-        const float wgt = (lane < d.n_spans) ? exp2f(m - M) / tot : 0.f;
-        if (d.S) {
+        if (lane < n_spans) zs[lane * NQ + qi] = (qi < nq) ? exp2f(m - M) / tot : 0.f;
+    }
+    __syncwarp();
+    if (d.S) {
+        for (int qi = 0; qi < nq; ++qi) {
             float* Srow = d.S + qi * d.S_qstride;
-            for (int sp = 0; sp < d.n_spans; ++sp) {
-                const float f = __shfl_sync(0xffffffffu, wgt, sp);
-                const int b = sp * span_len, e = min(d.len, b + span_len);
-                for (int j = b + lane; j < e; j += 32) Srow[j] = __ldcg(Srow + j) * f;
+            for (int j = lane; j < d.len; j += 32) Srow[j] = __ldcg(Srow + j) * zs[(j / span_len) * NQ + qi];
+        }
+    }
+    // every layer's output: E = pi*NQ*64 floats per span, four per lane per pass
+    const int E = d.pi * NQ * kDh;
+    for (int e0 = lane * 4; e0 < E; e0 += 128) {
+        const int qi = (e0 / kDh) % NQ;
+        if (qi >= nq) continue;
+        float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+        const float* src = row_part + HDR + e0;
+        int sp = 0;
+        for (; sp + 4 <= n_spans; sp += 4) {
+            float4 x[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) x[u] = __ldcg(reinterpret_cast<const float4*>(src + (long long)(sp + u) * stride));
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const float f = zs[(sp + u) * NQ + qi];
+                a.x = fmaf(f, x[u].x, a.x); a.y = fmaf(f, x[u].y, a.y); a.z = fmaf(f, x[u].z, a.z); a.w = fmaf(f, x[u].w, a.w);
             }
         }
-        for (int ly = 0; ly < d.pi; ++ly) {
-            float a0 = 0.f, a1 = 0.f;
-            for (int sp = 0; sp < d.n_spans; ++sp) {
-                const float f = __shfl_sync(0xffffffffu, wgt, sp);
-                const float* pp = row_part + (long long)sp * d.part_stride + 2 * NQ + ((long long)ly * NQ + qi) * kDh;
-                a0 = fmaf(f, __ldcg(pp + lane), a0);
-                a1 = fmaf(f, __ldcg(pp + 32 + lane), a1);
-            }
-            T* op = reinterpret_cast<T*>(d.O + ly * d.O_lstride + qi * d.O_qstride);
-            op[lane] = (T)a0;
-            op[32 + lane] = (T)a1;
+        for (; sp < n_spans; ++sp) {
+            const float4 x = __ldcg(reinterpret_cast<const float4*>(src + (long long)sp * stride));
+            const float f = zs[sp * NQ + qi];
+            a.x = fmaf(f, x.x, a.x); a.y = fmaf(f, x.y, a.y); a.z = fmaf(f, x.z, a.z); a.w = fmaf(f, x.w, a.w);
+        }
+        const int ly = e0 / (NQ * kDh), col = e0 % kDh;
+        char* op = d.O + ly * d.O_lstride + qi * d.O_qstride + col * (int)sizeof(T);
+        if (sizeof(T) == 2) {
+            __nv_bfloat162 lo = __floats2bfloat162_rn(a.x, a.y), hi = __floats2bfloat162_rn(a.z, a.w);
+            uint2 r; r.x = *reinterpret_cast<uint32_t*>(&lo); r.y = *reinterpret_cast<uint32_t*>(&hi);
+            *reinterpret_cast<uint2*>(op) = r;
+        } else {
+            *reinterpret_cast<float4*>(op) = a;
         }
     }
     if (lane == 0) p.tickets[d.row_id] = 0;
-    return true;
 }
 
 constexpr size_t fused_smem_bytes() {
@@ -496,6 +596,7 @@ constexpr size_t fused_smem_bytes() {
 template <typename T, int NQE>
 __global__ void __launch_bounds__(kFusedWarps * 32, 1) decode_step_kernel(const __grid_constant__ StepParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
+    __shared__ unsigned cta_next;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 
     // ---- AAN running average (Table 6 pairing): element-wise, every thread of the grid
@@ -537,32 +638,36 @@ __global__ void __launch_bounds__(kFusedWarps * 32, 1) decode_step_kernel(const 
     if (p.n_items == 0) return;
 
     // ---- attention items
+    if (threadIdx.x == 0) cta_next = kFusedWarps;   // slots 0..warps-1 are the warps' first items
+    __syncthreads();
     FusedWarp<T> w(p);
     char* base = reinterpret_cast<char*>(smem);
-    w.ring = base + (size_t)warp * kFusedStages * kStageBytes;
+    w.ring_g = base + (size_t)warp * kFusedStages * kStageBytes;
+    w.ring = smem_u32(w.ring_g);
     char* after = base + (size_t)kFusedWarps * kFusedStages * kStageBytes;
     w.zs = reinterpret_cast<float*>(after) + (size_t)warp * kZFloats;
     after += (size_t)kFusedWarps * kZFloats * sizeof(float);
     w.descs = reinterpret_cast<ItemDesc*>(after) + (size_t)warp * kDescSlots;
     after += (size_t)kFusedWarps * kDescSlots * sizeof(ItemDesc);
-    w.bars = reinterpret_cast<uint64_t*>(after) + (size_t)warp * kFusedStages;
+    uint64_t* bars_g = reinterpret_cast<uint64_t*>(after) + (size_t)warp * kFusedStages;
+    w.bars = smem_u32(bars_g);
+    w.cta_next = &cta_next;
     w.lane = lane; w.g = lane / RowGeom<T>::LPR; w.c = lane % RowGeom<T>::LPR;
-    w.stride = (long long)gridDim.x * kFusedWarps;
-    w.p_item = (long long)blockIdx.x * kFusedWarps + warp;   // neighbouring items go to different SMs' warps
-    w.p_tile = 0; w.p_seq = 0; w.p_n = 0; w.c_seq = 0; w.c_n = 0; w.dead = false;
+    w.p_seq = 0; w.p_n = 0; w.c_seq = 0; w.c_n = 0; w.dead = false; w.p_active = false;
     if (lane == 0) {
-        for (int s = 0; s < kFusedStages; ++s) mbar_init(w.bars + s, 1);
+        for (int s = 0; s < kFusedStages; ++s) mbar_init(bars_g + s, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncwarp();
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    w.fetch_meta(w.p_item, &w.pre_id, &w.pre_len);
+    w.nx_item = w.item_of_slot((unsigned)warp);
+    w.fetch_meta(w.nx_item, &w.nx_id, &w.nx_len);
+    w.nn_item = (w.nx_item < p.n_items) ? w.grab() : w.nx_item;
     w.next_item();
     for (int s = 0; s < kFusedStages; ++s) w.produce();
     while (w.c_n < w.p_n && !w.dead) {
         const ItemDesc& d = w.descs[w.c_n % kDescSlots];
-        const bool ok = d.kind ? w.template process<NQE>(d) : w.template process<1>(d);
-        (void)ok;
+        if (d.kind) w.template process<NQE>(d); else w.template process<1>(d);
         w.c_n += 1;
     }
     if (w.dead) w.drain();
