@@ -30,7 +30,11 @@
  *    s / beam (the beams of a sentence read the same encoder memory, Section 2).
  *
  * Cache layout inside the arena (head-major; every (id, head) panel is contiguous and
- * each row is 64 elements = 128 B bf16 / 256 B f32, 16-byte aligned):
+ * each row is 64 elements = 128 B bf16 / 256 B f32, 16-byte aligned).  bf16 rows are stored
+ * with their eight 16-byte chunks permuted: chunk c of the row at position pos sits at chunk
+ * c ^ (pos & 7), so that a tile of rows copied verbatim into shared memory can be read eight
+ * rows at a time without bank conflicts; callers never see this unless they read the arena
+ * directly.  float32 rows are stored in natural order.
  *    self K   [self block ][sequence][head][max_tgt_len][64]   (block-first layers only)
  *    self V   [layer      ][sequence][head][max_tgt_len][64]
  *    memory K [encdec block][sentence][head][max_src_len][64]

@@ -12,8 +12,9 @@
 // self-attention the newest position is not in the cache yet: its key/value rows are
 // copied from the caller's k_new/v_new into the last tile beside the cached rows, and
 // written to the cache from there.  S never leaves the chip between weights and apply
-// (it is also written out for the caller).  Arithmetic is float32 (packed two-wide FMAs)
-// on the CUDA cores.
+// (it is also written out for the caller).  bf16 items run on the tensor cores (mma.sync,
+// float32 accumulate) because the step is bound by instruction issue; float32 items use
+// packed two-wide FMAs on the CUDA cores.
 #pragma once
 
 #include "san_kernels.cuh"
@@ -107,6 +108,25 @@ __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity) {
         if (clock64() - t0 > 2000000000LL) return false;
     }
     return true;
+}
+
+// Four 8x8 b16 matrices from shared memory, one row address per lane (plain / transposed).
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr) : "memory");
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr) : "memory");
+}
+// D(16x8, f32) += A(16x16, bf16, row) * B(16x8, bf16, col)
+__device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
 }
 
 template <typename T> struct FusedGeom {
@@ -333,13 +353,41 @@ struct FusedWarp {
     }
     // Every lane is done with the tile: hand the stage back to the copy side.
     __device__ __forceinline__ void release() {
+        // the tensor-core path writes into its tiles (chunk-permuting the newest row, zeroing a
+        // ragged tail): order those writes ahead of the bulk copy that will reuse the stage
+        if (sizeof(T) == 2) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncwarp();
         c_seq += 1;
         produce();
     }
 
     template <int NQ> __device__ bool process(const ItemDesc& d);
+    template <int NQ> __device__ bool process_mma(const ItemDesc& d);
     template <int NQ> __device__ void combine(const ItemDesc& d);
+
+    // bf16 tiles only.  A tile's last row may be this step's new row, copied in natural chunk
+    // order from the caller's buffer: permute its chunks like a cached row (chunk c -> c ^ (pos & 7))
+    // and write it to the cache at `dst_row`.  Rows [r, next multiple of 16) are zeroed when
+    // `zero_tail` is set, so that a 16-row block never multiplies stale shared memory.
+    __device__ __forceinline__ void fix_tile(const char* st, int r, bool with_new, char* dst_row, bool zero_tail) {
+        if (with_new) {
+            char* row = const_cast<char*>(st) + (r - 1) * 128;
+            uint4 v = make_uint4(0, 0, 0, 0);
+            if (lane < 8) v = *reinterpret_cast<const uint4*>(row + lane * 16);
+            __syncwarp();
+            if (lane < 8) {
+                const int pc = lane ^ ((r - 1) & 7);
+                *reinterpret_cast<uint4*>(row + pc * 16) = v;
+                *reinterpret_cast<uint4*>(dst_row + pc * 16) = v;
+            }
+        }
+        if (zero_tail && (r & 15)) {
+            const int r16 = (r + 15) & ~15;
+            for (int j = r + (lane >> 3); j < r16; j += 4)
+                *reinterpret_cast<uint4*>(const_cast<char*>(st) + j * 128 + (lane & 7) * 16) = make_uint4(0, 0, 0, 0);
+        }
+        __syncwarp();
+    }
 
     // After a timeout: copies already issued may still land in this warp's stages, so give
     // each a last bounded chance to finish before the CTA's shared memory can go away.
@@ -526,6 +574,169 @@ __device__ bool FusedWarp<T>::process(const ItemDesc& d) {
     return true;
 }
 
+// bf16 items on the tensor cores (mma.sync m16n8k16, float32 accumulate).  Neither product
+// is a dense GEMM: the tensor cores are used because one 16-row block of a tile then costs
+// a handful of instructions (4 ldmatrix + 4 mma for the scores, 4 ldmatrix + 16 mma for one
+// layer's S.V) instead of a hundred or more unpack/FMA/shuffle instructions, and the step
+// is bound by instruction issue, not by tensor throughput.
+//   scores:  D[16 positions x 8 queries] = K_tile[16 x 64] . q^T          (queries padded to 8)
+//   apply:   D[16 queries x 8 dims]     += S[16 x 16 positions] . V_tile   (eight dim tiles)
+// S is split into a bf16 high part and a bf16 remainder (two MMAs) so that the weights keep
+// about 16 bits; products and sums are float32.
+template <typename T>
+template <int NQ>
+__device__ bool FusedWarp<T>::process_mma(const ItemDesc& d) {
+    static_assert(sizeof(T) == 2, "tensor-core path is for bf16 rows");
+    constexpr int ZQ = kZFloats / NQ;
+    constexpr int HDR = (2 * NQ + 3) / 4 * 4;
+    const int j0 = d.j0, n = d.j1 - d.j0, nq = d.nq, has_new = d.has_new, pi = d.pi;
+    const int tig = lane & 3, gid = lane >> 2;                 // mma fragment coordinates
+    const int lrow = (lane & 7) + ((lane >> 3) & 1) * 8;        // ldmatrix: row of the 16-row block this lane addresses
+    const int lx = lane & 7, lsel = lane >> 4;                  // its chunk permutation key and chunk of the pair
+
+    // ---- tile 0: the query rows as B fragments (k = dims, n = query), natural chunk order
+    uint32_t qb[4][2];
+    {
+        const char* st = acquire();
+        if (!st) return false;
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks) {
+            qb[ks][0] = 0u; qb[ks][1] = 0u;
+            if (gid < nq) {
+                qb[ks][0] = *reinterpret_cast<const uint32_t*>(st + gid * 128 + (16 * ks + 2 * tig) * 2);
+                qb[ks][1] = *reinterpret_cast<const uint32_t*>(st + gid * 128 + (16 * ks + 8 + 2 * tig) * 2);
+            }
+        }
+        release();
+    }
+
+    // ---- key tiles: scores into zs (log2 domain)
+    const float sc = p.scale_log2e;
+    for (int s0 = 0; s0 < n; s0 += TR) {
+        const char* st = acquire();
+        if (!st) return false;
+        const int r = min(TR, n - s0);
+        fix_tile(st, r, has_new && (s0 + r == n), const_cast<char*>(d.Kp) + (long long)(d.len - 1) * 128, false);
+        const uint32_t st_s = ring + (uint32_t)(st - ring_g);
+        for (int b0 = 0; b0 < r; b0 += 16) {
+            float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks) {
+                uint32_t a[4];
+                ldsm_x4(st_s + (b0 + lrow) * 128 + (((2 * ks + lsel) ^ lx) << 4), a);
+                mma_bf16(acc, a[0], a[1], a[2], a[3], qb[ks][0], qb[ks][1]);
+            }
+            // acc[0], acc[1]: position b0+gid, queries 2tig, 2tig+1; acc[2], acc[3]: position b0+gid+8
+            const int p0 = b0 + gid, p1 = b0 + gid + 8;
+            if (2 * tig < NQ) {
+                if (p0 < r) zs[(2 * tig) * ZQ + s0 + p0] = acc[0] * sc;
+                if (p1 < r) zs[(2 * tig) * ZQ + s0 + p1] = acc[2] * sc;
+            }
+            if (2 * tig + 1 < NQ) {
+                if (p0 < r) zs[(2 * tig + 1) * ZQ + s0 + p0] = acc[1] * sc;
+                if (p1 < r) zs[(2 * tig + 1) * ZQ + s0 + p1] = acc[3] * sc;
+            }
+        }
+        release();
+    }
+    __syncwarp();
+
+    // ---- softmax over the span (log2 domain)
+    float part_m[NQ], part_l[NQ];
+    const int n_spans = d.n_spans;
+    const int n16 = (n + 15) & ~15;
+#pragma unroll
+    for (int qi = 0; qi < NQ; ++qi) {
+        part_m[qi] = 0.f; part_l[qi] = 1.f;
+        if (qi < nq) {
+            float m = -INFINITY;
+            for (int jj = lane; jj < n; jj += 32) m = fmaxf(m, zs[qi * ZQ + jj]);
+            m = warp_max(m);
+            float s = 0.f;
+            for (int jj = lane; jj < n; jj += 32) { const float e = exp2f(zs[qi * ZQ + jj] - m); zs[qi * ZQ + jj] = e; s += e; }
+            s = warp_sum(s);
+            part_m[qi] = m; part_l[qi] = s;
+            float* Srow = d.S ? d.S + qi * d.S_qstride + j0 : nullptr;
+            if (n_spans == 1) {
+                const float inv = 1.0f / s;
+                for (int jj = lane; jj < n; jj += 32) {
+                    const float w = zs[qi * ZQ + jj] * inv;
+                    zs[qi * ZQ + jj] = w;
+                    if (Srow) Srow[jj] = w;
+                }
+            } else if (Srow) {
+                for (int jj = lane; jj < n; jj += 32) Srow[jj] = zs[qi * ZQ + jj];
+            }
+        }
+        // weights beyond the span's end (up to the next multiple of 16) must be exactly zero
+        for (int jj = n + lane; jj < n16; jj += 32) zs[qi * ZQ + jj] = 0.f;
+    }
+    __syncwarp();
+
+    // ---- value tiles, layer by layer
+    for (int l = 0; l < pi; ++l) {
+        float acc[8][4];
+#pragma unroll
+        for (int nt = 0; nt < 8; ++nt)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc[nt][e] = 0.f;
+        for (int s0 = 0; s0 < n; s0 += TR) {
+            const char* st = acquire();
+            if (!st) return false;
+            const int r = min(TR, n - s0);
+            fix_tile(st, r, has_new && (s0 + r == n),
+                     const_cast<char*>(d.Vp) + (long long)l * d.v_plane + (long long)(d.len - 1) * 128, true);
+            const uint32_t st_s = ring + (uint32_t)(st - ring_g);
+            for (int b0 = 0; b0 < r; b0 += 16) {
+                // A = weights of query gid at positions b0 + {2tig, 2tig+1, 2tig+8, 2tig+9}: high part + remainder
+                uint32_t ah0 = 0u, ah2 = 0u, al0 = 0u, al2 = 0u;
+                if (gid < NQ) {
+                    const float2 w0 = *reinterpret_cast<const float2*>(zs + gid * ZQ + s0 + b0 + 2 * tig);
+                    const float2 w1 = *reinterpret_cast<const float2*>(zs + gid * ZQ + s0 + b0 + 2 * tig + 8);
+                    ah0 = pack_bf16x2(w0.x, w0.y); ah2 = pack_bf16x2(w1.x, w1.y);
+                    al0 = pack_bf16x2(w0.x - __uint_as_float(ah0 << 16), w0.y - __uint_as_float(ah0 & 0xffff0000u));
+                    al2 = pack_bf16x2(w1.x - __uint_as_float(ah2 << 16), w1.y - __uint_as_float(ah2 & 0xffff0000u));
+                }
+#pragma unroll
+                for (int np = 0; np < 4; ++np) {
+                    uint32_t b[4];
+                    ldsm_x4_t(st_s + (b0 + lrow) * 128 + (((2 * np + lsel) ^ lx) << 4), b);
+                    mma_bf16(acc[2 * np], ah0, 0u, ah2, 0u, b[0], b[1]);
+                    mma_bf16(acc[2 * np + 1], ah0, 0u, ah2, 0u, b[2], b[3]);
+                    mma_bf16(acc[2 * np], al0, 0u, al2, 0u, b[0], b[1]);
+                    mma_bf16(acc[2 * np + 1], al0, 0u, al2, 0u, b[2], b[3]);
+                }
+            }
+            release();
+        }
+        // acc[nt][0], acc[nt][1]: query gid, dims 8nt + 2tig, +1
+        if (gid < nq) {
+            if (n_spans == 1) {
+                char* op = d.O + l * d.O_lstride + gid * d.O_qstride + 4 * tig;
+#pragma unroll
+                for (int nt = 0; nt < 8; ++nt) *reinterpret_cast<uint32_t*>(op + 16 * nt) = pack_bf16x2(acc[nt][0], acc[nt][1]);
+            } else {
+                float* pp = d.part + HDR + ((long long)l * NQ + gid) * kDh + 2 * tig;
+#pragma unroll
+                for (int nt = 0; nt < 8; ++nt) *reinterpret_cast<float2*>(pp + 8 * nt) = make_float2(acc[nt][0], acc[nt][1]);
+            }
+        }
+    }
+    if (n_spans == 1) return true;
+
+    if (lane == 0) {
+#pragma unroll
+        for (int qi = 0; qi < NQ; ++qi) { d.part[qi] = part_m[qi]; d.part[NQ + qi] = part_l[qi]; }
+    }
+    __threadfence();
+    __syncwarp();
+    int t = 0;
+    if (lane == 0) t = atomicAdd(p.tickets + d.row_id, 1);
+    t = __shfl_sync(0xffffffffu, t, 0);
+    if (t == n_spans - 1) combine<NQ>(d);
+    return true;
+}
+
 // The last span of a split row: softmax weights across spans, then S and every layer's O.
 template <typename T>
 template <int NQ>
@@ -667,7 +878,11 @@ __global__ void __launch_bounds__(kFusedWarps * 32, 1) decode_step_kernel(const 
     for (int s = 0; s < kFusedStages; ++s) w.produce();
     while (w.c_n < w.p_n && !w.dead) {
         const ItemDesc& d = w.descs[w.c_n % kDescSlots];
-        if (d.kind) w.template process<NQE>(d); else w.template process<1>(d);
+        if constexpr (sizeof(T) == 2) {
+            if (d.kind) w.template process_mma<NQE>(d); else w.template process_mma<1>(d);
+        } else {
+            if (d.kind) w.template process<NQE>(d); else w.template process<1>(d);
+        }
         w.c_n += 1;
     }
     if (w.dead) w.drain();

@@ -34,13 +34,20 @@ __device__ __forceinline__ void record_error(int* err, int tag, int item, int va
 
 // ---------------------------------------------------------------- row geometry per dtype
 template <typename T> struct RowGeom;
+// Cached bf16 rows are stored with their eight 16-byte chunks permuted: logical chunk c of
+// the row at position `pos` sits at chunk c ^ (pos & 7).  A tile of such rows copied
+// verbatim into shared memory (rows 128 bytes apart, tile starting at a multiple of 8
+// positions) can then be read eight rows at a time by ldmatrix without bank conflicts.
+// float32 rows (256 bytes) are stored in natural order.
 template <> struct RowGeom<__nv_bfloat16> {
     static constexpr int VEC = 8;   // elements per 16-byte load
     static constexpr int LPR = 8;   // lanes per 64-element row
+    static __device__ __forceinline__ int chunk(int c, int pos) { return c ^ (pos & 7); }
 };
 template <> struct RowGeom<float> {
     static constexpr int VEC = 4;
     static constexpr int LPR = 16;
+    static __device__ __forceinline__ int chunk(int c, int) { return c; }
 };
 
 __device__ __forceinline__ uint4 ld16_stream(const void* p) {
@@ -129,8 +136,9 @@ static __global__ void __launch_bounds__(256) append_kernel(const AppendParams p
     const int src_layer = is_k ? p.k_src[lr] : lr;
     const char* src = (is_k ? p.k_new : p.v_new) +
         ((((long long)src_layer * p.n_items + item) * p.rows_per_item + r) * p.H + h) * p.row_bytes + piece * 16;
+    const int dst_piece = (p.row_bytes == 128) ? (piece ^ ((pos + r) & 7)) : piece;   // bf16 rows are chunk-permuted
     char* dst = (is_k ? p.K + plane * p.k_plane_bytes : p.V + plane * p.v_plane_bytes) +
-        ((((long long)id * p.H + h) * p.cap_len) + pos + r) * p.row_bytes + piece * 16;
+        ((((long long)id * p.H + h) * p.cap_len) + pos + r) * p.row_bytes + dst_piece * 16;
     *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
 }
 
@@ -188,7 +196,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) weights_kernel(const Weight
         }
     }
 
-    const T* Kp = reinterpret_cast<const T*>(p.K) + (((long long)id * p.H + h) * p.cap_len) * kDh + c * VEC;
+    const T* Kp = reinterpret_cast<const T*>(p.K) + (((long long)id * p.H + h) * p.cap_len) * kDh;
     float (*zs)[kSub] = zs_all[warp];
     const bool one_pass = (j1 - j0) <= kSub;   // the whole span fits on chip: softmax from shared memory
     float run_max[NQ];
@@ -203,7 +211,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) weights_kernel(const Weight
 #pragma unroll
             for (int u = 0; u < UNROLL; ++u) {
                 const int j = jb + u * RPW + g;
-                kv[u] = (j < n) ? ld16_stream(Kp + (long long)(s0 + j) * kDh) : make_uint4(0, 0, 0, 0);
+                kv[u] = (j < n) ? ld16_stream(Kp + (long long)(s0 + j) * kDh + G::chunk(c, s0 + j) * VEC) : make_uint4(0, 0, 0, 0);
             }
 #pragma unroll
             for (int u = 0; u < UNROLL; ++u) {
@@ -338,7 +346,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) apply_kernel(const ApplyPar
 
     for (int l = l_begin; l < l_end; ++l) {
         const T* Vp = reinterpret_cast<const T*>(p.V) + (long long)l * p.plane_elems +
-                      (((long long)id * p.H + h) * p.cap_len) * kDh + c * VEC;
+                      (((long long)id * p.H + h) * p.cap_len) * kDh;
         float acc[NQ][VEC];
 #pragma unroll
         for (int qi = 0; qi < NQ; ++qi)
@@ -361,7 +369,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) apply_kernel(const ApplyPar
 #pragma unroll
                 for (int u = 0; u < UNROLL; ++u) {
                     const int j = jb + u * RPW + g;
-                    vv[u] = (j < n) ? ld16_stream(Vp + (long long)(s0 + j) * kDh) : make_uint4(0, 0, 0, 0);
+                    vv[u] = (j < n) ? ld16_stream(Vp + (long long)(s0 + j) * kDh + G::chunk(c, s0 + j) * VEC) : make_uint4(0, 0, 0, 0);
                 }
 #pragma unroll
                 for (int u = 0; u < UNROLL; ++u) {

@@ -135,3 +135,19 @@ def load_memory_for(o, w, shared_context):
         for g in range(w.n_sent):
             o.mem_set(l, g, K[g, :src[g]] if l in first else None, V[g, :src[g]])
     return src
+
+
+def cached_row_order(rows_bits: np.ndarray, pos, dtype: str) -> np.ndarray:
+    """How the library stores cache rows: bf16 rows have their eight 16-byte chunks permuted,
+    logical chunk c of the row at position ``pos`` sitting at chunk ``c ^ (pos & 7)``; float32
+    rows are stored as they are.  ``rows_bits``: [..., 64] bit patterns; ``pos``: broadcastable
+    to the leading axes."""
+    if dtype != synth.BF16:
+        return rows_bits
+    x = rows_bits.reshape(rows_bits.shape[:-1] + (8, 8))
+    pos = np.broadcast_to(np.asarray(pos), rows_bits.shape[:-1])
+    phys = np.arange(8)
+    src = phys[None, :] ^ (pos.reshape(-1, 1) & 7)            # physical chunk pc holds logical pc ^ (pos & 7)
+    flat = x.reshape(-1, 8, 8)
+    out = np.take_along_axis(flat, src[:, :, None], axis=1)
+    return out.reshape(rows_bits.shape)

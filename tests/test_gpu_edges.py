@@ -9,7 +9,7 @@ from paper_1906_11024_b200 import binding as B
 from paper_1906_11024_b200 import build as san_build
 from paper_1906_11024_b200 import synth
 from paper_1906_11024_b200.driver import Decoder, to_device, to_host_f32
-from tests.helpers import TOL, normwise_err, weights_err
+from tests.helpers import TOL, cached_row_order, normwise_err, weights_err
 
 pytestmark = pytest.mark.gpu
 
@@ -35,7 +35,8 @@ def _i32(x, dev):
 @pytest.mark.parametrize("dtype", [synth.BF16, synth.F32])
 def test_cache_contents_bit_exact_after_scripted_appends(dtype):
     """The arena layout is [self K planes][self V planes][memory K][memory V], each plane
-    [id][head][row][64]; after a scripted series of appends it equals a host-side scatter."""
+    [id][head][row][64] (bf16 rows chunk-permuted by position, see cached_row_order); after a
+    scripted series of appends it equals a host-side scatter."""
     w = _small(dtype)
     dec = Decoder(w)
     dev = dec.device
@@ -56,8 +57,8 @@ def test_cache_contents_bit_exact_after_scripted_appends(dtype):
                                 _i32(ids, dev), _i32(pos, dev), None, len(ids), 1)
         assert rc == B.SAN_OK
         for i, (s, p) in enumerate(zip(ids, pos)):
-            expK[:, s, :, p, :] = bits(k_new[:, i])
-            expV[:, s, :, p, :] = bits(v_new[:, i])
+            expK[:, s, :, p, :] = cached_row_order(bits(k_new[:, i]), p, dtype)
+            expV[:, s, :, p, :] = cached_row_order(bits(v_new[:, i]), p, dtype)
     torch.cuda.synchronize()
     assert dec.device_status()[0] == 0
     raw = dec.cache.cpu().numpy()
@@ -79,11 +80,12 @@ def test_cache_contents_bit_exact_after_scripted_appends(dtype):
         Km, Vm = synth.encoder_memory(w, l)
         for g in range(w.n_sent):
             L = src[g]
-            assert np.array_equal(gotVm[l, g, :, :L], bits(Vm[g, :L]).transpose(1, 0, 2))
+            rowpos = np.arange(L)[:, None]
+            assert np.array_equal(gotVm[l, g, :, :L], cached_row_order(bits(Vm[g, :L]), rowpos, dtype).transpose(1, 0, 2))
             assert not gotVm[l, g, :, L:].any()
             if l in dec.enc_first:
                 c = dec.enc_first.index(l)
-                assert np.array_equal(gotKm[c, g, :, :L], bits(Km[g, :L]).transpose(1, 0, 2))
+                assert np.array_equal(gotKm[c, g, :, :L], cached_row_order(bits(Km[g, :L]), rowpos, dtype).transpose(1, 0, 2))
                 assert not gotKm[c, g, :, L:].any()
     dec.close()
 
