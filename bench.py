@@ -337,6 +337,18 @@ def time_oracle(w, budget_s=12.0, n_sent_sample=8, max_steps=50, exact_steps=Non
             "ms_per_step": dt / steps * 1e3, "steps": steps}
 
 
+def whole_job(secs, units_per_rank, world, dist=None, device="cpu"):
+    """Replicas only: every rank runs the same workload on its own GPU and nothing is exchanged
+    on the data path.  The job's time is the slowest rank's, its throughput the units of all
+    ranks over that time.  Returns (max seconds over ranks, units per second of the whole job)."""
+    import torch
+    t = torch.tensor([secs], dtype=torch.float64, device=device)
+    if dist is not None and world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    secs_max = float(t.item())
+    return secs_max, units_per_rank * world / secs_max
+
+
 # ---------------------------------------------------------------------------------------- main
 def config_dict(w, extra=None):
     c = {"workload": f"{w.name}: {w.n_layers} layers, d_model {w.d_model}, {w.n_heads} heads, "
@@ -423,12 +435,7 @@ def main():
     err = [d.device_status()[0] for d in decs]
     assert not any(err), f"device check failed during the timed region: {err}"
 
-    t = torch.tensor([secs], dtype=torch.float64, device=device)
-    if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)      # max over ranks; every rank ran the same workload
-    secs_max = float(t.item())
-    tokens = w.n_seqs * args.steps * world
-    value = tokens / secs_max
+    secs_max, value = whole_job(secs, w.n_seqs * args.steps, world, dist, device)
 
     if fused:      # one kernel per step: its launch duration is the step time of the timed region
         dom_s, dom_per_step, dom_bytes, dom_name = secs / args.steps, 1, float(ab["total"]), "san_decode_step (decode_step_kernel)"

@@ -447,43 +447,58 @@ int32_t san_decode_step(san_ctx* ctx, const san_step_args* a, void* stream) {
     const int ns_self = do_self ? ceil_div(max_len, span_self) : 1, ns_enc = do_enc ? ceil_div(max_src, span_enc) : 1;
     if (ns_self > kMaxSpans || ns_enc > kMaxSpans) return SAN_ERR_UNSUPPORTED;
 
+    if ((long long)ctx->n_seqs * c.n_heads * c.n_layers >= (1ll << 31)) return SAN_ERR_UNSUPPORTED;   // 32-bit row indices
+    if (rows_enc * ns_enc + rows_self * ns_self > (1ll << 30)) return SAN_ERR_UNSUPPORTED;
     StepParams p;
     std::memset(&p, 0, sizeof(p));
-    p.q_self = static_cast<const char*>(a->d_q_self); p.k_new = static_cast<const char*>(a->d_k_new);
-    p.v_new = static_cast<const char*>(a->d_v_new);
-    p.seq_ids = a->d_seq_ids; p.pos = a->d_pos; p.S_self = a->d_S_self; p.ld_t = a->ld_t;
-    p.O_self = static_cast<char*>(a->d_O_self); p.n_seqs = n_seqs; p.max_len = max_len;
-    p.q_enc = static_cast<const char*>(a->d_q_enc); p.sent_ids = a->d_sent_ids; p.src_lens = a->d_src_lens;
-    p.S_enc = a->d_S_enc; p.ld_s = a->ld_s; p.O_enc = static_cast<char*>(a->d_O_enc); p.n_sent = n_sent; p.max_src = max_src;
-    if (aan && n_seqs > 0) {
-        p.x_aan = static_cast<const char*>(a->d_x_aan); p.t_aan = a->d_t;
-        p.aan_sum = reinterpret_cast<float*>(ctx->cache + ctx->off_aan); p.n_aan_layers = c.n_layers;
-    }
-    p.H = c.n_heads; p.beam = c.beam;
-    p.cap_tgt = c.max_tgt_len; p.cap_src = c.max_src_len; p.max_seqs = ctx->n_seqs; p.max_sent = c.max_sent;
-    p.enc_v_by_block = c.encdec_shared_context ? 1 : 0;
-    p.selfK = ctx->cache + ctx->off_self_k; p.selfV = ctx->cache + ctx->off_self_v;
-    p.memK = ctx->cache + ctx->off_mem_k; p.memV = ctx->cache + ctx->off_mem_v;
-    p.self_plane_bytes = (long long)ctx->self_plane_bytes; p.mem_plane_bytes = (long long)ctx->mem_plane_bytes;
-    p.self_span = span_self; p.self_nspans = ns_self; p.enc_span = span_enc; p.enc_nspans = ns_enc;
-    if (rows_enc * ns_enc + rows_self * ns_self > (1ll << 30)) return SAN_ERR_UNSUPPORTED;
+    p.H = c.n_heads;
     p.n_enc_items = (unsigned)(rows_enc * ns_enc); p.n_items = p.n_enc_items + (unsigned)(rows_self * ns_self);
-    p.n_enc_rows = (unsigned)rows_enc;
-    p.enc_div_span = make_fastdiv((unsigned)ns_enc); p.enc_div_h = make_fastdiv((unsigned)c.n_heads);
-    p.enc_div_item = make_fastdiv((unsigned)std::max(n_sent, 1));
-    p.self_div_span = make_fastdiv((unsigned)ns_self); p.self_div_h = make_fastdiv((unsigned)c.n_heads);
-    p.self_div_item = make_fastdiv((unsigned)std::max(n_seqs, 1));
-    p.enc_part_stride = stride_enc; p.self_part_stride = stride_self;
-    p.self_part_base = ns_enc > 1 ? rows_enc * ns_enc * stride_enc : 0;
     p.part = ctx->part; p.tickets = ctx->tickets; p.err = ctx->err;
     p.scale_log2e = (float)(1.4426950408889634 / std::sqrt((double)kDh));
-    for (int b = 0; b < ctx->self_pol.n_blocks; ++b) {
-        p.self_first[b] = (unsigned char)ctx->self_pol.first_layer_of_block[b];
-        p.self_size[b] = (unsigned char)ctx->self_pol.size_of_block[b];
+    {   // decoder self-attention
+        KindParams& k = p.k[0];
+        k.q = static_cast<const char*>(a->d_q_self); k.knew = static_cast<const char*>(a->d_k_new);
+        k.vnew = static_cast<const char*>(a->d_v_new);
+        k.K = ctx->cache + ctx->off_self_k; k.V = ctx->cache + ctx->off_self_v;
+        k.S = a->d_S_self; k.O = static_cast<char*>(a->d_O_self); k.ids = a->d_seq_ids; k.lens = a->d_pos;
+        k.plane_bytes = (long long)ctx->self_plane_bytes;
+        k.layer_bytes = (long long)n_seqs * c.n_heads * row_bytes;
+        k.S_ld = a->ld_t;
+        k.part_base = ns_enc > 1 ? rows_enc * ns_enc * stride_enc : 0;
+        k.panel_bytes = (unsigned)c.max_tgt_len * row_bytes;
+        k.n_it = (unsigned)std::max(n_seqs, 1); k.nq = 1; k.len_bias = 1; k.max_ids = (unsigned)ctx->n_seqs; k.bound = (unsigned)max_len;
+        k.span = (unsigned)span_self; k.nspans = (unsigned)ns_self; k.part_stride = (unsigned)stride_self; k.v_by_block = 0;
+        k.row_base = (unsigned)rows_enc;
+        k.div_span = make_fastdiv((unsigned)ns_self); k.div_h = make_fastdiv((unsigned)c.n_heads); k.div_item = make_fastdiv(k.n_it);
+        for (int b = 0; b < ctx->self_pol.n_blocks; ++b) {
+            k.first[b] = (unsigned char)ctx->self_pol.first_layer_of_block[b];
+            k.size[b] = (unsigned char)ctx->self_pol.size_of_block[b];
+        }
     }
-    for (int b = 0; b < ctx->enc_pol.n_blocks; ++b) {
-        p.enc_first[b] = (unsigned char)ctx->enc_pol.first_layer_of_block[b];
-        p.enc_size[b] = (unsigned char)ctx->enc_pol.size_of_block[b];
+    {   // encoder-decoder attention
+        KindParams& k = p.k[1];
+        k.q = static_cast<const char*>(a->d_q_enc); k.knew = nullptr; k.vnew = nullptr;
+        k.K = ctx->cache + ctx->off_mem_k; k.V = ctx->cache + ctx->off_mem_v;
+        k.S = a->d_S_enc; k.O = static_cast<char*>(a->d_O_enc); k.ids = a->d_sent_ids; k.lens = a->d_src_lens;
+        k.plane_bytes = (long long)ctx->mem_plane_bytes;
+        k.layer_bytes = (long long)n_sent * c.beam * c.n_heads * row_bytes;
+        k.S_ld = a->ld_s;
+        k.part_base = 0;
+        k.panel_bytes = (unsigned)c.max_src_len * row_bytes;
+        k.n_it = (unsigned)std::max(n_sent, 1); k.nq = (unsigned)c.beam; k.len_bias = 0; k.max_ids = (unsigned)c.max_sent; k.bound = (unsigned)max_src;
+        k.span = (unsigned)span_enc; k.nspans = (unsigned)ns_enc; k.part_stride = (unsigned)stride_enc;
+        k.v_by_block = c.encdec_shared_context ? 1 : 0;
+        k.row_base = 0;
+        k.div_span = make_fastdiv((unsigned)ns_enc); k.div_h = make_fastdiv((unsigned)c.n_heads); k.div_item = make_fastdiv(k.n_it);
+        for (int b = 0; b < ctx->enc_pol.n_blocks; ++b) {
+            k.first[b] = (unsigned char)ctx->enc_pol.first_layer_of_block[b];
+            k.size[b] = (unsigned char)ctx->enc_pol.size_of_block[b];
+        }
+    }
+    if (aan && n_seqs > 0) {
+        p.x_aan = static_cast<const char*>(a->d_x_aan); p.t_aan = a->d_t; p.aan_ids = a->d_seq_ids;
+        p.aan_sum = reinterpret_cast<float*>(ctx->cache + ctx->off_aan); p.aan_out = static_cast<char*>(a->d_O_self);
+        p.n_aan_layers = c.n_layers; p.n_aan_seqs = n_seqs; p.aan_max_seqs = ctx->n_seqs; p.aan_max_t = c.max_tgt_len;
     }
 
     const void* fn = nullptr;

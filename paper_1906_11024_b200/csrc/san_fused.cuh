@@ -40,46 +40,45 @@ struct FastDiv {
     }
 };
 
+// Everything that differs between the two attention kinds, filled by the host.
+struct KindParams {
+    const char* q; const char* K; const char* V;      // queries; key / value plane 0 of the kind
+    const char* knew; const char* vnew;               // this step's rows (self only, else null)
+    float* S; char* O;                                 // S may be null
+    const int* ids; const int* lens;                   // lens: source lengths (enc-dec) or write positions (self)
+    long long plane_bytes;                             // between cache planes
+    long long layer_bytes;                             // between layers in O and v_new / blocks in k_new: n_it*nq*H*row bytes
+    long long S_ld;                                    // floats between S rows
+    long long part_base;                               // float offset of the kind's partial sums
+    unsigned panel_bytes;                              // capacity * row bytes: one (id, head) panel
+    unsigned n_it, nq, len_bias, max_ids, bound;       // items, query rows per item, 1 if lens holds positions, limits
+    unsigned span, nspans, part_stride, v_by_block, row_base;
+    FastDiv div_span, div_h, div_item;
+    unsigned char first[SAN_MAX_LAYERS], size[SAN_MAX_LAYERS];   // per block
+};
+
 struct StepParams {
-    // decoder self-attention
-    const char* q_self; const char* k_new; const char* v_new;   // [N_s][n][H][64], same, [M][n][H][64]
-    const int* seq_ids; const int* pos;                         // row written this step; length = pos + 1
-    float* S_self; long long ld_t; char* O_self;                // S may be null
-    int n_seqs, max_len;
-    // encoder-decoder attention
-    const char* q_enc;                                          // [N_e][n_sent][beam][H][64]
-    const int* sent_ids; const int* src_lens;
-    float* S_enc; long long ld_s; char* O_enc;
-    int n_sent, max_src;
-    // AAN in place of self-attention (absent when x_aan == null)
-    const char* x_aan; const int* t_aan; float* aan_sum; int n_aan_layers;
-    // geometry
-    int H, beam, cap_tgt, cap_src, max_seqs, max_sent, enc_v_by_block;
-    char* selfK; char* selfV; char* memK; char* memV;
-    long long self_plane_bytes, mem_plane_bytes;
-    int self_span, self_nspans, enc_span, enc_nspans;           // positions per item, spans per row at the bound
-    unsigned n_enc_items, n_items;                              // enc items come first in the list
-    unsigned n_enc_rows;
-    long long self_part_base;                                   // float offset of the self rows' partials
-    int enc_part_stride, self_part_stride;                      // floats per (row, span)
-    FastDiv enc_div_span, enc_div_h, enc_div_item, self_div_span, self_div_h, self_div_item;
+    KindParams k[2];                                   // [0] decoder self-attention, [1] encoder-decoder attention
+    unsigned n_enc_items, n_items;                     // enc-dec items come first in the list
+    int H;
     float* part; int* tickets; int* err;
     float scale_log2e;
-    unsigned char self_first[SAN_MAX_LAYERS], self_size[SAN_MAX_LAYERS];
-    unsigned char enc_first[SAN_MAX_LAYERS], enc_size[SAN_MAX_LAYERS];
+    // AAN in place of self-attention (absent when x_aan == null)
+    const char* x_aan; const int* t_aan; const int* aan_ids; float* aan_sum; char* aan_out;
+    int n_aan_layers, n_aan_seqs, aan_max_seqs, aan_max_t;
 };
 
 // A decoded work item, kept in shared memory between the copy side and the math side.
 struct ItemDesc {
-    const char* q; long long q_stride;        // query row qi at q + qi*q_stride
+    const char* q;                            // query row 0
     const char* Kp;                           // key panel, row 0
-    const char* Vp; long long v_plane;        // value panel of the block's first layer, row 0
-    const char* knew; const char* vnew; long long vnew_stride;   // newest rows (self only)
-    float* S; long long S_qstride;            // S row of query 0 (may be null)
-    char* O; long long O_lstride, O_qstride;  // output of (first layer, query 0)
+    const char* Vp;                           // value panel of the block's first layer, row 0
+    const char* knew; const char* vnew;       // newest rows (self only)
+    float* S;                                 // S row of query 0 (may be null)
+    char* O;                                  // output of (first layer, query 0)
     float* part;                              // partial sums of this (row, span)
     unsigned row_id;                          // ticket index of the row
-    int kind, nq, pi, len, j0, j1, n_spans, span, has_new, part_stride;
+    int kind, nq, pi, len, j0, j1, n_spans, span, has_new;
 };
 
 // ------------------------------------------------------------------------------ PTX helpers
@@ -100,6 +99,15 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
                  : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
+}
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {     // never blocks
+    uint32_t ok;
+    asm volatile("{\n.reg .pred p;\nmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 // Bounded wait: gives up after about a second and reports it; never spins for ever.
 __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity) {
@@ -164,192 +172,183 @@ template <> struct Pairs<float> {
     }
 };
 
-// ------------------------------------------------------------------------------ the warp
+// ------------------------------------------------------------------------------ the copy side
+// One warp per CTA feeds all the others.  Lane i serves math warp i: it takes items from
+// the CTA's sequence, decodes them (32 items decoded side by side instead of one decode
+// repeated by 32 lanes), and issues the bulk copies of their tiles into warp i's ring as
+// its stages come free.  Nothing here blocks: a lane whose ring is full just polls again.
+template <typename T>
+struct TileProducer {
+    using F = FusedGeom<T>;
+    static constexpr int ROW_BYTES = F::ROW_BYTES, TR = F::TR, QROW = TR - 8;
+
+    const StepParams& p;
+    uint32_t ring, full, empty;   // shared-space addresses of the served warp's stages and barriers
+    ItemDesc* descs;
+    unsigned* cta_next;
+    bool active, finished;
+    unsigned n_dec, stage, issued;            // items decoded, next stage, tiles issued so far
+    int which, pi, n_pos, left, has_new, nq, kind;
+    const char* src;
+    unsigned nx_item; int nx_id, nx_len; unsigned nn_item;
+
+    __device__ TileProducer(const StepParams& pp) : p(pp) {}
+
+    __device__ __forceinline__ unsigned item_of_slot(unsigned k) const {
+        const unsigned long long it = (unsigned long long)k * gridDim.x + blockIdx.x;
+        return it < p.n_items ? (unsigned)it : p.n_items;
+    }
+    __device__ __forceinline__ unsigned grab() { return item_of_slot(atomicAdd(cta_next, 1u)); }
+
+    // ---- item list: [enc-dec items][self items]; within a kind: (((block, item), head), span)
+    __device__ __forceinline__ void fetch_meta(unsigned it, int* id, int* len) const {
+        *id = 0; *len = 0;
+        if (it >= p.n_items) return;
+        const int enc = it < p.n_enc_items;
+        const KindParams& kp = p.k[enc];
+        unsigned row, span, bi, h, block, item;
+        kp.div_span.divmod(enc ? it : it - p.n_enc_items, &row, &span);
+        kp.div_h.divmod(row, &bi, &h);
+        kp.div_item.divmod(bi, &block, &item);
+        *id = kp.ids[item]; *len = kp.lens[item] + (int)kp.len_bias;
+    }
+
+    // Decodes item `it` into *d; returns false if the item is to be skipped.
+    __device__ bool decode(unsigned it, int id, int len, ItemDesc* d) const {
+        const int enc = it < p.n_enc_items;
+        const KindParams& kp = p.k[enc];
+        unsigned row, span, bi, h, block, item;
+        kp.div_span.divmod(enc ? it : it - p.n_enc_items, &row, &span);
+        kp.div_h.divmod(row, &bi, &h);
+        kp.div_item.divmod(bi, &block, &item);
+        const bool reporter = (span == 0 && h == 0 && block == 0);
+        if ((unsigned)id >= kp.max_ids) { if (reporter) record_error(p.err, TAG_STEP, (int)item, id, (int)kp.max_ids); return false; }
+        if (len < 1 || len > (int)kp.bound) { if (reporter) record_error(p.err, TAG_STEP, (int)item, len, (int)kp.bound); return false; }
+        const int j0 = (int)(span * kp.span);
+        if (j0 >= len) return false;                      // a shorter row has fewer spans
+        const unsigned H = (unsigned)p.H;
+        const int j1 = min(len, j0 + (int)kp.span);
+        const unsigned first = kp.first[block];
+        const unsigned vplane = kp.v_by_block ? block : first;
+        const unsigned qrow = ((block * kp.n_it + item) * kp.nq) * H + h;          // row of query 0 in q and S
+        const unsigned long long panel = (unsigned long long)((unsigned)id * H + h) * kp.panel_bytes;
+        d->kind = enc; d->nq = (int)kp.nq; d->pi = kp.v_by_block ? 1 : kp.size[block];
+        d->len = len; d->j0 = j0; d->j1 = j1;
+        d->n_spans = (len + (int)kp.span - 1) / (int)kp.span; d->span = (int)span;
+        d->has_new = (kp.knew != nullptr && j1 == len) ? 1 : 0;
+        d->row_id = kp.row_base + row;
+        d->part = p.part + kp.part_base + (unsigned long long)(row * kp.nspans + span) * kp.part_stride;
+        d->q = kp.q + (unsigned long long)qrow * ROW_BYTES;
+        d->S = kp.S ? kp.S + (unsigned long long)qrow * (unsigned long long)kp.S_ld : nullptr;
+        d->Kp = kp.K + (unsigned long long)block * (unsigned long long)kp.plane_bytes + panel;
+        d->Vp = kp.V + (unsigned long long)vplane * (unsigned long long)kp.plane_bytes + panel;
+        d->O = kp.O + (unsigned long long)vplane * (unsigned long long)kp.layer_bytes +
+               (unsigned long long)((item * kp.nq) * H + h) * ROW_BYTES;
+        const unsigned long long in_row = (unsigned long long)(item * H + h) * ROW_BYTES;   // self: nq == 1
+        d->knew = kp.knew ? kp.knew + (unsigned long long)block * (unsigned long long)kp.layer_bytes + in_row : nullptr;
+        d->vnew = kp.vnew ? kp.vnew + (unsigned long long)first * (unsigned long long)kp.layer_bytes + in_row : nullptr;
+        return true;
+    }
+
+    // Makes the next item that is not skipped the one being issued.
+    __device__ void next_item() {
+        active = false;
+        while (nx_item < p.n_items) {
+            ItemDesc* d = &descs[n_dec % kDescSlots];
+            const bool ok = decode(nx_item, nx_id, nx_len, d);
+            nx_item = nn_item;                         // shift the look-ahead; its metadata loads start now
+            fetch_meta(nx_item, &nx_id, &nx_len);
+            nn_item = (nx_item < p.n_items) ? grab() : nx_item;
+            if (ok) {
+                n_dec += 1; active = true;
+                which = 0; pi = d->pi; n_pos = d->j1 - d->j0; left = n_pos; has_new = d->has_new;
+                nq = d->nq; kind = d->kind;
+                src = d->Kp + (long long)d->j0 * ROW_BYTES;
+                return;
+            }
+        }
+    }
+
+    // True if the stage the next tile goes to has been handed back by the math warp.
+    __device__ __forceinline__ bool stage_free() const {
+        if (issued < (unsigned)kFusedStages) return true;
+        return mbar_test_wait(empty + stage * 8, ((issued / kFusedStages) - 1) & 1);
+    }
+
+    // Issues one tile (or, when the items have run out, the end marker).  Call only when stage_free().
+    __device__ void issue() {
+        const uint32_t dst = ring + stage * kStageBytes;
+        const uint32_t bar = full + stage * 8;
+        if (!active) {      // no more items: an item slot with kind < 0 and an empty tile tell the math warp to stop
+            descs[n_dec % kDescSlots].kind = -1;
+            mbar_arrive(bar);
+            finished = true;
+        } else {
+            const ItemDesc& d = descs[(n_dec - 1) % kDescSlots];
+            const bool first = (which == 0 && left == n_pos);
+            const int r = min(first ? QROW : TR, left);
+            const bool with_new = has_new && (r == left);
+            const int r_cache = with_new ? r - 1 : r;
+            mbar_expect_tx(bar, (uint32_t)((r + (first ? nq : 0)) * ROW_BYTES));
+            if (r_cache > 0) bulk_g2s(dst, src, (uint32_t)(r_cache * ROW_BYTES), bar);
+            if (with_new) {     // this step's row of the panel: keys, or values of layer which - 1
+                const char* nsrc = which == 0 ? d.knew : d.vnew + (long long)(which - 1) * p.k[kind].layer_bytes;
+                bulk_g2s(dst + r_cache * ROW_BYTES, nsrc, ROW_BYTES, bar);
+            }
+            if (first) {        // the query rows ride behind the first key tile
+                const unsigned q_stride = (unsigned)p.H * ROW_BYTES;
+                for (int qi = 0; qi < nq; ++qi) bulk_g2s(dst + (QROW + qi) * ROW_BYTES, d.q + (size_t)qi * q_stride, ROW_BYTES, bar);
+            }
+            left -= r;
+            src += (long long)r * ROW_BYTES;
+            if (left <= 0) {
+                if (which == pi) next_item();
+                else {          // on to the value panel of layer `which`
+                    src = d.Vp + (long long)which * p.k[kind].plane_bytes + (long long)d.j0 * ROW_BYTES;
+                    which += 1;
+                    left = n_pos;
+                }
+            }
+        }
+        stage = (stage + 1 == (unsigned)kFusedStages) ? 0 : stage + 1;
+        issued += 1;
+    }
+};
+
+// ------------------------------------------------------------------------------ the math side
 template <typename T>
 struct FusedWarp {
     using G = RowGeom<T>;
     using F = FusedGeom<T>;
     using P = Pairs<T>;
     static constexpr int VEC = G::VEC, LPR = G::LPR, RPW = 32 / LPR, ROW_BYTES = F::ROW_BYTES, TR = F::TR;
+    static constexpr int QROW = TR - 8;      // the first key tile of an item holds key rows [0, QROW) and the
+                                             // query rows from row QROW on (at most 8 of them)
     static constexpr int NP = P::N;          // float pairs per 16 bytes
     static constexpr int BLK = 8;            // rows per inner block
     static constexpr int UN = BLK / RPW;     // loads per lane per block
 
     const StepParams& p;
-    uint32_t ring, bars;   // shared-space addresses: stages and their barriers
-    const char* ring_g;    // the same stages through a generic pointer
-    float* zs;             // kZFloats floats
-    ItemDesc* descs;       // kDescSlots
-    unsigned* cta_next;    // shared counter: next slot of this CTA's item sequence to hand out
+    uint32_t ring, full, empty;   // shared-space addresses: stages and their barriers
+    const char* ring_g;           // the same stages through a generic pointer
+    float* zs;                    // kZFloats floats
     int lane, g, c;
-    // copy side: the item being issued, the next one (metadata on its way), the one after
-    bool p_active;
-    unsigned p_seq, p_n;
-    int p_which, p_s0, p_j0, p_j1, p_pi, p_q_done;
-    const char* p_panel;
-    unsigned nx_item; int nx_id, nx_len;      // next item and its prefetched id / length
-    unsigned nn_item;                         // the item after that
-    // math side
-    unsigned c_seq, c_n;
-    bool dead;             // a wait ran out: stop issuing, drain, leave
+    unsigned c_stage, c_par;
+    bool dead;                    // a wait ran out: leave
 
     __device__ FusedWarp(const StepParams& pp) : p(pp) {}
 
-    __device__ __forceinline__ unsigned item_of_slot(unsigned k) const {
-        const unsigned long long it = (unsigned long long)k * gridDim.x + blockIdx.x;
-        return it < p.n_items ? (unsigned)it : p.n_items;
-    }
-    __device__ __forceinline__ unsigned grab() {
-        unsigned k = 0;
-        if (lane == 0) k = atomicAdd(cta_next, 1u);
-        return item_of_slot(__shfl_sync(0xffffffffu, k, 0));
-    }
-
-    // ---- item list: [enc items][self items]; within a kind: (((block, item), head), span)
-    __device__ __forceinline__ void split(unsigned it, bool* enc, unsigned* block, unsigned* item, unsigned* h, unsigned* span,
-                                          unsigned* row) const {
-        *enc = it < p.n_enc_items;
-        unsigned bi;
-        if (*enc) {
-            p.enc_div_span.divmod(it, row, span);
-            p.enc_div_h.divmod(*row, &bi, h);
-            p.enc_div_item.divmod(bi, block, item);
-        } else {
-            p.self_div_span.divmod(it - p.n_enc_items, row, span);
-            p.self_div_h.divmod(*row, &bi, h);
-            p.self_div_item.divmod(bi, block, item);
-        }
-    }
-    __device__ __forceinline__ void fetch_meta(unsigned it, int* id, int* len) const {
-        *id = 0; *len = 0;
-        if (it >= p.n_items) return;
-        bool enc; unsigned block, item, h, span, row;
-        split(it, &enc, &block, &item, &h, &span, &row);
-        if (enc) { *id = p.sent_ids[item]; *len = p.src_lens[item]; }
-        else { *id = p.seq_ids[item]; *len = p.pos[item] + 1; }
-    }
-
-    // Decodes item `it` into *d (lane 0 writes it); returns false if the item is to be skipped.
-    __device__ bool decode(unsigned it, int id, int len, ItemDesc* d) const {
-        bool enc; unsigned block, item, h, span, row;
-        split(it, &enc, &block, &item, &h, &span, &row);
-        const int span_len = enc ? p.enc_span : p.self_span;
-        const int max_ids = enc ? p.max_sent : p.max_seqs;
-        const int bound = enc ? p.max_src : p.max_len;
-        const bool reporter = (lane == 0 && span == 0 && h == 0 && block == 0);
-        if (id < 0 || id >= max_ids) { if (reporter) record_error(p.err, TAG_STEP, (int)item, id, max_ids); return false; }
-        if (len < 1 || len > bound) { if (reporter) record_error(p.err, TAG_STEP, (int)item, len, bound); return false; }
-        const int j0 = (int)span * span_len;
-        if (j0 >= len) return false;                      // a shorter row has fewer spans
-        if (lane != 0) return true;
-        const int j1 = min(len, j0 + span_len);
-        const int nq = enc ? p.beam : 1;
-        const int first = enc ? p.enc_first[block] : p.self_first[block];
-        const int pi = enc ? (p.enc_v_by_block ? 1 : p.enc_size[block]) : p.self_size[block];
-        const int cap = enc ? p.cap_src : p.cap_tgt;
-        const long long plane = enc ? p.mem_plane_bytes : p.self_plane_bytes;
-        const long long panel = (((long long)id * p.H + h) * cap) * ROW_BYTES;
-        const int nspans_max = enc ? p.enc_nspans : p.self_nspans;
-        d->kind = enc ? 1 : 0; d->nq = nq; d->pi = pi; d->len = len; d->j0 = j0; d->j1 = j1;
-        d->n_spans = (len + span_len - 1) / span_len; d->span = (int)span;
-        d->has_new = (!enc && j1 == len) ? 1 : 0;
-        d->row_id = enc ? row : p.n_enc_rows + row;
-        d->part_stride = enc ? p.enc_part_stride : p.self_part_stride;
-        d->part = p.part + (enc ? 0 : p.self_part_base) + ((long long)row * nspans_max + span) * (long long)d->part_stride;
-        d->v_plane = plane;
-        if (enc) {
-            d->q = p.q_enc + ((((long long)block * p.n_sent + item) * nq) * p.H + h) * ROW_BYTES;
-            d->q_stride = (long long)p.H * ROW_BYTES;
-            d->Kp = p.memK + block * plane + panel;
-            d->Vp = p.memV + (p.enc_v_by_block ? (int)block : first) * plane + panel;
-            d->knew = nullptr; d->vnew = nullptr; d->vnew_stride = 0;
-            d->S = p.S_enc ? p.S_enc + ((((long long)block * p.n_sent + item) * nq) * p.H + h) * p.ld_s : nullptr;
-            d->S_qstride = (long long)p.H * p.ld_s;
-            const int o_first = p.enc_v_by_block ? (int)block : first;
-            d->O = p.O_enc + ((((long long)o_first * p.n_sent + item) * nq) * p.H + h) * ROW_BYTES;
-            d->O_lstride = (long long)p.n_sent * nq * p.H * ROW_BYTES;
-            d->O_qstride = (long long)p.H * ROW_BYTES;
-        } else {
-            const long long in_row = ((long long)item * p.H + h) * ROW_BYTES;
-            const long long in_layer = (long long)p.n_seqs * p.H * ROW_BYTES;
-            d->q = p.q_self + block * in_layer + in_row; d->q_stride = 0;
-            d->Kp = p.selfK + block * plane + panel;
-            d->Vp = p.selfV + first * plane + panel;
-            d->knew = p.k_new + block * in_layer + in_row;
-            d->vnew = p.v_new + first * in_layer + in_row; d->vnew_stride = in_layer;
-            d->S = p.S_self ? p.S_self + (((long long)block * p.n_seqs + item) * p.H + h) * p.ld_t : nullptr;
-            d->S_qstride = 0;
-            d->O = p.O_self + first * in_layer + in_row;
-            d->O_lstride = in_layer; d->O_qstride = 0;
-        }
-        return true;
-    }
-
-    // Makes the next item that is not skipped the one being issued.
-    __device__ void next_item() {
-        p_active = false;
-        while (nx_item < p.n_items) {
-            ItemDesc* d = &descs[p_n % kDescSlots];
-            const bool ok = decode(nx_item, nx_id, nx_len, d);
-            // shift the look-ahead: the item after becomes next (its metadata loads start now)
-            nx_item = nn_item;
-            fetch_meta(nx_item, &nx_id, &nx_len);
-            nn_item = (nx_item < p.n_items) ? grab() : nx_item;
-            if (ok) {
-                __syncwarp();
-                p_n += 1; p_active = true;
-                p_q_done = 0; p_which = 0; p_j0 = d->j0; p_j1 = d->j1; p_pi = d->pi; p_s0 = p_j0;
-                p_panel = d->Kp;
-                return;
-            }
-        }
-    }
-
-    // Issues the copies of one tile of the item being issued, if any is left.
-    __device__ void produce() {
-        if (dead || !p_active) return;
-        const ItemDesc& d = descs[(p_n - 1) % kDescSlots];
-        const unsigned s = p_seq % kFusedStages;
-        if (lane == 0) {
-            const uint32_t dst = ring + s * kStageBytes;
-            const uint32_t bar = bars + s * 8;
-            if (!p_q_done) {
-                mbar_expect_tx(bar, (uint32_t)(d.nq * ROW_BYTES));
-                for (int qi = 0; qi < d.nq; ++qi) bulk_g2s(dst + qi * ROW_BYTES, d.q + qi * d.q_stride, ROW_BYTES, bar);
-            } else {
-                const int r = min(TR, p_j1 - p_s0);
-                const bool with_new = d.has_new && (p_s0 + r == p_j1);
-                const int r_cache = with_new ? r - 1 : r;
-                mbar_expect_tx(bar, (uint32_t)(r * ROW_BYTES));
-                if (r_cache > 0) bulk_g2s(dst, p_panel + (long long)p_s0 * ROW_BYTES, (uint32_t)(r_cache * ROW_BYTES), bar);
-                if (with_new) {
-                    const char* nsrc = p_which == 0 ? d.knew : d.vnew + (long long)(p_which - 1) * d.vnew_stride;
-                    bulk_g2s(dst + r_cache * ROW_BYTES, nsrc, ROW_BYTES, bar);
-                }
-            }
-        }
-        p_seq += 1;
-        if (!p_q_done) { p_q_done = 1; return; }
-        p_s0 += TR;
-        if (p_s0 >= p_j1) {
-            p_which += 1; p_s0 = p_j0;
-            if (p_which > p_pi) { next_item(); return; }
-            p_panel = d.Vp + (long long)(p_which - 1) * d.v_plane;
-        }
-    }
-
     // Waits for the next tile in order; returns its stage or null after a timeout.
     __device__ __forceinline__ const char* acquire() {
-        const unsigned s = c_seq % kFusedStages;
-        const uint32_t bar = bars + s * 8, par = (c_seq / kFusedStages) & 1;
-        if (!mbar_try_wait(bar, par)) {
-            if (!mbar_wait_slow(bar, par)) {
-                if (lane == 0 && atomicCAS(&p.err[0], 0, (int)SAN_ERR_TIMEOUT) == 0) { p.err[1] = TAG_STEP; p.err[2] = (int)c_seq; }
+        const uint32_t bar = full + c_stage * 8;
+        if (!mbar_try_wait(bar, c_par)) {
+            if (!mbar_wait_slow(bar, c_par)) {
+                if (lane == 0 && atomicCAS(&p.err[0], 0, (int)SAN_ERR_TIMEOUT) == 0) { p.err[1] = TAG_STEP; p.err[2] = (int)c_stage; }
                 dead = true;
                 return nullptr;
             }
         }
-        return ring_g + s * kStageBytes;
+        return ring_g + c_stage * kStageBytes;
     }
     // Every lane is done with the tile: hand the stage back to the copy side.
     __device__ __forceinline__ void release() {
@@ -357,13 +356,14 @@ struct FusedWarp {
         // ragged tail): order those writes ahead of the bulk copy that will reuse the stage
         if (sizeof(T) == 2) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncwarp();
-        c_seq += 1;
-        produce();
+        if (lane == 0) mbar_arrive(empty + c_stage * 8);
+        if (++c_stage == (unsigned)kFusedStages) { c_stage = 0; c_par ^= 1u; }
     }
 
     template <int NQ> __device__ bool process(const ItemDesc& d);
     template <int NQ> __device__ bool process_mma(const ItemDesc& d);
     template <int NQ> __device__ void combine(const ItemDesc& d);
+    template <int NQ> __device__ __forceinline__ void softmax_span(const ItemDesc& d, int n, int n_pad, float* part_m, float* part_l);
 
     // bf16 tiles only.  A tile's last row may be this step's new row, copied in natural chunk
     // order from the caller's buffer: permute its chunks like a cached row (chunk c -> c ^ (pos & 7))
@@ -386,54 +386,90 @@ struct FusedWarp {
             for (int j = r + (lane >> 3); j < r16; j += 4)
                 *reinterpret_cast<uint4*>(const_cast<char*>(st) + j * 128 + (lane & 7) * 16) = make_uint4(0, 0, 0, 0);
         }
-        __syncwarp();
-    }
-
-    // After a timeout: copies already issued may still land in this warp's stages, so give
-    // each a last bounded chance to finish before the CTA's shared memory can go away.
-    __device__ void drain() {
-        while (c_seq != p_seq) {
-            const unsigned s = c_seq % kFusedStages;
-            const uint32_t par = (c_seq / kFusedStages) & 1;
-            const long long t0 = clock64();
-            while (!mbar_try_wait(bars + s * 8, par)) { if (clock64() - t0 > 200000000LL) break; }
-            c_seq += 1;
-        }
+        if (with_new || (zero_tail && (r & 15))) __syncwarp();
     }
 };
 
+// Softmax of the n scores of a span held in zs (log2 domain), per query row.  A span that is
+// the whole row leaves normalised weights in zs and writes them to S; otherwise it leaves
+// exp2(z - max) and reports (max, sum) for the combine.  zs[n .. n_pad) is zeroed.
+template <typename T>
+template <int NQ>
+__device__ __forceinline__ void FusedWarp<T>::softmax_span(const ItemDesc& d, int n, int n_pad, float* part_m, float* part_l) {
+    constexpr int ZQ = kZFloats / NQ;
+    const int nq = d.nq, n_spans = d.n_spans;
+    const long long S_qstride = (long long)p.H * p.k[d.kind].S_ld;
+#pragma unroll
+    for (int qi = 0; qi < NQ; ++qi) {
+        part_m[qi] = 0.f; part_l[qi] = 1.f;
+        float* zq = zs + qi * ZQ;
+        if (qi < nq) {
+            float* Srow = d.S ? d.S + qi * S_qstride + d.j0 : nullptr;
+            if (n <= 32) {      // one score per lane: no loops
+                const float z = lane < n ? zq[lane] : -INFINITY;
+                const float m = warp_max(z);
+                const float e = lane < n ? exp2f(z - m) : 0.f;
+                const float s = warp_sum(e);
+                part_m[qi] = m; part_l[qi] = s;
+                const float w = (n_spans == 1) ? e * (1.0f / s) : e;
+                if (lane < n_pad) zq[lane] = w;
+                if (Srow && lane < n) Srow[lane] = w;
+            } else {
+                float m = -INFINITY;
+                for (int jj = lane; jj < n; jj += 32) m = fmaxf(m, zq[jj]);
+                m = warp_max(m);
+                float s = 0.f;
+                for (int jj = lane; jj < n; jj += 32) { const float e = exp2f(zq[jj] - m); zq[jj] = e; s += e; }
+                s = warp_sum(s);
+                part_m[qi] = m; part_l[qi] = s;
+                if (n_spans == 1) {
+                    const float inv = 1.0f / s;
+                    for (int jj = lane; jj < n; jj += 32) {
+                        const float w = zq[jj] * inv;
+                        zq[jj] = w;
+                        if (Srow) Srow[jj] = w;
+                    }
+                } else if (Srow) {
+                    for (int jj = lane; jj < n; jj += 32) Srow[jj] = zq[jj];
+                }
+                for (int jj = n + lane; jj < n_pad; jj += 32) zq[jj] = 0.f;
+            }
+        } else {
+            for (int jj = lane; jj < n_pad; jj += 32) zq[jj] = 0.f;     // absent query rows weigh nothing
+        }
+    }
+    __syncwarp();
+}
+
+// float32 items: packed two-wide FMAs on the CUDA cores (rows in natural chunk order).
 template <typename T>
 template <int NQ>
 __device__ bool FusedWarp<T>::process(const ItemDesc& d) {
     constexpr int ZQ = kZFloats / NQ;          // score slots per query row
     constexpr int HDR = (2 * NQ + 3) / 4 * 4;  // (max, sum) per query ahead of a span's partial sums
-    const int j0 = d.j0, n = d.j1 - d.j0, nq = d.nq, has_new = d.has_new, pi = d.pi;
+    const KindParams& kp = p.k[d.kind];
+    const int n = d.j1 - d.j0, nq = d.nq, has_new = d.has_new, pi = d.pi;
 
-    // ---- tile 0: the query rows, scaled into the log2 domain
+    // ---- key tiles: scores into zs.  The first tile also carries the query rows.
     float2 q2[NQ][NP];
-    {
+    for (int s0 = 0; s0 < n;) {
         const char* st = acquire();
         if (!st) return false;
-        const float sc = p.scale_log2e;
+        const int r = min(s0 == 0 ? QROW : TR, n - s0);
+        if (s0 == 0) {
+            const float sc = p.scale_log2e;
 #pragma unroll
-        for (int qi = 0; qi < NQ; ++qi) {
-            if (qi < nq) {
-                P::load(*reinterpret_cast<const uint4*>(st + qi * ROW_BYTES + c * 16), q2[qi]);
+            for (int qi = 0; qi < NQ; ++qi) {
+                if (qi < nq) {
+                    P::load(*reinterpret_cast<const uint4*>(st + (QROW + qi) * ROW_BYTES + c * 16), q2[qi]);
 #pragma unroll
-                for (int e = 0; e < NP; ++e) { q2[qi][e].x *= sc; q2[qi][e].y *= sc; }
-            } else {
+                    for (int e = 0; e < NP; ++e) { q2[qi][e].x *= sc; q2[qi][e].y *= sc; }
+                } else {
 #pragma unroll
-                for (int e = 0; e < NP; ++e) q2[qi][e] = make_float2(0.f, 0.f);
+                    for (int e = 0; e < NP; ++e) q2[qi][e] = make_float2(0.f, 0.f);
+                }
             }
         }
-        release();
-    }
-
-    // ---- key tiles: scores into zs
-    for (int s0 = 0; s0 < n; s0 += TR) {
-        const char* st = acquire();
-        if (!st) return false;
-        const int r = min(TR, n - s0);
         const bool with_new = has_new && (s0 + r == n);
         for (int jb = 0; jb < r; jb += BLK) {
             uint4 kv[UN];
@@ -462,39 +498,17 @@ __device__ bool FusedWarp<T>::process(const ItemDesc& d) {
                     *reinterpret_cast<uint4*>(const_cast<char*>(d.Kp) + (long long)(d.len - 1) * ROW_BYTES + c * 16) = kv[u];
             }
         }
+        s0 += r;
         release();
-    }
-
-    // ---- softmax over the span (log2 domain)
-    float part_m[NQ], part_l[NQ];
-    const int n_spans = d.n_spans;
-#pragma unroll
-    for (int qi = 0; qi < NQ; ++qi) {
-        part_m[qi] = 0.f; part_l[qi] = 1.f;
-        if (qi < nq) {
-            float m = -INFINITY;
-            for (int jj = lane; jj < n; jj += 32) m = fmaxf(m, zs[qi * ZQ + jj]);
-            m = warp_max(m);
-            float s = 0.f;
-            for (int jj = lane; jj < n; jj += 32) { const float e = exp2f(zs[qi * ZQ + jj] - m); zs[qi * ZQ + jj] = e; s += e; }
-            s = warp_sum(s);
-            part_m[qi] = m; part_l[qi] = s;
-            float* Srow = d.S ? d.S + qi * d.S_qstride + j0 : nullptr;
-            if (n_spans == 1) {
-                const float inv = 1.0f / s;
-                for (int jj = lane; jj < n; jj += 32) {
-                    const float w = zs[qi * ZQ + jj] * inv;
-                    zs[qi * ZQ + jj] = w;
-                    if (Srow) Srow[jj] = w;
-                }
-            } else if (Srow) {
-                for (int jj = lane; jj < n; jj += 32) Srow[jj] = zs[qi * ZQ + jj];
-            }
-        }
     }
     __syncwarp();
 
+    float part_m[NQ], part_l[NQ];
+    const int n_spans = d.n_spans;
+    softmax_span<NQ>(d, n, n, part_m, part_l);
+
     // ---- value tiles, layer by layer (score rows of absent queries hold zeros)
+    const long long O_qstride = (long long)p.H * ROW_BYTES;
     for (int l = 0; l < pi; ++l) {
         float2 acc[NQ][NP];
 #pragma unroll
@@ -527,7 +541,7 @@ __device__ bool FusedWarp<T>::process(const ItemDesc& d) {
                             for (int e = 0; e < NP; ++e) acc[qi][e] = __ffma2_rn(ss, v2[e], acc[qi][e]);
                         }
                         if (with_new && j == r - 1)
-                            *reinterpret_cast<uint4*>(const_cast<char*>(d.Vp) + (long long)l * d.v_plane +
+                            *reinterpret_cast<uint4*>(const_cast<char*>(d.Vp) + (long long)l * kp.plane_bytes +
                                                       (long long)(d.len - 1) * ROW_BYTES + c * 16) = vv[u];
                     }
                 }
@@ -548,7 +562,7 @@ __device__ bool FusedWarp<T>::process(const ItemDesc& d) {
             for (int qi = 0; qi < NQ; ++qi) {
                 if (qi < nq) {
                     if (n_spans == 1) {
-                        *reinterpret_cast<uint4*>(d.O + l * d.O_lstride + qi * d.O_qstride + c * 16) = P::store(acc[qi]);
+                        *reinterpret_cast<uint4*>(d.O + l * kp.layer_bytes + qi * O_qstride + c * 16) = P::store(acc[qi]);
                     } else {
                         float2* pp = reinterpret_cast<float2*>(d.part + HDR + ((long long)l * NQ + qi) * kDh + c * VEC);
 #pragma unroll
@@ -589,33 +603,30 @@ __device__ bool FusedWarp<T>::process_mma(const ItemDesc& d) {
     static_assert(sizeof(T) == 2, "tensor-core path is for bf16 rows");
     constexpr int ZQ = kZFloats / NQ;
     constexpr int HDR = (2 * NQ + 3) / 4 * 4;
-    const int j0 = d.j0, n = d.j1 - d.j0, nq = d.nq, has_new = d.has_new, pi = d.pi;
+    const KindParams& kp = p.k[d.kind];
+    const int n = d.j1 - d.j0, nq = d.nq, has_new = d.has_new, pi = d.pi;
     const int tig = lane & 3, gid = lane >> 2;                 // mma fragment coordinates
     const int lrow = (lane & 7) + ((lane >> 3) & 1) * 8;        // ldmatrix: row of the 16-row block this lane addresses
     const int lx = lane & 7, lsel = lane >> 4;                  // its chunk permutation key and chunk of the pair
 
-    // ---- tile 0: the query rows as B fragments (k = dims, n = query), natural chunk order
+    // ---- key tiles: scores into zs (log2 domain).  The first tile also carries the query rows
+    // (natural chunk order), read as B fragments (k = dims, n = query).
     uint32_t qb[4][2];
-    {
+    const float sc = p.scale_log2e;
+    for (int s0 = 0; s0 < n;) {
         const char* st = acquire();
         if (!st) return false;
+        const int r = min(s0 == 0 ? QROW : TR, n - s0);
+        if (s0 == 0) {
 #pragma unroll
-        for (int ks = 0; ks < 4; ++ks) {
-            qb[ks][0] = 0u; qb[ks][1] = 0u;
-            if (gid < nq) {
-                qb[ks][0] = *reinterpret_cast<const uint32_t*>(st + gid * 128 + (16 * ks + 2 * tig) * 2);
-                qb[ks][1] = *reinterpret_cast<const uint32_t*>(st + gid * 128 + (16 * ks + 8 + 2 * tig) * 2);
+            for (int ks = 0; ks < 4; ++ks) {
+                qb[ks][0] = 0u; qb[ks][1] = 0u;
+                if (gid < nq) {
+                    qb[ks][0] = *reinterpret_cast<const uint32_t*>(st + (QROW + gid) * 128 + (16 * ks + 2 * tig) * 2);
+                    qb[ks][1] = *reinterpret_cast<const uint32_t*>(st + (QROW + gid) * 128 + (16 * ks + 8 + 2 * tig) * 2);
+                }
             }
         }
-        release();
-    }
-
-    // ---- key tiles: scores into zs (log2 domain)
-    const float sc = p.scale_log2e;
-    for (int s0 = 0; s0 < n; s0 += TR) {
-        const char* st = acquire();
-        if (!st) return false;
-        const int r = min(TR, n - s0);
         fix_tile(st, r, has_new && (s0 + r == n), const_cast<char*>(d.Kp) + (long long)(d.len - 1) * 128, false);
         const uint32_t st_s = ring + (uint32_t)(st - ring_g);
         for (int b0 = 0; b0 < r; b0 += 16) {
@@ -637,43 +648,17 @@ __device__ bool FusedWarp<T>::process_mma(const ItemDesc& d) {
                 if (p1 < r) zs[(2 * tig + 1) * ZQ + s0 + p1] = acc[3] * sc;
             }
         }
+        s0 += r;
         release();
     }
     __syncwarp();
 
-    // ---- softmax over the span (log2 domain)
     float part_m[NQ], part_l[NQ];
     const int n_spans = d.n_spans;
-    const int n16 = (n + 15) & ~15;
-#pragma unroll
-    for (int qi = 0; qi < NQ; ++qi) {
-        part_m[qi] = 0.f; part_l[qi] = 1.f;
-        if (qi < nq) {
-            float m = -INFINITY;
-            for (int jj = lane; jj < n; jj += 32) m = fmaxf(m, zs[qi * ZQ + jj]);
-            m = warp_max(m);
-            float s = 0.f;
-            for (int jj = lane; jj < n; jj += 32) { const float e = exp2f(zs[qi * ZQ + jj] - m); zs[qi * ZQ + jj] = e; s += e; }
-            s = warp_sum(s);
-            part_m[qi] = m; part_l[qi] = s;
-            float* Srow = d.S ? d.S + qi * d.S_qstride + j0 : nullptr;
-            if (n_spans == 1) {
-                const float inv = 1.0f / s;
-                for (int jj = lane; jj < n; jj += 32) {
-                    const float w = zs[qi * ZQ + jj] * inv;
-                    zs[qi * ZQ + jj] = w;
-                    if (Srow) Srow[jj] = w;
-                }
-            } else if (Srow) {
-                for (int jj = lane; jj < n; jj += 32) Srow[jj] = zs[qi * ZQ + jj];
-            }
-        }
-        // weights beyond the span's end (up to the next multiple of 16) must be exactly zero
-        for (int jj = n + lane; jj < n16; jj += 32) zs[qi * ZQ + jj] = 0.f;
-    }
-    __syncwarp();
+    softmax_span<NQ>(d, n, (n + 15) & ~15, part_m, part_l);   // weights up to the next multiple of 16 are exact zeros
 
     // ---- value tiles, layer by layer
+    const long long O_qstride = (long long)p.H * 128;
     for (int l = 0; l < pi; ++l) {
         float acc[8][4];
 #pragma unroll
@@ -685,7 +670,7 @@ __device__ bool FusedWarp<T>::process_mma(const ItemDesc& d) {
             if (!st) return false;
             const int r = min(TR, n - s0);
             fix_tile(st, r, has_new && (s0 + r == n),
-                     const_cast<char*>(d.Vp) + (long long)l * d.v_plane + (long long)(d.len - 1) * 128, true);
+                     const_cast<char*>(d.Vp) + (long long)l * kp.plane_bytes + (long long)(d.len - 1) * 128, true);
             const uint32_t st_s = ring + (uint32_t)(st - ring_g);
             for (int b0 = 0; b0 < r; b0 += 16) {
                 // A = weights of query gid at positions b0 + {2tig, 2tig+1, 2tig+8, 2tig+9}: high part + remainder
@@ -712,7 +697,7 @@ __device__ bool FusedWarp<T>::process_mma(const ItemDesc& d) {
         // acc[nt][0], acc[nt][1]: query gid, dims 8nt + 2tig, +1
         if (gid < nq) {
             if (n_spans == 1) {
-                char* op = d.O + l * d.O_lstride + gid * d.O_qstride + 4 * tig;
+                char* op = d.O + l * kp.layer_bytes + gid * O_qstride + 4 * tig;
 #pragma unroll
                 for (int nt = 0; nt < 8; ++nt) *reinterpret_cast<uint32_t*>(op + 16 * nt) = pack_bf16x2(acc[nt][0], acc[nt][1]);
             } else {
@@ -743,9 +728,11 @@ template <int NQ>
 __device__ void FusedWarp<T>::combine(const ItemDesc& d) {
     constexpr int HDR = (2 * NQ + 3) / 4 * 4;
     __threadfence();
-    const int n_spans = d.n_spans, nq = d.nq, stride = d.part_stride;
+    const KindParams& kp = p.k[d.kind];
+    const int n_spans = d.n_spans, nq = d.nq, stride = (int)kp.part_stride;
     const float* row_part = d.part - (long long)d.span * stride;
-    const int span_len = d.kind ? p.enc_span : p.self_span;
+    const int span_len = (int)kp.span;
+    const long long S_qstride = (long long)p.H * kp.S_ld, O_qstride = (long long)p.H * ROW_BYTES;
     // zs[sp * NQ + qi] = exp2(m_sp - M) / total  (zs is free: every layer of this span is done)
     __syncwarp();
     for (int qi = 0; qi < NQ; ++qi) {
@@ -759,7 +746,7 @@ __device__ void FusedWarp<T>::combine(const ItemDesc& d) {
     __syncwarp();
     if (d.S) {
         for (int qi = 0; qi < nq; ++qi) {
-            float* Srow = d.S + qi * d.S_qstride;
+            float* Srow = d.S + qi * S_qstride;
             for (int j = lane; j < d.len; j += 32) Srow[j] = __ldcg(Srow + j) * zs[(j / span_len) * NQ + qi];
         }
     }
@@ -787,7 +774,7 @@ __device__ void FusedWarp<T>::combine(const ItemDesc& d) {
             a.x = fmaf(f, x.x, a.x); a.y = fmaf(f, x.y, a.y); a.z = fmaf(f, x.z, a.z); a.w = fmaf(f, x.w, a.w);
         }
         const int ly = e0 / (NQ * kDh), col = e0 % kDh;
-        char* op = d.O + ly * d.O_lstride + qi * d.O_qstride + col * (int)sizeof(T);
+        char* op = d.O + ly * kp.layer_bytes + qi * O_qstride + col * (int)sizeof(T);
         if (sizeof(T) == 2) {
             __nv_bfloat162 lo = __floats2bfloat162_rn(a.x, a.y), hi = __floats2bfloat162_rn(a.z, a.w);
             uint2 r; r.x = *reinterpret_cast<uint32_t*>(&lo); r.y = *reinterpret_cast<uint32_t*>(&hi);
@@ -799,9 +786,10 @@ __device__ void FusedWarp<T>::combine(const ItemDesc& d) {
     if (lane == 0) p.tickets[d.row_id] = 0;
 }
 
+constexpr int kMathWarps = kFusedWarps - 1;     // the last warp of the CTA is the copy warp
 constexpr size_t fused_smem_bytes() {
-    return (size_t)kFusedWarps * (kFusedStages * kStageBytes + kZFloats * sizeof(float) + kDescSlots * sizeof(ItemDesc) +
-                                  kFusedStages * sizeof(uint64_t)) + 128;
+    return (size_t)kMathWarps * (kFusedStages * kStageBytes + kZFloats * sizeof(float) + kDescSlots * sizeof(ItemDesc) +
+                                 2 * kFusedStages * sizeof(uint64_t)) + 128;
 }
 
 template <typename T, int NQE>
@@ -813,15 +801,15 @@ __global__ void __launch_bounds__(kFusedWarps * 32, 1) decode_step_kernel(const 
     // ---- AAN running average (Table 6 pairing): element-wise, every thread of the grid
     if (p.x_aan) {
         const int d = p.H * kDh, d4 = d >> 2;
-        const long long total = (long long)p.n_aan_layers * p.n_seqs * d4;
+        const long long total = (long long)p.n_aan_layers * p.n_aan_seqs * d4;
         for (long long u = (long long)blockIdx.x * blockDim.x + threadIdx.x; u < total; u += (long long)gridDim.x * blockDim.x) {
             const int c4 = (int)(u % d4);
-            const int item = (int)((u / d4) % p.n_seqs);
-            const int lr = (int)(u / ((long long)d4 * p.n_seqs));
-            const int id = p.seq_ids[item], t = p.t_aan[item];
-            if (id < 0 || id >= p.max_seqs) { if (c4 == 0 && lr == 0) record_error(p.err, TAG_AAN, item, id, p.max_seqs); continue; }
-            if (t < 1 || t > p.cap_tgt) { if (c4 == 0 && lr == 0) record_error(p.err, TAG_AAN, item, t, p.cap_tgt); continue; }
-            const long long io = ((long long)lr * p.n_seqs + item) * d + c4 * 4;
+            const int item = (int)((u / d4) % p.n_aan_seqs);
+            const int lr = (int)(u / ((long long)d4 * p.n_aan_seqs));
+            const int id = p.aan_ids[item], t = p.t_aan[item];
+            if (id < 0 || id >= p.aan_max_seqs) { if (c4 == 0 && lr == 0) record_error(p.err, TAG_AAN, item, id, p.aan_max_seqs); continue; }
+            if (t < 1 || t > p.aan_max_t) { if (c4 == 0 && lr == 0) record_error(p.err, TAG_AAN, item, t, p.aan_max_t); continue; }
+            const long long io = ((long long)lr * p.n_aan_seqs + item) * d + c4 * 4;
             float xv[4];
             if (sizeof(T) == 2) {
                 const uint2 raw = *reinterpret_cast<const uint2*>(p.x_aan + io * 2);
@@ -831,7 +819,7 @@ __global__ void __launch_bounds__(kFusedWarps * 32, 1) decode_step_kernel(const 
                 const float4 raw = *reinterpret_cast<const float4*>(p.x_aan + io * 4);
                 xv[0] = raw.x; xv[1] = raw.y; xv[2] = raw.z; xv[3] = raw.w;
             }
-            float4* sp = reinterpret_cast<float4*>(p.aan_sum + ((long long)lr * p.max_seqs + id) * d + c4 * 4);
+            float4* sp = reinterpret_cast<float4*>(p.aan_sum + ((long long)lr * p.aan_max_seqs + id) * d + c4 * 4);
             float4 s = (t == 1) ? make_float4(0.f, 0.f, 0.f, 0.f) : *sp;
             s.x += xv[0]; s.y += xv[1]; s.z += xv[2]; s.w += xv[3];
             *sp = s;
@@ -840,52 +828,84 @@ __global__ void __launch_bounds__(kFusedWarps * 32, 1) decode_step_kernel(const 
             if (sizeof(T) == 2) {
                 __nv_bfloat162 a = __floats2bfloat162_rn(o[0], o[1]), b = __floats2bfloat162_rn(o[2], o[3]);
                 uint2 r; r.x = *reinterpret_cast<uint32_t*>(&a); r.y = *reinterpret_cast<uint32_t*>(&b);
-                *reinterpret_cast<uint2*>(p.O_self + io * 2) = r;
+                *reinterpret_cast<uint2*>(p.aan_out + io * 2) = r;
             } else {
-                *reinterpret_cast<float4*>(p.O_self + io * 4) = make_float4(o[0], o[1], o[2], o[3]);
+                *reinterpret_cast<float4*>(p.aan_out + io * 4) = make_float4(o[0], o[1], o[2], o[3]);
             }
         }
     }
     if (p.n_items == 0) return;
 
-    // ---- attention items
-    if (threadIdx.x == 0) cta_next = kFusedWarps;   // slots 0..warps-1 are the warps' first items
-    __syncthreads();
-    FusedWarp<T> w(p);
+    // ---- attention items: warps 0 .. kMathWarps-1 do the arithmetic, the last warp copies for them
     char* base = reinterpret_cast<char*>(smem);
-    w.ring_g = base + (size_t)warp * kFusedStages * kStageBytes;
-    w.ring = smem_u32(w.ring_g);
-    char* after = base + (size_t)kFusedWarps * kFusedStages * kStageBytes;
-    w.zs = reinterpret_cast<float*>(after) + (size_t)warp * kZFloats;
-    after += (size_t)kFusedWarps * kZFloats * sizeof(float);
-    w.descs = reinterpret_cast<ItemDesc*>(after) + (size_t)warp * kDescSlots;
-    after += (size_t)kFusedWarps * kDescSlots * sizeof(ItemDesc);
-    uint64_t* bars_g = reinterpret_cast<uint64_t*>(after) + (size_t)warp * kFusedStages;
-    w.bars = smem_u32(bars_g);
-    w.cta_next = &cta_next;
-    w.lane = lane; w.g = lane / RowGeom<T>::LPR; w.c = lane % RowGeom<T>::LPR;
-    w.p_seq = 0; w.p_n = 0; w.c_seq = 0; w.c_n = 0; w.dead = false; w.p_active = false;
-    if (lane == 0) {
-        for (int s = 0; s < kFusedStages; ++s) mbar_init(bars_g + s, 1);
+    char* rings = base;
+    float* zs_all = reinterpret_cast<float*>(base + (size_t)kMathWarps * kFusedStages * kStageBytes);
+    ItemDesc* descs_all = reinterpret_cast<ItemDesc*>(reinterpret_cast<char*>(zs_all) + (size_t)kMathWarps * kZFloats * sizeof(float));
+    uint64_t* bars_all = reinterpret_cast<uint64_t*>(reinterpret_cast<char*>(descs_all) + (size_t)kMathWarps * kDescSlots * sizeof(ItemDesc));
+    // per math warp: full[kFusedStages] then empty[kFusedStages]
+    if (threadIdx.x < kMathWarps) {
+        uint64_t* b = bars_all + (size_t)threadIdx.x * 2 * kFusedStages;
+        for (int s = 0; s < 2 * kFusedStages; ++s) mbar_init(b + s, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    __syncwarp();
+    if (threadIdx.x == 0) cta_next = kMathWarps;   // slots 0..kMathWarps-1 are the math warps' first items
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    w.nx_item = w.item_of_slot((unsigned)warp);
-    w.fetch_meta(w.nx_item, &w.nx_id, &w.nx_len);
-    w.nn_item = (w.nx_item < p.n_items) ? w.grab() : w.nx_item;
-    w.next_item();
-    for (int s = 0; s < kFusedStages; ++s) w.produce();
-    while (w.c_n < w.p_n && !w.dead) {
-        const ItemDesc& d = w.descs[w.c_n % kDescSlots];
+    __syncthreads();
+
+    if (warp == kMathWarps) {
+        // ------------------------------------------------------------ the copy warp
+        TileProducer<T> pr(p);
+        const int mw = lane < kMathWarps ? lane : 0;
+        pr.ring = smem_u32(rings + (size_t)mw * kFusedStages * kStageBytes);
+        pr.full = smem_u32(bars_all + (size_t)mw * 2 * kFusedStages);
+        pr.empty = pr.full + kFusedStages * 8;
+        pr.descs = descs_all + (size_t)mw * kDescSlots;
+        pr.cta_next = &cta_next;
+        pr.n_dec = 0; pr.stage = 0; pr.issued = 0; pr.active = false;
+        pr.finished = lane >= kMathWarps;
+        if (!pr.finished) {
+            pr.nx_item = pr.item_of_slot((unsigned)lane);
+            pr.fetch_meta(pr.nx_item, &pr.nx_id, &pr.nx_len);
+            pr.nn_item = (pr.nx_item < p.n_items) ? pr.grab() : pr.nx_item;
+            pr.next_item();
+        }
+        long long t_idle = clock64();
+        while (true) {
+            bool progressed = false;
+            if (!pr.finished && pr.stage_free()) { pr.issue(); progressed = true; }
+            if (__all_sync(0xffffffffu, pr.finished)) break;
+            if (__any_sync(0xffffffffu, progressed)) { t_idle = clock64(); continue; }
+            // every ring is full: the math warps are busy.  Give up after about a second of no progress.
+            if (clock64() - t_idle > 2000000000LL) {
+                if (lane == 0 && atomicCAS(&p.err[0], 0, (int)SAN_ERR_TIMEOUT) == 0) { p.err[1] = TAG_STEP; p.err[2] = -1; }
+                break;
+            }
+            __nanosleep(64);
+        }
+        return;
+    }
+
+    // ---------------------------------------------------------------- a math warp
+    FusedWarp<T> w(p);
+    w.ring_g = rings + (size_t)warp * kFusedStages * kStageBytes;
+    w.ring = smem_u32(w.ring_g);
+    w.full = smem_u32(bars_all + (size_t)warp * 2 * kFusedStages);
+    w.empty = w.full + kFusedStages * 8;
+    w.zs = zs_all + (size_t)warp * kZFloats;
+    w.lane = lane; w.g = lane / RowGeom<T>::LPR; w.c = lane % RowGeom<T>::LPR;
+    w.c_stage = 0; w.c_par = 0; w.dead = false;
+    const ItemDesc* descs = descs_all + (size_t)warp * kDescSlots;
+    for (unsigned c_n = 0; !w.dead; ++c_n) {
+        // an item's descriptor becomes visible with its first tile (or with the end marker)
+        if (!w.acquire()) break;
+        const ItemDesc& d = descs[c_n % kDescSlots];
+        if (d.kind < 0) break;
         if constexpr (sizeof(T) == 2) {
             if (d.kind) w.template process_mma<NQE>(d); else w.template process_mma<1>(d);
         } else {
             if (d.kind) w.template process<NQE>(d); else w.template process<1>(d);
         }
-        w.c_n += 1;
     }
-    if (w.dead) w.drain();
 }
 
 }  // namespace san
