@@ -423,7 +423,7 @@ int32_t san_decode_step(san_ctx* ctx, const san_step_args* a, void* stream) {
     auto items = [&]() {
         return rows_self * ceil_div(max_len, span_self) + rows_enc * ceil_div(max_src, span_enc);
     };
-    while (items() < 3 * warps) {
+    while (items() < 2 * warps) {
         const long long bs = do_self ? (long long)span_self * (1 + pi_self) : 0;
         const long long be = do_enc ? (long long)span_enc * (1 + pi_enc) : 0;
         if (bs >= be && span_self > 32 && ceil_div(max_len, span_self) < ceil_div(max_len, 32)) span_self = std::max(32, (int)align_up((size_t)ceil_div(span_self, 2), TR));

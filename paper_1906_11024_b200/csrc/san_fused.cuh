@@ -100,15 +100,6 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
                  : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {     // never blocks
-    uint32_t ok;
-    asm volatile("{\n.reg .pred p;\nmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
-                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
 // Bounded wait: gives up after about a second and reports it; never spins for ever.
 __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity) {
     const long long t0 = clock64();
@@ -172,150 +163,50 @@ template <> struct Pairs<float> {
     }
 };
 
-// ------------------------------------------------------------------------------ the copy side
-// One warp per CTA feeds all the others.  Lane i serves math warp i: it takes items from
-// the CTA's sequence, decodes them (32 items decoded side by side instead of one decode
-// repeated by 32 lanes), and issues the bulk copies of their tiles into warp i's ring as
-// its stages come free.  Nothing here blocks: a lane whose ring is full just polls again.
-template <typename T>
-struct TileProducer {
-    using F = FusedGeom<T>;
-    static constexpr int ROW_BYTES = F::ROW_BYTES, TR = F::TR, QROW = TR - 8;
+// ------------------------------------------------------------------------------ decoding
+// Item `it` of the list ([enc-dec items][self items]; within a kind (((block, item), head),
+// span)) into *d.  Returns false if the item is to be skipped (a failed device check, which
+// is recorded, or a span beyond the row's length).  Called by one thread per item: a CTA
+// decodes its whole share of the list side by side before any arithmetic starts.
+template <int ROW_BYTES>
+__device__ bool decode_item(const StepParams& p, unsigned it, ItemDesc* d) {
+    const int enc = it < p.n_enc_items;
+    const KindParams& kp = p.k[enc];
+    unsigned row, span, bi, h, block, item;
+    kp.div_span.divmod(enc ? it : it - p.n_enc_items, &row, &span);
+    kp.div_h.divmod(row, &bi, &h);
+    kp.div_item.divmod(bi, &block, &item);
+    const int id = kp.ids[item], len = kp.lens[item] + (int)kp.len_bias;
+    const bool reporter = (span == 0 && h == 0 && block == 0);
+    if ((unsigned)id >= kp.max_ids) { if (reporter) record_error(p.err, TAG_STEP, (int)item, id, (int)kp.max_ids); return false; }
+    if (len < 1 || len > (int)kp.bound) { if (reporter) record_error(p.err, TAG_STEP, (int)item, len, (int)kp.bound); return false; }
+    const int j0 = (int)(span * kp.span);
+    if (j0 >= len) return false;                      // a shorter row has fewer spans
+    const unsigned H = (unsigned)p.H;
+    const int j1 = min(len, j0 + (int)kp.span);
+    const unsigned first = kp.first[block];
+    const unsigned vplane = kp.v_by_block ? block : first;
+    const unsigned qrow = ((block * kp.n_it + item) * kp.nq) * H + h;          // row of query 0 in q and S
+    const unsigned long long panel = (unsigned long long)((unsigned)id * H + h) * kp.panel_bytes;
+    d->kind = enc; d->nq = (int)kp.nq; d->pi = kp.v_by_block ? 1 : kp.size[block];
+    d->len = len; d->j0 = j0; d->j1 = j1;
+    d->n_spans = (len + (int)kp.span - 1) / (int)kp.span; d->span = (int)span;
+    d->has_new = (kp.knew != nullptr && j1 == len) ? 1 : 0;
+    d->row_id = kp.row_base + row;
+    d->part = p.part + kp.part_base + (unsigned long long)(row * kp.nspans + span) * kp.part_stride;
+    d->q = kp.q + (unsigned long long)qrow * ROW_BYTES;
+    d->S = kp.S ? kp.S + (unsigned long long)qrow * (unsigned long long)kp.S_ld : nullptr;
+    d->Kp = kp.K + (unsigned long long)block * (unsigned long long)kp.plane_bytes + panel;
+    d->Vp = kp.V + (unsigned long long)vplane * (unsigned long long)kp.plane_bytes + panel;
+    d->O = kp.O + (unsigned long long)vplane * (unsigned long long)kp.layer_bytes +
+           (unsigned long long)((item * kp.nq) * H + h) * ROW_BYTES;
+    const unsigned long long in_row = (unsigned long long)(item * H + h) * ROW_BYTES;   // self: nq == 1
+    d->knew = kp.knew ? kp.knew + (unsigned long long)block * (unsigned long long)kp.layer_bytes + in_row : nullptr;
+    d->vnew = kp.vnew ? kp.vnew + (unsigned long long)first * (unsigned long long)kp.layer_bytes + in_row : nullptr;
+    return true;
+}
 
-    const StepParams& p;
-    uint32_t ring, full, empty;   // shared-space addresses of the served warp's stages and barriers
-    ItemDesc* descs;
-    unsigned* cta_next;
-    bool active, finished;
-    unsigned n_dec, stage, issued;            // items decoded, next stage, tiles issued so far
-    int which, pi, n_pos, left, has_new, nq, kind;
-    const char* src;
-    unsigned nx_item; int nx_id, nx_len; unsigned nn_item;
-
-    __device__ TileProducer(const StepParams& pp) : p(pp) {}
-
-    __device__ __forceinline__ unsigned item_of_slot(unsigned k) const {
-        const unsigned long long it = (unsigned long long)k * gridDim.x + blockIdx.x;
-        return it < p.n_items ? (unsigned)it : p.n_items;
-    }
-    __device__ __forceinline__ unsigned grab() { return item_of_slot(atomicAdd(cta_next, 1u)); }
-
-    // ---- item list: [enc-dec items][self items]; within a kind: (((block, item), head), span)
-    __device__ __forceinline__ void fetch_meta(unsigned it, int* id, int* len) const {
-        *id = 0; *len = 0;
-        if (it >= p.n_items) return;
-        const int enc = it < p.n_enc_items;
-        const KindParams& kp = p.k[enc];
-        unsigned row, span, bi, h, block, item;
-        kp.div_span.divmod(enc ? it : it - p.n_enc_items, &row, &span);
-        kp.div_h.divmod(row, &bi, &h);
-        kp.div_item.divmod(bi, &block, &item);
-        *id = kp.ids[item]; *len = kp.lens[item] + (int)kp.len_bias;
-    }
-
-    // Decodes item `it` into *d; returns false if the item is to be skipped.
-    __device__ bool decode(unsigned it, int id, int len, ItemDesc* d) const {
-        const int enc = it < p.n_enc_items;
-        const KindParams& kp = p.k[enc];
-        unsigned row, span, bi, h, block, item;
-        kp.div_span.divmod(enc ? it : it - p.n_enc_items, &row, &span);
-        kp.div_h.divmod(row, &bi, &h);
-        kp.div_item.divmod(bi, &block, &item);
-        const bool reporter = (span == 0 && h == 0 && block == 0);
-        if ((unsigned)id >= kp.max_ids) { if (reporter) record_error(p.err, TAG_STEP, (int)item, id, (int)kp.max_ids); return false; }
-        if (len < 1 || len > (int)kp.bound) { if (reporter) record_error(p.err, TAG_STEP, (int)item, len, (int)kp.bound); return false; }
-        const int j0 = (int)(span * kp.span);
-        if (j0 >= len) return false;                      // a shorter row has fewer spans
-        const unsigned H = (unsigned)p.H;
-        const int j1 = min(len, j0 + (int)kp.span);
-        const unsigned first = kp.first[block];
-        const unsigned vplane = kp.v_by_block ? block : first;
-        const unsigned qrow = ((block * kp.n_it + item) * kp.nq) * H + h;          // row of query 0 in q and S
-        const unsigned long long panel = (unsigned long long)((unsigned)id * H + h) * kp.panel_bytes;
-        d->kind = enc; d->nq = (int)kp.nq; d->pi = kp.v_by_block ? 1 : kp.size[block];
-        d->len = len; d->j0 = j0; d->j1 = j1;
-        d->n_spans = (len + (int)kp.span - 1) / (int)kp.span; d->span = (int)span;
-        d->has_new = (kp.knew != nullptr && j1 == len) ? 1 : 0;
-        d->row_id = kp.row_base + row;
-        d->part = p.part + kp.part_base + (unsigned long long)(row * kp.nspans + span) * kp.part_stride;
-        d->q = kp.q + (unsigned long long)qrow * ROW_BYTES;
-        d->S = kp.S ? kp.S + (unsigned long long)qrow * (unsigned long long)kp.S_ld : nullptr;
-        d->Kp = kp.K + (unsigned long long)block * (unsigned long long)kp.plane_bytes + panel;
-        d->Vp = kp.V + (unsigned long long)vplane * (unsigned long long)kp.plane_bytes + panel;
-        d->O = kp.O + (unsigned long long)vplane * (unsigned long long)kp.layer_bytes +
-               (unsigned long long)((item * kp.nq) * H + h) * ROW_BYTES;
-        const unsigned long long in_row = (unsigned long long)(item * H + h) * ROW_BYTES;   // self: nq == 1
-        d->knew = kp.knew ? kp.knew + (unsigned long long)block * (unsigned long long)kp.layer_bytes + in_row : nullptr;
-        d->vnew = kp.vnew ? kp.vnew + (unsigned long long)first * (unsigned long long)kp.layer_bytes + in_row : nullptr;
-        return true;
-    }
-
-    // Makes the next item that is not skipped the one being issued.
-    __device__ void next_item() {
-        active = false;
-        while (nx_item < p.n_items) {
-            ItemDesc* d = &descs[n_dec % kDescSlots];
-            const bool ok = decode(nx_item, nx_id, nx_len, d);
-            nx_item = nn_item;                         // shift the look-ahead; its metadata loads start now
-            fetch_meta(nx_item, &nx_id, &nx_len);
-            nn_item = (nx_item < p.n_items) ? grab() : nx_item;
-            if (ok) {
-                n_dec += 1; active = true;
-                which = 0; pi = d->pi; n_pos = d->j1 - d->j0; left = n_pos; has_new = d->has_new;
-                nq = d->nq; kind = d->kind;
-                src = d->Kp + (long long)d->j0 * ROW_BYTES;
-                return;
-            }
-        }
-    }
-
-    // True if the stage the next tile goes to has been handed back by the math warp.
-    __device__ __forceinline__ bool stage_free() const {
-        if (issued < (unsigned)kFusedStages) return true;
-        return mbar_test_wait(empty + stage * 8, ((issued / kFusedStages) - 1) & 1);
-    }
-
-    // Issues one tile (or, when the items have run out, the end marker).  Call only when stage_free().
-    __device__ void issue() {
-        const uint32_t dst = ring + stage * kStageBytes;
-        const uint32_t bar = full + stage * 8;
-        if (!active) {      // no more items: an item slot with kind < 0 and an empty tile tell the math warp to stop
-            descs[n_dec % kDescSlots].kind = -1;
-            mbar_arrive(bar);
-            finished = true;
-        } else {
-            const ItemDesc& d = descs[(n_dec - 1) % kDescSlots];
-            const bool first = (which == 0 && left == n_pos);
-            const int r = min(first ? QROW : TR, left);
-            const bool with_new = has_new && (r == left);
-            const int r_cache = with_new ? r - 1 : r;
-            mbar_expect_tx(bar, (uint32_t)((r + (first ? nq : 0)) * ROW_BYTES));
-            if (r_cache > 0) bulk_g2s(dst, src, (uint32_t)(r_cache * ROW_BYTES), bar);
-            if (with_new) {     // this step's row of the panel: keys, or values of layer which - 1
-                const char* nsrc = which == 0 ? d.knew : d.vnew + (long long)(which - 1) * p.k[kind].layer_bytes;
-                bulk_g2s(dst + r_cache * ROW_BYTES, nsrc, ROW_BYTES, bar);
-            }
-            if (first) {        // the query rows ride behind the first key tile
-                const unsigned q_stride = (unsigned)p.H * ROW_BYTES;
-                for (int qi = 0; qi < nq; ++qi) bulk_g2s(dst + (QROW + qi) * ROW_BYTES, d.q + (size_t)qi * q_stride, ROW_BYTES, bar);
-            }
-            left -= r;
-            src += (long long)r * ROW_BYTES;
-            if (left <= 0) {
-                if (which == pi) next_item();
-                else {          // on to the value panel of layer `which`
-                    src = d.Vp + (long long)which * p.k[kind].plane_bytes + (long long)d.j0 * ROW_BYTES;
-                    which += 1;
-                    left = n_pos;
-                }
-            }
-        }
-        stage = (stage + 1 == (unsigned)kFusedStages) ? 0 : stage + 1;
-        issued += 1;
-    }
-};
-
-// ------------------------------------------------------------------------------ the math side
+// ------------------------------------------------------------------------------ the warp
 template <typename T>
 struct FusedWarp {
     using G = RowGeom<T>;
@@ -329,18 +220,84 @@ struct FusedWarp {
     static constexpr int UN = BLK / RPW;     // loads per lane per block
 
     const StepParams& p;
-    uint32_t ring, full, empty;   // shared-space addresses: stages and their barriers
+    uint32_t ring, bars;          // shared-space addresses: stages and their barriers
     const char* ring_g;           // the same stages through a generic pointer
     float* zs;                    // kZFloats floats
+    const ItemDesc* descs;        // the CTA's decoded items
+    unsigned* q_next;             // shared counter: next of them to hand out
+    unsigned n_valid;             // how many there are
     int lane, g, c;
+    // copy side: the item whose tiles are being issued, and the one after (taken ahead)
+    bool p_active;
+    unsigned p_idx, nx_idx, p_stage;
+    int p_which, p_pi, p_n_pos, p_left, p_has_new, p_nq, p_kind;
+    const char* p_src;
+    // math side
     unsigned c_stage, c_par;
+    unsigned long long fifo;      // items whose tiles are (being) issued and whose arithmetic is still to do,
+    int fifo_n;                   // oldest in the low byte (item indices are below kCtaItems <= 255)
     bool dead;                    // a wait ran out: leave
 
     __device__ FusedWarp(const StepParams& pp) : p(pp) {}
 
+    __device__ __forceinline__ unsigned grab() {
+        unsigned k = 0;
+        if (lane == 0) k = atomicAdd(q_next, 1u);
+        return __shfl_sync(0xffffffffu, k, 0);
+    }
+
+    // The copy side moves on to the item taken ahead, and takes the one after.
+    __device__ __forceinline__ void next_item() {
+        p_idx = nx_idx;
+        p_active = p_idx < n_valid;
+        if (!p_active) return;
+        fifo |= (unsigned long long)p_idx << (8 * fifo_n);
+        fifo_n += 1;
+        nx_idx = grab();
+        const ItemDesc& d = descs[p_idx];
+        p_which = 0; p_pi = d.pi; p_n_pos = d.j1 - d.j0; p_left = p_n_pos; p_has_new = d.has_new;
+        p_nq = d.nq; p_kind = d.kind;
+        p_src = d.Kp + (long long)d.j0 * ROW_BYTES;
+    }
+
+    // Issues the copies of one tile of the item being issued, if any is left.  The first key
+    // tile of an item has room for QROW key rows and carries the query rows behind them.
+    __device__ __forceinline__ void produce() {
+        if (!p_active) return;
+        const bool first = (p_which == 0 && p_left == p_n_pos);
+        const int r = min(first ? QROW : TR, p_left);
+        if (lane == 0) {
+            const ItemDesc& d = descs[p_idx];
+            const uint32_t dst = ring + p_stage * kStageBytes;
+            const uint32_t bar = bars + p_stage * 8;
+            const bool with_new = p_has_new && (r == p_left);
+            const int r_cache = with_new ? r - 1 : r;
+            mbar_expect_tx(bar, (uint32_t)((r + (first ? p_nq : 0)) * ROW_BYTES));
+            if (r_cache > 0) bulk_g2s(dst, p_src, (uint32_t)(r_cache * ROW_BYTES), bar);
+            if (with_new) {     // this step's row of the panel: keys, or values of layer p_which - 1
+                const char* nsrc = p_which == 0 ? d.knew : d.vnew + (long long)(p_which - 1) * p.k[p_kind].layer_bytes;
+                bulk_g2s(dst + r_cache * ROW_BYTES, nsrc, ROW_BYTES, bar);
+            }
+            if (first) {        // the query rows ride behind the first key tile
+                const unsigned q_stride = (unsigned)p.H * ROW_BYTES;
+                for (int qi = 0; qi < p_nq; ++qi) bulk_g2s(dst + (QROW + qi) * ROW_BYTES, d.q + (size_t)qi * q_stride, ROW_BYTES, bar);
+            }
+        }
+        p_stage = (p_stage + 1 == (unsigned)kFusedStages) ? 0 : p_stage + 1;
+        p_left -= r;
+        p_src += (long long)r * ROW_BYTES;
+        if (p_left <= 0) {
+            if (p_which == p_pi) { next_item(); return; }
+            const ItemDesc& d = descs[p_idx];                       // on to the value panel of layer p_which
+            p_src = d.Vp + (long long)p_which * p.k[p_kind].plane_bytes + (long long)d.j0 * ROW_BYTES;
+            p_which += 1;
+            p_left = p_n_pos;
+        }
+    }
+
     // Waits for the next tile in order; returns its stage or null after a timeout.
     __device__ __forceinline__ const char* acquire() {
-        const uint32_t bar = full + c_stage * 8;
+        const uint32_t bar = bars + c_stage * 8;
         if (!mbar_try_wait(bar, c_par)) {
             if (!mbar_wait_slow(bar, c_par)) {
                 if (lane == 0 && atomicCAS(&p.err[0], 0, (int)SAN_ERR_TIMEOUT) == 0) { p.err[1] = TAG_STEP; p.err[2] = (int)c_stage; }
@@ -350,14 +307,14 @@ struct FusedWarp {
         }
         return ring_g + c_stage * kStageBytes;
     }
-    // Every lane is done with the tile: hand the stage back to the copy side.
+    // Every lane is done with the tile: its stage takes the next tile to be issued.
     __device__ __forceinline__ void release() {
         // the tensor-core path writes into its tiles (chunk-permuting the newest row, zeroing a
         // ragged tail): order those writes ahead of the bulk copy that will reuse the stage
         if (sizeof(T) == 2) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncwarp();
-        if (lane == 0) mbar_arrive(empty + c_stage * 8);
         if (++c_stage == (unsigned)kFusedStages) { c_stage = 0; c_par ^= 1u; }
+        produce();
     }
 
     template <int NQ> __device__ bool process(const ItemDesc& d);
@@ -786,10 +743,10 @@ __device__ void FusedWarp<T>::combine(const ItemDesc& d) {
     if (lane == 0) p.tickets[d.row_id] = 0;
 }
 
-constexpr int kMathWarps = kFusedWarps - 1;     // the last warp of the CTA is the copy warp
+constexpr int kCtaItems = 144;      // decoded items a CTA holds at a time (at most 255: the warps queue them by byte)
 constexpr size_t fused_smem_bytes() {
-    return (size_t)kMathWarps * (kFusedStages * kStageBytes + kZFloats * sizeof(float) + kDescSlots * sizeof(ItemDesc) +
-                                 2 * kFusedStages * sizeof(uint64_t)) + 128;
+    return (size_t)kFusedWarps * (kFusedStages * kStageBytes + kZFloats * sizeof(float) + kFusedStages * sizeof(uint64_t)) +
+           (size_t)kCtaItems * sizeof(ItemDesc) + 128;
 }
 
 template <typename T, int NQE>
@@ -836,75 +793,60 @@ __global__ void __launch_bounds__(kFusedWarps * 32, 1) decode_step_kernel(const 
     }
     if (p.n_items == 0) return;
 
-    // ---- attention items: warps 0 .. kMathWarps-1 do the arithmetic, the last warp copies for them
+    // ---- attention items.  CTA b owns list slots b, b + G, b + 2G, ...  It takes them in rounds
+    // of kCtaItems slots: every thread decodes one slot, the survivors are packed in list order
+    // (big items first), then the warps drain them through a shared counter.
+    __shared__ unsigned q_next, n_valid, warp_count[kFusedWarps];
     char* base = reinterpret_cast<char*>(smem);
-    char* rings = base;
-    float* zs_all = reinterpret_cast<float*>(base + (size_t)kMathWarps * kFusedStages * kStageBytes);
-    ItemDesc* descs_all = reinterpret_cast<ItemDesc*>(reinterpret_cast<char*>(zs_all) + (size_t)kMathWarps * kZFloats * sizeof(float));
-    uint64_t* bars_all = reinterpret_cast<uint64_t*>(reinterpret_cast<char*>(descs_all) + (size_t)kMathWarps * kDescSlots * sizeof(ItemDesc));
-    // per math warp: full[kFusedStages] then empty[kFusedStages]
-    if (threadIdx.x < kMathWarps) {
-        uint64_t* b = bars_all + (size_t)threadIdx.x * 2 * kFusedStages;
-        for (int s = 0; s < 2 * kFusedStages; ++s) mbar_init(b + s, 1);
+    float* zs_all = reinterpret_cast<float*>(base + (size_t)kFusedWarps * kFusedStages * kStageBytes);
+    uint64_t* bars_all = reinterpret_cast<uint64_t*>(reinterpret_cast<char*>(zs_all) + (size_t)kFusedWarps * kZFloats * sizeof(float));
+    ItemDesc* descs = reinterpret_cast<ItemDesc*>(reinterpret_cast<char*>(bars_all) + (size_t)kFusedWarps * kFusedStages * sizeof(uint64_t));
+
+    FusedWarp<T> w(p);
+    w.ring_g = base + (size_t)warp * kFusedStages * kStageBytes;
+    w.ring = smem_u32(w.ring_g);
+    w.bars = smem_u32(bars_all + (size_t)warp * kFusedStages);
+    w.zs = zs_all + (size_t)warp * kZFloats;
+    w.descs = descs; w.q_next = &q_next;
+    w.lane = lane; w.g = lane / RowGeom<T>::LPR; w.c = lane % RowGeom<T>::LPR;
+    w.p_stage = 0; w.c_stage = 0; w.c_par = 0; w.dead = false; w.p_active = false;
+    if (lane == 0) {
+        for (int s = 0; s < kFusedStages; ++s) mbar_init(bars_all + (size_t)warp * kFusedStages + s, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (threadIdx.x == 0) cta_next = kMathWarps;   // slots 0..kMathWarps-1 are the math warps' first items
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    __syncthreads();
 
-    if (warp == kMathWarps) {
-        // ------------------------------------------------------------ the copy warp
-        TileProducer<T> pr(p);
-        const int mw = lane < kMathWarps ? lane : 0;
-        pr.ring = smem_u32(rings + (size_t)mw * kFusedStages * kStageBytes);
-        pr.full = smem_u32(bars_all + (size_t)mw * 2 * kFusedStages);
-        pr.empty = pr.full + kFusedStages * 8;
-        pr.descs = descs_all + (size_t)mw * kDescSlots;
-        pr.cta_next = &cta_next;
-        pr.n_dec = 0; pr.stage = 0; pr.issued = 0; pr.active = false;
-        pr.finished = lane >= kMathWarps;
-        if (!pr.finished) {
-            pr.nx_item = pr.item_of_slot((unsigned)lane);
-            pr.fetch_meta(pr.nx_item, &pr.nx_id, &pr.nx_len);
-            pr.nn_item = (pr.nx_item < p.n_items) ? pr.grab() : pr.nx_item;
-            pr.next_item();
-        }
-        long long t_idle = clock64();
-        while (true) {
-            bool progressed = false;
-            if (!pr.finished && pr.stage_free()) { pr.issue(); progressed = true; }
-            if (__all_sync(0xffffffffu, pr.finished)) break;
-            if (__any_sync(0xffffffffu, progressed)) { t_idle = clock64(); continue; }
-            // every ring is full: the math warps are busy.  Give up after about a second of no progress.
-            if (clock64() - t_idle > 2000000000LL) {
-                if (lane == 0 && atomicCAS(&p.err[0], 0, (int)SAN_ERR_TIMEOUT) == 0) { p.err[1] = TAG_STEP; p.err[2] = -1; }
-                break;
+    const unsigned long long my_slots = (p.n_items > blockIdx.x) ? ((unsigned long long)p.n_items - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+    for (unsigned long long k0 = 0; k0 < my_slots; k0 += kCtaItems) {
+        // -- decode: thread t takes slot k0 + t; survivors keep their order
+        ItemDesc mine;
+        bool ok = false;
+        if (threadIdx.x < kCtaItems && k0 + threadIdx.x < my_slots)
+            ok = decode_item<FusedGeom<T>::ROW_BYTES>(p, (unsigned)((k0 + threadIdx.x) * gridDim.x + blockIdx.x), &mine);
+        const unsigned ballot = __ballot_sync(0xffffffffu, ok);
+        if (lane == 0) warp_count[warp] = __popc(ballot);
+        if (threadIdx.x == 0) q_next = kFusedWarps;      // the first kFusedWarps items go to the warps directly
+        __syncthreads();                                 // also: every warp is done with the previous round's items
+        unsigned before = 0, total = 0;
+        for (int i = 0; i < kFusedWarps; ++i) { const unsigned cnt = warp_count[i]; if (i < warp) before += cnt; total += cnt; }
+        if (ok) descs[before + __popc(ballot & ((1u << lane) - 1u))] = mine;
+        __syncthreads();
+        // -- drain
+        w.n_valid = w.dead ? 0u : total;
+        w.nx_idx = (unsigned)warp;
+        w.fifo = 0ull; w.fifo_n = 0;
+        w.next_item();
+        for (int s = 0; s < kFusedStages; ++s) w.produce();
+        while (w.fifo_n > 0 && !w.dead) {
+            const ItemDesc& d = descs[(unsigned)(w.fifo & 0xffull)];
+            w.fifo >>= 8; w.fifo_n -= 1;
+            if constexpr (sizeof(T) == 2) {
+                if (d.kind) w.template process_mma<NQE>(d); else w.template process_mma<1>(d);
+            } else {
+                if (d.kind) w.template process<NQE>(d); else w.template process<1>(d);
             }
-            __nanosleep(64);
         }
-        return;
-    }
-
-    // ---------------------------------------------------------------- a math warp
-    FusedWarp<T> w(p);
-    w.ring_g = rings + (size_t)warp * kFusedStages * kStageBytes;
-    w.ring = smem_u32(w.ring_g);
-    w.full = smem_u32(bars_all + (size_t)warp * 2 * kFusedStages);
-    w.empty = w.full + kFusedStages * 8;
-    w.zs = zs_all + (size_t)warp * kZFloats;
-    w.lane = lane; w.g = lane / RowGeom<T>::LPR; w.c = lane % RowGeom<T>::LPR;
-    w.c_stage = 0; w.c_par = 0; w.dead = false;
-    const ItemDesc* descs = descs_all + (size_t)warp * kDescSlots;
-    for (unsigned c_n = 0; !w.dead; ++c_n) {
-        // an item's descriptor becomes visible with its first tile (or with the end marker)
-        if (!w.acquire()) break;
-        const ItemDesc& d = descs[c_n % kDescSlots];
-        if (d.kind < 0) break;
-        if constexpr (sizeof(T) == 2) {
-            if (d.kind) w.template process_mma<NQE>(d); else w.template process_mma<1>(d);
-        } else {
-            if (d.kind) w.template process<NQE>(d); else w.template process<1>(d);
-        }
+        // a warp whose wait ran out stops working but keeps meeting the CTA at the barriers above
     }
 }
 
