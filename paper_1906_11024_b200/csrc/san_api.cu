@@ -412,33 +412,52 @@ int32_t san_decode_step(san_ctx* ctx, const san_step_args* a, void* stream) {
 
     // positions per item: what the on-chip score buffer holds, then smaller while items are
     // fat (long tails) or too few to fill the persistent warps
-    auto first_span = [&](int bound, int cap_z, int pi) {
-        int sp = std::min(cap_z, (int)align_up((size_t)bound, (size_t)TR));
-        while (sp > 32 && (long long)sp * (1 + pi) * row_bytes > (128 << 10)) sp = std::max(32, (int)align_up((size_t)ceil_div(sp, 2), TR));
-        return sp;
+    // Work per item.  An item is one warp's serial chain of tiles (key panel, then the value
+    // panels of its layers), so its length bounds both the step time and the balance: keep it
+    // to about half of a warp's share of all tiles, never under kMinTiles.  A long chain
+    // is first cut by layers: a block's layers go to several items, each of which recomputes
+    // the block's S from the keys (extra key reads, nothing to combine; never fewer than two
+    // layers per item, or sharing would buy nothing), or by positions: spans of a row whose
+    // partial sums the last span to finish combines.  Spans are multiples of 16 rows and
+    // at most what the on-chip score buffer holds.
+    constexpr long long kMinTiles = 8;
+    const int QR = TR - 8;                                           // key rows beside the queries in an item's first tile
+    auto tiles_of = [&](int span, int layers) {
+        const int k_tiles = span <= QR ? 1 : 1 + ceil_div(span - QR, TR);
+        return (long long)k_tiles + (long long)layers * ceil_div(span, TR);
     };
-    int span_self = first_span(max_len, kZFloats, pi_self);
-    int span_enc = first_span(max_src, kZFloats / nqe, pi_enc);
     const long long warps = (long long)ctx->sm_count * kFusedWarps;
-    auto items = [&]() {
-        return rows_self * ceil_div(max_len, span_self) + rows_enc * ceil_div(max_src, span_enc);
+    const int cap_self = std::min(kZFloats, (int)align_up((size_t)max_len, 16)), cap_enc = std::min(kZFloats / nqe, (int)align_up((size_t)max_src, 16));
+    const long long total_tiles = (do_self ? rows_self * ceil_div(max_len, cap_self) * tiles_of(cap_self, pi_self) : 0) +
+                                  (do_enc ? rows_enc * ceil_div(max_src, cap_enc) * tiles_of(cap_enc, pi_enc) : 0);
+    const long long budget = std::max<long long>(kMinTiles, total_tiles / (2 * warps));
+    auto pick = [&](int cap, int pi, int nq, int* span, int* lg_size) {
+        int sp = cap, lg = pi;
+        if (nq == 1) {      // one query row: partial sums are small and quick to combine, so cut positions first
+            while (sp > 64 && tiles_of(sp, lg) > budget) sp = std::max(64, (int)align_up((size_t)ceil_div(sp, 2), 16));
+            while (lg > 2 && tiles_of(sp, lg) > budget) lg = std::max(2, ceil_div(lg, 2));
+        } else {            // several query rows share a tile: partial sums are nq times bigger, so cut layers first
+            while (lg > 2 && tiles_of(sp, lg) > budget) lg = std::max(2, ceil_div(lg, 2));
+            while (sp > 32 && tiles_of(sp, lg) > 2 * budget) sp = std::max(32, (int)align_up((size_t)ceil_div(sp, 2), 16));
+        }
+        *span = sp; *lg_size = lg;
     };
-    while (items() < 2 * warps) {
-        const long long bs = do_self ? (long long)span_self * (1 + pi_self) : 0;
-        const long long be = do_enc ? (long long)span_enc * (1 + pi_enc) : 0;
-        if (bs >= be && span_self > 32 && ceil_div(max_len, span_self) < ceil_div(max_len, 32)) span_self = std::max(32, (int)align_up((size_t)ceil_div(span_self, 2), TR));
-        else if (be > 0 && span_enc > 32 && ceil_div(max_src, span_enc) < ceil_div(max_src, 32)) span_enc = std::max(32, (int)align_up((size_t)ceil_div(span_enc, 2), TR));
-        else if (bs > 0 && span_self > 32 && ceil_div(max_len, span_self) < ceil_div(max_len, 32)) span_self = std::max(32, (int)align_up((size_t)ceil_div(span_self, 2), TR));
-        else break;
-    }
-    const int stride_self = part_header_floats(1) + pi_self * kDh, stride_enc = part_header_floats(nqe) + pi_enc * nqe * kDh;
+    int span_self = cap_self, span_enc = cap_enc, lg_self = pi_self, lg_enc = pi_enc;
+    pick(cap_self, pi_self, 1, &span_self, &lg_self);
+    pick(cap_enc, pi_enc, c.beam, &span_enc, &lg_enc);
+    while (ceil_div(max_len, span_self) > kMaxSpans) span_self = std::min(kZFloats, span_self * 2);
+    while (ceil_div(max_src, span_enc) > kMaxSpans) span_enc = std::min(kZFloats / nqe, span_enc * 2);
+    const int nlg_self = ceil_div(pi_self, lg_self), nlg_enc = ceil_div(pi_enc, lg_enc);
+    const long long rl_self = rows_self * nlg_self, rl_enc = rows_enc * nlg_enc;      // (row, layer group) pairs
+    if ((size_t)(rl_self + rl_enc) > ctx->n_tickets) return SAN_ERR_CAPACITY;
+    const int stride_self = part_header_floats(1) + lg_self * kDh, stride_enc = part_header_floats(nqe) + lg_enc * nqe * kDh;
     auto part_need = [&]() {
         const int ns = ceil_div(max_len, span_self), ne = ceil_div(max_src, span_enc);
-        return (ns > 1 ? rows_self * ns * stride_self : 0) + (ne > 1 ? rows_enc * ne * stride_enc : 0);
+        return (ns > 1 ? rl_self * ns * stride_self : 0) + (ne > 1 ? rl_enc * ne * stride_enc : 0);
     };
     while (part_need() > (long long)ctx->part_floats) {   // fewer, longer spans until the partial sums fit
         if (span_self < kZFloats && ceil_div(max_len, span_self) > 1 &&
-            (long long)rows_self * stride_self * ceil_div(max_len, span_self) >= (long long)rows_enc * stride_enc * ceil_div(max_src, span_enc))
+            (long long)rl_self * stride_self * ceil_div(max_len, span_self) >= (long long)rl_enc * stride_enc * ceil_div(max_src, span_enc))
             span_self = std::min(kZFloats, span_self * 2);
         else if (span_enc < kZFloats / nqe && ceil_div(max_src, span_enc) > 1) span_enc = std::min(kZFloats / nqe, span_enc * 2);
         else if (span_self < kZFloats && ceil_div(max_len, span_self) > 1) span_self = std::min(kZFloats, span_self * 2);
@@ -448,11 +467,11 @@ int32_t san_decode_step(san_ctx* ctx, const san_step_args* a, void* stream) {
     if (ns_self > kMaxSpans || ns_enc > kMaxSpans) return SAN_ERR_UNSUPPORTED;
 
     if ((long long)ctx->n_seqs * c.n_heads * c.n_layers >= (1ll << 31)) return SAN_ERR_UNSUPPORTED;   // 32-bit row indices
-    if (rows_enc * ns_enc + rows_self * ns_self > (1ll << 30)) return SAN_ERR_UNSUPPORTED;
+    if (rl_enc * ns_enc + rl_self * ns_self > (1ll << 30)) return SAN_ERR_UNSUPPORTED;
     StepParams p;
     std::memset(&p, 0, sizeof(p));
     p.H = c.n_heads;
-    p.n_enc_items = (unsigned)(rows_enc * ns_enc); p.n_items = p.n_enc_items + (unsigned)(rows_self * ns_self);
+    p.n_enc_items = (unsigned)(rl_enc * ns_enc); p.n_items = p.n_enc_items + (unsigned)(rl_self * ns_self);
     p.part = ctx->part; p.tickets = ctx->tickets; p.err = ctx->err;
     p.scale_log2e = (float)(1.4426950408889634 / std::sqrt((double)kDh));
     {   // decoder self-attention
@@ -464,11 +483,12 @@ int32_t san_decode_step(san_ctx* ctx, const san_step_args* a, void* stream) {
         k.plane_bytes = (long long)ctx->self_plane_bytes;
         k.layer_bytes = (long long)n_seqs * c.n_heads * row_bytes;
         k.S_ld = a->ld_t;
-        k.part_base = ns_enc > 1 ? rows_enc * ns_enc * stride_enc : 0;
+        k.part_base = ns_enc > 1 ? rl_enc * ns_enc * stride_enc : 0;
         k.panel_bytes = (unsigned)c.max_tgt_len * row_bytes;
         k.n_it = (unsigned)std::max(n_seqs, 1); k.nq = 1; k.len_bias = 1; k.max_ids = (unsigned)ctx->n_seqs; k.bound = (unsigned)max_len;
         k.span = (unsigned)span_self; k.nspans = (unsigned)ns_self; k.part_stride = (unsigned)stride_self; k.v_by_block = 0;
-        k.row_base = (unsigned)rows_enc;
+        k.row_base = (unsigned)rl_enc;
+        k.lg_size = (unsigned)lg_self; k.n_lg = (unsigned)nlg_self; k.div_lg = make_fastdiv((unsigned)nlg_self);
         k.div_span = make_fastdiv((unsigned)ns_self); k.div_h = make_fastdiv((unsigned)c.n_heads); k.div_item = make_fastdiv(k.n_it);
         for (int b = 0; b < ctx->self_pol.n_blocks; ++b) {
             k.first[b] = (unsigned char)ctx->self_pol.first_layer_of_block[b];
@@ -489,6 +509,7 @@ int32_t san_decode_step(san_ctx* ctx, const san_step_args* a, void* stream) {
         k.span = (unsigned)span_enc; k.nspans = (unsigned)ns_enc; k.part_stride = (unsigned)stride_enc;
         k.v_by_block = c.encdec_shared_context ? 1 : 0;
         k.row_base = 0;
+        k.lg_size = (unsigned)lg_enc; k.n_lg = (unsigned)nlg_enc; k.div_lg = make_fastdiv((unsigned)nlg_enc);
         k.div_span = make_fastdiv((unsigned)ns_enc); k.div_h = make_fastdiv((unsigned)c.n_heads); k.div_item = make_fastdiv(k.n_it);
         for (int b = 0; b < ctx->enc_pol.n_blocks; ++b) {
             k.first[b] = (unsigned char)ctx->enc_pol.first_layer_of_block[b];

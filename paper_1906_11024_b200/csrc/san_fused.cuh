@@ -53,7 +53,8 @@ struct KindParams {
     unsigned panel_bytes;                              // capacity * row bytes: one (id, head) panel
     unsigned n_it, nq, len_bias, max_ids, bound;       // items, query rows per item, 1 if lens holds positions, limits
     unsigned span, nspans, part_stride, v_by_block, row_base;
-    FastDiv div_span, div_h, div_item;
+    unsigned lg_size, n_lg;                            // layers per item (a block is cut into groups), groups per block at most
+    FastDiv div_span, div_lg, div_h, div_item;
     unsigned char first[SAN_MAX_LAYERS], size[SAN_MAX_LAYERS];   // per block
 };
 
@@ -78,7 +79,7 @@ struct ItemDesc {
     char* O;                                  // output of (first layer, query 0)
     float* part;                              // partial sums of this (row, span)
     unsigned row_id;                          // ticket index of the row
-    int kind, nq, pi, len, j0, j1, n_spans, span, has_new;
+    int kind, nq, pi, len, j0, j1, n_spans, span, has_new, lead;
 };
 
 // ------------------------------------------------------------------------------ PTX helpers
@@ -172,30 +173,35 @@ template <int ROW_BYTES>
 __device__ bool decode_item(const StepParams& p, unsigned it, ItemDesc* d) {
     const int enc = it < p.n_enc_items;
     const KindParams& kp = p.k[enc];
-    unsigned row, span, bi, h, block, item;
-    kp.div_span.divmod(enc ? it : it - p.n_enc_items, &row, &span);
+    unsigned row, span, bi, h, block, item, rl, lg;
+    kp.div_span.divmod(enc ? it : it - p.n_enc_items, &rl, &span);    // rl = (row, layer group)
+    kp.div_lg.divmod(rl, &row, &lg);
     kp.div_h.divmod(row, &bi, &h);
     kp.div_item.divmod(bi, &block, &item);
     const int id = kp.ids[item], len = kp.lens[item] + (int)kp.len_bias;
-    const bool reporter = (span == 0 && h == 0 && block == 0);
+    const bool reporter = (span == 0 && lg == 0 && h == 0 && block == 0);
     if ((unsigned)id >= kp.max_ids) { if (reporter) record_error(p.err, TAG_STEP, (int)item, id, (int)kp.max_ids); return false; }
     if (len < 1 || len > (int)kp.bound) { if (reporter) record_error(p.err, TAG_STEP, (int)item, len, (int)kp.bound); return false; }
     const int j0 = (int)(span * kp.span);
     if (j0 >= len) return false;                      // a shorter row has fewer spans
+    const unsigned size = kp.v_by_block ? 1u : kp.size[block];
+    const unsigned l0 = lg * kp.lg_size;              // first layer of the group, relative to the block
+    if (l0 >= size) return false;                     // a smaller block has fewer layer groups
     const unsigned H = (unsigned)p.H;
     const int j1 = min(len, j0 + (int)kp.span);
-    const unsigned first = kp.first[block];
-    const unsigned vplane = kp.v_by_block ? block : first;
+    const unsigned first = kp.first[block] + l0;      // every group recomputes S from the block's keys
+    const unsigned vplane = (kp.v_by_block ? block : kp.first[block]) + l0;
     const unsigned qrow = ((block * kp.n_it + item) * kp.nq) * H + h;          // row of query 0 in q and S
     const unsigned long long panel = (unsigned long long)((unsigned)id * H + h) * kp.panel_bytes;
-    d->kind = enc; d->nq = (int)kp.nq; d->pi = kp.v_by_block ? 1 : kp.size[block];
+    d->kind = enc; d->nq = (int)kp.nq; d->pi = (int)min(kp.lg_size, size - l0);
     d->len = len; d->j0 = j0; d->j1 = j1;
     d->n_spans = (len + (int)kp.span - 1) / (int)kp.span; d->span = (int)span;
     d->has_new = (kp.knew != nullptr && j1 == len) ? 1 : 0;
-    d->row_id = kp.row_base + row;
-    d->part = p.part + kp.part_base + (unsigned long long)(row * kp.nspans + span) * kp.part_stride;
+    d->lead = (lg == 0) ? 1 : 0;                      // the group that also stores S and this step's key row
+    d->row_id = kp.row_base + rl;
+    d->part = p.part + kp.part_base + (unsigned long long)(rl * kp.nspans + span) * kp.part_stride;
     d->q = kp.q + (unsigned long long)qrow * ROW_BYTES;
-    d->S = kp.S ? kp.S + (unsigned long long)qrow * (unsigned long long)kp.S_ld : nullptr;
+    d->S = (kp.S && lg == 0) ? kp.S + (unsigned long long)qrow * (unsigned long long)kp.S_ld : nullptr;
     d->Kp = kp.K + (unsigned long long)block * (unsigned long long)kp.plane_bytes + panel;
     d->Vp = kp.V + (unsigned long long)vplane * (unsigned long long)kp.plane_bytes + panel;
     d->O = kp.O + (unsigned long long)vplane * (unsigned long long)kp.layer_bytes +
@@ -237,6 +243,7 @@ struct FusedWarp {
     unsigned long long fifo;      // items whose tiles are (being) issued and whose arithmetic is still to do,
     int fifo_n;                   // oldest in the low byte (item indices are below kCtaItems <= 255)
     bool dead;                    // a wait ran out: leave
+    bool tile_written;            // the math side wrote into the current tile (see release)
 
     __device__ FusedWarp(const StepParams& pp) : p(pp) {}
 
@@ -311,7 +318,7 @@ struct FusedWarp {
     __device__ __forceinline__ void release() {
         // the tensor-core path writes into its tiles (chunk-permuting the newest row, zeroing a
         // ragged tail): order those writes ahead of the bulk copy that will reuse the stage
-        if (sizeof(T) == 2) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        if (tile_written) { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); tile_written = false; }
         __syncwarp();
         if (++c_stage == (unsigned)kFusedStages) { c_stage = 0; c_par ^= 1u; }
         produce();
@@ -320,13 +327,14 @@ struct FusedWarp {
     template <int NQ> __device__ bool process(const ItemDesc& d);
     template <int NQ> __device__ bool process_mma(const ItemDesc& d);
     template <int NQ> __device__ void combine(const ItemDesc& d);
-    template <int NQ> __device__ __forceinline__ void softmax_span(const ItemDesc& d, int n, int n_pad, float* part_m, float* part_l);
+    template <int NQ, bool PACK> __device__ __forceinline__ void softmax_span(const ItemDesc& d, int n, int n_pad, float* part_m, float* part_l);
 
     // bf16 tiles only.  A tile's last row may be this step's new row, copied in natural chunk
     // order from the caller's buffer: permute its chunks like a cached row (chunk c -> c ^ (pos & 7))
     // and write it to the cache at `dst_row`.  Rows [r, next multiple of 16) are zeroed when
     // `zero_tail` is set, so that a 16-row block never multiplies stale shared memory.
     __device__ __forceinline__ void fix_tile(const char* st, int r, bool with_new, char* dst_row, bool zero_tail) {
+        tile_written = true;
         if (with_new) {
             char* row = const_cast<char*>(st) + (r - 1) * 128;
             uint4 v = make_uint4(0, 0, 0, 0);
@@ -335,7 +343,7 @@ struct FusedWarp {
             if (lane < 8) {
                 const int pc = lane ^ ((r - 1) & 7);
                 *reinterpret_cast<uint4*>(row + pc * 16) = v;
-                *reinterpret_cast<uint4*>(dst_row + pc * 16) = v;
+                if (dst_row) *reinterpret_cast<uint4*>(dst_row + pc * 16) = v;
             }
         }
         if (zero_tail && (r & 15)) {
@@ -348,10 +356,13 @@ struct FusedWarp {
 };
 
 // Softmax of the n scores of a span held in zs (log2 domain), per query row.  A span that is
-// the whole row leaves normalised weights in zs and writes them to S; otherwise it leaves
-// exp2(z - max) and reports (max, sum) for the combine.  zs[n .. n_pad) is zeroed.
+// the whole row produces normalised weights and writes them to S; otherwise it produces
+// exp2(z - max) and reports (max, sum) for the combine.  With PACK == false the weights are
+// left in zs as floats (entries n .. n_pad zeroed).  With PACK == true (tensor-core path) they
+// are left as bf16 pairs: positions 2j, 2j+1 of a query row become word 2j = their bf16 high
+// parts and word 2j+1 = the bf16 remainders (w - high), zero beyond n up to n_pad.
 template <typename T>
-template <int NQ>
+template <int NQ, bool PACK>
 __device__ __forceinline__ void FusedWarp<T>::softmax_span(const ItemDesc& d, int n, int n_pad, float* part_m, float* part_l) {
     constexpr int ZQ = kZFloats / NQ;
     const int nq = d.nq, n_spans = d.n_spans;
@@ -359,40 +370,54 @@ __device__ __forceinline__ void FusedWarp<T>::softmax_span(const ItemDesc& d, in
 #pragma unroll
     for (int qi = 0; qi < NQ; ++qi) {
         part_m[qi] = 0.f; part_l[qi] = 1.f;
+        if (qi >= nq) break;                 // rows of absent queries are never stored
         float* zq = zs + qi * ZQ;
-        if (qi < nq) {
-            float* Srow = d.S ? d.S + qi * S_qstride + d.j0 : nullptr;
-            if (n <= 32) {      // one score per lane: no loops
-                const float z = lane < n ? zq[lane] : -INFINITY;
-                const float m = warp_max(z);
-                const float e = lane < n ? exp2f(z - m) : 0.f;
-                const float s = warp_sum(e);
-                part_m[qi] = m; part_l[qi] = s;
-                const float w = (n_spans == 1) ? e * (1.0f / s) : e;
-                if (lane < n_pad) zq[lane] = w;
-                if (Srow && lane < n) Srow[lane] = w;
-            } else {
-                float m = -INFINITY;
-                for (int jj = lane; jj < n; jj += 32) m = fmaxf(m, zq[jj]);
-                m = warp_max(m);
-                float s = 0.f;
-                for (int jj = lane; jj < n; jj += 32) { const float e = exp2f(zq[jj] - m); zq[jj] = e; s += e; }
-                s = warp_sum(s);
-                part_m[qi] = m; part_l[qi] = s;
-                if (n_spans == 1) {
-                    const float inv = 1.0f / s;
-                    for (int jj = lane; jj < n; jj += 32) {
-                        const float w = zq[jj] * inv;
-                        zq[jj] = w;
-                        if (Srow) Srow[jj] = w;
-                    }
-                } else if (Srow) {
-                    for (int jj = lane; jj < n; jj += 32) Srow[jj] = zq[jj];
+        unsigned short* zh = reinterpret_cast<unsigned short*>(zq);
+        float* Srow = d.S ? d.S + qi * S_qstride + d.j0 : nullptr;
+        if (n <= 32) {      // one score per lane: no loops
+            const float z = lane < n ? zq[lane] : -INFINITY;
+            const float m = warp_max(z);
+            const float e = lane < n ? exp2f(z - m) : 0.f;
+            const float s = warp_sum(e);
+            part_m[qi] = m; part_l[qi] = s;
+            const float w = (n_spans == 1) ? e * (1.0f / s) : e;
+            if (Srow && lane < n) Srow[lane] = w;
+            if (PACK) {
+                __syncwarp();                // every lane has read its score: the words may be reused
+                if (lane < n_pad) {
+                    const __nv_bfloat16 hi = __float2bfloat16_rn(w);
+                    const __nv_bfloat16 lo = __float2bfloat16_rn(w - __bfloat162float(hi));
+                    zh[(lane >> 1) * 4 + (lane & 1)] = *reinterpret_cast<const unsigned short*>(&hi);
+                    zh[(lane >> 1) * 4 + 2 + (lane & 1)] = *reinterpret_cast<const unsigned short*>(&lo);
                 }
-                for (int jj = n + lane; jj < n_pad; jj += 32) zq[jj] = 0.f;
+            } else if (lane < n_pad) {
+                zq[lane] = w;
             }
         } else {
-            for (int jj = lane; jj < n_pad; jj += 32) zq[jj] = 0.f;     // absent query rows weigh nothing
+            float m = -INFINITY;
+            for (int jj = lane; jj < n; jj += 32) m = fmaxf(m, zq[jj]);
+            m = warp_max(m);
+            float s = 0.f;
+            for (int jj = lane; jj < n; jj += 32) { const float e = exp2f(zq[jj] - m); zq[jj] = e; s += e; }
+            s = warp_sum(s);
+            part_m[qi] = m; part_l[qi] = s;
+            const float inv = (n_spans == 1) ? 1.0f / s : 1.0f;
+            for (int j0 = 0; j0 < n_pad; j0 += 32) {      // warp-uniform trip count
+                const int jj = j0 + lane;
+                const float w = jj < n ? zq[jj] * inv : 0.f;
+                if (Srow && jj < n) Srow[jj] = w;
+                if (PACK) {
+                    __syncwarp();
+                    if (jj < n_pad) {
+                        const __nv_bfloat16 hi = __float2bfloat16_rn(w);
+                        const __nv_bfloat16 lo = __float2bfloat16_rn(w - __bfloat162float(hi));
+                        zh[(jj >> 1) * 4 + (jj & 1)] = *reinterpret_cast<const unsigned short*>(&hi);
+                        zh[(jj >> 1) * 4 + 2 + (jj & 1)] = *reinterpret_cast<const unsigned short*>(&lo);
+                    }
+                } else if (jj < n_pad) {
+                    zq[jj] = w;
+                }
+            }
         }
     }
     __syncwarp();
@@ -451,7 +476,7 @@ __device__ bool FusedWarp<T>::process(const ItemDesc& d) {
                     if (c == 0 && j < r) zs[qi * ZQ + s0 + j] = dot;
                 }
                 // the newest key row goes into the cache from here
-                if (with_new && j == r - 1)
+                if (with_new && d.lead && j == r - 1)
                     *reinterpret_cast<uint4*>(const_cast<char*>(d.Kp) + (long long)(d.len - 1) * ROW_BYTES + c * 16) = kv[u];
             }
         }
@@ -462,7 +487,7 @@ __device__ bool FusedWarp<T>::process(const ItemDesc& d) {
 
     float part_m[NQ], part_l[NQ];
     const int n_spans = d.n_spans;
-    softmax_span<NQ>(d, n, n, part_m, part_l);
+    softmax_span<NQ, false>(d, n, n, part_m, part_l);
 
     // ---- value tiles, layer by layer (score rows of absent queries hold zeros)
     const long long O_qstride = (long long)p.H * ROW_BYTES;
@@ -552,57 +577,61 @@ __device__ bool FusedWarp<T>::process(const ItemDesc& d) {
 // is bound by instruction issue, not by tensor throughput.
 //   scores:  D[16 positions x 8 queries] = K_tile[16 x 64] . q^T          (queries padded to 8)
 //   apply:   D[16 queries x 8 dims]     += S[16 x 16 positions] . V_tile   (eight dim tiles)
-// S is split into a bf16 high part and a bf16 remainder (two MMAs) so that the weights keep
-// about 16 bits; products and sums are float32.
+// S is used as a bf16 high part plus a bf16 remainder (two MMAs), packed once per item by
+// the softmax, so that the weights keep about 16 bits; products and sums are float32.
+// Rows of D that belong to padding queries are computed from whatever the padding lanes
+// load and are never stored.
 template <typename T>
 template <int NQ>
 __device__ bool FusedWarp<T>::process_mma(const ItemDesc& d) {
     static_assert(sizeof(T) == 2, "tensor-core path is for bf16 rows");
     constexpr int ZQ = kZFloats / NQ;
     constexpr int HDR = (2 * NQ + 3) / 4 * 4;
-    const KindParams& kp = p.k[d.kind];
     const int n = d.j1 - d.j0, nq = d.nq, has_new = d.has_new, pi = d.pi;
     const int tig = lane & 3, gid = lane >> 2;                 // mma fragment coordinates
-    const int lrow = (lane & 7) + ((lane >> 3) & 1) * 8;        // ldmatrix: row of the 16-row block this lane addresses
-    const int lx = lane & 7, lsel = lane >> 4;                  // its chunk permutation key and chunk of the pair
+    // ldmatrix: this lane addresses row (lane & 7) + 8 * ((lane >> 3) & 1) of a 16-row block and,
+    // for the pair of 16-byte chunks 2x, 2x+1, the chunk 2x + (lane >> 4), permuted by the row
+    uint32_t ld_off[4];
+#pragma unroll
+    for (int x = 0; x < 4; ++x)
+        ld_off[x] = (uint32_t)(((lane & 7) + ((lane >> 3) & 1) * 8) * 128 + (((2 * x + (lane >> 4)) ^ (lane & 7)) << 4));
 
     // ---- key tiles: scores into zs (log2 domain).  The first tile also carries the query rows
     // (natural chunk order), read as B fragments (k = dims, n = query).
     uint32_t qb[4][2];
     const float sc = p.scale_log2e;
+    float* zk = zs + (2 * tig) * ZQ + gid;        // this lane's score slots: queries 2tig, 2tig+1; positions gid, gid+8
     for (int s0 = 0; s0 < n;) {
         const char* st = acquire();
         if (!st) return false;
         const int r = min(s0 == 0 ? QROW : TR, n - s0);
         if (s0 == 0) {
+            const char* qrow = st + (QROW + (gid < nq ? gid : 0)) * 128 + 4 * tig;
 #pragma unroll
             for (int ks = 0; ks < 4; ++ks) {
-                qb[ks][0] = 0u; qb[ks][1] = 0u;
-                if (gid < nq) {
-                    qb[ks][0] = *reinterpret_cast<const uint32_t*>(st + (QROW + gid) * 128 + (16 * ks + 2 * tig) * 2);
-                    qb[ks][1] = *reinterpret_cast<const uint32_t*>(st + (QROW + gid) * 128 + (16 * ks + 8 + 2 * tig) * 2);
-                }
+                qb[ks][0] = *reinterpret_cast<const uint32_t*>(qrow + 32 * ks);
+                qb[ks][1] = *reinterpret_cast<const uint32_t*>(qrow + 32 * ks + 16);
             }
         }
-        fix_tile(st, r, has_new && (s0 + r == n), const_cast<char*>(d.Kp) + (long long)(d.len - 1) * 128, false);
+        if (has_new && s0 + r == n) fix_tile(st, r, true, d.lead ? const_cast<char*>(d.Kp) + (long long)(d.len - 1) * 128 : nullptr, false);
         const uint32_t st_s = ring + (uint32_t)(st - ring_g);
         for (int b0 = 0; b0 < r; b0 += 16) {
             float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int ks = 0; ks < 4; ++ks) {
                 uint32_t a[4];
-                ldsm_x4(st_s + (b0 + lrow) * 128 + (((2 * ks + lsel) ^ lx) << 4), a);
+                ldsm_x4(st_s + b0 * 128 + ld_off[ks], a);
                 mma_bf16(acc, a[0], a[1], a[2], a[3], qb[ks][0], qb[ks][1]);
             }
             // acc[0], acc[1]: position b0+gid, queries 2tig, 2tig+1; acc[2], acc[3]: position b0+gid+8
-            const int p0 = b0 + gid, p1 = b0 + gid + 8;
+            float* z = zk + s0 + b0;
             if (2 * tig < NQ) {
-                if (p0 < r) zs[(2 * tig) * ZQ + s0 + p0] = acc[0] * sc;
-                if (p1 < r) zs[(2 * tig) * ZQ + s0 + p1] = acc[2] * sc;
+                if (b0 + gid < r) z[0] = acc[0] * sc;
+                if (b0 + gid + 8 < r) z[8] = acc[2] * sc;
             }
             if (2 * tig + 1 < NQ) {
-                if (p0 < r) zs[(2 * tig + 1) * ZQ + s0 + p0] = acc[1] * sc;
-                if (p1 < r) zs[(2 * tig + 1) * ZQ + s0 + p1] = acc[3] * sc;
+                if (b0 + gid < r) z[ZQ] = acc[1] * sc;
+                if (b0 + gid + 8 < r) z[ZQ + 8] = acc[3] * sc;
             }
         }
         s0 += r;
@@ -612,10 +641,16 @@ __device__ bool FusedWarp<T>::process_mma(const ItemDesc& d) {
 
     float part_m[NQ], part_l[NQ];
     const int n_spans = d.n_spans;
-    softmax_span<NQ>(d, n, (n + 15) & ~15, part_m, part_l);   // weights up to the next multiple of 16 are exact zeros
+    softmax_span<NQ, true>(d, n, (n + 15) & ~15, part_m, part_l);
 
     // ---- value tiles, layer by layer
-    const long long O_qstride = (long long)p.H * 128;
+    // A fragments: the weights of query gid at positions b0 + {2tig, 2tig+1} and b0 + {2tig+8, 2tig+9},
+    // high parts and remainders, straight from the packed words
+    const uint2* za = reinterpret_cast<const uint2*>(zs + (gid < NQ ? gid : 0) * ZQ) + tig;
+    const KindParams& kp = p.k[d.kind];
+    const long long plane_bytes = kp.plane_bytes, layer_bytes = kp.layer_bytes;
+    char* vlast = const_cast<char*>(d.Vp) + (long long)(d.len - 1) * 128;      // where this step's value row goes
+    char* op = d.O + gid * ((long long)p.H * 128) + 4 * tig;
     for (int l = 0; l < pi; ++l) {
         float acc[8][4];
 #pragma unroll
@@ -626,27 +661,19 @@ __device__ bool FusedWarp<T>::process_mma(const ItemDesc& d) {
             const char* st = acquire();
             if (!st) return false;
             const int r = min(TR, n - s0);
-            fix_tile(st, r, has_new && (s0 + r == n),
-                     const_cast<char*>(d.Vp) + (long long)l * kp.plane_bytes + (long long)(d.len - 1) * 128, true);
+            const bool with_new = has_new && (s0 + r == n);
+            if (with_new || (r & 15)) fix_tile(st, r, with_new, vlast, true);
             const uint32_t st_s = ring + (uint32_t)(st - ring_g);
             for (int b0 = 0; b0 < r; b0 += 16) {
-                // A = weights of query gid at positions b0 + {2tig, 2tig+1, 2tig+8, 2tig+9}: high part + remainder
-                uint32_t ah0 = 0u, ah2 = 0u, al0 = 0u, al2 = 0u;
-                if (gid < NQ) {
-                    const float2 w0 = *reinterpret_cast<const float2*>(zs + gid * ZQ + s0 + b0 + 2 * tig);
-                    const float2 w1 = *reinterpret_cast<const float2*>(zs + gid * ZQ + s0 + b0 + 2 * tig + 8);
-                    ah0 = pack_bf16x2(w0.x, w0.y); ah2 = pack_bf16x2(w1.x, w1.y);
-                    al0 = pack_bf16x2(w0.x - __uint_as_float(ah0 << 16), w0.y - __uint_as_float(ah0 & 0xffff0000u));
-                    al2 = pack_bf16x2(w1.x - __uint_as_float(ah2 << 16), w1.y - __uint_as_float(ah2 & 0xffff0000u));
-                }
+                const uint2 w0 = za[(s0 + b0) >> 1], w1 = za[((s0 + b0) >> 1) + 4];    // (high, remainder) x 2
 #pragma unroll
-                for (int np = 0; np < 4; ++np) {
+                for (int x = 0; x < 4; ++x) {
                     uint32_t b[4];
-                    ldsm_x4_t(st_s + (b0 + lrow) * 128 + (((2 * np + lsel) ^ lx) << 4), b);
-                    mma_bf16(acc[2 * np], ah0, 0u, ah2, 0u, b[0], b[1]);
-                    mma_bf16(acc[2 * np + 1], ah0, 0u, ah2, 0u, b[2], b[3]);
-                    mma_bf16(acc[2 * np], al0, 0u, al2, 0u, b[0], b[1]);
-                    mma_bf16(acc[2 * np + 1], al0, 0u, al2, 0u, b[2], b[3]);
+                    ldsm_x4_t(st_s + b0 * 128 + ld_off[x], b);
+                    mma_bf16(acc[2 * x], w0.x, 0u, w1.x, 0u, b[0], b[1]);
+                    mma_bf16(acc[2 * x + 1], w0.x, 0u, w1.x, 0u, b[2], b[3]);
+                    mma_bf16(acc[2 * x], w0.y, 0u, w1.y, 0u, b[0], b[1]);
+                    mma_bf16(acc[2 * x + 1], w0.y, 0u, w1.y, 0u, b[2], b[3]);
                 }
             }
             release();
@@ -654,7 +681,6 @@ __device__ bool FusedWarp<T>::process_mma(const ItemDesc& d) {
         // acc[nt][0], acc[nt][1]: query gid, dims 8nt + 2tig, +1
         if (gid < nq) {
             if (n_spans == 1) {
-                char* op = d.O + l * kp.layer_bytes + gid * O_qstride + 4 * tig;
 #pragma unroll
                 for (int nt = 0; nt < 8; ++nt) *reinterpret_cast<uint32_t*>(op + 16 * nt) = pack_bf16x2(acc[nt][0], acc[nt][1]);
             } else {
@@ -663,6 +689,8 @@ __device__ bool FusedWarp<T>::process_mma(const ItemDesc& d) {
                 for (int nt = 0; nt < 8; ++nt) *reinterpret_cast<float2*>(pp + 8 * nt) = make_float2(acc[nt][0], acc[nt][1]);
             }
         }
+        vlast += plane_bytes;
+        op += layer_bytes;
     }
     if (n_spans == 1) return true;
 
@@ -809,7 +837,7 @@ __global__ void __launch_bounds__(kFusedWarps * 32, 1) decode_step_kernel(const 
     w.zs = zs_all + (size_t)warp * kZFloats;
     w.descs = descs; w.q_next = &q_next;
     w.lane = lane; w.g = lane / RowGeom<T>::LPR; w.c = lane % RowGeom<T>::LPR;
-    w.p_stage = 0; w.c_stage = 0; w.c_par = 0; w.dead = false; w.p_active = false;
+    w.p_stage = 0; w.c_stage = 0; w.c_par = 0; w.dead = false; w.p_active = false; w.tile_written = false;
     if (lane == 0) {
         for (int s = 0; s < kFusedStages; ++s) mbar_init(bars_all + (size_t)warp * kFusedStages + s, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
