@@ -853,8 +853,8 @@ __global__ void __launch_bounds__(kFusedWarps * 32, 1) decode_step_kernel(const 
             ok = decode_item<FusedGeom<T>::ROW_BYTES>(p, (unsigned)((k0 + threadIdx.x) * gridDim.x + blockIdx.x), &mine);
         const unsigned ballot = __ballot_sync(0xffffffffu, ok);
         if (lane == 0) warp_count[warp] = __popc(ballot);
-        if (threadIdx.x == 0) q_next = kFusedWarps;      // the first kFusedWarps items go to the warps directly
         __syncthreads();                                 // also: every warp is done with the previous round's items
+        if (threadIdx.x == 0) q_next = kFusedWarps;      // the first kFusedWarps items go to the warps directly
         unsigned before = 0, total = 0;
         for (int i = 0; i < kFusedWarps; ++i) { const unsigned cnt = warp_count[i]; if (i < warp) before += cnt; total += cnt; }
         if (ok) descs[before + __popc(ballot & ((1u << lane) - 1u))] = mine;

@@ -146,6 +146,12 @@ def test_aan_bf16_full_size_sampled_steps():
     _run(synth.WORKLOADS["aan"], check_steps={0, 1, 40, 79})
 
 
+def test_learned_policy_blocks_separate_calls():
+    """Uneven blocks, as the policy learner of Section 3.3 produces on the paper's Figure 2."""
+    _run(dataclasses.replace(synth.scaled(synth.WORKLOADS["base"], 6), self_blocks=(1, 5), encdec_blocks=(4, 2),
+                             name="learned"), max_steps=12)
+
+
 def test_encdec_shared_context_eq5():
     """Eq. 5: one output per enc-dec block; upper layers of the block reuse it."""
     _run(synth.scaled(synth.WORKLOADS["base"], 4), max_steps=6, shared_context=True)
@@ -179,6 +185,11 @@ FUSED_CASES = {
     "long-full": lambda: _run(synth.WORKLOADS["long"], jumps=[(0, 2), (63, 3), (255, 3), (510, 2)], fused=True),
     "aan-scaled": lambda: _run(synth.scaled(synth.WORKLOADS["aan"], 8), max_steps=80, fused=True),
     "aan-full": lambda: _run(synth.WORKLOADS["aan"], check_steps={0, 1, 40, 79}, fused=True),
+    # the policies the paper's Figure 2 leads to: layer 1 alone then layers 2-6 (self), {4,2} (enc-dec)
+    "learned-policy-blocks": lambda: _run(dataclasses.replace(synth.scaled(synth.WORKLOADS["base"], 6), self_blocks=(1, 5),
+                                                              encdec_blocks=(4, 2), name="learned"), max_steps=12, fused=True),
+    # sharing off on the big shape: about 500 list slots per CTA, so every CTA decodes and drains in rounds
+    "big-unshared-many-rounds": lambda: _run(synth.unshared(synth.WORKLOADS["big"]), check_steps={0, 3}, max_steps=4, fused=True),
     "eq5-shared-context": lambda: _run(synth.scaled(synth.WORKLOADS["base"], 4), max_steps=6, shared_context=True,
                                        fused=True),
     "fp32-long-rows": lambda: _run(dataclasses.replace(synth.WORKLOADS["tiny"], name="tiny-long", src_lo=300, src_hi=300,
