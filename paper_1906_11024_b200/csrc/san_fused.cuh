@@ -232,7 +232,7 @@ struct FusedWarp {
     const ItemDesc* descs;        // the CTA's decoded items
     unsigned* q_next;             // shared counter: next of them to hand out
     unsigned n_valid;             // how many there are
-    int lane, g, c;
+    int lane;
     // copy side: the item whose tiles are being issued, and the one after (taken ahead)
     bool p_active;
     unsigned p_idx, nx_idx, p_stage;
@@ -327,7 +327,7 @@ struct FusedWarp {
     template <int NQ> __device__ bool process(const ItemDesc& d);
     template <int NQ> __device__ bool process_mma(const ItemDesc& d);
     template <int NQ> __device__ void combine(const ItemDesc& d);
-    template <int NQ, bool PACK> __device__ __forceinline__ void softmax_span(const ItemDesc& d, int n, int n_pad, float* part_m, float* part_l);
+    template <int NQ, bool PACK> __device__ __forceinline__ void softmax_span(const ItemDesc& d, int n, int n_pad);
 
     // bf16 tiles only.  A tile's last row may be this step's new row, copied in natural chunk
     // order from the caller's buffer: permute its chunks like a cached row (chunk c -> c ^ (pos & 7))
@@ -357,19 +357,18 @@ struct FusedWarp {
 
 // Softmax of the n scores of a span held in zs (log2 domain), per query row.  A span that is
 // the whole row produces normalised weights and writes them to S; otherwise it produces
-// exp2(z - max) and reports (max, sum) for the combine.  With PACK == false the weights are
+// exp2(z - max) and parks (max, sum) in the span's partial-sum record for the combine.  With PACK == false the weights are
 // left in zs as floats (entries n .. n_pad zeroed).  With PACK == true (tensor-core path) they
 // are left as bf16 pairs: positions 2j, 2j+1 of a query row become word 2j = their bf16 high
 // parts and word 2j+1 = the bf16 remainders (w - high), zero beyond n up to n_pad.
 template <typename T>
 template <int NQ, bool PACK>
-__device__ __forceinline__ void FusedWarp<T>::softmax_span(const ItemDesc& d, int n, int n_pad, float* part_m, float* part_l) {
+__device__ __forceinline__ void FusedWarp<T>::softmax_span(const ItemDesc& d, int n, int n_pad) {
     constexpr int ZQ = kZFloats / NQ;
     const int nq = d.nq, n_spans = d.n_spans;
     const long long S_qstride = (long long)p.H * p.k[d.kind].S_ld;
 #pragma unroll
     for (int qi = 0; qi < NQ; ++qi) {
-        part_m[qi] = 0.f; part_l[qi] = 1.f;
         if (qi >= nq) break;                 // rows of absent queries are never stored
         float* zq = zs + qi * ZQ;
         unsigned short* zh = reinterpret_cast<unsigned short*>(zq);
@@ -379,7 +378,7 @@ __device__ __forceinline__ void FusedWarp<T>::softmax_span(const ItemDesc& d, in
             const float m = warp_max(z);
             const float e = lane < n ? exp2f(z - m) : 0.f;
             const float s = warp_sum(e);
-            part_m[qi] = m; part_l[qi] = s;
+            if (n_spans > 1 && lane == 0) { d.part[qi] = m; d.part[NQ + qi] = s; }     // for the combine
             const float w = (n_spans == 1) ? e * (1.0f / s) : e;
             if (Srow && lane < n) Srow[lane] = w;
             if (PACK) {
@@ -400,7 +399,7 @@ __device__ __forceinline__ void FusedWarp<T>::softmax_span(const ItemDesc& d, in
             float s = 0.f;
             for (int jj = lane; jj < n; jj += 32) { const float e = exp2f(zq[jj] - m); zq[jj] = e; s += e; }
             s = warp_sum(s);
-            part_m[qi] = m; part_l[qi] = s;
+            if (n_spans > 1 && lane == 0) { d.part[qi] = m; d.part[NQ + qi] = s; }
             const float inv = (n_spans == 1) ? 1.0f / s : 1.0f;
             for (int j0 = 0; j0 < n_pad; j0 += 32) {      // warp-uniform trip count
                 const int jj = j0 + lane;
@@ -431,6 +430,7 @@ __device__ bool FusedWarp<T>::process(const ItemDesc& d) {
     constexpr int HDR = (2 * NQ + 3) / 4 * 4;  // (max, sum) per query ahead of a span's partial sums
     const KindParams& kp = p.k[d.kind];
     const int n = d.j1 - d.j0, nq = d.nq, has_new = d.has_new, pi = d.pi;
+    const int g = lane / LPR, c = lane % LPR;   // row of a block this lane reads, and its 16-byte chunk
 
     // ---- key tiles: scores into zs.  The first tile also carries the query rows.
     float2 q2[NQ][NP];
@@ -485,9 +485,8 @@ __device__ bool FusedWarp<T>::process(const ItemDesc& d) {
     }
     __syncwarp();
 
-    float part_m[NQ], part_l[NQ];
     const int n_spans = d.n_spans;
-    softmax_span<NQ, false>(d, n, n, part_m, part_l);
+    softmax_span<NQ, false>(d, n, n);
 
     // ---- value tiles, layer by layer (score rows of absent queries hold zeros)
     const long long O_qstride = (long long)p.H * ROW_BYTES;
@@ -557,10 +556,6 @@ __device__ bool FusedWarp<T>::process(const ItemDesc& d) {
     if (n_spans == 1) return true;
 
     // ---- split row: park (max, sum); the last span to arrive combines all of them
-    if (lane == 0) {
-#pragma unroll
-        for (int qi = 0; qi < NQ; ++qi) { d.part[qi] = part_m[qi]; d.part[NQ + qi] = part_l[qi]; }
-    }
     __threadfence();
     __syncwarp();
     int t = 0;
@@ -639,9 +634,8 @@ __device__ bool FusedWarp<T>::process_mma(const ItemDesc& d) {
     }
     __syncwarp();
 
-    float part_m[NQ], part_l[NQ];
     const int n_spans = d.n_spans;
-    softmax_span<NQ, true>(d, n, (n + 15) & ~15, part_m, part_l);
+    softmax_span<NQ, true>(d, n, (n + 15) & ~15);
 
     // ---- value tiles, layer by layer
     // A fragments: the weights of query gid at positions b0 + {2tig, 2tig+1} and b0 + {2tig+8, 2tig+9},
@@ -666,14 +660,20 @@ __device__ bool FusedWarp<T>::process_mma(const ItemDesc& d) {
             const uint32_t st_s = ring + (uint32_t)(st - ring_g);
             for (int b0 = 0; b0 < r; b0 += 16) {
                 const uint2 w0 = za[(s0 + b0) >> 1], w1 = za[((s0 + b0) >> 1) + 4];    // (high, remainder) x 2
+                // the A operand of an MMA is four consecutive registers: build the two quads (high parts,
+                // remainders) once per block; rows 8..15 of A (registers 1 and 3) are padding queries
+                uint32_t ah[4], al[4];
+                ah[0] = w0.x; ah[2] = w1.x; al[0] = w0.y; al[2] = w1.y;
+                asm volatile("mov.b32 %0, 0;\n\tmov.b32 %1, 0;\n\tmov.b32 %2, 0;\n\tmov.b32 %3, 0;"
+                             : "=r"(ah[1]), "=r"(ah[3]), "=r"(al[1]), "=r"(al[3]));
 #pragma unroll
                 for (int x = 0; x < 4; ++x) {
                     uint32_t b[4];
                     ldsm_x4_t(st_s + b0 * 128 + ld_off[x], b);
-                    mma_bf16(acc[2 * x], w0.x, 0u, w1.x, 0u, b[0], b[1]);
-                    mma_bf16(acc[2 * x + 1], w0.x, 0u, w1.x, 0u, b[2], b[3]);
-                    mma_bf16(acc[2 * x], w0.y, 0u, w1.y, 0u, b[0], b[1]);
-                    mma_bf16(acc[2 * x + 1], w0.y, 0u, w1.y, 0u, b[2], b[3]);
+                    mma_bf16(acc[2 * x], ah[0], ah[1], ah[2], ah[3], b[0], b[1]);
+                    mma_bf16(acc[2 * x + 1], ah[0], ah[1], ah[2], ah[3], b[2], b[3]);
+                    mma_bf16(acc[2 * x], al[0], al[1], al[2], al[3], b[0], b[1]);
+                    mma_bf16(acc[2 * x + 1], al[0], al[1], al[2], al[3], b[2], b[3]);
                 }
             }
             release();
@@ -694,10 +694,6 @@ __device__ bool FusedWarp<T>::process_mma(const ItemDesc& d) {
     }
     if (n_spans == 1) return true;
 
-    if (lane == 0) {
-#pragma unroll
-        for (int qi = 0; qi < NQ; ++qi) { d.part[qi] = part_m[qi]; d.part[NQ + qi] = part_l[qi]; }
-    }
     __threadfence();
     __syncwarp();
     int t = 0;
@@ -836,7 +832,7 @@ __global__ void __launch_bounds__(kFusedWarps * 32, 1) decode_step_kernel(const 
     w.bars = smem_u32(bars_all + (size_t)warp * kFusedStages);
     w.zs = zs_all + (size_t)warp * kZFloats;
     w.descs = descs; w.q_next = &q_next;
-    w.lane = lane; w.g = lane / RowGeom<T>::LPR; w.c = lane % RowGeom<T>::LPR;
+    w.lane = lane;
     w.p_stage = 0; w.c_stage = 0; w.c_par = 0; w.dead = false; w.p_active = false; w.tile_written = false;
     if (lane == 0) {
         for (int s = 0; s < kFusedStages; ++s) mbar_init(bars_all + (size_t)warp * kFusedStages + s, 1);
