@@ -82,6 +82,12 @@ struct ItemDesc {
     int kind, nq, pi, len, j0, j1, n_spans, span, has_new, lead;
 };
 
+// The kernel's dynamic shared memory.  Everything a warp keeps there is addressed by a 32-bit
+// byte offset into this array, so that the compiler emits shared-space loads and stores with
+// 32-bit address arithmetic instead of generic 64-bit pointers.
+extern __shared__ __align__(128) unsigned char san_smem[];
+template <typename U> __device__ __forceinline__ U* sp(uint32_t off) { return reinterpret_cast<U*>(san_smem + off); }
+
 // ------------------------------------------------------------------------------ PTX helpers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -226,10 +232,10 @@ struct FusedWarp {
     static constexpr int UN = BLK / RPW;     // loads per lane per block
 
     const StepParams& p;
-    uint32_t ring, bars;          // shared-space addresses: stages and their barriers
-    const char* ring_g;           // the same stages through a generic pointer
-    float* zs;                    // kZFloats floats
-    const ItemDesc* descs;        // the CTA's decoded items
+    uint32_t sm_base;             // shared-space address of san_smem (for PTX operands: address = sm_base + offset)
+    uint32_t ring, bars;          // offsets of this warp's stages and of their barriers
+    uint32_t zs_off;              // offset of its kZFloats score slots
+    uint32_t descs_off;           // offset of the CTA's decoded items
     unsigned* q_next;             // shared counter: next of them to hand out
     unsigned n_valid;             // how many there are
     int lane;
@@ -261,7 +267,7 @@ struct FusedWarp {
         fifo |= (unsigned long long)p_idx << (8 * fifo_n);
         fifo_n += 1;
         nx_idx = grab();
-        const ItemDesc& d = descs[p_idx];
+        const ItemDesc& d = *sp<ItemDesc>(descs_off + p_idx * (uint32_t)sizeof(ItemDesc));
         p_which = 0; p_pi = d.pi; p_n_pos = d.j1 - d.j0; p_left = p_n_pos; p_has_new = d.has_new;
         p_nq = d.nq; p_kind = d.kind;
         p_src = d.Kp + (long long)d.j0 * ROW_BYTES;
@@ -274,9 +280,9 @@ struct FusedWarp {
         const bool first = (p_which == 0 && p_left == p_n_pos);
         const int r = min(first ? QROW : TR, p_left);
         if (lane == 0) {
-            const ItemDesc& d = descs[p_idx];
-            const uint32_t dst = ring + p_stage * kStageBytes;
-            const uint32_t bar = bars + p_stage * 8;
+            const ItemDesc& d = *sp<ItemDesc>(descs_off + p_idx * (uint32_t)sizeof(ItemDesc));
+            const uint32_t dst = sm_base + ring + p_stage * kStageBytes;
+            const uint32_t bar = sm_base + bars + p_stage * 8;
             const bool with_new = p_has_new && (r == p_left);
             const int r_cache = with_new ? r - 1 : r;
             mbar_expect_tx(bar, (uint32_t)((r + (first ? p_nq : 0)) * ROW_BYTES));
@@ -295,24 +301,25 @@ struct FusedWarp {
         p_src += (long long)r * ROW_BYTES;
         if (p_left <= 0) {
             if (p_which == p_pi) { next_item(); return; }
-            const ItemDesc& d = descs[p_idx];                       // on to the value panel of layer p_which
+            const ItemDesc& d = *sp<ItemDesc>(descs_off + p_idx * (uint32_t)sizeof(ItemDesc));   // on to the value panel of layer p_which
             p_src = d.Vp + (long long)p_which * p.k[p_kind].plane_bytes + (long long)d.j0 * ROW_BYTES;
             p_which += 1;
             p_left = p_n_pos;
         }
     }
 
-    // Waits for the next tile in order; returns its stage or null after a timeout.
-    __device__ __forceinline__ const char* acquire() {
-        const uint32_t bar = bars + c_stage * 8;
+    // Waits for the next tile in order; returns the offset of its stage, or kNoTile after a timeout.
+    static constexpr uint32_t kNoTile = 0xffffffffu;
+    __device__ __forceinline__ uint32_t acquire() {
+        const uint32_t bar = sm_base + bars + c_stage * 8;
         if (!mbar_try_wait(bar, c_par)) {
             if (!mbar_wait_slow(bar, c_par)) {
                 if (lane == 0 && atomicCAS(&p.err[0], 0, (int)SAN_ERR_TIMEOUT) == 0) { p.err[1] = TAG_STEP; p.err[2] = (int)c_stage; }
                 dead = true;
-                return nullptr;
+                return kNoTile;
             }
         }
-        return ring_g + c_stage * kStageBytes;
+        return ring + c_stage * kStageBytes;
     }
     // Every lane is done with the tile: its stage takes the next tile to be issued.
     __device__ __forceinline__ void release() {
@@ -333,25 +340,29 @@ struct FusedWarp {
     // order from the caller's buffer: permute its chunks like a cached row (chunk c -> c ^ (pos & 7))
     // and write it to the cache at `dst_row`.  Rows [r, next multiple of 16) are zeroed when
     // `zero_tail` is set, so that a 16-row block never multiplies stale shared memory.
-    __device__ __forceinline__ void fix_tile(const char* st, int r, bool with_new, char* dst_row, bool zero_tail) {
+    __device__ __forceinline__ void fix_tile(uint32_t st, int r, bool with_new, char* dst_row, bool zero_tail) {
         tile_written = true;
         if (with_new) {
-            char* row = const_cast<char*>(st) + (r - 1) * 128;
+            const uint32_t row = st + (r - 1) * 128;
             uint4 v = make_uint4(0, 0, 0, 0);
-            if (lane < 8) v = *reinterpret_cast<const uint4*>(row + lane * 16);
+            if (lane < 8) v = *sp<uint4>(row + lane * 16);
             __syncwarp();
             if (lane < 8) {
                 const int pc = lane ^ ((r - 1) & 7);
-                *reinterpret_cast<uint4*>(row + pc * 16) = v;
+                *sp<uint4>(row + pc * 16) = v;
                 if (dst_row) *reinterpret_cast<uint4*>(dst_row + pc * 16) = v;
             }
         }
-        if (zero_tail && (r & 15)) {
+        if (zero_tail && (r & 15)) {     // at most 15 rows: four rows per pass, 8 lanes per row
             const int r16 = (r + 15) & ~15;
-            for (int j = r + (lane >> 3); j < r16; j += 4)
-                *reinterpret_cast<uint4*>(const_cast<char*>(st) + j * 128 + (lane & 7) * 16) = make_uint4(0, 0, 0, 0);
+            const uint32_t at = st + (lane >> 3) * 128 + (lane & 7) * 16;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int j = r + 4 * k + (lane >> 3);
+                if (j < r16) *sp<uint4>(at + (r + 4 * k) * 128) = make_uint4(0, 0, 0, 0);
+            }
         }
-        if (with_new || (zero_tail && (r & 15))) __syncwarp();
+        __syncwarp();
     }
 };
 
@@ -370,7 +381,7 @@ __device__ __forceinline__ void FusedWarp<T>::softmax_span(const ItemDesc& d, in
 #pragma unroll
     for (int qi = 0; qi < NQ; ++qi) {
         if (qi >= nq) break;                 // rows of absent queries are never stored
-        float* zq = zs + qi * ZQ;
+        float* zq = sp<float>(zs_off + qi * ZQ * 4);
         unsigned short* zh = reinterpret_cast<unsigned short*>(zq);
         float* Srow = d.S ? d.S + qi * S_qstride + d.j0 : nullptr;
         if (n <= 32) {      // one score per lane: no loops
@@ -431,12 +442,14 @@ __device__ bool FusedWarp<T>::process(const ItemDesc& d) {
     const KindParams& kp = p.k[d.kind];
     const int n = d.j1 - d.j0, nq = d.nq, has_new = d.has_new, pi = d.pi;
     const int g = lane / LPR, c = lane % LPR;   // row of a block this lane reads, and its 16-byte chunk
+    float* zs = sp<float>(zs_off);
 
     // ---- key tiles: scores into zs.  The first tile also carries the query rows.
     float2 q2[NQ][NP];
     for (int s0 = 0; s0 < n;) {
-        const char* st = acquire();
-        if (!st) return false;
+        const uint32_t st_o = acquire();
+        if (st_o == kNoTile) return false;
+        const char* st = sp<char>(st_o);
         const int r = min(s0 == 0 ? QROW : TR, n - s0);
         if (s0 == 0) {
             const float sc = p.scale_log2e;
@@ -497,8 +510,9 @@ __device__ bool FusedWarp<T>::process(const ItemDesc& d) {
 #pragma unroll
             for (int e = 0; e < NP; ++e) acc[qi][e] = make_float2(0.f, 0.f);
         for (int s0 = 0; s0 < n; s0 += TR) {
-            const char* st = acquire();
-            if (!st) return false;
+            const uint32_t st_o = acquire();
+            if (st_o == kNoTile) return false;
+            const char* st = sp<char>(st_o);
             const int r = min(TR, n - s0);
             const bool with_new = has_new && (s0 + r == n);
             for (int jb = 0; jb < r; jb += BLK) {
@@ -595,21 +609,21 @@ __device__ bool FusedWarp<T>::process_mma(const ItemDesc& d) {
     // (natural chunk order), read as B fragments (k = dims, n = query).
     uint32_t qb[4][2];
     const float sc = p.scale_log2e;
-    float* zk = zs + (2 * tig) * ZQ + gid;        // this lane's score slots: queries 2tig, 2tig+1; positions gid, gid+8
+    const uint32_t zk = zs_off + ((2 * tig) * ZQ + gid) * 4;   // this lane's score slots: queries 2tig, 2tig+1; positions gid, gid+8
     for (int s0 = 0; s0 < n;) {
-        const char* st = acquire();
-        if (!st) return false;
+        const uint32_t st = acquire();
+        if (st == kNoTile) return false;
         const int r = min(s0 == 0 ? QROW : TR, n - s0);
         if (s0 == 0) {
-            const char* qrow = st + (QROW + (gid < nq ? gid : 0)) * 128 + 4 * tig;
+            const uint32_t qrow = st + (QROW + (gid < nq ? gid : 0)) * 128 + 4 * tig;
 #pragma unroll
             for (int ks = 0; ks < 4; ++ks) {
-                qb[ks][0] = *reinterpret_cast<const uint32_t*>(qrow + 32 * ks);
-                qb[ks][1] = *reinterpret_cast<const uint32_t*>(qrow + 32 * ks + 16);
+                qb[ks][0] = *sp<uint32_t>(qrow + 32 * ks);
+                qb[ks][1] = *sp<uint32_t>(qrow + 32 * ks + 16);
             }
         }
         if (has_new && s0 + r == n) fix_tile(st, r, true, d.lead ? const_cast<char*>(d.Kp) + (long long)(d.len - 1) * 128 : nullptr, false);
-        const uint32_t st_s = ring + (uint32_t)(st - ring_g);
+        const uint32_t st_s = sm_base + st;
         for (int b0 = 0; b0 < r; b0 += 16) {
             float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
@@ -619,7 +633,7 @@ __device__ bool FusedWarp<T>::process_mma(const ItemDesc& d) {
                 mma_bf16(acc, a[0], a[1], a[2], a[3], qb[ks][0], qb[ks][1]);
             }
             // acc[0], acc[1]: position b0+gid, queries 2tig, 2tig+1; acc[2], acc[3]: position b0+gid+8
-            float* z = zk + s0 + b0;
+            float* z = sp<float>(zk + (s0 + b0) * 4);
             if (2 * tig < NQ) {
                 if (b0 + gid < r) z[0] = acc[0] * sc;
                 if (b0 + gid + 8 < r) z[8] = acc[2] * sc;
@@ -640,7 +654,7 @@ __device__ bool FusedWarp<T>::process_mma(const ItemDesc& d) {
     // ---- value tiles, layer by layer
     // A fragments: the weights of query gid at positions b0 + {2tig, 2tig+1} and b0 + {2tig+8, 2tig+9},
     // high parts and remainders, straight from the packed words
-    const uint2* za = reinterpret_cast<const uint2*>(zs + (gid < NQ ? gid : 0) * ZQ) + tig;
+    const uint32_t za = zs_off + (gid < NQ ? gid : 0) * ZQ * 4 + tig * 8;
     const KindParams& kp = p.k[d.kind];
     const long long plane_bytes = kp.plane_bytes, layer_bytes = kp.layer_bytes;
     char* vlast = const_cast<char*>(d.Vp) + (long long)(d.len - 1) * 128;      // where this step's value row goes
@@ -652,14 +666,14 @@ __device__ bool FusedWarp<T>::process_mma(const ItemDesc& d) {
 #pragma unroll
             for (int e = 0; e < 4; ++e) acc[nt][e] = 0.f;
         for (int s0 = 0; s0 < n; s0 += TR) {
-            const char* st = acquire();
-            if (!st) return false;
+            const uint32_t st = acquire();
+            if (st == kNoTile) return false;
             const int r = min(TR, n - s0);
             const bool with_new = has_new && (s0 + r == n);
             if (with_new || (r & 15)) fix_tile(st, r, with_new, vlast, true);
-            const uint32_t st_s = ring + (uint32_t)(st - ring_g);
+            const uint32_t st_s = sm_base + st;
             for (int b0 = 0; b0 < r; b0 += 16) {
-                const uint2 w0 = za[(s0 + b0) >> 1], w1 = za[((s0 + b0) >> 1) + 4];    // (high, remainder) x 2
+                const uint2 w0 = *sp<uint2>(za + (s0 + b0) * 4), w1 = *sp<uint2>(za + (s0 + b0) * 4 + 32);    // (high, remainder) x 2
                 // the A operand of an MMA is four consecutive registers: build the two quads (high parts,
                 // remainders) once per block; rows 8..15 of A (registers 1 and 3) are padding queries
                 uint32_t ah[4], al[4];
@@ -715,6 +729,7 @@ __device__ void FusedWarp<T>::combine(const ItemDesc& d) {
     const int span_len = (int)kp.span;
     const long long S_qstride = (long long)p.H * kp.S_ld, O_qstride = (long long)p.H * ROW_BYTES;
     // zs[sp * NQ + qi] = exp2(m_sp - M) / total  (zs is free: every layer of this span is done)
+    float* zs = sp<float>(zs_off);
     __syncwarp();
     for (int qi = 0; qi < NQ; ++qi) {
         float m = -INFINITY, l = 0.f;
@@ -738,20 +753,20 @@ __device__ void FusedWarp<T>::combine(const ItemDesc& d) {
         if (qi >= nq) continue;
         float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
         const float* src = row_part + HDR + e0;
-        int sp = 0;
-        for (; sp + 4 <= n_spans; sp += 4) {
+        int sn = 0;
+        for (; sn + 4 <= n_spans; sn += 4) {
             float4 x[4];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) x[u] = __ldcg(reinterpret_cast<const float4*>(src + (long long)(sp + u) * stride));
+            for (int u = 0; u < 4; ++u) x[u] = __ldcg(reinterpret_cast<const float4*>(src + (long long)(sn + u) * stride));
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
-                const float f = zs[(sp + u) * NQ + qi];
+                const float f = zs[(sn + u) * NQ + qi];
                 a.x = fmaf(f, x[u].x, a.x); a.y = fmaf(f, x[u].y, a.y); a.z = fmaf(f, x[u].z, a.z); a.w = fmaf(f, x[u].w, a.w);
             }
         }
-        for (; sp < n_spans; ++sp) {
-            const float4 x = __ldcg(reinterpret_cast<const float4*>(src + (long long)sp * stride));
-            const float f = zs[sp * NQ + qi];
+        for (; sn < n_spans; ++sn) {
+            const float4 x = __ldcg(reinterpret_cast<const float4*>(src + (long long)sn * stride));
+            const float f = zs[sn * NQ + qi];
             a.x = fmaf(f, x.x, a.x); a.y = fmaf(f, x.y, a.y); a.z = fmaf(f, x.z, a.z); a.w = fmaf(f, x.w, a.w);
         }
         const int ly = e0 / (NQ * kDh), col = e0 % kDh;
@@ -775,8 +790,6 @@ constexpr size_t fused_smem_bytes() {
 
 template <typename T, int NQE>
 __global__ void __launch_bounds__(kFusedWarps * 32, 1) decode_step_kernel(const __grid_constant__ StepParams p) {
-    extern __shared__ __align__(128) unsigned char smem[];
-    __shared__ unsigned cta_next;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 
     // ---- AAN running average (Table 6 pairing): element-wise, every thread of the grid
@@ -800,10 +813,10 @@ __global__ void __launch_bounds__(kFusedWarps * 32, 1) decode_step_kernel(const 
                 const float4 raw = *reinterpret_cast<const float4*>(p.x_aan + io * 4);
                 xv[0] = raw.x; xv[1] = raw.y; xv[2] = raw.z; xv[3] = raw.w;
             }
-            float4* sp = reinterpret_cast<float4*>(p.aan_sum + ((long long)lr * p.aan_max_seqs + id) * d + c4 * 4);
-            float4 s = (t == 1) ? make_float4(0.f, 0.f, 0.f, 0.f) : *sp;
+            float4* sum = reinterpret_cast<float4*>(p.aan_sum + ((long long)lr * p.aan_max_seqs + id) * d + c4 * 4);
+            float4 s = (t == 1) ? make_float4(0.f, 0.f, 0.f, 0.f) : *sum;
             s.x += xv[0]; s.y += xv[1]; s.z += xv[2]; s.w += xv[3];
-            *sp = s;
+            *sum = s;
             const float ft = (float)t;
             const float o[4] = {s.x / ft, s.y / ft, s.z / ft, s.w / ft};
             if (sizeof(T) == 2) {
@@ -821,21 +834,22 @@ __global__ void __launch_bounds__(kFusedWarps * 32, 1) decode_step_kernel(const 
     // of kCtaItems slots: every thread decodes one slot, the survivors are packed in list order
     // (big items first), then the warps drain them through a shared counter.
     __shared__ unsigned q_next, n_valid, warp_count[kFusedWarps];
-    char* base = reinterpret_cast<char*>(smem);
-    float* zs_all = reinterpret_cast<float*>(base + (size_t)kFusedWarps * kFusedStages * kStageBytes);
-    uint64_t* bars_all = reinterpret_cast<uint64_t*>(reinterpret_cast<char*>(zs_all) + (size_t)kFusedWarps * kZFloats * sizeof(float));
-    ItemDesc* descs = reinterpret_cast<ItemDesc*>(reinterpret_cast<char*>(bars_all) + (size_t)kFusedWarps * kFusedStages * sizeof(uint64_t));
+    // layout of san_smem: the warps' rings, their score slots, their barriers, the CTA's items
+    constexpr uint32_t kZsAll = kFusedWarps * kFusedStages * kStageBytes;
+    constexpr uint32_t kBarsAll = kZsAll + kFusedWarps * kZFloats * (uint32_t)sizeof(float);
+    constexpr uint32_t kDescsAll = kBarsAll + kFusedWarps * kFusedStages * (uint32_t)sizeof(uint64_t);
+    ItemDesc* descs = sp<ItemDesc>(kDescsAll);
 
     FusedWarp<T> w(p);
-    w.ring_g = base + (size_t)warp * kFusedStages * kStageBytes;
-    w.ring = smem_u32(w.ring_g);
-    w.bars = smem_u32(bars_all + (size_t)warp * kFusedStages);
-    w.zs = zs_all + (size_t)warp * kZFloats;
-    w.descs = descs; w.q_next = &q_next;
+    w.sm_base = smem_u32(san_smem);
+    w.ring = (uint32_t)warp * kFusedStages * kStageBytes;
+    w.bars = kBarsAll + (uint32_t)warp * kFusedStages * 8;
+    w.zs_off = kZsAll + (uint32_t)warp * kZFloats * 4;
+    w.descs_off = kDescsAll; w.q_next = &q_next;
     w.lane = lane;
     w.p_stage = 0; w.c_stage = 0; w.c_par = 0; w.dead = false; w.p_active = false; w.tile_written = false;
     if (lane == 0) {
-        for (int s = 0; s < kFusedStages; ++s) mbar_init(bars_all + (size_t)warp * kFusedStages + s, 1);
+        for (int s = 0; s < kFusedStages; ++s) mbar_init(sp<uint64_t>(w.bars + s * 8), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
