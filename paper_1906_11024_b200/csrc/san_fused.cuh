@@ -72,14 +72,18 @@ struct StepParams {
 // A decoded work item, kept in shared memory between the copy side and the math side.
 struct ItemDesc {
     const char* q;                            // query row 0
-    const char* Kp;                           // key panel, row 0
-    const char* Vp;                           // value panel of the block's first layer, row 0
-    const char* knew; const char* vnew;       // newest rows (self only)
-    float* S;                                 // S row of query 0 (may be null)
+    const char* srcK;                         // key panel, first row of the span
+    const char* srcV;                         // value panel of the item's first layer, first row of the span
+    const char* knew; const char* vnew;       // newest rows (self only): key row; value row of the item's first layer
+    float* S;                                 // S row of query 0 at the span's first position (null: not stored)
     char* O;                                  // output of (first layer, query 0)
     float* part;                              // partial sums of this (row, span)
     unsigned row_id;                          // ticket index of the row
-    int kind, nq, pi, len, j0, j1, n_spans, span, has_new, lead;
+    int n;                                    // positions in the span
+    int len;                                  // positions in the whole row
+    int kind, nq, pi, n_spans, span;
+    int has_new;                              // the span's last position is this step's row, not yet in the cache
+    int lead;                                 // this item also stores the key row of the step
 };
 
 // The kernel's dynamic shared memory.  Everything a warp keeps there is addressed by a 32-bit
@@ -200,16 +204,16 @@ __device__ bool decode_item(const StepParams& p, unsigned it, ItemDesc* d) {
     const unsigned qrow = ((block * kp.n_it + item) * kp.nq) * H + h;          // row of query 0 in q and S
     const unsigned long long panel = (unsigned long long)((unsigned)id * H + h) * kp.panel_bytes;
     d->kind = enc; d->nq = (int)kp.nq; d->pi = (int)min(kp.lg_size, size - l0);
-    d->len = len; d->j0 = j0; d->j1 = j1;
+    d->len = len; d->n = j1 - j0;
     d->n_spans = (len + (int)kp.span - 1) / (int)kp.span; d->span = (int)span;
     d->has_new = (kp.knew != nullptr && j1 == len) ? 1 : 0;
     d->lead = (lg == 0) ? 1 : 0;                      // the group that also stores S and this step's key row
     d->row_id = kp.row_base + rl;
     d->part = p.part + kp.part_base + (unsigned long long)(rl * kp.nspans + span) * kp.part_stride;
     d->q = kp.q + (unsigned long long)qrow * ROW_BYTES;
-    d->S = (kp.S && lg == 0) ? kp.S + (unsigned long long)qrow * (unsigned long long)kp.S_ld : nullptr;
-    d->Kp = kp.K + (unsigned long long)block * (unsigned long long)kp.plane_bytes + panel;
-    d->Vp = kp.V + (unsigned long long)vplane * (unsigned long long)kp.plane_bytes + panel;
+    d->S = (kp.S && lg == 0) ? kp.S + (unsigned long long)qrow * (unsigned long long)kp.S_ld + j0 : nullptr;
+    d->srcK = kp.K + (unsigned long long)block * (unsigned long long)kp.plane_bytes + panel + (unsigned)j0 * ROW_BYTES;
+    d->srcV = kp.V + (unsigned long long)vplane * (unsigned long long)kp.plane_bytes + panel + (unsigned)j0 * ROW_BYTES;
     d->O = kp.O + (unsigned long long)vplane * (unsigned long long)kp.layer_bytes +
            (unsigned long long)((item * kp.nq) * H + h) * ROW_BYTES;
     const unsigned long long in_row = (unsigned long long)(item * H + h) * ROW_BYTES;   // self: nq == 1
@@ -219,6 +223,9 @@ __device__ bool decode_item(const StepParams& p, unsigned it, ItemDesc* d) {
 }
 
 // ------------------------------------------------------------------------------ the warp
+template <typename T, int NQ>
+__device__ void combine_spans(const StepParams& p, const ItemDesc& d, uint32_t zs_off, int lane);
+
 template <typename T>
 struct FusedWarp {
     using G = RowGeom<T>;
@@ -236,22 +243,29 @@ struct FusedWarp {
     uint32_t ring, bars;          // offsets of this warp's stages and of their barriers
     uint32_t zs_off;              // offset of its kZFloats score slots
     uint32_t descs_off;           // offset of the CTA's decoded items
+    uint32_t zero_row;            // shared-space address of 128 zero bytes
     unsigned* q_next;             // shared counter: next of them to hand out
     unsigned n_valid;             // how many there are
     int lane;
     // copy side: the item whose tiles are being issued, and the one after (taken ahead)
     bool p_active;
+    bool p_first;                 // the next tile is the item's first key tile
     unsigned p_idx, nx_idx, p_stage;
-    int p_which, p_pi, p_n_pos, p_left, p_has_new, p_nq, p_kind;
-    const char* p_src;
+    int p_which;                  // panel being issued: 0 = keys, l + 1 = values of the item's layer l
+    int p_pi, p_n, p_left, p_has_new, p_nq, p_kind;
+    const char* p_src;            // next rows of the panel
+    const char* p_new;            // this step's row of the panel (self only)
     // math side
     unsigned c_stage, c_par;
     unsigned long long fifo;      // items whose tiles are (being) issued and whose arithmetic is still to do,
     int fifo_n;                   // oldest in the low byte (item indices are below kCtaItems <= 255)
     bool dead;                    // a wait ran out: leave
-    bool tile_written;            // the math side wrote into the current tile (see release)
 
     __device__ FusedWarp(const StepParams& pp) : p(pp) {}
+
+    __device__ __forceinline__ const ItemDesc& desc(unsigned idx) const {
+        return *sp<ItemDesc>(descs_off + idx * (uint32_t)sizeof(ItemDesc));
+    }
 
     __device__ __forceinline__ unsigned grab() {
         unsigned k = 0;
@@ -267,44 +281,47 @@ struct FusedWarp {
         fifo |= (unsigned long long)p_idx << (8 * fifo_n);
         fifo_n += 1;
         nx_idx = grab();
-        const ItemDesc& d = *sp<ItemDesc>(descs_off + p_idx * (uint32_t)sizeof(ItemDesc));
-        p_which = 0; p_pi = d.pi; p_n_pos = d.j1 - d.j0; p_left = p_n_pos; p_has_new = d.has_new;
+        const ItemDesc& d = desc(p_idx);
+        p_which = 0; p_first = true; p_pi = d.pi; p_n = d.n; p_left = p_n; p_has_new = d.has_new;
         p_nq = d.nq; p_kind = d.kind;
-        p_src = d.Kp + (long long)d.j0 * ROW_BYTES;
+        p_src = d.srcK; p_new = d.knew;
     }
 
     // Issues the copies of one tile of the item being issued, if any is left.  The first key
     // tile of an item has room for QROW key rows and carries the query rows behind them.
     __device__ __forceinline__ void produce() {
         if (!p_active) return;
-        const bool first = (p_which == 0 && p_left == p_n_pos);
-        const int r = min(first ? QROW : TR, p_left);
+        const int r = min(p_first ? QROW : TR, p_left);
+        const bool with_new = p_has_new && (r == p_left);      // this step's row closes the panel
+        const uint32_t cache_bytes = (uint32_t)(r - (with_new ? 1 : 0)) * ROW_BYTES;
         if (lane == 0) {
-            const ItemDesc& d = *sp<ItemDesc>(descs_off + p_idx * (uint32_t)sizeof(ItemDesc));
             const uint32_t dst = sm_base + ring + p_stage * kStageBytes;
             const uint32_t bar = sm_base + bars + p_stage * 8;
-            const bool with_new = p_has_new && (r == p_left);
-            const int r_cache = with_new ? r - 1 : r;
-            mbar_expect_tx(bar, (uint32_t)((r + (first ? p_nq : 0)) * ROW_BYTES));
-            if (r_cache > 0) bulk_g2s(dst, p_src, (uint32_t)(r_cache * ROW_BYTES), bar);
-            if (with_new) {     // this step's row of the panel: keys, or values of layer p_which - 1
-                const char* nsrc = p_which == 0 ? d.knew : d.vnew + (long long)(p_which - 1) * p.k[p_kind].layer_bytes;
-                bulk_g2s(dst + r_cache * ROW_BYTES, nsrc, ROW_BYTES, bar);
-            }
-            if (first) {        // the query rows ride behind the first key tile
+            mbar_expect_tx(bar, (uint32_t)(r + (p_first ? p_nq : 0)) * ROW_BYTES);
+            if (cache_bytes) bulk_g2s(dst, p_src, cache_bytes, bar);
+            if (with_new) bulk_g2s(dst + cache_bytes, p_new, ROW_BYTES, bar);
+            if (p_first) {      // the query rows ride behind the first key tile
+                const char* q = desc(p_idx).q;
                 const unsigned q_stride = (unsigned)p.H * ROW_BYTES;
-                for (int qi = 0; qi < p_nq; ++qi) bulk_g2s(dst + (QROW + qi) * ROW_BYTES, d.q + (size_t)qi * q_stride, ROW_BYTES, bar);
+#pragma unroll 1
+                for (int qi = 0; qi < p_nq; ++qi, q += q_stride) bulk_g2s(dst + (QROW + qi) * ROW_BYTES, q, ROW_BYTES, bar);
             }
         }
+        p_first = false;
         p_stage = (p_stage + 1 == (unsigned)kFusedStages) ? 0 : p_stage + 1;
         p_left -= r;
-        p_src += (long long)r * ROW_BYTES;
+        p_src += (uint32_t)r * ROW_BYTES;
         if (p_left <= 0) {
             if (p_which == p_pi) { next_item(); return; }
-            const ItemDesc& d = *sp<ItemDesc>(descs_off + p_idx * (uint32_t)sizeof(ItemDesc));   // on to the value panel of layer p_which
-            p_src = d.Vp + (long long)p_which * p.k[p_kind].plane_bytes + (long long)d.j0 * ROW_BYTES;
+            if (p_which == 0) {                                 // on to the value panel of the item's first layer
+                const ItemDesc& d = desc(p_idx);
+                p_src = d.srcV; p_new = d.vnew;
+            } else {                                            // the same rows of the next layer's plane
+                p_src += p.k[p_kind].plane_bytes - (long long)((uint32_t)p_n * ROW_BYTES);
+                p_new += p.k[p_kind].layer_bytes;
+            }
             p_which += 1;
-            p_left = p_n_pos;
+            p_left = p_n;
         }
     }
 
@@ -321,11 +338,9 @@ struct FusedWarp {
         }
         return ring + c_stage * kStageBytes;
     }
-    // Every lane is done with the tile: its stage takes the next tile to be issued.
+    // Every lane is done with the tile (tiles are only ever read): its stage takes the next
+    // tile to be issued.
     __device__ __forceinline__ void release() {
-        // the tensor-core path writes into its tiles (chunk-permuting the newest row, zeroing a
-        // ragged tail): order those writes ahead of the bulk copy that will reuse the stage
-        if (tile_written) { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); tile_written = false; }
         __syncwarp();
         if (++c_stage == (unsigned)kFusedStages) { c_stage = 0; c_par ^= 1u; }
         produce();
@@ -333,37 +348,7 @@ struct FusedWarp {
 
     template <int NQ> __device__ bool process(const ItemDesc& d);
     template <int NQ> __device__ bool process_mma(const ItemDesc& d);
-    template <int NQ> __device__ void combine(const ItemDesc& d);
     template <int NQ, bool PACK> __device__ __forceinline__ void softmax_span(const ItemDesc& d, int n, int n_pad);
-
-    // bf16 tiles only.  A tile's last row may be this step's new row, copied in natural chunk
-    // order from the caller's buffer: permute its chunks like a cached row (chunk c -> c ^ (pos & 7))
-    // and write it to the cache at `dst_row`.  Rows [r, next multiple of 16) are zeroed when
-    // `zero_tail` is set, so that a 16-row block never multiplies stale shared memory.
-    __device__ __forceinline__ void fix_tile(uint32_t st, int r, bool with_new, char* dst_row, bool zero_tail) {
-        tile_written = true;
-        if (with_new) {
-            const uint32_t row = st + (r - 1) * 128;
-            uint4 v = make_uint4(0, 0, 0, 0);
-            if (lane < 8) v = *sp<uint4>(row + lane * 16);
-            __syncwarp();
-            if (lane < 8) {
-                const int pc = lane ^ ((r - 1) & 7);
-                *sp<uint4>(row + pc * 16) = v;
-                if (dst_row) *reinterpret_cast<uint4*>(dst_row + pc * 16) = v;
-            }
-        }
-        if (zero_tail && (r & 15)) {     // at most 15 rows: four rows per pass, 8 lanes per row
-            const int r16 = (r + 15) & ~15;
-            const uint32_t at = st + (lane >> 3) * 128 + (lane & 7) * 16;
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const int j = r + 4 * k + (lane >> 3);
-                if (j < r16) *sp<uint4>(at + (r + 4 * k) * 128) = make_uint4(0, 0, 0, 0);
-            }
-        }
-        __syncwarp();
-    }
 };
 
 // Softmax of the n scores of a span held in zs (log2 domain), per query row.  A span that is
@@ -383,7 +368,7 @@ __device__ __forceinline__ void FusedWarp<T>::softmax_span(const ItemDesc& d, in
         if (qi >= nq) break;                 // rows of absent queries are never stored
         float* zq = sp<float>(zs_off + qi * ZQ * 4);
         unsigned short* zh = reinterpret_cast<unsigned short*>(zq);
-        float* Srow = d.S ? d.S + qi * S_qstride + d.j0 : nullptr;
+        float* Srow = d.S ? d.S + qi * S_qstride : nullptr;
         if (n <= 32) {      // one score per lane: no loops
             const float z = lane < n ? zq[lane] : -INFINITY;
             const float m = warp_max(z);
@@ -405,13 +390,16 @@ __device__ __forceinline__ void FusedWarp<T>::softmax_span(const ItemDesc& d, in
             }
         } else {
             float m = -INFINITY;
+#pragma unroll 1
             for (int jj = lane; jj < n; jj += 32) m = fmaxf(m, zq[jj]);
             m = warp_max(m);
             float s = 0.f;
+#pragma unroll 1
             for (int jj = lane; jj < n; jj += 32) { const float e = exp2f(zq[jj] - m); zq[jj] = e; s += e; }
             s = warp_sum(s);
             if (n_spans > 1 && lane == 0) { d.part[qi] = m; d.part[NQ + qi] = s; }
             const float inv = (n_spans == 1) ? 1.0f / s : 1.0f;
+#pragma unroll 1
             for (int j0 = 0; j0 < n_pad; j0 += 32) {      // warp-uniform trip count
                 const int jj = j0 + lane;
                 const float w = jj < n ? zq[jj] * inv : 0.f;
@@ -440,7 +428,7 @@ __device__ bool FusedWarp<T>::process(const ItemDesc& d) {
     constexpr int ZQ = kZFloats / NQ;          // score slots per query row
     constexpr int HDR = (2 * NQ + 3) / 4 * 4;  // (max, sum) per query ahead of a span's partial sums
     const KindParams& kp = p.k[d.kind];
-    const int n = d.j1 - d.j0, nq = d.nq, has_new = d.has_new, pi = d.pi;
+    const int n = d.n, nq = d.nq, has_new = d.has_new, pi = d.pi;
     const int g = lane / LPR, c = lane % LPR;   // row of a block this lane reads, and its 16-byte chunk
     float* zs = sp<float>(zs_off);
 
@@ -490,7 +478,7 @@ __device__ bool FusedWarp<T>::process(const ItemDesc& d) {
                 }
                 // the newest key row goes into the cache from here
                 if (with_new && d.lead && j == r - 1)
-                    *reinterpret_cast<uint4*>(const_cast<char*>(d.Kp) + (long long)(d.len - 1) * ROW_BYTES + c * 16) = kv[u];
+                    *reinterpret_cast<uint4*>(const_cast<char*>(d.srcK) + (n - 1) * ROW_BYTES + c * 16) = kv[u];
             }
         }
         s0 += r;
@@ -536,8 +524,8 @@ __device__ bool FusedWarp<T>::process(const ItemDesc& d) {
                             for (int e = 0; e < NP; ++e) acc[qi][e] = __ffma2_rn(ss, v2[e], acc[qi][e]);
                         }
                         if (with_new && j == r - 1)
-                            *reinterpret_cast<uint4*>(const_cast<char*>(d.Vp) + (long long)l * kp.plane_bytes +
-                                                      (long long)(d.len - 1) * ROW_BYTES + c * 16) = vv[u];
+                            *reinterpret_cast<uint4*>(const_cast<char*>(d.srcV) + (long long)l * kp.plane_bytes +
+                                                      (n - 1) * ROW_BYTES + c * 16) = vv[u];
                     }
                 }
             }
@@ -575,7 +563,7 @@ __device__ bool FusedWarp<T>::process(const ItemDesc& d) {
     int t = 0;
     if (lane == 0) t = atomicAdd(p.tickets + d.row_id, 1);
     t = __shfl_sync(0xffffffffu, t, 0);
-    if (t == n_spans - 1) combine<NQ>(d);
+    if (t == n_spans - 1) combine_spans<T, NQ>(p, d, zs_off, lane);
     return true;
 }
 
@@ -596,14 +584,17 @@ __device__ bool FusedWarp<T>::process_mma(const ItemDesc& d) {
     static_assert(sizeof(T) == 2, "tensor-core path is for bf16 rows");
     constexpr int ZQ = kZFloats / NQ;
     constexpr int HDR = (2 * NQ + 3) / 4 * 4;
-    const int n = d.j1 - d.j0, nq = d.nq, has_new = d.has_new, pi = d.pi;
+    const int n = d.n, nq = d.nq, has_new = d.has_new, pi = d.pi;
     const int tig = lane & 3, gid = lane >> 2;                 // mma fragment coordinates
-    // ldmatrix: this lane addresses row (lane & 7) + 8 * ((lane >> 3) & 1) of a 16-row block and,
-    // for the pair of 16-byte chunks 2x, 2x+1, the chunk 2x + (lane >> 4), permuted by the row
+    // ldmatrix: this lane addresses row lrow of a 16-row block and, for the pair of 16-byte
+    // chunks 2x, 2x+1, the chunk 2x + (lane >> 4).  Cached rows keep chunk c at c ^ (row & 7)
+    // (row & 7 == lane & 7 here); this step's own row arrives in natural order, so a lane that
+    // addresses it takes the permutation out again (new_fix).
+    const int lrow = (lane & 7) + ((lane >> 3) & 1) * 8;
+    const uint32_t new_fix = (uint32_t)(lane & 7) << 4;
     uint32_t ld_off[4];
 #pragma unroll
-    for (int x = 0; x < 4; ++x)
-        ld_off[x] = (uint32_t)(((lane & 7) + ((lane >> 3) & 1) * 8) * 128 + (((2 * x + (lane >> 4)) ^ (lane & 7)) << 4));
+    for (int x = 0; x < 4; ++x) ld_off[x] = (uint32_t)(lrow * 128 + (((2 * x + (lane >> 4)) ^ (lane & 7)) << 4));
 
     // ---- key tiles: scores into zs (log2 domain).  The first tile also carries the query rows
     // (natural chunk order), read as B fragments (k = dims, n = query).
@@ -622,25 +613,33 @@ __device__ bool FusedWarp<T>::process_mma(const ItemDesc& d) {
                 qb[ks][1] = *sp<uint32_t>(qrow + 32 * ks + 16);
             }
         }
-        if (has_new && s0 + r == n) fix_tile(st, r, true, d.lead ? const_cast<char*>(d.Kp) + (long long)(d.len - 1) * 128 : nullptr, false);
+        const int new_row = (has_new && s0 + r == n) ? r - 1 : -1;     // where this step's key row sits in the tile
+        if (new_row >= 0 && d.lead && lane < 8)                        // into the cache, chunk-permuted
+            *reinterpret_cast<uint4*>(const_cast<char*>(d.srcK) + (n - 1) * 128 + ((lane ^ (new_row & 7)) << 4)) =
+                *sp<uint4>(st + new_row * 128 + lane * 16);
         const uint32_t st_s = sm_base + st;
+#pragma unroll 1
         for (int b0 = 0; b0 < r; b0 += 16) {
+            const uint32_t fix = (b0 + lrow == new_row) ? new_fix : 0u;
             float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int ks = 0; ks < 4; ++ks) {
                 uint32_t a[4];
-                ldsm_x4(st_s + b0 * 128 + ld_off[ks], a);
+                ldsm_x4(st_s + b0 * 128 + (ld_off[ks] ^ fix), a);
                 mma_bf16(acc, a[0], a[1], a[2], a[3], qb[ks][0], qb[ks][1]);
             }
-            // acc[0], acc[1]: position b0+gid, queries 2tig, 2tig+1; acc[2], acc[3]: position b0+gid+8
+            // acc[0], acc[1]: position b0+gid, queries 2tig, 2tig+1; acc[2], acc[3]: position b0+gid+8.
+            // Rows of the block at or beyond r (the query rows of a first tile, stale bytes) give
+            // scores that the next tile overwrites; nothing is stored beyond the span.
+            const int pos = s0 + b0 + gid;
             float* z = sp<float>(zk + (s0 + b0) * 4);
             if (2 * tig < NQ) {
-                if (b0 + gid < r) z[0] = acc[0] * sc;
-                if (b0 + gid + 8 < r) z[8] = acc[2] * sc;
+                if (pos < n) z[0] = acc[0] * sc;
+                if (pos + 8 < n) z[8] = acc[2] * sc;
             }
             if (2 * tig + 1 < NQ) {
-                if (b0 + gid < r) z[ZQ] = acc[1] * sc;
-                if (b0 + gid + 8 < r) z[ZQ + 8] = acc[3] * sc;
+                if (pos < n) z[ZQ] = acc[1] * sc;
+                if (pos + 8 < n) z[ZQ + 8] = acc[3] * sc;
             }
         }
         s0 += r;
@@ -657,21 +656,25 @@ __device__ bool FusedWarp<T>::process_mma(const ItemDesc& d) {
     const uint32_t za = zs_off + (gid < NQ ? gid : 0) * ZQ * 4 + tig * 8;
     const KindParams& kp = p.k[d.kind];
     const long long plane_bytes = kp.plane_bytes, layer_bytes = kp.layer_bytes;
-    char* vlast = const_cast<char*>(d.Vp) + (long long)(d.len - 1) * 128;      // where this step's value row goes
+    char* vlast = const_cast<char*>(d.srcV) + (n - 1) * 128;      // where this step's value row goes
     char* op = d.O + gid * ((long long)p.H * 128) + 4 * tig;
+#pragma unroll 1
     for (int l = 0; l < pi; ++l) {
         float acc[8][4];
 #pragma unroll
         for (int nt = 0; nt < 8; ++nt)
 #pragma unroll
             for (int e = 0; e < 4; ++e) acc[nt][e] = 0.f;
+#pragma unroll 1
         for (int s0 = 0; s0 < n; s0 += TR) {
             const uint32_t st = acquire();
             if (st == kNoTile) return false;
             const int r = min(TR, n - s0);
-            const bool with_new = has_new && (s0 + r == n);
-            if (with_new || (r & 15)) fix_tile(st, r, with_new, vlast, true);
+            const int new_row = (has_new && s0 + r == n) ? r - 1 : -1;
+            if (new_row >= 0 && lane < 8)
+                *reinterpret_cast<uint4*>(vlast + ((lane ^ (new_row & 7)) << 4)) = *sp<uint4>(st + new_row * 128 + lane * 16);
             const uint32_t st_s = sm_base + st;
+#pragma unroll 1
             for (int b0 = 0; b0 < r; b0 += 16) {
                 const uint2 w0 = *sp<uint2>(za + (s0 + b0) * 4), w1 = *sp<uint2>(za + (s0 + b0) * 4 + 32);    // (high, remainder) x 2
                 // the A operand of an MMA is four consecutive registers: build the two quads (high parts,
@@ -680,10 +683,15 @@ __device__ bool FusedWarp<T>::process_mma(const ItemDesc& d) {
                 ah[0] = w0.x; ah[2] = w1.x; al[0] = w0.y; al[2] = w1.y;
                 asm volatile("mov.b32 %0, 0;\n\tmov.b32 %1, 0;\n\tmov.b32 %2, 0;\n\tmov.b32 %3, 0;"
                              : "=r"(ah[1]), "=r"(ah[3]), "=r"(al[1]), "=r"(al[3]));
+                // rows at or beyond r hold stale bytes: their weights are zero, but 0 x NaN would not be,
+                // so those lanes address a row of zeros instead
+                const int row = b0 + lrow;
+                const uint32_t fix = (row == new_row) ? new_fix : 0u;
+                const uint32_t blk = st_s + b0 * 128;
 #pragma unroll
                 for (int x = 0; x < 4; ++x) {
                     uint32_t b[4];
-                    ldsm_x4_t(st_s + b0 * 128 + ld_off[x], b);
+                    ldsm_x4_t(row < r ? blk + (ld_off[x] ^ fix) : zero_row, b);
                     mma_bf16(acc[2 * x], ah[0], ah[1], ah[2], ah[3], b[0], b[1]);
                     mma_bf16(acc[2 * x + 1], ah[0], ah[1], ah[2], ah[3], b[2], b[3]);
                     mma_bf16(acc[2 * x], al[0], al[1], al[2], al[3], b[0], b[1]);
@@ -713,15 +721,16 @@ __device__ bool FusedWarp<T>::process_mma(const ItemDesc& d) {
     int t = 0;
     if (lane == 0) t = atomicAdd(p.tickets + d.row_id, 1);
     t = __shfl_sync(0xffffffffu, t, 0);
-    if (t == n_spans - 1) combine<NQ>(d);
+    if (t == n_spans - 1) combine_spans<T, NQ>(p, d, zs_off, lane);
     return true;
 }
 
 // The last span of a split row: softmax weights across spans, then S and every layer's O.
-template <typename T>
-template <int NQ>
-__device__ void FusedWarp<T>::combine(const ItemDesc& d) {
+// Rare (split rows only) and long: kept out of line so that the hot loops stay small.
+template <typename T, int NQ>
+__device__ __noinline__ void combine_spans(const StepParams& p, const ItemDesc& d, uint32_t zs_off, int lane) {
     constexpr int HDR = (2 * NQ + 3) / 4 * 4;
+    constexpr int ROW_BYTES = FusedGeom<T>::ROW_BYTES;
     __threadfence();
     const KindParams& kp = p.k[d.kind];
     const int n_spans = d.n_spans, nq = d.nq, stride = (int)kp.part_stride;
@@ -742,18 +751,21 @@ __device__ void FusedWarp<T>::combine(const ItemDesc& d) {
     __syncwarp();
     if (d.S) {
         for (int qi = 0; qi < nq; ++qi) {
-            float* Srow = d.S + qi * S_qstride;
+            float* Srow = d.S - d.span * span_len + qi * S_qstride;      // d.S starts at this span's first position
+#pragma unroll 1
             for (int j = lane; j < d.len; j += 32) Srow[j] = __ldcg(Srow + j) * zs[(j / span_len) * NQ + qi];
         }
     }
     // every layer's output: E = pi*NQ*64 floats per span, four per lane per pass
     const int E = d.pi * NQ * kDh;
+#pragma unroll 1
     for (int e0 = lane * 4; e0 < E; e0 += 128) {
         const int qi = (e0 / kDh) % NQ;
         if (qi >= nq) continue;
         float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
         const float* src = row_part + HDR + e0;
         int sn = 0;
+#pragma unroll 1
         for (; sn + 4 <= n_spans; sn += 4) {
             float4 x[4];
 #pragma unroll
@@ -764,6 +776,7 @@ __device__ void FusedWarp<T>::combine(const ItemDesc& d) {
                 a.x = fmaf(f, x[u].x, a.x); a.y = fmaf(f, x[u].y, a.y); a.z = fmaf(f, x[u].z, a.z); a.w = fmaf(f, x[u].w, a.w);
             }
         }
+#pragma unroll 1
         for (; sn < n_spans; ++sn) {
             const float4 x = __ldcg(reinterpret_cast<const float4*>(src + (long long)sn * stride));
             const float f = zs[sn * NQ + qi];
@@ -785,7 +798,7 @@ __device__ void FusedWarp<T>::combine(const ItemDesc& d) {
 constexpr int kCtaItems = 144;      // decoded items a CTA holds at a time (at most 255: the warps queue them by byte)
 constexpr size_t fused_smem_bytes() {
     return (size_t)kFusedWarps * (kFusedStages * kStageBytes + kZFloats * sizeof(float) + kFusedStages * sizeof(uint64_t)) +
-           (size_t)kCtaItems * sizeof(ItemDesc) + 128;
+           128 /* a row of zeros */ + (size_t)kCtaItems * sizeof(ItemDesc);
 }
 
 template <typename T, int NQE>
@@ -833,21 +846,23 @@ __global__ void __launch_bounds__(kFusedWarps * 32, 1) decode_step_kernel(const 
     // ---- attention items.  CTA b owns list slots b, b + G, b + 2G, ...  It takes them in rounds
     // of kCtaItems slots: every thread decodes one slot, the survivors are packed in list order
     // (big items first), then the warps drain them through a shared counter.
-    __shared__ unsigned q_next, n_valid, warp_count[kFusedWarps];
+    __shared__ unsigned q_next, warp_count[kFusedWarps];
     // layout of san_smem: the warps' rings, their score slots, their barriers, the CTA's items
     constexpr uint32_t kZsAll = kFusedWarps * kFusedStages * kStageBytes;
     constexpr uint32_t kBarsAll = kZsAll + kFusedWarps * kZFloats * (uint32_t)sizeof(float);
-    constexpr uint32_t kDescsAll = kBarsAll + kFusedWarps * kFusedStages * (uint32_t)sizeof(uint64_t);
+    constexpr uint32_t kZeroRow = kBarsAll + kFusedWarps * kFusedStages * (uint32_t)sizeof(uint64_t);
+    constexpr uint32_t kDescsAll = kZeroRow + 128;
     ItemDesc* descs = sp<ItemDesc>(kDescsAll);
+    if (threadIdx.x < 32) *sp<uint32_t>(kZeroRow + threadIdx.x * 4) = 0u;      // read after the first barrier below
 
     FusedWarp<T> w(p);
     w.sm_base = smem_u32(san_smem);
     w.ring = (uint32_t)warp * kFusedStages * kStageBytes;
     w.bars = kBarsAll + (uint32_t)warp * kFusedStages * 8;
     w.zs_off = kZsAll + (uint32_t)warp * kZFloats * 4;
-    w.descs_off = kDescsAll; w.q_next = &q_next;
+    w.descs_off = kDescsAll; w.q_next = &q_next; w.zero_row = w.sm_base + kZeroRow;
     w.lane = lane;
-    w.p_stage = 0; w.c_stage = 0; w.c_par = 0; w.dead = false; w.p_active = false; w.tile_written = false;
+    w.p_stage = 0; w.c_stage = 0; w.c_par = 0; w.dead = false; w.p_active = false;
     if (lane == 0) {
         for (int s = 0; s < kFusedStages; ++s) mbar_init(sp<uint64_t>(w.bars + s * 8), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -874,14 +889,15 @@ __global__ void __launch_bounds__(kFusedWarps * 32, 1) decode_step_kernel(const 
         w.nx_idx = (unsigned)warp;
         w.fifo = 0ull; w.fifo_n = 0;
         w.next_item();
+#pragma unroll 1
         for (int s = 0; s < kFusedStages; ++s) w.produce();
         while (w.fifo_n > 0 && !w.dead) {
-            const ItemDesc& d = descs[(unsigned)(w.fifo & 0xffull)];
+            const ItemDesc& d = w.desc((unsigned)(w.fifo & 0xffull));
             w.fifo >>= 8; w.fifo_n -= 1;
             if constexpr (sizeof(T) == 2) {
-                if (d.kind) w.template process_mma<NQE>(d); else w.template process_mma<1>(d);
+                if (NQE > 1 && d.kind) w.template process_mma<NQE>(d); else w.template process_mma<1>(d);
             } else {
-                if (d.kind) w.template process<NQE>(d); else w.template process<1>(d);
+                if (NQE > 1 && d.kind) w.template process<NQE>(d); else w.template process<1>(d);
             }
         }
         // a warp whose wait ran out stops working but keeps meeting the CTA at the barriers above
