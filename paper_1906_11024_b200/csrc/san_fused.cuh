@@ -351,12 +351,21 @@ struct FusedWarp {
     template <int NQ, bool PACK> __device__ __forceinline__ void softmax_span(const ItemDesc& d, int n, int n_pad);
 };
 
+// Where the bf16 high part of position `pos` goes in a packed score row, as a 16-bit index
+// (the remainder sits 4 further): see softmax_span.
+__device__ __forceinline__ int packed_slot(int pos) {
+    const int jp = (pos >> 1) & 7;       // pair of positions within the block of 16
+    return (((pos >> 4) << 4) + ((jp & 3) << 2) + (jp >> 2)) * 2 + (pos & 1);
+}
+
 // Softmax of the n scores of a span held in zs (log2 domain), per query row.  A span that is
 // the whole row produces normalised weights and writes them to S; otherwise it produces
 // exp2(z - max) and parks (max, sum) in the span's partial-sum record for the combine.  With PACK == false the weights are
 // left in zs as floats (entries n .. n_pad zeroed).  With PACK == true (tensor-core path) they
-// are left as bf16 pairs: positions 2j, 2j+1 of a query row become word 2j = their bf16 high
-// parts and word 2j+1 = the bf16 remainders (w - high), zero beyond n up to n_pad.
+// are left as bf16 pairs, split into a bf16 high part and a bf16 remainder (w - high), zero
+// beyond n up to n_pad, in the order the MMA's B fragments want them: the 16 positions of a
+// block take 16 words; thread-in-group t owns words 4t .. 4t+3 = high parts of positions
+// (2t, 2t+1), high parts of (2t+8, 2t+9), remainders of (2t, 2t+1), remainders of (2t+8, 2t+9).
 template <typename T>
 template <int NQ, bool PACK>
 __device__ __forceinline__ void FusedWarp<T>::softmax_span(const ItemDesc& d, int n, int n_pad) {
@@ -382,8 +391,9 @@ __device__ __forceinline__ void FusedWarp<T>::softmax_span(const ItemDesc& d, in
                 if (lane < n_pad) {
                     const __nv_bfloat16 hi = __float2bfloat16_rn(w);
                     const __nv_bfloat16 lo = __float2bfloat16_rn(w - __bfloat162float(hi));
-                    zh[(lane >> 1) * 4 + (lane & 1)] = *reinterpret_cast<const unsigned short*>(&hi);
-                    zh[(lane >> 1) * 4 + 2 + (lane & 1)] = *reinterpret_cast<const unsigned short*>(&lo);
+                    const int at = packed_slot(lane);
+                    zh[at] = *reinterpret_cast<const unsigned short*>(&hi);
+                    zh[at + 4] = *reinterpret_cast<const unsigned short*>(&lo);
                 }
             } else if (lane < n_pad) {
                 zq[lane] = w;
@@ -409,8 +419,9 @@ __device__ __forceinline__ void FusedWarp<T>::softmax_span(const ItemDesc& d, in
                     if (jj < n_pad) {
                         const __nv_bfloat16 hi = __float2bfloat16_rn(w);
                         const __nv_bfloat16 lo = __float2bfloat16_rn(w - __bfloat162float(hi));
-                        zh[(jj >> 1) * 4 + (jj & 1)] = *reinterpret_cast<const unsigned short*>(&hi);
-                        zh[(jj >> 1) * 4 + 2 + (jj & 1)] = *reinterpret_cast<const unsigned short*>(&lo);
+                        const int at = packed_slot(jj);
+                        zh[at] = *reinterpret_cast<const unsigned short*>(&hi);
+                        zh[at + 4] = *reinterpret_cast<const unsigned short*>(&lo);
                     }
                 } else if (jj < n_pad) {
                     zq[jj] = w;
@@ -572,11 +583,11 @@ __device__ bool FusedWarp<T>::process(const ItemDesc& d) {
 // a handful of instructions (4 ldmatrix + 4 mma for the scores, 4 ldmatrix + 16 mma for one
 // layer's S.V) instead of a hundred or more unpack/FMA/shuffle instructions, and the step
 // is bound by instruction issue, not by tensor throughput.
-//   scores:  D[16 positions x 8 queries] = K_tile[16 x 64] . q^T          (queries padded to 8)
-//   apply:   D[16 queries x 8 dims]     += S[16 x 16 positions] . V_tile   (eight dim tiles)
+//   scores:  D[16 positions x 8 queries] = K_tile[16 x 64] . q^T              (queries padded to 8)
+//   apply:   D[16 dims x 8 queries]     += V_tile^T[16 x 16 positions] . S^T   (four dim tiles)
 // S is used as a bf16 high part plus a bf16 remainder (two MMAs), packed once per item by
 // the softmax, so that the weights keep about 16 bits; products and sums are float32.
-// Rows of D that belong to padding queries are computed from whatever the padding lanes
+// Columns of D that belong to padding queries are computed from whatever the padding lanes
 // load and are never stored.
 template <typename T>
 template <int NQ>
@@ -651,20 +662,30 @@ __device__ bool FusedWarp<T>::process_mma(const ItemDesc& d) {
     softmax_span<NQ, true>(d, n, (n + 15) & ~15);
 
     // ---- value tiles, layer by layer
-    // A fragments: the weights of query gid at positions b0 + {2tig, 2tig+1} and b0 + {2tig+8, 2tig+9},
-    // high parts and remainders, straight from the packed words
-    const uint32_t za = zs_off + (gid < NQ ? gid : 0) * ZQ * 4 + tig * 8;
+    // B fragments: the weights of query gid at positions b0 + {2tig, 2tig+1} and b0 + {2tig+8, 2tig+9},
+    // high parts and remainders, one 16-byte load per block straight from the packed words.
+    // A fragments: the tile transposed by ldmatrix; this lane addresses position vrow of a block
+    // and, for the dim tile x, the 16-byte chunk 2x + ((lane >> 3) & 1).
+    const uint32_t za = zs_off + (gid < NQ ? gid : 0) * ZQ * 4 + tig * 16;
+    const int vrow = (lane & 7) + ((lane >> 4) << 3);
+    uint32_t vd_off[4];
+#pragma unroll
+    for (int x = 0; x < 4; ++x) vd_off[x] = (uint32_t)(vrow * 128 + (((2 * x + ((lane >> 3) & 1)) ^ (lane & 7)) << 4));
     const KindParams& kp = p.k[d.kind];
     const long long plane_bytes = kp.plane_bytes, layer_bytes = kp.layer_bytes;
     char* vlast = const_cast<char*>(d.srcV) + (n - 1) * 128;      // where this step's value row goes
-    char* op = d.O + gid * ((long long)p.H * 128) + 4 * tig;
+    // output: this lane ends up with a pair of adjacent dims of one query (see below)
+    const int odd = gid & 1;
+    const int q_mine = NQ == 1 ? 0 : 2 * tig + odd;
+    const bool q_store = NQ == 1 ? (tig == 0 && !odd) : (q_mine < nq);
+    char* op = d.O + q_mine * ((long long)p.H * 128) + (gid - odd) * 2;
 #pragma unroll 1
     for (int l = 0; l < pi; ++l) {
-        float acc[8][4];
+        float acc[4][4];
 #pragma unroll
-        for (int nt = 0; nt < 8; ++nt)
+        for (int x = 0; x < 4; ++x)
 #pragma unroll
-            for (int e = 0; e < 4; ++e) acc[nt][e] = 0.f;
+            for (int e = 0; e < 4; ++e) acc[x][e] = 0.f;
 #pragma unroll 1
         for (int s0 = 0; s0 < n; s0 += TR) {
             const uint32_t st = acquire();
@@ -676,40 +697,49 @@ __device__ bool FusedWarp<T>::process_mma(const ItemDesc& d) {
             const uint32_t st_s = sm_base + st;
 #pragma unroll 1
             for (int b0 = 0; b0 < r; b0 += 16) {
-                const uint2 w0 = *sp<uint2>(za + (s0 + b0) * 4), w1 = *sp<uint2>(za + (s0 + b0) * 4 + 32);    // (high, remainder) x 2
-                // the A operand of an MMA is four consecutive registers: build the two quads (high parts,
-                // remainders) once per block; rows 8..15 of A (registers 1 and 3) are padding queries
-                uint32_t ah[4], al[4];
-                ah[0] = w0.x; ah[2] = w1.x; al[0] = w0.y; al[2] = w1.y;
-                asm volatile("mov.b32 %0, 0;\n\tmov.b32 %1, 0;\n\tmov.b32 %2, 0;\n\tmov.b32 %3, 0;"
-                             : "=r"(ah[1]), "=r"(ah[3]), "=r"(al[1]), "=r"(al[3]));
+                const uint4 w = *sp<uint4>(za + (s0 + b0) * 4);      // (high b0, high b1, remainder b0, remainder b1)
                 // rows at or beyond r hold stale bytes: their weights are zero, but 0 x NaN would not be,
                 // so those lanes address a row of zeros instead
-                const int row = b0 + lrow;
+                const int row = b0 + vrow;
                 const uint32_t fix = (row == new_row) ? new_fix : 0u;
                 const uint32_t blk = st_s + b0 * 128;
 #pragma unroll
                 for (int x = 0; x < 4; ++x) {
-                    uint32_t b[4];
-                    ldsm_x4_t(row < r ? blk + (ld_off[x] ^ fix) : zero_row, b);
-                    mma_bf16(acc[2 * x], ah[0], ah[1], ah[2], ah[3], b[0], b[1]);
-                    mma_bf16(acc[2 * x + 1], ah[0], ah[1], ah[2], ah[3], b[2], b[3]);
-                    mma_bf16(acc[2 * x], al[0], al[1], al[2], al[3], b[0], b[1]);
-                    mma_bf16(acc[2 * x + 1], al[0], al[1], al[2], al[3], b[2], b[3]);
+                    uint32_t a[4];
+                    ldsm_x4_t(row < r ? blk + (vd_off[x] ^ fix) : zero_row, a);
+                    mma_bf16(acc[x], a[0], a[1], a[2], a[3], w.x, w.y);
+                    mma_bf16(acc[x], a[0], a[1], a[2], a[3], w.z, w.w);
                 }
             }
             release();
         }
-        // acc[nt][0], acc[nt][1]: query gid, dims 8nt + 2tig, +1
-        if (gid < nq) {
-            if (n_spans == 1) {
+        // acc[x][0], [1]: dim 16x + gid of queries 2tig, 2tig+1; acc[x][2], [3]: dim 16x + gid + 8
+        if (n_spans == 1) {
+            // lanes gid and gid ^ 1 hold adjacent dims: the even one collects the pair of query 2tig,
+            // the odd one the pair of query 2tig + 1 (one query: only the even lanes of tig 0 store)
 #pragma unroll
-                for (int nt = 0; nt < 8; ++nt) *reinterpret_cast<uint32_t*>(op + 16 * nt) = pack_bf16x2(acc[nt][0], acc[nt][1]);
-            } else {
-                float* pp = d.part + HDR + ((long long)l * NQ + gid) * kDh + 2 * tig;
+            for (int x = 0; x < 4; ++x)
 #pragma unroll
-                for (int nt = 0; nt < 8; ++nt) *reinterpret_cast<float2*>(pp + 8 * nt) = make_float2(acc[nt][0], acc[nt][1]);
-            }
+                for (int h = 0; h < 2; ++h) {
+                    uint32_t packed;
+                    if (NQ == 1) {
+                        const float up = __shfl_down_sync(0xffffffffu, acc[x][2 * h], 4);
+                        packed = pack_bf16x2(acc[x][2 * h], up);
+                    } else {
+                        const float got = __shfl_xor_sync(0xffffffffu, odd ? acc[x][2 * h] : acc[x][2 * h + 1], 4);
+                        packed = odd ? pack_bf16x2(got, acc[x][2 * h + 1]) : pack_bf16x2(acc[x][2 * h], got);
+                    }
+                    if (q_store) *reinterpret_cast<uint32_t*>(op + (16 * x + 8 * h) * 2) = packed;
+                }
+        } else {
+            float* pp = d.part + HDR + ((long long)l * NQ + 2 * tig) * kDh + gid;
+#pragma unroll
+            for (int x = 0; x < 4; ++x)
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    if (2 * tig < nq) pp[16 * x + 8 * h] = acc[x][2 * h];
+                    if (2 * tig + 1 < nq) pp[kDh + 16 * x + 8 * h] = acc[x][2 * h + 1];
+                }
         }
         vlast += plane_bytes;
         op += layer_bytes;
