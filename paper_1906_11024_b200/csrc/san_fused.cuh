@@ -372,60 +372,101 @@ __device__ __forceinline__ void FusedWarp<T>::softmax_span(const ItemDesc& d, in
     constexpr int ZQ = kZFloats / NQ;
     const int nq = d.nq, n_spans = d.n_spans;
     const long long S_qstride = (long long)p.H * p.k[d.kind].S_ld;
+    if (n <= 64) {
+        // At most two scores per lane and no loops; the query rows go through the reductions side
+        // by side, so that their shuffles overlap.  Rows of absent queries (padding up to NQ) hold
+        // finite scores of a repeated query row: they are carried along and never stored.
+        const bool two = n > 32;                       // warp-uniform
+        const bool in0 = lane < n, in1 = lane + 32 < n;
+        float z0[NQ], z1[NQ], m[NQ], sum[NQ];
 #pragma unroll
-    for (int qi = 0; qi < NQ; ++qi) {
-        if (qi >= nq) break;                 // rows of absent queries are never stored
-        float* zq = sp<float>(zs_off + qi * ZQ * 4);
-        unsigned short* zh = reinterpret_cast<unsigned short*>(zq);
-        float* Srow = d.S ? d.S + qi * S_qstride : nullptr;
-        if (n <= 32) {      // one score per lane: no loops
-            const float z = lane < n ? zq[lane] : -INFINITY;
-            const float m = warp_max(z);
-            const float e = lane < n ? exp2f(z - m) : 0.f;
-            const float s = warp_sum(e);
-            if (n_spans > 1 && lane == 0) { d.part[qi] = m; d.part[NQ + qi] = s; }     // for the combine
-            const float w = (n_spans == 1) ? e * (1.0f / s) : e;
-            if (Srow && lane < n) Srow[lane] = w;
+        for (int qi = 0; qi < NQ; ++qi) {
+            const float* zq = sp<float>(zs_off + qi * ZQ * 4);
+            z0[qi] = in0 ? zq[lane] : -INFINITY;
+            z1[qi] = (two && in1) ? zq[lane + 32] : -INFINITY;
+            m[qi] = fmaxf(z0[qi], z1[qi]);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+            for (int qi = 0; qi < NQ; ++qi) m[qi] = fmaxf(m[qi], __shfl_xor_sync(0xffffffffu, m[qi], o));
+#pragma unroll
+        for (int qi = 0; qi < NQ; ++qi) {
+            z0[qi] = exp2f(z0[qi] - m[qi]);             // exp2(-inf) = 0 for the lanes beyond n
+            z1[qi] = exp2f(z1[qi] - m[qi]);
+            sum[qi] = z0[qi] + z1[qi];
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+            for (int qi = 0; qi < NQ; ++qi) sum[qi] += __shfl_xor_sync(0xffffffffu, sum[qi], o);
+        __syncwarp();                                   // every lane has read its scores: the words may be reused
+#pragma unroll
+        for (int qi = 0; qi < NQ; ++qi) {
+            float* zq = sp<float>(zs_off + qi * ZQ * 4);
+            unsigned short* zh = reinterpret_cast<unsigned short*>(zq);
+            if (n_spans > 1 && lane == 0 && qi < nq) { d.part[qi] = m[qi]; d.part[NQ + qi] = sum[qi]; }     // for the combine
+            const float inv = (n_spans == 1) ? 1.0f / sum[qi] : 1.0f;
+            const float w0 = z0[qi] * inv, w1 = z1[qi] * inv;
+            if (d.S && qi < nq) {
+                float* Srow = d.S + qi * S_qstride;
+                if (in0) Srow[lane] = w0;
+                if (two && in1) Srow[lane + 32] = w1;
+            }
             if (PACK) {
-                __syncwarp();                // every lane has read its score: the words may be reused
                 if (lane < n_pad) {
-                    const __nv_bfloat16 hi = __float2bfloat16_rn(w);
-                    const __nv_bfloat16 lo = __float2bfloat16_rn(w - __bfloat162float(hi));
+                    const __nv_bfloat16 hi = __float2bfloat16_rn(w0);
+                    const __nv_bfloat16 lo = __float2bfloat16_rn(w0 - __bfloat162float(hi));
                     const int at = packed_slot(lane);
                     zh[at] = *reinterpret_cast<const unsigned short*>(&hi);
                     zh[at + 4] = *reinterpret_cast<const unsigned short*>(&lo);
                 }
-            } else if (lane < n_pad) {
-                zq[lane] = w;
-            }
-        } else {
-            float m = -INFINITY;
-#pragma unroll 1
-            for (int jj = lane; jj < n; jj += 32) m = fmaxf(m, zq[jj]);
-            m = warp_max(m);
-            float s = 0.f;
-#pragma unroll 1
-            for (int jj = lane; jj < n; jj += 32) { const float e = exp2f(zq[jj] - m); zq[jj] = e; s += e; }
-            s = warp_sum(s);
-            if (n_spans > 1 && lane == 0) { d.part[qi] = m; d.part[NQ + qi] = s; }
-            const float inv = (n_spans == 1) ? 1.0f / s : 1.0f;
-#pragma unroll 1
-            for (int j0 = 0; j0 < n_pad; j0 += 32) {      // warp-uniform trip count
-                const int jj = j0 + lane;
-                const float w = jj < n ? zq[jj] * inv : 0.f;
-                if (Srow && jj < n) Srow[jj] = w;
-                if (PACK) {
-                    __syncwarp();
-                    if (jj < n_pad) {
-                        const __nv_bfloat16 hi = __float2bfloat16_rn(w);
-                        const __nv_bfloat16 lo = __float2bfloat16_rn(w - __bfloat162float(hi));
-                        const int at = packed_slot(jj);
-                        zh[at] = *reinterpret_cast<const unsigned short*>(&hi);
-                        zh[at + 4] = *reinterpret_cast<const unsigned short*>(&lo);
-                    }
-                } else if (jj < n_pad) {
-                    zq[jj] = w;
+                if (two && lane + 32 < n_pad) {
+                    const __nv_bfloat16 hi = __float2bfloat16_rn(w1);
+                    const __nv_bfloat16 lo = __float2bfloat16_rn(w1 - __bfloat162float(hi));
+                    const int at = packed_slot(lane + 32);
+                    zh[at] = *reinterpret_cast<const unsigned short*>(&hi);
+                    zh[at + 4] = *reinterpret_cast<const unsigned short*>(&lo);
                 }
+            } else {
+                if (lane < n_pad) zq[lane] = w0;
+                if (two && lane + 32 < n_pad) zq[lane + 32] = w1;
+            }
+        }
+        __syncwarp();
+        return;
+    }
+#pragma unroll 1
+    for (int qi = 0; qi < nq; ++qi) {        // long spans: row by row; rows of absent queries are never stored
+        float* zq = sp<float>(zs_off + qi * ZQ * 4);
+        unsigned short* zh = reinterpret_cast<unsigned short*>(zq);
+        float* Srow = d.S ? d.S + qi * S_qstride : nullptr;
+        float m = -INFINITY;
+#pragma unroll 1
+        for (int jj = lane; jj < n; jj += 32) m = fmaxf(m, zq[jj]);
+        m = warp_max(m);
+        float s = 0.f;
+#pragma unroll 1
+        for (int jj = lane; jj < n; jj += 32) { const float e = exp2f(zq[jj] - m); zq[jj] = e; s += e; }
+        s = warp_sum(s);
+        if (n_spans > 1 && lane == 0) { d.part[qi] = m; d.part[NQ + qi] = s; }
+        const float inv = (n_spans == 1) ? 1.0f / s : 1.0f;
+#pragma unroll 1
+        for (int j0 = 0; j0 < n_pad; j0 += 32) {      // warp-uniform trip count
+            const int jj = j0 + lane;
+            const float w = jj < n ? zq[jj] * inv : 0.f;
+            if (Srow && jj < n) Srow[jj] = w;
+            if (PACK) {
+                __syncwarp();
+                if (jj < n_pad) {
+                    const __nv_bfloat16 hi = __float2bfloat16_rn(w);
+                    const __nv_bfloat16 lo = __float2bfloat16_rn(w - __bfloat162float(hi));
+                    const int at = packed_slot(jj);
+                    zh[at] = *reinterpret_cast<const unsigned short*>(&hi);
+                    zh[at + 4] = *reinterpret_cast<const unsigned short*>(&lo);
+                }
+            } else if (jj < n_pad) {
+                zq[jj] = w;
             }
         }
     }
@@ -910,8 +951,15 @@ __global__ void __launch_bounds__(kFusedWarps * 32, 1) decode_step_kernel(const 
         if (lane == 0) warp_count[warp] = __popc(ballot);
         __syncthreads();                                 // also: every warp is done with the previous round's items
         if (threadIdx.x == 0) q_next = kFusedWarps;      // the first kFusedWarps items go to the warps directly
-        unsigned before = 0, total = 0;
-        for (int i = 0; i < kFusedWarps; ++i) { const unsigned cnt = warp_count[i]; if (i < warp) before += cnt; total += cnt; }
+        // lane i holds warp i's count: survivors ahead of this warp's, and all of them
+        static_assert(kFusedWarps <= 32, "one lane per warp");
+        const unsigned cnt = lane < kFusedWarps ? warp_count[lane] : 0u;
+        unsigned before = lane < warp ? cnt : 0u, total = cnt;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            before += __shfl_xor_sync(0xffffffffu, before, o);
+            total += __shfl_xor_sync(0xffffffffu, total, o);
+        }
         if (ok) descs[before + __popc(ballot & ((1u << lane) - 1u))] = mine;
         __syncthreads();
         // -- drain
