@@ -23,9 +23,11 @@ namespace san {
 
 constexpr int kStageBytes = 4096;   // one tile: 32 bf16 rows or 16 float32 rows
 constexpr int kFusedWarps = 16;
-constexpr int kFusedStages = 3;
-constexpr int kZFloats = 256;       // scores a warp keeps on chip: span <= kZFloats / NQ
-constexpr int kDescSlots = 6;       // decoded items a warp keeps (in flight, being finished, being decoded)
+// Two stages per warp keep the copies ahead of the arithmetic as well as three did (measured),
+// and leave the shared memory for longer spans: a row of up to kZFloats / NQ positions needs
+// no partial sums and no combine.
+constexpr int kFusedStages = 2;
+constexpr int kZFloats = 1024;      // scores a warp keeps on chip: span <= kZFloats / NQ
 constexpr int kMaxSpans = 32;
 
 enum { TAG_STEP = 6 };
@@ -131,7 +133,7 @@ __device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t (&r)[4]) {
 }
 // D(16x8, f32) += A(16x16, bf16, row) * B(16x8, bf16, col)
 __device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                  : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
@@ -674,12 +676,11 @@ __device__ bool FusedWarp<T>::process_mma(const ItemDesc& d) {
         for (int b0 = 0; b0 < r; b0 += 16) {
             const uint32_t fix = (b0 + lrow == new_row) ? new_fix : 0u;
             float acc[4] = {0.f, 0.f, 0.f, 0.f};
+            uint32_t a[4][4];          // all four loads first: their latencies overlap
 #pragma unroll
-            for (int ks = 0; ks < 4; ++ks) {
-                uint32_t a[4];
-                ldsm_x4(st_s + b0 * 128 + (ld_off[ks] ^ fix), a);
-                mma_bf16(acc, a[0], a[1], a[2], a[3], qb[ks][0], qb[ks][1]);
-            }
+            for (int ks = 0; ks < 4; ++ks) ldsm_x4(st_s + b0 * 128 + (ld_off[ks] ^ fix), a[ks]);
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks) mma_bf16(acc, a[ks][0], a[ks][1], a[ks][2], a[ks][3], qb[ks][0], qb[ks][1]);
             // acc[0], acc[1]: position b0+gid, queries 2tig, 2tig+1; acc[2], acc[3]: position b0+gid+8.
             // Rows of the block at or beyond r (the query rows of a first tile, stale bytes) give
             // scores that the next tile overwrites; nothing is stored beyond the span.
@@ -744,13 +745,13 @@ __device__ bool FusedWarp<T>::process_mma(const ItemDesc& d) {
                 const int row = b0 + vrow;
                 const uint32_t fix = (row == new_row) ? new_fix : 0u;
                 const uint32_t blk = st_s + b0 * 128;
+                uint32_t a[4][4];      // all four loads first: their latencies overlap
 #pragma unroll
-                for (int x = 0; x < 4; ++x) {
-                    uint32_t a[4];
-                    ldsm_x4_t(row < r ? blk + (vd_off[x] ^ fix) : zero_row, a);
-                    mma_bf16(acc[x], a[0], a[1], a[2], a[3], w.x, w.y);
-                    mma_bf16(acc[x], a[0], a[1], a[2], a[3], w.z, w.w);
-                }
+                for (int x = 0; x < 4; ++x) ldsm_x4_t(row < r ? blk + (vd_off[x] ^ fix) : zero_row, a[x]);
+#pragma unroll
+                for (int x = 0; x < 4; ++x) mma_bf16(acc[x], a[x][0], a[x][1], a[x][2], a[x][3], w.x, w.y);
+#pragma unroll
+                for (int x = 0; x < 4; ++x) mma_bf16(acc[x], a[x][0], a[x][1], a[x][2], a[x][3], w.z, w.w);
             }
             release();
         }
