@@ -535,8 +535,17 @@ int32_t san_decode_step(san_ctx* ctx, const san_step_args* a, void* stream) {
     long long ctas = std::min<long long>(ctx->sm_count, (p.n_items + kFusedWarps - 1) / kFusedWarps);
     if (p.x_aan) ctas = ctx->sm_count;     // the running average is spread over every thread of the grid
     if (ctas < 1) ctas = 1;
+    // Programmatic stream serialization: the grid may be scheduled while the preceding kernel of
+    // the stream is finishing; the kernel touches no global memory before that kernel is complete.
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)ctas); cfg.blockDim = dim3(kFusedWarps * 32);
+    cfg.dynamicSmemBytes = smem; cfg.stream = static_cast<cudaStream_t>(stream);
+    cfg.attrs = &attr; cfg.numAttrs = 1;
     void* args[] = {&p};
-    cudaError_t e = cudaLaunchKernel(fn, dim3((unsigned)ctas), dim3(kFusedWarps * 32), args, smem, static_cast<cudaStream_t>(stream));
+    cudaError_t e = cudaLaunchKernelExC(&cfg, fn, args);
     return cuda_status(e);
 }
 

@@ -877,6 +877,25 @@ template <typename T, int NQE>
 __global__ void __launch_bounds__(kFusedWarps * 32, 1) decode_step_kernel(const __grid_constant__ StepParams p) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 
+    // The launch allows programmatic stream serialization: the next kernel of the stream may be
+    // scheduled onto SMs as this grid leaves them, and this grid may have been scheduled while
+    // its predecessor was still finishing.  Nothing is read from or written to global memory
+    // until the predecessor has completed and its writes are visible (the wait below); only the
+    // set-up of shared memory runs ahead of it.  Without the launch attribute both are no-ops.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // layout of san_smem: the warps' rings, their score slots, their barriers, a row of zeros, the CTA's items
+    constexpr uint32_t kZsAll = kFusedWarps * kFusedStages * kStageBytes;
+    constexpr uint32_t kBarsAll = kZsAll + kFusedWarps * kZFloats * (uint32_t)sizeof(float);
+    constexpr uint32_t kZeroRow = kBarsAll + kFusedWarps * kFusedStages * (uint32_t)sizeof(uint64_t);
+    constexpr uint32_t kDescsAll = kZeroRow + 128;
+    if (threadIdx.x < 32) *sp<uint32_t>(kZeroRow + threadIdx.x * 4) = 0u;      // read after the first CTA barrier
+    if (lane == 0) {
+        for (int s = 0; s < kFusedStages; ++s) mbar_init(sp<uint64_t>(kBarsAll + ((uint32_t)warp * kFusedStages + s) * 8), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+
     // ---- AAN running average (Table 6 pairing): element-wise, every thread of the grid
     if (p.x_aan) {
         const int d = p.H * kDh, d4 = d >> 2;
@@ -919,13 +938,7 @@ __global__ void __launch_bounds__(kFusedWarps * 32, 1) decode_step_kernel(const 
     // of kCtaItems slots: every thread decodes one slot, the survivors are packed in list order
     // (big items first), then the warps drain them through a shared counter.
     __shared__ unsigned q_next, warp_count[kFusedWarps];
-    // layout of san_smem: the warps' rings, their score slots, their barriers, the CTA's items
-    constexpr uint32_t kZsAll = kFusedWarps * kFusedStages * kStageBytes;
-    constexpr uint32_t kBarsAll = kZsAll + kFusedWarps * kZFloats * (uint32_t)sizeof(float);
-    constexpr uint32_t kZeroRow = kBarsAll + kFusedWarps * kFusedStages * (uint32_t)sizeof(uint64_t);
-    constexpr uint32_t kDescsAll = kZeroRow + 128;
     ItemDesc* descs = sp<ItemDesc>(kDescsAll);
-    if (threadIdx.x < 32) *sp<uint32_t>(kZeroRow + threadIdx.x * 4) = 0u;      // read after the first barrier below
 
     FusedWarp<T> w(p);
     w.sm_base = smem_u32(san_smem);
@@ -935,11 +948,6 @@ __global__ void __launch_bounds__(kFusedWarps * 32, 1) decode_step_kernel(const 
     w.descs_off = kDescsAll; w.q_next = &q_next; w.zero_row = w.sm_base + kZeroRow;
     w.lane = lane;
     w.p_stage = 0; w.c_stage = 0; w.c_par = 0; w.dead = false; w.p_active = false;
-    if (lane == 0) {
-        for (int s = 0; s < kFusedStages; ++s) mbar_init(sp<uint64_t>(w.bars + s * 8), 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 
     const unsigned long long my_slots = (p.n_items > blockIdx.x) ? ((unsigned long long)p.n_items - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
     for (unsigned long long k0 = 0; k0 < my_slots; k0 += kCtaItems) {
