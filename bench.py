@@ -34,6 +34,28 @@ L2_BYTES = 126e6
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 
+# DRAM bytes read + written per launch of the step kernel, from the ncu capture summarised in
+# profiles/decode_step_base_long.md, and the digest of the kernel sources they were taken
+# with: once those sources change the counters no longer describe the kernel and the bench
+# line reports null until a new capture is recorded here.
+KERNEL_SOURCES = ("san_fused.cuh", "san_api.cu", "san_kernels.cuh")
+NCU_TRAFFIC = {"digest": "f7a74a902b0d071a", "fused": {"base": 70.2e6, "long": 762.2e6}}
+
+
+def kernel_digest():
+    import hashlib
+    h = hashlib.sha256()
+    for f in KERNEL_SOURCES:
+        with open(os.path.join(ROOT, "paper_1906_11024_b200", "csrc", f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
+def ncu_traffic(path, workload):
+    if kernel_digest() != NCU_TRAFFIC["digest"]:
+        return None
+    return NCU_TRAFFIC.get(path, {}).get(workload)
+
 
 # ------------------------------------------------------------------------------- workload state
 def state_positions(w):
@@ -489,7 +511,7 @@ def main():
         "roofline": {"bound": "hbm", "kernel": dom_name, "achieved": dom_bytes / dom_s / 1e9,
                      "peak": peak, "unit": "GB/s", "frac": dom_bytes / dom_s / 1e9 / peak, "peak_kind": peak_kind,
                      "bytes_per_launch": dom_bytes, "us_per_launch": dom_s * 1e6, "launches_per_step": dom_per_step,
-                     "traffic": None},
+                     "traffic": ncu_traffic(args.path, w.name)},
         "e2e": {"value": w.n_seqs * e2e_steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": e2e_s / e2e_steps * 1e3},
         "clocks": clocks,
