@@ -203,6 +203,44 @@ typedef struct {
 } san_step_args;
 int32_t san_decode_step(san_ctx* ctx, const san_step_args* args, void* stream);
 
+/* Beam-search cache reorder (Section 4.1: decoding runs a beam of hypotheses per sentence;
+ * after a step each surviving hypothesis continues the attention cache of the hypothesis it
+ * extends).  For item i = sentence d_sent_ids[i] and beam slot s, the sequence
+ * sentence*beam + s takes over the first d_lens[i*beam + s] cached rows of the sequence
+ * sentence*beam + d_parent[i*beam + s], in every self-attention key plane (one per block:
+ * Section 3.2, shared layers keep no keys, so sharing shrinks this step too) and every
+ * value plane; with self_is_aan it takes over the parent's running sum instead (when the
+ * length is > 0).  d_parent holds beam slots 0..beam-1 of the SAME sentence, which is what
+ * lets the gather run in place: all rows are read before any is written, as if copied
+ * through a snapshot.  Slots with d_parent == s keep their rows and cost nothing.
+ * Encoder memory is per sentence and is not touched.  max_len is a host bound on d_lens
+ * (0 = capacity).  A parent outside 0..beam-1, a length outside 0..max_len or a sentence id
+ * out of range skips that slot and is reported through san_device_status.  Bit copy. */
+int32_t san_beam_reorder(san_ctx* ctx, const int32_t* d_sent_ids, const int32_t* d_parent,
+                         const int32_t* d_lens, int32_t n_sent, int32_t max_len, void* stream);
+
+/* Policy learning (Section 3.1, Section 3.3, Eq. 6).
+ *
+ * san_js_matrix: the Jensen-Shannon divergence between the attention weights of every pair
+ * of layers, JS(p,q) = (KL(p||m) + KL(q||m))/2 with m = (p+q)/2 and natural logarithms, one
+ * value per (row, head) distribution and averaged over all of them (heads count as separate
+ * channels).  d_S holds the weights of n_layers layers of an unshared model (block size 1) as
+ * the decode step writes them: layer l at d_S + l*layer_stride, each [n_rows][n_heads][ld_s]
+ * float32 with d_lens[row] valid positions (clamped to 0..ld_s).  d_js receives the
+ * n_layers x n_layers symmetric matrix (float64, zero diagonal); it is cleared first.  Needs
+ * no context and allocates nothing.
+ *
+ * san_block_similarity (host): Eq. 6 for the block of layers m..n (0-based, m < n),
+ *   sim(m,n) = sum_{i != j in m..n} (ln 2 - JS(i,j)) / ((n-m+1)(n-m)).
+ * san_policy_search (host): the bottom-up search of Section 3.3; starting at the lowest layer
+ * a block grows while the similarity of the block with the next layer added is >= theta and
+ * closes at the first failure (a block of one layer always qualifies); sizes[] (room for
+ * n_layers entries) receives {pi_i}, ready for san_policy_set_sizes. js is a HOST matrix. */
+int32_t san_js_matrix(int32_t n_layers, const float* d_S, int64_t layer_stride, int64_t ld_s,
+                      int32_t n_rows, int32_t n_heads, const int32_t* d_lens, double* d_js, void* stream);
+int32_t san_block_similarity(const double* js, int32_t n_layers, int32_t m, int32_t n, double* sim);
+int32_t san_policy_search(const double* js, int32_t n_layers, double theta, int32_t* sizes, int32_t* n_blocks);
+
 /* Reads (and clears) the device error word: *first_error = SAN_OK or the first
  * device-check error since the last read; detail[0..3] (optional) = kernel tag, item,
  * offending value, limit.  Synchronises `stream`. */

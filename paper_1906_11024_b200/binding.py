@@ -29,6 +29,7 @@ EXPORTS = (
     "san_policy_set_sizes", "san_policy_set_map", "san_policy_get_map",
     "san_cache_append", "san_attn_weights", "san_attn_apply", "san_aan_step",
     "san_device_status", "san_status_string", "san_attn_weights_static", "san_decode_step",
+    "san_beam_reorder", "san_js_matrix", "san_block_similarity", "san_policy_search",
 )
 
 
@@ -83,6 +84,10 @@ def lib():
     L.san_device_status.argtypes = [vp, _I32P, _I32P, vp]
     L.san_attn_weights_static.argtypes = [i32, i32, i32, vp, vp, i32, i32, vp, vp, i32, i32, vp, i64, vp, vp]
     L.san_decode_step.argtypes = [vp, C.POINTER(san_step_args), vp]
+    L.san_beam_reorder.argtypes = [vp, vp, vp, vp, i32, i32, vp]
+    L.san_js_matrix.argtypes = [i32, vp, i64, i64, i32, i32, vp, vp, vp]
+    L.san_block_similarity.argtypes = [C.POINTER(C.c_double), i32, i32, i32, C.POINTER(C.c_double)]
+    L.san_policy_search.argtypes = [C.POINTER(C.c_double), i32, C.c_double, _I32P, _I32P]
     L.san_status_string.argtypes = [i32]
     L.san_status_string.restype = C.c_char_p
     for name in EXPORTS:
@@ -212,3 +217,37 @@ def san_decode_step(ctx, *, d_q_self=None, d_k_new=None, d_v_new=None, d_seq_ids
                       _ptr(d_S_self), ld_t, _ptr(d_O_self), _ptr(d_q_enc), _ptr(d_sent_ids), _ptr(d_src_lens),
                       n_sent, max_src, _ptr(d_S_enc), ld_s, _ptr(d_O_enc), _ptr(d_x_aan), _ptr(d_t))
     return lib().san_decode_step(ctx, C.byref(a), _stream(stream))
+
+
+def san_beam_reorder(ctx, d_sent_ids, d_parent, d_lens, n_sent, max_len=0, stream=None) -> int:
+    """Beam-search cache reorder: every beam slot takes over its parent's cached rows, in place."""
+    return lib().san_beam_reorder(ctx, _ptr(d_sent_ids), _ptr(d_parent), _ptr(d_lens), n_sent, max_len,
+                                  _stream(stream))
+
+
+def san_js_matrix(n_layers, d_S, layer_stride, ld_s, n_rows, n_heads, d_lens, d_js, stream=None) -> int:
+    """Pairwise Jensen-Shannon divergence of the layers' attention weights into d_js [M][M] float64."""
+    return lib().san_js_matrix(n_layers, _ptr(d_S), layer_stride, ld_s, n_rows, n_heads, _ptr(d_lens), _ptr(d_js),
+                               _stream(stream))
+
+
+def _f64_matrix(js, n_layers):
+    flat = [float(x) for row in js for x in row] if not isinstance(js, (bytes, bytearray)) else js
+    if len(flat) != n_layers * n_layers:
+        raise ValueError("js must be n_layers x n_layers")
+    return (C.c_double * len(flat))(*flat)
+
+
+def san_block_similarity(js, n_layers, m, n):
+    """Eq. 6 on a host matrix (nested sequences).  Returns (status, sim)."""
+    out = C.c_double(0.0)
+    rc = lib().san_block_similarity(_f64_matrix(js, n_layers), n_layers, m, n, C.byref(out))
+    return rc, out.value
+
+
+def san_policy_search(js, n_layers, theta):
+    """Section 3.3 search on a host matrix.  Returns (status, block sizes bottom-up)."""
+    sizes = (C.c_int32 * max(n_layers, 1))()
+    nb = C.c_int32(0)
+    rc = lib().san_policy_search(_f64_matrix(js, n_layers), n_layers, float(theta), sizes, C.byref(nb))
+    return rc, list(sizes[:nb.value]) if rc == SAN_OK else []

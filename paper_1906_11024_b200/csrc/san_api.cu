@@ -9,6 +9,8 @@
 #include "san_ctx.h"
 #include "san_kernels.cuh"
 #include "san_fused.cuh"
+#include "san_reorder.cuh"
+#include "san_learn.cuh"
 
 using namespace san;
 
@@ -547,6 +549,90 @@ int32_t san_decode_step(san_ctx* ctx, const san_step_args* a, void* stream) {
     void* args[] = {&p};
     cudaError_t e = cudaLaunchKernelExC(&cfg, fn, args);
     return cuda_status(e);
+}
+
+int32_t san_beam_reorder(san_ctx* ctx, const int32_t* d_sent_ids, const int32_t* d_parent,
+                         const int32_t* d_lens, int32_t n_sent, int32_t max_len, void* stream) {
+    if (!ctx || !d_sent_ids || !d_parent || !d_lens) return SAN_ERR_NULL;
+    const san_config& c = ctx->cfg;
+    if (n_sent < 0 || n_sent > c.max_sent) return SAN_ERR_SHAPE;
+    if (max_len == 0) max_len = c.max_tgt_len;
+    if (max_len < 1 || max_len > c.max_tgt_len) return SAN_ERR_SHAPE;
+    if (n_sent == 0) return SAN_OK;
+    ReorderParams p;
+    std::memset(&p, 0, sizeof(p));
+    p.sent_ids = d_sent_ids; p.parent = d_parent; p.lens = d_lens;
+    p.n_sent = n_sent; p.beam = c.beam; p.max_sent = c.max_sent; p.err = ctx->err;
+    const int per_beam = kReorderTile / c.beam;
+    if (c.self_is_aan) {       // the running sums [layer][sequence][H*64] float32
+        p.base = ctx->cache + ctx->off_aan; p.plane_bytes = (long long)ctx->aan_plane_bytes;
+        p.n_planes = c.n_layers; p.n_heads = 1; p.head_bytes = 0;
+        p.fixed_bytes = c.n_heads * kDh * (int)sizeof(float);
+        p.seq_bytes = p.fixed_bytes; p.unit_bytes = 0; p.max_units = max_len;
+        p.tiles_per_panel = ceil_div(p.fixed_bytes / 16, per_beam);
+    } else {                   // key planes of the blocks, then value planes of the layers: adjacent in the arena
+        const int row_bytes = kDh * ctx->elem_bytes;
+        p.base = ctx->cache + ctx->off_self_k; p.plane_bytes = (long long)ctx->self_plane_bytes;
+        p.n_planes = ctx->self_pol.n_blocks + ctx->n_self_v_planes; p.n_heads = c.n_heads;
+        p.head_bytes = (long long)c.max_tgt_len * row_bytes;
+        p.seq_bytes = p.head_bytes * c.n_heads;
+        p.unit_bytes = row_bytes; p.fixed_bytes = 0; p.max_units = max_len;
+        p.tiles_per_panel = ceil_div(max_len * (row_bytes / 16), per_beam);
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (!c.self_is_aan && ctx->self_pol.n_blocks < ctx->n_self_k_planes) {
+        // the policy in force uses fewer key planes than the arena holds: the unused planes lie
+        // between the used key planes and the value planes, so the two runs are launched apart
+        ReorderParams pk = p;
+        pk.n_planes = ctx->self_pol.n_blocks;
+        const long long gk = (long long)pk.n_planes * n_sent * pk.n_heads * pk.tiles_per_panel;
+        if (gk > 0x7fffffffLL) return SAN_ERR_SHAPE;
+        beam_reorder_kernel<<<(unsigned)gk, kReorderThreads, 0, st>>>(pk);
+        if (cudaGetLastError() != cudaSuccess) return SAN_ERR_CUDA;
+        p.base = ctx->cache + ctx->off_self_v; p.n_planes = ctx->n_self_v_planes;
+    }
+    const long long grid = (long long)p.n_planes * n_sent * p.n_heads * p.tiles_per_panel;
+    if (grid > 0x7fffffffLL) return SAN_ERR_SHAPE;
+    beam_reorder_kernel<<<(unsigned)grid, kReorderThreads, 0, st>>>(p);
+    return cuda_status(cudaGetLastError());
+}
+
+int32_t san_js_matrix(int32_t n_layers, const float* d_S, int64_t layer_stride, int64_t ld_s,
+                      int32_t n_rows, int32_t n_heads, const int32_t* d_lens, double* d_js, void* stream) {
+    if (!d_S || !d_lens || !d_js) return SAN_ERR_NULL;
+    if (n_layers < 1 || n_layers > SAN_MAX_LAYERS) return SAN_ERR_SHAPE;
+    if (n_rows < 0 || n_heads < 1 || ld_s < 1 || layer_stride < 0) return SAN_ERR_SHAPE;
+    if (n_layers > 1 && layer_stride < (int64_t)n_rows * n_heads * ld_s) return SAN_ERR_SHAPE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaMemsetAsync(d_js, 0, sizeof(double) * n_layers * n_layers, st) != cudaSuccess) return SAN_ERR_CUDA;
+    const long long warps = (long long)n_rows * n_heads;
+    if (warps > 0 && n_layers > 1) {
+        JsParams p;
+        p.S = d_S; p.layer_stride = layer_stride; p.ld = ld_s; p.lens = d_lens;
+        p.n_layers = n_layers; p.n_rows = n_rows; p.n_heads = n_heads; p.js = d_js;
+        const long long grid = (warps + 7) / 8;
+        if (grid > 0x7fffffffLL) return SAN_ERR_SHAPE;
+        js_pairs_kernel<<<(unsigned)grid, 256, 0, st>>>(p);
+        if (cudaGetLastError() != cudaSuccess) return SAN_ERR_CUDA;
+    }
+    js_finish_kernel<<<n_layers, n_layers, 0, st>>>(d_js, n_layers, (double)warps);
+    return cuda_status(cudaGetLastError());
+}
+
+int32_t san_block_similarity(const double* js, int32_t n_layers, int32_t m, int32_t n, double* sim) {
+    if (!js || !sim) return SAN_ERR_NULL;
+    if (n_layers < 1 || n_layers > SAN_MAX_LAYERS) return SAN_ERR_SHAPE;
+    if (m < 0 || n >= n_layers || m >= n) return SAN_ERR_RANGE;
+    *sim = block_similarity(js, n_layers, m, n);
+    return SAN_OK;
+}
+
+int32_t san_policy_search(const double* js, int32_t n_layers, double theta, int32_t* sizes, int32_t* n_blocks) {
+    if (!js || !sizes || !n_blocks) return SAN_ERR_NULL;
+    if (n_layers < 1 || n_layers > SAN_MAX_LAYERS) return SAN_ERR_SHAPE;
+    if (!(theta == theta)) return SAN_ERR_RANGE;      // NaN compares false with everything
+    *n_blocks = search_policy(js, n_layers, theta, sizes);
+    return SAN_OK;
 }
 
 int32_t san_device_status(san_ctx* ctx, int32_t* first_error, int32_t* detail, void* stream) {

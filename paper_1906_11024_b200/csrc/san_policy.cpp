@@ -1,5 +1,7 @@
 #include "san_policy.h"
 
+#include <cmath>
+
 namespace san {
 
 int32_t policy_from_sizes(const int32_t* sizes, int32_t n_blocks, int32_t n_layers, Policy* out) {
@@ -44,6 +46,27 @@ int32_t policy_from_map(const int32_t* block_of_layer, int32_t n_layers, Policy*
     }
     *out = p;
     return SAN_OK;
+}
+
+double block_similarity(const double* js, int32_t n_layers, int32_t m, int32_t n) {
+    const double ln2 = std::log(2.0);
+    double mu = 0.0;
+    for (int32_t i = m; i <= n; ++i)
+        for (int32_t j = m; j <= n; ++j)
+            if (i != j) mu += ln2 - js[(int64_t)i * n_layers + j];
+    const double layers = (double)(n - m + 1);
+    return mu / (layers * (layers - 1.0));           // ordered pairs i != j inside the block
+}
+
+int32_t search_policy(const double* js, int32_t n_layers, double theta, int32_t* sizes) {
+    int32_t n_blocks = 0;
+    for (int32_t m = 0; m < n_layers;) {
+        int32_t top = m;                               // a block of one layer always qualifies
+        while (top + 1 < n_layers && block_similarity(js, n_layers, m, top + 1) >= theta) ++top;
+        sizes[n_blocks++] = top - m + 1;
+        m = top + 1;
+    }
+    return n_blocks;
 }
 
 }  // namespace san
