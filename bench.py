@@ -37,9 +37,10 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes read + written per launch of the step kernel, from the ncu capture summarised in
 # profiles/decode_step_base_long.md, and the digest of the kernel sources they were taken
 # with: once those sources change the counters no longer describe the kernel and the bench
-# line reports null until a new capture is recorded here.
-KERNEL_SOURCES = ("san_fused.cuh", "san_api.cu", "san_kernels.cuh")
-NCU_TRAFFIC = {"digest": "f7a74a902b0d071a", "fused": {"base": 70.2e6, "long": 762.2e6}}
+# line reports null until a new capture is recorded here.  (The choice of spans and layer
+# groups lives in san_api.cu; a change there calls for a new capture as well.)
+KERNEL_SOURCES = ("san_fused.cuh", "san_kernels.cuh")
+NCU_TRAFFIC = {"digest": "bc56d6bb56dcf9ab", "fused": {"base": 70.2e6, "long": 762.2e6}}
 
 
 def kernel_digest():
@@ -276,22 +277,27 @@ def dominant_kernel_bytes(w, pos):
 
 def time_e2e(w, dec, sb, steps, device, fused=True):
     """The same step with HOST buffers: every step copies its inputs from pinned host memory
-    to the device, runs the library calls, and reads the outputs back."""
+    to the device, runs the library, and reads the outputs back.  On the one-launch path this
+    is a single C-ABI call, san_decode_step_host, which issues the copies itself."""
     import torch
-    names_in = ["x_aan", "t_aan"] if w.self_is_aan else ["q_self", "k_new", "v_new"]
-    names_in += ["q_enc", "ids", "pos", "lens", "sent_ids", "src_lens"]
-    names_out = ["O_self", "O_enc"]
-    host_in = {k: getattr(sb, k).cpu().pin_memory() for k in names_in}
-    host_out = {k: torch.empty_like(getattr(sb, k), device="cpu").pin_memory() for k in names_out}
-    h2d = sum(t.numel() * t.element_size() for t in host_in.values())
-    d2h = sum(t.numel() * t.element_size() for t in host_out.values())
+    hb = dec.host_buffers(sb)
+    lens_host = sb.lens.cpu().pin_memory()           # the separate calls take lengths, the one-launch step positions
+    h2d = sum(hb[k].numel() * hb[k].element_size() for k in hb["_in"]) + (0 if fused else lens_host.numel() * 4)
+    d2h = sum(hb[k].numel() * hb[k].element_size() for k in hb["_out"])
+    dev_of = {"d_seq_ids": "ids", "d_pos": "pos", "d_sent_ids": "sent_ids", "d_src_lens": "src_lens",
+              "d_q_enc": "q_enc", "d_q_self": "q_self", "d_k_new": "k_new", "d_v_new": "v_new",
+              "d_x_aan": "x_aan", "d_t": "t_aan", "d_O_self": "O_self", "d_O_enc": "O_enc"}
 
     def one():
-        for k, t in host_in.items():
-            getattr(sb, k).copy_(t, non_blocking=True)
-        dec.step_fused(sb) if fused else dec.step(sb)
-        for k, t in host_out.items():
-            t.copy_(getattr(sb, k), non_blocking=True)
+        if fused:
+            dec.step_fused_host(sb, hb)
+            return
+        for k in hb["_in"]:
+            getattr(sb, dev_of[k]).copy_(hb[k], non_blocking=True)
+        sb.lens.copy_(lens_host, non_blocking=True)
+        dec.step(sb)
+        for k in hb["_out"]:
+            hb[k].copy_(getattr(sb, dev_of[k]), non_blocking=True)
 
     for _ in range(3):
         one()
@@ -303,6 +309,74 @@ def time_e2e(w, dec, sb, steps, device, fused=True):
     e1.record()
     torch.cuda.synchronize(device)
     return e0.elapsed_time(e1) * 1e-3, h2d, d2h
+
+
+def time_beam_reorder(w, decs, sbs, pos, device, peak, reps=10):
+    """The step next to the path in a beam-search decoder: san_beam_reorder with every beam
+    taking over the whole history of its neighbour (parent = slot + 1 mod beam), so that every
+    cached row of every self-attention plane moves; launches rotate over the replicas."""
+    import torch
+    from paper_1906_11024_b200 import binding as B
+    R = len(decs)
+    sent = torch.arange(w.n_sent, dtype=torch.int32, device=device)
+    parent = ((torch.arange(w.beam, dtype=torch.int32, device=device) + 1) % w.beam).repeat(w.n_sent, 1).contiguous()
+    lens = torch.from_numpy((pos + 1).astype(np.int32)).to(device).view(w.n_sent, w.beam).contiguous()
+    max_len = int(pos.max()) + 1
+
+    def all_replicas():
+        for r in range(R):
+            B.check(B.san_beam_reorder(decs[r].ctx, sent, parent, lens, w.n_sent, max_len), "san_beam_reorder")
+
+    g = capture(all_replicas, device)
+    for _ in range(3):
+        g.replay()
+    torch.cuda.synchronize(device)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        g.replay()
+    e1.record()
+    torch.cuda.synchronize(device)
+    secs = e0.elapsed_time(e1) * 1e-3 / (reps * R)
+    if w.self_is_aan:
+        moved = w.n_layers * w.n_seqs * w.d_model * 4
+    else:
+        moved = (len(w.self_blocks) + w.n_layers) * int((pos.astype(np.int64) + 1).sum()) * w.d_model * w.elem_bytes
+    gbs = 2 * moved / secs / 1e9                      # every piece is read once and written once
+    return {"call": "san_beam_reorder", "us_per_launch": secs * 1e6, "bytes_per_launch": 2 * moved,
+            "achieved_gbs": gbs, "frac_of_peak": gbs / peak, "bound": "hbm",
+            "note": "all beams change parent; launches of the AAN workload move only the running sums"}
+
+
+def time_js_matrix(w, dec, sb, pos, device, reps=50):
+    """Policy learner, device part: san_js_matrix over the self-attention weights that an
+    unshared decode step wrote (one S per layer)."""
+    import torch
+    from paper_1906_11024_b200 import binding as B
+    if w.self_is_aan or sb.S_self is None or sb.S_self.shape[0] < 2:
+        return None
+    M = sb.S_self.shape[0]
+    lens = torch.from_numpy((pos + 1).astype(np.int32)).to(device)
+    djs = torch.zeros(M, M, dtype=torch.float64, device=device)
+
+    def one():
+        B.check(B.san_js_matrix(M, sb.S_self, sb.S_self.stride(0), dec.ld_t, w.n_seqs, w.n_heads, lens, djs), "san_js_matrix")
+
+    g = capture(one, device)
+    for _ in range(3):
+        g.replay()
+    torch.cuda.synchronize(device)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        g.replay()
+    e1.record()
+    torch.cuda.synchronize(device)
+    secs = e0.elapsed_time(e1) * 1e-3 / reps
+    nbytes = M * w.n_heads * int((pos.astype(np.int64) + 1).sum()) * 4
+    return {"call": "san_js_matrix", "layers": M, "us_per_call": secs * 1e6, "bytes_per_call": nbytes,
+            "achieved_gbs": nbytes / secs / 1e9,
+            "note": "three launches (clear, pairs, finish) over weights that fit in L2: launch-bound, not a roofline case"}
 
 
 # ------------------------------------------------------------------------- the CPU oracle arm
@@ -466,6 +540,9 @@ def main():
         dom_bytes, dom_name = dominant_kernel_bytes(w, pos), "san_attn_apply (apply_kernel)"
     e2e_s, h2d, d2h = time_e2e(w, decs[0], sbs[0], min(args.steps, 100), device, fused)
     e2e_steps = min(args.steps, 100)
+    next_rows = {}
+    if rank == 0:
+        next_rows["beam_reorder"] = time_beam_reorder(w, decs, sbs, pos, device, peak)
 
     unshared = None
     if not args.no_unshared and rank == 0:
@@ -480,6 +557,9 @@ def main():
         unshared = {"value": wu.n_seqs * args.steps / su, "unit": UNIT, "ms_per_step": su / args.steps * 1e3,
                     "kv_bytes_per_step": abu["kv"], "bytes_per_step": abu["total"],
                     "hbm_gbs": abu["total"] / (su / args.steps) / 1e9, "gpu_launches_per_step": lu}
+        js = time_js_matrix(wu, decs_u[0], sbs_u[0], pos, device)
+        if js is not None:
+            next_rows["policy_learner"] = js
         for d in decs_u:
             d.close()
         del decs_u, sbs_u
@@ -516,6 +596,8 @@ def main():
                 "d2h_bytes_per_step": d2h, "ms_per_step": e2e_s / e2e_steps * 1e3},
         "clocks": clocks,
     }
+    if next_rows:
+        line["next_rows"] = next_rows
     if unshared is not None:
         unshared["speedup_from_sharing"] = value / world / unshared["value"]
         unshared["kv_bytes_ratio_shared_over_unshared"] = ab["kv"] / unshared["kv_bytes_per_step"]

@@ -203,6 +203,18 @@ typedef struct {
 } san_step_args;
 int32_t san_decode_step(san_ctx* ctx, const san_step_args* args, void* stream);
 
+/* san_decode_step for a caller whose step inputs and outputs live in HOST memory (pinned
+ * memory if the copies are to overlap anything): the same step (Eq. 1-5, Section 4.1) with
+ * the transfers issued by the library on `stream`, in order: every input array named in
+ * `host` is copied into the array of the same field in `dev`, san_decode_step(ctx, dev) is
+ * launched, then O_self and O_enc (and S_self / S_enc where both structs name a buffer) are
+ * copied back into `host`.  `dev` is a complete argument block of caller-owned device
+ * buffers and carries the counts, bounds and leading dimensions; the pointer fields of
+ * `host` are HOST pointers of the same shapes (its scalar fields are ignored).  Nothing is
+ * allocated and the host is not synchronised: `host` outputs are valid once `stream` has
+ * reached this point, and `host` inputs must stay untouched until then. */
+int32_t san_decode_step_host(san_ctx* ctx, const san_step_args* host, const san_step_args* dev, void* stream);
+
 /* Beam-search cache reorder (Section 4.1: decoding runs a beam of hypotheses per sentence;
  * after a step each surviving hypothesis continues the attention cache of the hypothesis it
  * extends).  For item i = sentence d_sent_ids[i] and beam slot s, the sequence

@@ -29,7 +29,7 @@ EXPORTS = (
     "san_policy_set_sizes", "san_policy_set_map", "san_policy_get_map",
     "san_cache_append", "san_attn_weights", "san_attn_apply", "san_aan_step",
     "san_device_status", "san_status_string", "san_attn_weights_static", "san_decode_step",
-    "san_beam_reorder", "san_js_matrix", "san_block_similarity", "san_policy_search",
+    "san_decode_step_host", "san_beam_reorder", "san_js_matrix", "san_block_similarity", "san_policy_search",
 )
 
 
@@ -84,6 +84,7 @@ def lib():
     L.san_device_status.argtypes = [vp, _I32P, _I32P, vp]
     L.san_attn_weights_static.argtypes = [i32, i32, i32, vp, vp, i32, i32, vp, vp, i32, i32, vp, i64, vp, vp]
     L.san_decode_step.argtypes = [vp, C.POINTER(san_step_args), vp]
+    L.san_decode_step_host.argtypes = [vp, C.POINTER(san_step_args), C.POINTER(san_step_args), vp]
     L.san_beam_reorder.argtypes = [vp, vp, vp, vp, i32, i32, vp]
     L.san_js_matrix.argtypes = [i32, vp, i64, i64, i32, i32, vp, vp, vp]
     L.san_block_similarity.argtypes = [C.POINTER(C.c_double), i32, i32, i32, C.POINTER(C.c_double)]
@@ -251,3 +252,22 @@ def san_policy_search(js, n_layers, theta):
     nb = C.c_int32(0)
     rc = lib().san_policy_search(_f64_matrix(js, n_layers), n_layers, float(theta), sizes, C.byref(nb))
     return rc, list(sizes[:nb.value]) if rc == SAN_OK else []
+
+
+def step_args(**kw) -> san_step_args:
+    """A san_step_args block from keyword arguments named like its fields (tensors, addresses or None)."""
+    a = san_step_args()
+    for name, _ in san_step_args._fields_:
+        v = kw.pop(name, None)
+        if name in ("n_seqs", "max_len", "n_sent", "max_src", "ld_t", "ld_s"):
+            setattr(a, name, int(v or 0))
+        else:
+            setattr(a, name, _ptr(v))
+    if kw:
+        raise TypeError(f"unknown san_step_args fields: {sorted(kw)}")
+    return a
+
+
+def san_decode_step_host(ctx, host: san_step_args, dev: san_step_args, stream=None) -> int:
+    """san_decode_step with host-resident inputs and outputs: copies in, one launch, copies out."""
+    return lib().san_decode_step_host(ctx, C.byref(host), C.byref(dev), _stream(stream))

@@ -551,6 +551,53 @@ int32_t san_decode_step(san_ctx* ctx, const san_step_args* a, void* stream) {
     return cuda_status(e);
 }
 
+int32_t san_decode_step_host(san_ctx* ctx, const san_step_args* h, const san_step_args* d, void* stream) {
+    if (!ctx || !h || !d) return SAN_ERR_NULL;
+    const san_config& c = ctx->cfg;
+    const bool aan = c.self_is_aan != 0;
+    const int n_seqs = d->n_seqs, n_sent = d->n_sent;
+    if (n_seqs < 0 || n_seqs > ctx->n_seqs || n_sent < 0 || n_sent > c.max_sent) return SAN_ERR_SHAPE;
+    const size_t row = (size_t)c.n_heads * kDh * ctx->elem_bytes;           // one sequence, all heads
+    const size_t Ns = (size_t)ctx->self_pol.n_blocks, Ne = (size_t)ctx->enc_pol.n_blocks, M = (size_t)c.n_layers;
+    const size_t n_enc_out = c.encdec_shared_context ? Ne : M;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    struct Copy { const void* from; const void* to; size_t bytes; };
+    // inputs: host -> the caller's device buffers
+    const Copy in[] = {
+        {h->d_seq_ids, d->d_seq_ids, n_seqs * sizeof(int32_t)},
+        {aan ? nullptr : h->d_pos, d->d_pos, n_seqs * sizeof(int32_t)},
+        {aan ? nullptr : h->d_q_self, d->d_q_self, Ns * n_seqs * row},
+        {aan ? nullptr : h->d_k_new, d->d_k_new, Ns * n_seqs * row},
+        {aan ? nullptr : h->d_v_new, d->d_v_new, M * n_seqs * row},
+        {aan ? h->d_x_aan : nullptr, d->d_x_aan, M * n_seqs * row},
+        {aan ? h->d_t : nullptr, d->d_t, n_seqs * sizeof(int32_t)},
+        {h->d_sent_ids, d->d_sent_ids, n_sent * sizeof(int32_t)},
+        {h->d_src_lens, d->d_src_lens, n_sent * sizeof(int32_t)},
+        {h->d_q_enc, d->d_q_enc, Ne * n_sent * c.beam * row},
+    };
+    for (const Copy& cp : in) {
+        if (cp.bytes == 0 || (!cp.from && !cp.to)) continue;
+        if (!cp.from || !cp.to) return SAN_ERR_NULL;
+    }
+    const Copy out[] = {
+        {d->d_O_self, h->d_O_self, M * n_seqs * row},
+        {d->d_O_enc, h->d_O_enc, n_enc_out * n_sent * c.beam * row},
+        {d->d_S_self, h->d_S_self, aan ? 0 : Ns * n_seqs * c.n_heads * (size_t)d->ld_t * sizeof(float)},
+        {d->d_S_enc, h->d_S_enc, Ne * n_sent * c.beam * c.n_heads * (size_t)d->ld_s * sizeof(float)},
+    };
+    for (int i = 0; i < 2; ++i)
+        if (out[i].bytes && (!out[i].from || !out[i].to)) return SAN_ERR_NULL;
+    for (const Copy& cp : in)
+        if (cp.bytes && cp.from && cudaMemcpyAsync(const_cast<void*>(cp.to), cp.from, cp.bytes, cudaMemcpyHostToDevice, st) != cudaSuccess)
+            return SAN_ERR_CUDA;
+    const int32_t rc = san_decode_step(ctx, d, stream);
+    if (rc != SAN_OK) return rc;
+    for (const Copy& cp : out)      // S comes back only if the host asked for it and the device step stored it
+        if (cp.bytes && cp.from && cp.to && cudaMemcpyAsync(const_cast<void*>(cp.to), cp.from, cp.bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+            return SAN_ERR_CUDA;
+    return SAN_OK;
+}
+
 int32_t san_beam_reorder(san_ctx* ctx, const int32_t* d_sent_ids, const int32_t* d_parent,
                          const int32_t* d_lens, int32_t n_sent, int32_t max_len, void* stream) {
     if (!ctx || !d_sent_ids || !d_parent || !d_lens) return SAN_ERR_NULL;
@@ -562,39 +609,40 @@ int32_t san_beam_reorder(san_ctx* ctx, const int32_t* d_sent_ids, const int32_t*
     ReorderParams p;
     std::memset(&p, 0, sizeof(p));
     p.sent_ids = d_sent_ids; p.parent = d_parent; p.lens = d_lens;
-    p.n_sent = n_sent; p.beam = c.beam; p.max_sent = c.max_sent; p.err = ctx->err;
-    const int per_beam = kReorderTile / c.beam;
+    p.n_sent = n_sent; p.beam = c.beam; p.max_sent = c.max_sent; p.max_units = max_len; p.err = ctx->err;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    auto launch = [&](const ReorderParams& q) -> int32_t {
+        const long long gx = (long long)q.tiles_per_panel * q.n_heads * q.n_sent;
+        if (gx > 0x7fffffffLL || q.n_planes > 65535) return SAN_ERR_SHAPE;
+        beam_reorder_kernel<<<dim3((unsigned)gx, (unsigned)q.n_planes), kReorderThreads, 0, st>>>(q);
+        return cuda_status(cudaGetLastError());
+    };
     if (c.self_is_aan) {       // the running sums [layer][sequence][H*64] float32
         p.base = ctx->cache + ctx->off_aan; p.plane_bytes = (long long)ctx->aan_plane_bytes;
         p.n_planes = c.n_layers; p.n_heads = 1; p.head_bytes = 0;
-        p.fixed_bytes = c.n_heads * kDh * (int)sizeof(float);
-        p.seq_bytes = p.fixed_bytes; p.unit_bytes = 0; p.max_units = max_len;
-        p.tiles_per_panel = ceil_div(p.fixed_bytes / 16, per_beam);
-    } else {                   // key planes of the blocks, then value planes of the layers: adjacent in the arena
-        const int row_bytes = kDh * ctx->elem_bytes;
-        p.base = ctx->cache + ctx->off_self_k; p.plane_bytes = (long long)ctx->self_plane_bytes;
-        p.n_planes = ctx->self_pol.n_blocks + ctx->n_self_v_planes; p.n_heads = c.n_heads;
-        p.head_bytes = (long long)c.max_tgt_len * row_bytes;
-        p.seq_bytes = p.head_bytes * c.n_heads;
-        p.unit_bytes = row_bytes; p.fixed_bytes = 0; p.max_units = max_len;
-        p.tiles_per_panel = ceil_div(max_len * (row_bytes / 16), per_beam);
+        p.fixed_pieces = c.n_heads * kDh * (int)sizeof(float) / 16;
+        p.seq_bytes = (long long)p.fixed_pieces * 16;
+        p.tiles_per_panel = ceil_div(p.fixed_pieces, kReorderThreads);
+        return launch(p);
     }
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (!c.self_is_aan && ctx->self_pol.n_blocks < ctx->n_self_k_planes) {
+    // key planes of the blocks and value planes of the layers, same geometry
+    const int row_bytes = kDh * ctx->elem_bytes;
+    p.n_heads = c.n_heads; p.plane_bytes = (long long)ctx->self_plane_bytes;
+    p.head_bytes = (long long)c.max_tgt_len * row_bytes;
+    p.seq_bytes = p.head_bytes * c.n_heads;
+    p.unit_pieces = row_bytes / 16;
+    if ((long long)max_len * p.unit_pieces > 0x7fffffffLL) return SAN_ERR_SHAPE;
+    p.tiles_per_panel = ceil_div(max_len * p.unit_pieces, kReorderThreads);
+    p.base = ctx->cache + ctx->off_self_k; p.n_planes = ctx->self_pol.n_blocks + ctx->n_self_v_planes;
+    if (ctx->self_pol.n_blocks < ctx->n_self_k_planes) {
         // the policy in force uses fewer key planes than the arena holds: the unused planes lie
         // between the used key planes and the value planes, so the two runs are launched apart
-        ReorderParams pk = p;
-        pk.n_planes = ctx->self_pol.n_blocks;
-        const long long gk = (long long)pk.n_planes * n_sent * pk.n_heads * pk.tiles_per_panel;
-        if (gk > 0x7fffffffLL) return SAN_ERR_SHAPE;
-        beam_reorder_kernel<<<(unsigned)gk, kReorderThreads, 0, st>>>(pk);
-        if (cudaGetLastError() != cudaSuccess) return SAN_ERR_CUDA;
+        p.n_planes = ctx->self_pol.n_blocks;
+        const int32_t rc = launch(p);
+        if (rc != SAN_OK) return rc;
         p.base = ctx->cache + ctx->off_self_v; p.n_planes = ctx->n_self_v_planes;
     }
-    const long long grid = (long long)p.n_planes * n_sent * p.n_heads * p.tiles_per_panel;
-    if (grid > 0x7fffffffLL) return SAN_ERR_SHAPE;
-    beam_reorder_kernel<<<(unsigned)grid, kReorderThreads, 0, st>>>(p);
-    return cuda_status(cudaGetLastError());
+    return launch(p);
 }
 
 int32_t san_js_matrix(int32_t n_layers, const float* d_S, int64_t layer_stride, int64_t ld_s,

@@ -17,9 +17,7 @@
 
 namespace san {
 
-constexpr int kReorderThreads = 256;
-constexpr int kReorderPieces = 4;                                      // 16-byte pieces per thread
-constexpr int kReorderTile = kReorderThreads * kReorderPieces;         // pieces per tile, all beams together
+constexpr int kReorderThreads = 256;      // one 16-byte piece per thread and beam: a tile is 4 KB of every beam
 
 // The tile is written later in the same kernel, so the read-only (non-coherent) path is not
 // allowed here: an ordinary load, kept out of L1 because every piece is read once.
@@ -37,49 +35,52 @@ struct ReorderParams {
     long long head_bytes;          // between the heads of a sequence (unused when n_heads == 1)
     const int* sent_ids; const int* parent; const int* lens;    // [n_sent], [n_sent][beam], [n_sent][beam]
     int n_planes, n_sent, n_heads, beam, max_sent;
-    int unit_bytes;                // bytes per unit of lens (a cached row)
-    int fixed_bytes;               // > 0: every beam with lens > 0 moves this many bytes (AAN sums)
+    int unit_pieces;               // 16-byte pieces per unit of lens (a cached row)
+    int fixed_pieces;              // > 0: every beam with lens > 0 moves this many pieces (AAN sums)
     int max_units;                 // limit of lens (row capacity)
     int tiles_per_panel;           // tiles covering the longest run the host allows
     int* err;
 };
 
-// grid = n_planes * n_sent * n_heads * tiles_per_panel CTAs
+// grid = (tiles_per_panel * n_heads * n_sent, n_planes).  Thread t of tile k owns piece
+// k * 256 + t of the (plane, sentence, head) panel in every beam: it loads the piece of each
+// beam's parent, the CTA meets at a barrier, it stores.  The address arithmetic that does not
+// depend on the beam is done once per thread; the copy itself is a handful of instructions
+// per piece, so that the kernel is bound by HBM and not by instruction issue.
 static __global__ void __launch_bounds__(kReorderThreads) beam_reorder_kernel(const ReorderParams p) {
     unsigned u = blockIdx.x;
     const int tile = (int)(u % (unsigned)p.tiles_per_panel); u /= (unsigned)p.tiles_per_panel;
-    const int h = (int)(u % (unsigned)p.n_heads); u /= (unsigned)p.n_heads;
-    const int item = (int)(u % (unsigned)p.n_sent);
-    const int plane = (int)(u / (unsigned)p.n_sent);
-    const int per_beam = kReorderTile / p.beam;            // pieces of one beam in a tile
+    const int h = (int)(u % (unsigned)p.n_heads);
+    const int item = (int)(u / (unsigned)p.n_heads);
+    const int plane = blockIdx.y;
     const int sent = p.sent_ids[item];
-    const bool reporter = (plane == 0 && h == 0 && tile == 0);
-    const bool sent_ok = sent >= 0 && sent < p.max_sent;
-    if (!sent_ok && reporter && threadIdx.x == 0) record_error(p.err, TAG_REORDER, item, sent, p.max_sent);
-
-    uint4 v[kReorderPieces];
-    char* dst[kReorderPieces];
+    const bool reporter = (plane == 0 && h == 0 && tile == 0 && threadIdx.x == 0);
+    if (sent < 0 || sent >= p.max_sent) {                  // uniform over the CTA
+        if (reporter) record_error(p.err, TAG_REORDER, item, sent, p.max_sent);
+        return;
+    }
+    const int piece = tile * kReorderThreads + (int)threadIdx.x;
+    char* panel = p.base + (long long)plane * p.plane_bytes + (long long)h * p.head_bytes +
+                  (long long)sent * p.beam * p.seq_bytes + (long long)piece * 16;
+    const int* parent = p.parent + item * p.beam;
+    const int* lens = p.lens + item * p.beam;
+    uint4 v[SAN_MAX_BEAM];
+    unsigned take = 0;                                     // beams whose piece this thread moves
 #pragma unroll
-    for (int r = 0; r < kReorderPieces; ++r) {
-        dst[r] = nullptr;
-        const int e = r * kReorderThreads + (int)threadIdx.x;      // consecutive threads: consecutive pieces of a beam
-        const int s = e / per_beam, k = e - s * per_beam;
-        if (!sent_ok || s >= p.beam) continue;
-        const int par = p.parent[item * p.beam + s], len = p.lens[item * p.beam + s];
-        if (par < 0 || par >= p.beam) { if (reporter && k == 0) record_error(p.err, TAG_REORDER, item * p.beam + s, par, p.beam); continue; }
-        if (len < 0 || len > p.max_units) { if (reporter && k == 0) record_error(p.err, TAG_REORDER, item * p.beam + s, len, p.max_units); continue; }
-        if (par == s) continue;                                    // keeps its own history
-        const long long bytes = p.fixed_bytes > 0 ? (len > 0 ? (long long)p.fixed_bytes : 0) : (long long)len * p.unit_bytes;
-        const long long off = ((long long)tile * per_beam + k) * 16;
-        if (off >= bytes) continue;
-        char* panel = p.base + (long long)plane * p.plane_bytes + (long long)h * p.head_bytes + off;
-        v[r] = ld16_once(panel + ((long long)sent * p.beam + par) * p.seq_bytes);
-        dst[r] = panel + ((long long)sent * p.beam + s) * p.seq_bytes;
+    for (int s = 0; s < SAN_MAX_BEAM; ++s) {
+        if (s >= p.beam) break;
+        const int par = parent[s], len = lens[s];
+        if (par < 0 || par >= p.beam) { if (reporter) record_error(p.err, TAG_REORDER, item * p.beam + s, par, p.beam); continue; }
+        if (len < 0 || len > p.max_units) { if (reporter) record_error(p.err, TAG_REORDER, item * p.beam + s, len, p.max_units); continue; }
+        const int pieces = p.fixed_pieces > 0 ? (len > 0 ? p.fixed_pieces : 0) : len * p.unit_pieces;
+        if (par == s || piece >= pieces) continue;         // keeps its own history / beyond the rows taken
+        v[s] = ld16_once(panel + par * p.seq_bytes);
+        take |= 1u << s;
     }
     __syncthreads();            // every piece of the tile that is needed has been read
 #pragma unroll
-    for (int r = 0; r < kReorderPieces; ++r)
-        if (dst[r]) *reinterpret_cast<uint4*>(dst[r]) = v[r];
+    for (int s = 0; s < SAN_MAX_BEAM; ++s)
+        if (take & (1u << s)) *reinterpret_cast<uint4*>(panel + s * p.seq_bytes) = v[s];
 }
 
 }  // namespace san

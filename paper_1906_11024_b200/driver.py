@@ -209,6 +209,45 @@ class Decoder:
         B.check(B.san_decode_step(self.ctx, **kw), "san_decode_step")
         return 1
 
+    def _dev_step_args(self, sb: StepBuffers) -> dict:
+        w = self.w
+        n, n_sent = sb.ids.shape[0], sb.sent_ids.shape[0]
+        kw = dict(d_seq_ids=sb.ids, n_seqs=n, max_len=sb.max_len, d_O_self=sb.O_self,
+                  d_q_enc=sb.q_enc, d_sent_ids=sb.sent_ids, d_src_lens=sb.src_lens, n_sent=n_sent, max_src=sb.max_src,
+                  d_S_enc=sb.S_enc, ld_s=self.ld_s, d_O_enc=sb.O_enc)
+        if w.self_is_aan:
+            kw.update(d_x_aan=sb.x_aan, d_t=sb.t_aan)
+        else:
+            kw.update(d_q_self=sb.q_self, d_k_new=sb.k_new, d_v_new=sb.v_new, d_pos=sb.pos, d_S_self=sb.S_self,
+                      ld_t=self.ld_t)
+        return kw
+
+    def host_buffers(self, sb: StepBuffers, want_S: bool = False) -> dict:
+        """Pinned host copies of the step's inputs and pinned room for its outputs, keyed by
+        the san_step_args field they stand for."""
+        names_in = {"d_seq_ids": sb.ids, "d_sent_ids": sb.sent_ids, "d_src_lens": sb.src_lens, "d_q_enc": sb.q_enc}
+        if self.w.self_is_aan:
+            names_in.update(d_x_aan=sb.x_aan, d_t=sb.t_aan)
+        else:
+            names_in.update(d_pos=sb.pos, d_q_self=sb.q_self, d_k_new=sb.k_new, d_v_new=sb.v_new)
+        names_out = {"d_O_self": sb.O_self, "d_O_enc": sb.O_enc}
+        if want_S:
+            names_out["d_S_enc"] = sb.S_enc
+            if sb.S_self is not None:
+                names_out["d_S_self"] = sb.S_self
+        hb = {k: t.cpu().pin_memory() for k, t in names_in.items()}
+        hb.update({k: torch.empty_like(t, device="cpu").pin_memory() for k, t in names_out.items()})
+        hb["_in"], hb["_out"] = list(names_in), list(names_out)
+        return hb
+
+    def step_fused_host(self, sb: StepBuffers, hb: dict, stream=None) -> int:
+        """The decode step through san_decode_step_host: inputs come from and outputs go to the
+        pinned host tensors of ``hb``; the library issues the copies around its one launch."""
+        host = B.step_args(**{k: hb[k] for k in hb["_in"] + hb["_out"]})
+        dev = B.step_args(**self._dev_step_args(sb))
+        B.check(B.san_decode_step_host(self.ctx, host, dev, stream), "san_decode_step_host")
+        return 1
+
     def device_status(self, stream=None):
         rc, first_error, detail = B.san_device_status(self.ctx, stream)
         B.check(rc, "san_device_status")

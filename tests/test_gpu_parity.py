@@ -228,3 +228,37 @@ def test_one_launch_step_writes_the_cache_like_append():
     assert a.device_status()[0] == 0 and b.device_status()[0] == 0
     assert torch.equal(a.cache, b.cache)
     a.close(); b.close()
+
+
+@pytest.mark.parametrize("name", ["tiny", "aan"])
+def test_host_buffer_step_equals_oracle(name):
+    """san_decode_step_host: inputs in pinned host memory, outputs read back by the library."""
+    w = synth.WORKLOADS[name] if name == "tiny" else synth.scaled(synth.WORKLOADS[name], 3)
+    dec = Decoder(w)
+    orc = OracleRun(w)
+    dec.load_encoder_memory()
+    ids = np.arange(w.n_seqs, dtype=np.int32)
+    tol = TOL[w.dtype]
+    for step in range(5):
+        pos = np.full(w.n_seqs, step, np.int32)
+        sb = dec.new_step_buffers()
+        host = dec.fill_step_inputs(sb, step, ids, pos)
+        hb = dec.host_buffers(sb, want_S=True)
+        for k in hb["_in"]:                       # the device copies of the inputs must come from the host side
+            if hb[k].dtype != torch.int32:
+                getattr(sb, {"d_q_enc": "q_enc", "d_q_self": "q_self", "d_k_new": "k_new", "d_v_new": "v_new",
+                             "d_x_aan": "x_aan"}[k]).zero_()
+        dec.step_fused_host(sb, hb)
+        torch.cuda.synchronize()
+        assert dec.device_status()[0] == 0
+        ref = orc.step(host, ids, pos)
+        for key, want in (("d_O_self", ref["O_self"]), ("d_O_enc", ref["O_enc"])):
+            assert normwise_err(hb[key].to(torch.float32).numpy(), want) <= tol, (name, step, key)
+        L = step + 1
+        if not w.self_is_aan:
+            assert weights_err(hb["d_S_self"].numpy()[..., :L], ref["S_self"][..., :L]) <= TOL_S
+        src_seq = np.repeat(w.src_lens(), w.beam)
+        S = hb["d_S_enc"].numpy()
+        for i in range(S.shape[1]):
+            assert weights_err(S[:, i, :, :src_seq[i]], ref["S_enc"][:, i, :, :src_seq[i]]) <= TOL_S
+    dec.close()
