@@ -231,6 +231,24 @@ int32_t san_decode_step_host(san_ctx* ctx, const san_step_args* host, const san_
 int32_t san_beam_reorder(san_ctx* ctx, const int32_t* d_sent_ids, const int32_t* d_parent,
                          const int32_t* d_lens, int32_t n_sent, int32_t max_len, void* stream);
 
+/* Full-sequence shared attention (the encoder-side use of Table 5; with causal != 0 the
+ * prefill of a decoder prompt): for every sequence i and head, the l x l weights
+ *   S = Softmax(Q.K^T / sqrt(64)),  l = d_lens[i],  query row a over keys 0..l-1 (0..a when causal)
+ * are computed once from the queries and keys of the block's lowest layer (Eq. 1, Eq. 3) and
+ * applied to the values of each of the block's n_layers layers (Eq. 2, Eq. 4) in the same
+ * launch.  Needs no context and allocates nothing.
+ *   d_q, d_k  [n_seq][cap_len][n_heads][64]            (the order a projection writes them)
+ *   d_v       [n_layers][n_seq][cap_len][n_heads][64]
+ *   d_out     [n_layers][n_seq][cap_len][n_heads][64]  rows at or beyond d_lens[i] are not written
+ *   d_S       optional [n_seq][n_heads][cap_len][ld_s] float32; entries a row does not attend
+ *             to (causal) are written as 0, entries at or beyond d_lens[i] are not written
+ * dtype must be SAN_BF16 (SAN_F32 is refused with SAN_ERR_UNSUPPORTED: tensor-core products
+ * of float32 inputs would not meet the float32 tolerance).  max_len is a host bound on d_lens
+ * (0 = cap_len); a longer length is cut to max_len; max_len above 512 is SAN_ERR_UNSUPPORTED. */
+int32_t san_full_block(int32_t dtype, int32_t n_heads, int32_t n_layers, int32_t causal, const void* d_q,
+                       const void* d_k, const void* d_v, const int32_t* d_lens, int32_t n_seq, int32_t cap_len,
+                       int32_t max_len, float* d_S, int64_t ld_s, void* d_out, void* stream);
+
 /* Policy learning (Section 3.1, Section 3.3, Eq. 6).
  *
  * san_js_matrix: the Jensen-Shannon divergence between the attention weights of every pair

@@ -29,7 +29,7 @@ EXPORTS = (
     "san_policy_set_sizes", "san_policy_set_map", "san_policy_get_map",
     "san_cache_append", "san_attn_weights", "san_attn_apply", "san_aan_step",
     "san_device_status", "san_status_string", "san_attn_weights_static", "san_decode_step",
-    "san_decode_step_host", "san_beam_reorder", "san_js_matrix", "san_block_similarity", "san_policy_search",
+    "san_decode_step_host", "san_full_block", "san_beam_reorder", "san_js_matrix", "san_block_similarity", "san_policy_search",
 )
 
 
@@ -85,6 +85,7 @@ def lib():
     L.san_attn_weights_static.argtypes = [i32, i32, i32, vp, vp, i32, i32, vp, vp, i32, i32, vp, i64, vp, vp]
     L.san_decode_step.argtypes = [vp, C.POINTER(san_step_args), vp]
     L.san_decode_step_host.argtypes = [vp, C.POINTER(san_step_args), C.POINTER(san_step_args), vp]
+    L.san_full_block.argtypes = [i32, i32, i32, i32, vp, vp, vp, vp, i32, i32, i32, vp, i64, vp, vp]
     L.san_beam_reorder.argtypes = [vp, vp, vp, vp, i32, i32, vp]
     L.san_js_matrix.argtypes = [i32, vp, i64, i64, i32, i32, vp, vp, vp]
     L.san_block_similarity.argtypes = [C.POINTER(C.c_double), i32, i32, i32, C.POINTER(C.c_double)]
@@ -271,3 +272,10 @@ def step_args(**kw) -> san_step_args:
 def san_decode_step_host(ctx, host: san_step_args, dev: san_step_args, stream=None) -> int:
     """san_decode_step with host-resident inputs and outputs: copies in, one launch, copies out."""
     return lib().san_decode_step_host(ctx, C.byref(host), C.byref(dev), _stream(stream))
+
+
+def san_full_block(dtype, n_heads, n_layers, causal, d_q, d_k, d_v, d_lens, n_seq, cap_len, max_len, d_S, ld_s,
+                   d_out, stream=None) -> int:
+    """Full-sequence shared attention: S once per block, applied to every layer's values."""
+    return lib().san_full_block(dtype, n_heads, n_layers, int(causal), _ptr(d_q), _ptr(d_k), _ptr(d_v), _ptr(d_lens),
+                                n_seq, cap_len, max_len, _ptr(d_S), ld_s, _ptr(d_out), _stream(stream))

@@ -11,6 +11,7 @@
 #include "san_fused.cuh"
 #include "san_reorder.cuh"
 #include "san_learn.cuh"
+#include "san_full.cuh"
 
 using namespace san;
 
@@ -643,6 +644,37 @@ int32_t san_beam_reorder(san_ctx* ctx, const int32_t* d_sent_ids, const int32_t*
         p.base = ctx->cache + ctx->off_self_v; p.n_planes = ctx->n_self_v_planes;
     }
     return launch(p);
+}
+
+int32_t san_full_block(int32_t dtype, int32_t n_heads, int32_t n_layers, int32_t causal, const void* d_q,
+                       const void* d_k, const void* d_v, const int32_t* d_lens, int32_t n_seq, int32_t cap_len,
+                       int32_t max_len, float* d_S, int64_t ld_s, void* d_out, void* stream) {
+    if (!d_q || !d_k || !d_v || !d_lens || !d_out) return SAN_ERR_NULL;
+    if (dtype != SAN_BF16) return dtype == SAN_F32 ? SAN_ERR_UNSUPPORTED : SAN_ERR_DTYPE;
+    if (n_heads < 1 || n_heads > 65535 || n_layers < 1 || n_layers > SAN_MAX_LAYERS) return SAN_ERR_SHAPE;
+    if (n_seq < 0 || n_seq > 65535 || cap_len < 1) return SAN_ERR_SHAPE;
+    if (max_len == 0) max_len = cap_len;
+    if (max_len < 1 || max_len > cap_len) return SAN_ERR_SHAPE;
+    if (max_len > kFullMaxLen) return SAN_ERR_UNSUPPORTED;
+    if (d_S && ld_s < max_len) return SAN_ERR_SHAPE;
+    if (n_seq == 0) return SAN_OK;
+    FullParams p;
+    p.q = static_cast<const __nv_bfloat16*>(d_q); p.k = static_cast<const __nv_bfloat16*>(d_k);
+    p.v = static_cast<const __nv_bfloat16*>(d_v); p.out = static_cast<__nv_bfloat16*>(d_out);
+    p.S = d_S; p.ld_s = ld_s; p.lens = d_lens;
+    p.layer_elems = (long long)n_seq * cap_len * n_heads * kDh;
+    p.n_seq = n_seq; p.H = n_heads; p.cap = cap_len; p.max_len = max_len; p.n_layers = n_layers; p.causal = causal ? 1 : 0;
+    p.strip_ld = (int)align_up((size_t)max_len, kFullChunk) + 8;
+    p.scale_log2e = (float)(1.4426950408889634 / std::sqrt((double)kDh));
+    const size_t smem = (size_t)kFullChunk * kFullRowBytes + (size_t)4 * 16 * p.strip_ld * sizeof(float);
+    static size_t smem_set = 0;      // largest opt-in so far (the attribute only ever needs to grow)
+    if (smem > smem_set) {
+        if (cudaFuncSetAttribute(full_block_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return SAN_ERR_CUDA;
+        smem_set = smem;
+    }
+    const dim3 grid((unsigned)ceil_div(max_len, kFullQ), (unsigned)n_heads, (unsigned)n_seq);
+    full_block_kernel<<<grid, 128, smem, static_cast<cudaStream_t>(stream)>>>(p);
+    return cuda_status(cudaGetLastError());
 }
 
 int32_t san_js_matrix(int32_t n_layers, const float* d_S, int64_t layer_stride, int64_t ld_s,

@@ -293,6 +293,17 @@ struct FusedWarp {
     // tile of an item has room for QROW key rows and carries the query rows behind them.
     __device__ __forceinline__ void produce() {
         if (!p_active) return;
+        if (!p_first && p_left > TR) {      // a whole tile from the middle of a panel: nothing else to decide
+            if (lane == 0) {
+                const uint32_t bar = sm_base + bars + p_stage * 8;
+                mbar_expect_tx(bar, (uint32_t)kStageBytes);
+                bulk_g2s(sm_base + ring + p_stage * kStageBytes, p_src, (uint32_t)kStageBytes, bar);
+            }
+            p_stage = (p_stage + 1 == (unsigned)kFusedStages) ? 0 : p_stage + 1;
+            p_left -= TR;
+            p_src += kStageBytes;
+            return;
+        }
         const int r = min(p_first ? QROW : TR, p_left);
         const bool with_new = p_has_new && (r == p_left);      // this step's row closes the panel
         const uint32_t cache_bytes = (uint32_t)(r - (with_new ? 1 : 0)) * ROW_BYTES;
