@@ -379,6 +379,54 @@ def time_js_matrix(w, dec, sb, pos, device, reps=50):
             "note": "three launches (clear, pairs, finish) over weights that fit in L2: launch-bound, not a roofline case"}
 
 
+def time_full_block(w, device, peak, reps=5):
+    """Full-sequence shared attention (encoder-side use): one san_full_block launch over the
+    workload's sentences at their source lengths, a block of self_blocks[0] layers (AAN
+    workload: encdec_blocks[0]).  Launches rotate over input replicas larger than L2."""
+    import torch
+    from paper_1906_11024_b200 import binding as B
+    if w.dtype != "bf16":
+        return None
+    src = w.src_lens().astype(np.int64)
+    cap = int(src.max())
+    if cap > 512:
+        return None
+    pi = int((w.encdec_blocks if w.self_is_aan else w.self_blocks)[0])
+    H, n = w.n_heads, w.n_sent
+    per_rep = (2 + 2 * pi) * n * cap * H * 64 * 2
+    R = int(min(32, max(2, math.ceil(3 * L2_BYTES / per_rep))))
+    gen = torch.Generator(device=device)
+    gen.manual_seed(77)
+    mk = lambda *shape: torch.randn(*shape, generator=gen, device=device, dtype=torch.float32).to(torch.bfloat16)
+    reps_in = [(mk(n, cap, H, 64), mk(n, cap, H, 64), mk(pi, n, cap, H, 64)) for _ in range(R)]
+    out = torch.empty(pi, n, cap, H, 64, dtype=torch.bfloat16, device=device)
+    lens = torch.from_numpy(src.astype(np.int32)).to(device)
+
+    def all_replicas():
+        for q, k, v in reps_in:
+            B.check(B.san_full_block(B.SAN_BF16, H, pi, 0, q, k, v, lens, n, cap, cap, None, 0, out), "san_full_block")
+
+    g = capture(all_replicas, device)
+    for _ in range(3):
+        g.replay()
+    torch.cuda.synchronize(device)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        g.replay()
+    e1.record()
+    torch.cuda.synchronize(device)
+    secs = e0.elapsed_time(e1) * 1e-3 / (reps * R)
+    rows = int(src.sum())
+    nbytes = (2 + 2 * pi) * rows * H * 64 * 2                       # Q, K, pi value panels in; pi outputs out
+    flops = float((2 + 2 * pi) * (src * src).sum() * H * 64)        # 2 l^2 d_h for the scores and per layer of S.V
+    return {"call": "san_full_block", "layers_in_block": pi, "us_per_launch": secs * 1e6,
+            "bytes_per_launch": nbytes, "achieved_gbs": nbytes / secs / 1e9, "frac_of_hbm_peak": nbytes / secs / 1e9 / peak,
+            "flops_per_launch": flops, "achieved_tflops": flops / secs / 1e12, "bound": "hbm",
+            "note": "sentences of 10-100 positions: Q, K and V are read once and the l x l products are small, "
+                    "so the launch is bound by HBM and latency, not by the tensor pipe"}
+
+
 # ------------------------------------------------------------------------- the CPU oracle arm
 def oracle_sample(w, n_sent_sample):
     """Oracle state for the first sentences of the workload at the benchmarked positions."""
@@ -543,6 +591,9 @@ def main():
     next_rows = {}
     if rank == 0:
         next_rows["beam_reorder"] = time_beam_reorder(w, decs, sbs, pos, device, peak)
+        fb = time_full_block(w, device, peak)
+        if fb is not None:
+            next_rows["full_sequence"] = fb
 
     unshared = None
     if not args.no_unshared and rank == 0:

@@ -45,20 +45,28 @@ __device__ __forceinline__ uint32_t full_pack(float lo, float hi) {
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
-// 64 rows of 64 bf16 from global memory (row stride H*64 elements) into a padded chunk;
-// rows at or beyond `rows` are zero-filled.
-__device__ __forceinline__ void full_load_chunk(unsigned char* dst, const __nv_bfloat16* src, long long row_elems, int rows) {
-    for (int u = threadIdx.x; u < kFullChunk * 8; u += blockDim.x) {
-        const int r = u >> 3, c = u & 7;
-        uint4 val = make_uint4(0, 0, 0, 0);
-        if (r < rows) val = *reinterpret_cast<const uint4*>(src + (long long)r * row_elems + c * 8);
-        *reinterpret_cast<uint4*>(dst + r * kFullRowBytes + c * 16) = val;
+// A chunk = 64 rows of 64 bf16 (row stride H*64 elements in global memory).  Its 512 pieces
+// of 16 bytes are fetched into registers, four per thread, one chunk ahead of their use, and
+// stored into the padded shared-memory chunk when the previous chunk has been consumed; rows
+// at or beyond `rows` read as zero.
+__device__ __forceinline__ void full_fetch(uint4 (&pre)[4], const __nv_bfloat16* src, long long row_elems, int rows) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int u = (int)threadIdx.x + i * 128, r = u >> 3, c = u & 7;
+        pre[i] = r < rows ? ld16_stream(src + (long long)r * row_elems + c * 8) : make_uint4(0, 0, 0, 0);
+    }
+}
+__device__ __forceinline__ void full_store(unsigned char* chunk, const uint4 (&pre)[4]) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int u = (int)threadIdx.x + i * 128, r = u >> 3, c = u & 7;
+        *reinterpret_cast<uint4*>(chunk + r * kFullRowBytes + c * 16) = pre[i];
     }
 }
 
 extern __shared__ __align__(16) unsigned char full_smem[];
 
-static __global__ void __launch_bounds__(128) full_block_kernel(const FullParams p) {
+static __global__ void __launch_bounds__(128, 4) full_block_kernel(const FullParams p) {
     const int seq = blockIdx.z, h = blockIdx.y, q0 = blockIdx.x * kFullQ;
     const int len = min(p.lens[seq], p.max_len);       // the strips are sized for max_len: longer sequences are cut there
     if (q0 >= len) return;
@@ -69,6 +77,12 @@ static __global__ void __launch_bounds__(128) full_block_kernel(const FullParams
     float* strip = reinterpret_cast<float*>(full_smem + kFullChunk * kFullRowBytes) + (long long)warp * 16 * p.strip_ld;
     const int qa = q0 + warp * 16 + gid, qb = qa + 8;                                    // this lane's two query rows
     const int n_keys = p.causal ? min(len, q0 + kFullQ) : len;                           // keys any query of the tile sees
+    const int n_chunks = (n_keys + kFullChunk - 1) / kFullChunk;
+    const int n_pad = n_chunks * kFullChunk;
+
+    // the first key chunk is on its way while the query fragments are read
+    uint4 pre[4];
+    full_fetch(pre, p.k + seq_off, row_elems, min(kFullChunk, len));
 
     // query fragments (A operand, 16 queries x 64 dims): rows beyond the sequence read as zero
     uint32_t qf[4][4];
@@ -83,72 +97,89 @@ static __global__ void __launch_bounds__(128) full_block_kernel(const FullParams
             qf[ks][3] = qb < len ? *reinterpret_cast<const uint32_t*>(qr_b + 16 * ks + 2 * tig + 8) : 0u;
         }
     }
-
-    // ---- 1. scores (log2 domain) into the strip; masked keys get -inf
-    for (int k0 = 0; k0 < n_keys; k0 += kFullChunk) {
-        __syncthreads();                                   // the chunk is free
-        full_load_chunk(chunk, p.k + seq_off + (long long)k0 * row_elems, row_elems, min(kFullChunk, len - k0));
-        __syncthreads();
-#pragma unroll
-        for (int nt = 0; nt < kFullChunk / 8; ++nt) {      // 8 keys per MMA
-            float acc[4] = {0.f, 0.f, 0.f, 0.f};
-            const unsigned char* krow = chunk + (nt * 8 + gid) * kFullRowBytes + 4 * tig;     // key nt*8+gid, dims 2tig..
-#pragma unroll
-            for (int ks = 0; ks < 4; ++ks) {
-                const uint32_t b0 = *reinterpret_cast<const uint32_t*>(krow + 32 * ks);
-                const uint32_t b1 = *reinterpret_cast<const uint32_t*>(krow + 32 * ks + 16);
-                full_mma(acc, qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3], b0, b1);
-            }
-            const int key = k0 + nt * 8 + 2 * tig;         // acc[0], acc[1]: query qa, keys key, key+1; acc[2], acc[3]: query qb
-            float2 za, zb;
-            za.x = (key < len && (!p.causal || key <= qa)) ? acc[0] * p.scale_log2e : -INFINITY;
-            za.y = (key + 1 < len && (!p.causal || key + 1 <= qa)) ? acc[1] * p.scale_log2e : -INFINITY;
-            zb.x = (key < len && (!p.causal || key <= qb)) ? acc[2] * p.scale_log2e : -INFINITY;
-            zb.y = (key + 1 < len && (!p.causal || key + 1 <= qb)) ? acc[3] * p.scale_log2e : -INFINITY;
-            *reinterpret_cast<float2*>(strip + gid * p.strip_ld + key) = za;
-            *reinterpret_cast<float2*>(strip + (gid + 8) * p.strip_ld + key) = zb;
-        }
-    }
-    __syncwarp();
-
-    // ---- 2. softmax of the warp's 16 rows over keys [0, n_pad), n_pad = scored keys (a multiple of 64)
-    const int n_pad = (n_keys + kFullChunk - 1) / kFullChunk * kFullChunk;
-    for (int r = 0; r < 16; ++r) {
-        float* row = strip + r * p.strip_ld;
-        const int qrow = q0 + warp * 16 + r;
-        float m = -INFINITY;
-        for (int j = lane; j < n_pad; j += 32) m = fmaxf(m, row[j]);
-        m = warp_max(m);
-        if (qrow >= len) m = 0.f;                          // a row outside the sequence: all keys masked; weights become 0
-        float s = 0.f;
-        for (int j = lane; j < n_pad; j += 32) { const float e = exp2f(row[j] - m); row[j] = e; s += e; }
-        s = warp_sum(s);
-        const float inv = s > 0.f ? 1.0f / s : 0.f;
-        float* Srow = (p.S && qrow < len) ? p.S + (((long long)seq * p.H + h) * p.cap + qrow) * p.ld_s : nullptr;
-        for (int j = lane; j < n_pad; j += 32) {
-            const float w = row[j] * inv;
-            row[j] = w;
-            if (Srow && j < len) Srow[j] = w;              // masked keys of a causal row are stored as 0
-        }
-        if (Srow && p.causal) for (int j = n_pad + lane; j < len; j += 32) Srow[j] = 0.f;
-    }
-    __syncwarp();
-
-    // ---- 3. apply to every layer's values
     const int vrow_l = (lane & 7) + ((lane >> 3) & 1) * 8;          // ldmatrix.trans: key row this lane addresses in a 16-key block
-    const int vcol_l = (lane >> 4) * 8;                             // and its dim offset inside a 16-dim pair of tiles
+    const int vcol_l = (lane >> 4) * 8;                             // and its dim offset inside a pair of 8-dim tiles
     const uint32_t chunk_s = (uint32_t)__cvta_generic_to_shared(chunk);
-    for (int l = 0; l < p.n_layers; ++l) {
-        float acc[8][4];
-#pragma unroll
-        for (int x = 0; x < 8; ++x)
-#pragma unroll
-            for (int e = 0; e < 4; ++e) acc[x][e] = 0.f;
-        const __nv_bfloat16* vbase = p.v + (long long)l * p.layer_elems + seq_off;
-        for (int k0 = 0; k0 < n_keys; k0 += kFullChunk) {
+    float acc[8][4];
+
+    // Panels in order: the keys, then the values of each layer; every panel in chunks of 64 rows.
+    // panel 0 fills the strip with scores and ends with the softmax; panel l+1 applies the strip
+    // to layer l's values and ends with that layer's output.
+    for (int panel = 0; panel <= p.n_layers; ++panel) {
+        for (int kc = 0; kc < n_chunks; ++kc) {
+            const int k0 = kc * kFullChunk;
+            __syncthreads();                                   // every warp is done with the previous chunk
+            full_store(chunk, pre);
             __syncthreads();
-            full_load_chunk(chunk, vbase + (long long)k0 * row_elems, row_elems, min(kFullChunk, len - k0));
-            __syncthreads();
+            {   // fetch the chunk after this one
+                int np = panel, nkc = kc + 1;
+                if (nkc == n_chunks) { np += 1; nkc = 0; }
+                if (np <= p.n_layers) {
+                    const __nv_bfloat16* base = np == 0 ? p.k : p.v + (long long)(np - 1) * p.layer_elems;
+                    full_fetch(pre, base + seq_off + (long long)nkc * kFullChunk * row_elems, row_elems,
+                               min(kFullChunk, len - nkc * kFullChunk));
+                }
+            }
+            if (panel == 0) {
+                // ---- scores (log2 domain) into the strip; masked keys get -inf
+#pragma unroll
+                for (int nt = 0; nt < kFullChunk / 8; ++nt) {      // 8 keys per MMA
+                    float sc[4] = {0.f, 0.f, 0.f, 0.f};
+                    const unsigned char* krow = chunk + (nt * 8 + gid) * kFullRowBytes + 4 * tig;     // key nt*8+gid, dims 2tig..
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks) {
+                        const uint32_t b0 = *reinterpret_cast<const uint32_t*>(krow + 32 * ks);
+                        const uint32_t b1 = *reinterpret_cast<const uint32_t*>(krow + 32 * ks + 16);
+                        full_mma(sc, qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3], b0, b1);
+                    }
+                    const int key = k0 + nt * 8 + 2 * tig;         // sc[0], sc[1]: query qa, keys key, key+1; sc[2], sc[3]: query qb
+                    float2 za, zb;
+                    za.x = (key < len && (!p.causal || key <= qa)) ? sc[0] * p.scale_log2e : -INFINITY;
+                    za.y = (key + 1 < len && (!p.causal || key + 1 <= qa)) ? sc[1] * p.scale_log2e : -INFINITY;
+                    zb.x = (key < len && (!p.causal || key <= qb)) ? sc[2] * p.scale_log2e : -INFINITY;
+                    zb.y = (key + 1 < len && (!p.causal || key + 1 <= qb)) ? sc[3] * p.scale_log2e : -INFINITY;
+                    *reinterpret_cast<float2*>(strip + gid * p.strip_ld + key) = za;
+                    *reinterpret_cast<float2*>(strip + (gid + 8) * p.strip_ld + key) = zb;
+                }
+                if (kc + 1 < n_chunks) continue;
+                // ---- softmax of the warp's 16 rows over the scored keys [0, n_pad): eight lanes per
+                // row, four rows side by side (lane i of a row takes keys i, i + 8, ...: with a row
+                // stride of 8 mod 32 words the 32 lanes touch 32 different banks)
+                __syncwarp();
+                const int sub = lane & 7;
+#pragma unroll
+                for (int rg = 0; rg < 4; ++rg) {
+                    const int r = rg * 4 + (lane >> 3);
+                    float* row = strip + r * p.strip_ld;
+                    const int qrow = q0 + warp * 16 + r;
+                    float m = -INFINITY;
+                    for (int j = sub; j < n_pad; j += 8) m = fmaxf(m, row[j]);
+#pragma unroll
+                    for (int o = 4; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+                    if (qrow >= len) m = 0.f;                  // a row outside the sequence is never stored; keep it finite
+                    float s = 0.f;
+                    for (int j = sub; j < n_pad; j += 8) { const float e = exp2f(row[j] - m); row[j] = e; s += e; }
+#pragma unroll
+                    for (int o = 4; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+                    const float inv = s > 0.f ? 1.0f / s : 0.f;
+                    float* Srow = (p.S && qrow < len) ? p.S + (((long long)seq * p.H + h) * p.cap + qrow) * p.ld_s : nullptr;
+                    for (int j = sub; j < n_pad; j += 8) {
+                        const float w = row[j] * inv;
+                        row[j] = w;
+                        if (Srow && j < len) Srow[j] = w;      // masked keys of a causal row are stored as 0
+                    }
+                    if (Srow && p.causal) for (int j = n_pad + sub; j < len; j += 8) Srow[j] = 0.f;
+                }
+                __syncwarp();
+                continue;
+            }
+            // ---- apply the strip to this chunk of the layer's values
+            if (kc == 0) {
+#pragma unroll
+                for (int x = 0; x < 8; ++x)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) acc[x][e] = 0.f;
+            }
 #pragma unroll
             for (int kb = 0; kb < kFullChunk; kb += 16) {           // 16 keys per MMA
                 // A = weights of queries (gid, gid+8) at keys k0+kb + {2tig, 2tig+1, 2tig+8, 2tig+9}
@@ -174,14 +205,16 @@ static __global__ void __launch_bounds__(128) full_block_kernel(const FullParams
                     full_mma(acc[2 * dp + 1], r0, r1, r2, r3, b[2], b[3]);
                 }
             }
-        }
-        // acc[x][0], [1]: query qa, dims 8x + 2tig, +1; acc[x][2], [3]: query qb
-        __nv_bfloat16* oa = p.out + (long long)l * p.layer_elems + seq_off + (long long)qa * row_elems + 2 * tig;
-        __nv_bfloat16* ob = p.out + (long long)l * p.layer_elems + seq_off + (long long)qb * row_elems + 2 * tig;
+            if (kc + 1 < n_chunks) continue;
+            // acc[x][0], [1]: query qa, dims 8x + 2tig, +1; acc[x][2], [3]: query qb
+            const long long lo = (long long)(panel - 1) * p.layer_elems + seq_off + 2 * tig;
+            __nv_bfloat16* oa = p.out + lo + (long long)qa * row_elems;
+            __nv_bfloat16* ob = p.out + lo + (long long)qb * row_elems;
 #pragma unroll
-        for (int x = 0; x < 8; ++x) {
-            if (qa < len) *reinterpret_cast<uint32_t*>(oa + 8 * x) = full_pack(acc[x][0], acc[x][1]);
-            if (qb < len) *reinterpret_cast<uint32_t*>(ob + 8 * x) = full_pack(acc[x][2], acc[x][3]);
+            for (int x = 0; x < 8; ++x) {
+                if (qa < len) *reinterpret_cast<uint32_t*>(oa + 8 * x) = full_pack(acc[x][0], acc[x][1]);
+                if (qb < len) *reinterpret_cast<uint32_t*>(ob + 8 * x) = full_pack(acc[x][2], acc[x][3]);
+            }
         }
     }
 }
