@@ -4,6 +4,9 @@
 #include <algorithm>
 #include <cmath>
 #include <cstring>
+#include <functional>
+#include <queue>
+#include <vector>
 #include <new>
 
 #include "san_ctx.h"
@@ -96,6 +99,40 @@ void pick_spans(const san_ctx* ctx, long long units, int max_len, long long part
     }
     *span_len = sl;
     *n_spans = ns;
+}
+
+// Estimated length of a step of the one-launch kernel for one way of cutting the rows, in
+// tiles: a CTA's share of the item list (encoder-memory items first, as in the list) handed to
+// its warps greedily, each item to the warp that is free first; the step is as long as the
+// busiest warp.  Every row is taken at the host's length bound.
+struct CutShape { long long rows; int bound, pi, nq, span, lg; };
+double step_makespan(const CutShape& enc, const CutShape& self, int ctas, int tile_rows) {
+    constexpr double kItemCost = 1.0;            // tiles' worth of work per item that is not tile arithmetic
+    constexpr double kSplitCost = 2.0;           // per span of a split row: partial sums out, ticket, share of the combine
+    const int QR = tile_rows - 8;
+    auto cost_and_count = [&](const CutShape& c, double* cost, long long* per_cta) {
+        if (c.rows == 0) { *cost = 0.0; *per_cta = 0; return; }
+        const int ns = ceil_div(c.bound, c.span), nlg = ceil_div(c.pi, c.lg);
+        const int span = std::min(c.span, c.bound);
+        const int k_tiles = span <= QR ? 1 : 1 + ceil_div(span - QR, tile_rows);
+        *cost = k_tiles + (double)c.lg * ceil_div(span, tile_rows) + kItemCost +
+                (ns > 1 ? kSplitCost * (1.0 + c.lg * c.nq / 4.0) : 0.0);
+        *per_cta = (c.rows * nlg * ns + ctas - 1) / ctas;
+    };
+    double cost[2]; long long count[2];
+    cost_and_count(enc, &cost[0], &count[0]);
+    cost_and_count(self, &cost[1], &count[1]);
+    std::priority_queue<double, std::vector<double>, std::greater<double>> warps;
+    for (int w = 0; w < kFusedWarps; ++w) warps.push(0.0);
+    double longest = 0.0;
+    for (int k = 0; k < 2; ++k)
+        for (long long i = 0; i < count[k]; ++i) {
+            const double t = warps.top() + cost[k];
+            warps.pop();
+            warps.push(t);
+            longest = std::max(longest, t);
+        }
+    return longest;
 }
 
 template <typename T>
@@ -196,6 +233,7 @@ int32_t san_policy_set_sizes(san_ctx* ctx, int32_t kind, const int32_t* sizes, i
                                         : ctx->n_enc_k_planes;
     if (p.n_blocks > planes) return SAN_ERR_CAPACITY;
     (kind == SAN_SELF ? ctx->self_pol : ctx->enc_pol) = p;
+    ctx->policy_epoch += 1;
     return SAN_OK;
 }
 
@@ -448,6 +486,49 @@ int32_t san_decode_step(san_ctx* ctx, const san_step_args* a, void* stream) {
     int span_self = cap_self, span_enc = cap_enc, lg_self = pi_self, lg_enc = pi_enc;
     pick(cap_self, pi_self, 1, &span_self, &lg_self);
     pick(cap_enc, pi_enc, c.beam, &span_enc, &lg_enc);
+    // The rule above looks at one item at a time.  Where it cuts anything, compare it with the other
+    // ways of cutting (halved spans, halved layer groups, or no cut at all) by the estimated length
+    // of the step: items of equal size that divide evenly over the warps beat smaller items that
+    // leave a warp with one more than its neighbours.  The choice is remembered per launch shape.
+    if (span_self < cap_self || lg_self < pi_self || span_enc < cap_enc || lg_enc < pi_enc) {
+        const int len_b = std::min(c.max_tgt_len, (int)align_up((size_t)max_len, TR)), src_b = std::min(c.max_src_len, (int)align_up((size_t)max_src, TR));
+        san_ctx::StepPlan* plan = nullptr;
+        for (auto& pl : ctx->plans)
+            if (pl.valid && pl.epoch == ctx->policy_epoch && pl.n_seqs == n_seqs && pl.n_sent == n_sent &&
+                pl.len_bound == len_b && pl.src_bound == src_b) plan = &pl;
+        if (!plan) {
+            const int ctas = (int)std::max<long long>(1, std::min<long long>(ctx->sm_count, (rows_self + rows_enc + kFusedWarps - 1) / kFusedWarps));
+            CutShape ce{rows_enc, src_b, pi_enc, c.beam, span_enc, lg_enc}, cs{rows_self, len_b, pi_self, 1, span_self, lg_self};
+            double best = step_makespan(ce, cs, ctas, TR);
+            int b_ss = span_self, b_ls = lg_self, b_se = span_enc, b_le = lg_enc;
+            auto halvings = [](int from, int floor_, int align, std::vector<int>* out) {
+                for (int v = from;; v = std::max(floor_, (int)align_up((size_t)ceil_div(v, 2), align))) {
+                    out->push_back(v);
+                    if (v <= floor_) break;
+                }
+            };
+            std::vector<int> ss, ls, se, le;
+            halvings(cap_self, std::min(cap_self, 64), 16, &ss); halvings(pi_self, std::min(pi_self, 2), 1, &ls);
+            halvings(cap_enc, std::min(cap_enc, 32), 16, &se);   halvings(pi_enc, std::min(pi_enc, 2), 1, &le);
+            if (!do_self) { ss.assign(1, span_self); ls.assign(1, lg_self); }
+            if (!do_enc) { se.assign(1, span_enc); le.assign(1, lg_enc); }
+            for (int a : ss) for (int b : ls) for (int d : se) for (int e : le) {
+                if (ceil_div(len_b, a) > kMaxSpans || ceil_div(src_b, d) > kMaxSpans) continue;
+                const long long need = (ceil_div(len_b, a) > 1 ? rows_self * ceil_div(pi_self, b) * ceil_div(len_b, a) * (part_header_floats(1) + b * kDh) : 0) +
+                                       (ceil_div(src_b, d) > 1 ? rows_enc * ceil_div(pi_enc, e) * ceil_div(src_b, d) * (part_header_floats(nqe) + e * nqe * kDh) : 0);
+                if (need > (long long)ctx->part_floats) continue;
+                cs.span = a; cs.lg = b; ce.span = d; ce.lg = e;
+                const double t = step_makespan(ce, cs, ctas, TR);
+                if (t < 0.97 * best) { best = t; b_ss = a; b_ls = b; b_se = d; b_le = e; }
+            }
+            plan = &ctx->plans[ctx->plan_next];
+            ctx->plan_next = (ctx->plan_next + 1) % san_ctx::kPlans;
+            plan->valid = true; plan->epoch = ctx->policy_epoch; plan->n_seqs = n_seqs; plan->n_sent = n_sent;
+            plan->len_bound = len_b; plan->src_bound = src_b;
+            plan->span_self = b_ss; plan->lg_self = b_ls; plan->span_enc = b_se; plan->lg_enc = b_le;
+        }
+        span_self = plan->span_self; lg_self = plan->lg_self; span_enc = plan->span_enc; lg_enc = plan->lg_enc;
+    }
     while (ceil_div(max_len, span_self) > kMaxSpans) span_self = std::min(kZFloats, span_self * 2);
     while (ceil_div(max_src, span_enc) > kMaxSpans) span_enc = std::min(kZFloats / nqe, span_enc * 2);
     const int nlg_self = ceil_div(pi_self, lg_self), nlg_enc = ceil_div(pi_enc, lg_enc);

@@ -28,4 +28,18 @@ struct san_ctx {
     int* tickets = nullptr;
     float* part = nullptr;
     bool fused_attr_set = false;   // shared-memory opt-in of the one-launch step kernel done
+
+    // How the one-launch step cuts long rows (positions per item, layers per item), remembered
+    // per launch shape: the search that balances the items over the warps costs more than a
+    // short step, and a decode loop repeats the same shape for many steps.
+    struct StepPlan {
+        bool valid = false;
+        unsigned epoch = 0;                      // policy_epoch it was made for
+        int n_seqs = 0, n_sent = 0, len_bound = 0, src_bound = 0;
+        int span_self = 0, lg_self = 0, span_enc = 0, lg_enc = 0;
+    };
+    static constexpr int kPlans = 8;
+    StepPlan plans[kPlans];
+    int plan_next = 0;
+    unsigned policy_epoch = 0;     // raised whenever a sharing policy changes
 };
