@@ -40,7 +40,8 @@ FALLBACK_HBM_GBS = 6650.0
 # line reports null until a new capture is recorded here.  (The choice of spans and layer
 # groups lives in san_api.cu; a change there calls for a new capture as well.)
 KERNEL_SOURCES = ("san_fused.cuh", "san_kernels.cuh")
-NCU_TRAFFIC = {"digest": "55c777fde63b549e", "fused": {"base": 70.3e6, "long": 762.4e6}}
+NCU_TRAFFIC = {"digest": "55c777fde63b549e", "fused": {"base": 70.3e6, "long": 762.4e6,
+                                                          "base-unshared": 102.6e6, "long-unshared": 1317.0e6}}
 
 
 def kernel_digest():
@@ -529,10 +530,15 @@ def main():
                     help="fused: san_decode_step, one launch per step; calls: append/weights/apply launches")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-unshared", action="store_true")
+    ap.add_argument("--sharing", default="on", choices=["on", "off"],
+                    help="off: time the workload with every block size 1 as the main arm (for byte counts of the unshared path)")
     args = ap.parse_args()
 
     from paper_1906_11024_b200 import synth
     w = synth.WORKLOADS[args.workload]
+    if args.sharing == "off":
+        w = synth.unshared(w)
+        args.no_unshared = True
     if args.impl == "reference":
         run_reference(args, w)
         return
@@ -607,7 +613,8 @@ def main():
         su, lu, _ = time_steps(decs_u, sbs_u, args.steps, args.warmup, device, lambda: None, fused)
         unshared = {"value": wu.n_seqs * args.steps / su, "unit": UNIT, "ms_per_step": su / args.steps * 1e3,
                     "kv_bytes_per_step": abu["kv"], "bytes_per_step": abu["total"],
-                    "hbm_gbs": abu["total"] / (su / args.steps) / 1e9, "gpu_launches_per_step": lu}
+                    "hbm_gbs": abu["total"] / (su / args.steps) / 1e9, "gpu_launches_per_step": lu,
+                    "traffic": ncu_traffic(args.path, wu.name)}
         js = time_js_matrix(wu, decs_u[0], sbs_u[0], pos, device)
         if js is not None:
             next_rows["policy_learner"] = js
