@@ -748,10 +748,17 @@ int32_t san_full_block(int32_t dtype, int32_t n_heads, int32_t n_layers, int32_t
     p.strip_ld = (int)align_up((size_t)max_len, kFullChunk) + 8;
     p.scale_log2e = (float)(1.4426950408889634 / std::sqrt((double)kDh));
     const size_t smem = (size_t)kFullChunk * kFullRowBytes + (size_t)4 * 16 * p.strip_ld * sizeof(float);
-    static size_t smem_set = 0;      // largest opt-in so far (the attribute only ever needs to grow)
-    if (smem > smem_set) {
-        if (cudaFuncSetAttribute(full_block_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return SAN_ERR_CUDA;
-        smem_set = smem;
+    // the opt-in above 48 KB is a per-device attribute of the kernel: remember the largest
+    // value set on each device (it only ever needs to grow)
+    if (smem > 48 * 1024) {
+        static size_t smem_set[64] = {};
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess) return SAN_ERR_CUDA;
+        if (dev < 0 || dev >= 64 || smem > smem_set[dev]) {
+            if (cudaFuncSetAttribute(full_block_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+                return SAN_ERR_CUDA;
+            if (dev >= 0 && dev < 64) smem_set[dev] = smem;
+        }
     }
     const dim3 grid((unsigned)ceil_div(max_len, kFullQ), (unsigned)n_heads, (unsigned)n_seq);
     full_block_kernel<<<grid, 128, smem, static_cast<cudaStream_t>(stream)>>>(p);

@@ -78,7 +78,7 @@ static __global__ void __launch_bounds__(128, 4) full_block_kernel(const FullPar
     const int qa = q0 + warp * 16 + gid, qb = qa + 8;                                    // this lane's two query rows
     const int n_keys = p.causal ? min(len, q0 + kFullQ) : len;                           // keys any query of the tile sees
     const int n_chunks = (n_keys + kFullChunk - 1) / kFullChunk;
-    const int n_pad = n_chunks * kFullChunk;
+    const int n_pad = (n_keys + 15) & ~15;             // keys that are scored, normalised and applied: whole 16-key MMA blocks
 
     // the first key chunk is on its way while the query fragments are read
     uint4 pre[4];
@@ -124,6 +124,7 @@ static __global__ void __launch_bounds__(128, 4) full_block_kernel(const FullPar
                 // ---- scores (log2 domain) into the strip; masked keys get -inf
 #pragma unroll
                 for (int nt = 0; nt < kFullChunk / 8; ++nt) {      // 8 keys per MMA
+                    if (k0 + nt * 8 >= n_pad) break;
                     float sc[4] = {0.f, 0.f, 0.f, 0.f};
                     const unsigned char* krow = chunk + (nt * 8 + gid) * kFullRowBytes + 4 * tig;     // key nt*8+gid, dims 2tig..
 #pragma unroll
@@ -182,6 +183,7 @@ static __global__ void __launch_bounds__(128, 4) full_block_kernel(const FullPar
             }
 #pragma unroll
             for (int kb = 0; kb < kFullChunk; kb += 16) {           // 16 keys per MMA
+                if (k0 + kb >= n_pad) break;
                 // A = weights of queries (gid, gid+8) at keys k0+kb + {2tig, 2tig+1, 2tig+8, 2tig+9}
                 const float2 wa0 = *reinterpret_cast<const float2*>(strip + gid * p.strip_ld + k0 + kb + 2 * tig);
                 const float2 wb0 = *reinterpret_cast<const float2*>(strip + (gid + 8) * p.strip_ld + k0 + kb + 2 * tig);
