@@ -15,6 +15,7 @@
 #include "san_reorder.cuh"
 #include "san_learn.cuh"
 #include "san_full.cuh"
+#include "san_full_tc5.cuh"
 
 using namespace san;
 
@@ -747,21 +748,33 @@ int32_t san_full_block(int32_t dtype, int32_t n_heads, int32_t n_layers, int32_t
     p.n_seq = n_seq; p.H = n_heads; p.cap = cap_len; p.max_len = max_len; p.n_layers = n_layers; p.causal = causal ? 1 : 0;
     p.strip_ld = (int)align_up((size_t)max_len, kFullChunk) + 8;
     p.scale_log2e = (float)(1.4426950408889634 / std::sqrt((double)kDh));
-    const size_t smem = (size_t)kFullChunk * kFullRowBytes + (size_t)4 * 16 * p.strip_ld * sizeof(float);
-    // the opt-in above 48 KB is a per-device attribute of the kernel: remember the largest
-    // value set on each device (it only ever needs to grow)
-    if (smem > 48 * 1024) {
-        static size_t smem_set[64] = {};
+    // the opt-in above 48 KB of dynamic shared memory is a per-device attribute of a kernel:
+    // remember the largest value set on each device (it only ever needs to grow)
+    auto opt_in = [](const void* fn, size_t bytes, size_t* set_per_device) -> bool {
+        if (bytes <= 48 * 1024) return true;
         int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess) return SAN_ERR_CUDA;
-        if (dev < 0 || dev >= 64 || smem > smem_set[dev]) {
-            if (cudaFuncSetAttribute(full_block_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-                return SAN_ERR_CUDA;
-            if (dev >= 0 && dev < 64) smem_set[dev] = smem;
+        if (cudaGetDevice(&dev) != cudaSuccess) return false;
+        if (dev < 0 || dev >= 64 || bytes > set_per_device[dev]) {
+            if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess) return false;
+            if (dev >= 0 && dev < 64) set_per_device[dev] = bytes;
         }
+        return true;
+    };
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (max_len >= kTcQ && n_layers <= kTcMaxLayers) {
+        // sequences that fill a 128-query tile: tcgen05 path, accumulators in tensor memory
+        static size_t set_tc5[64] = {};
+        const size_t smem = full_tc5_smem_bytes();
+        if (!opt_in((const void*)full_block_tc5_kernel, smem, set_tc5)) return SAN_ERR_CUDA;
+        const dim3 grid((unsigned)ceil_div(max_len, kTcQ), (unsigned)n_heads, (unsigned)n_seq);
+        full_block_tc5_kernel<<<grid, kTcQ, smem, st>>>(p);
+        return cuda_status(cudaGetLastError());
     }
+    static size_t set_mma[64] = {};
+    const size_t smem = (size_t)kFullChunk * kFullRowBytes + (size_t)4 * 16 * p.strip_ld * sizeof(float);
+    if (!opt_in((const void*)full_block_kernel, smem, set_mma)) return SAN_ERR_CUDA;
     const dim3 grid((unsigned)ceil_div(max_len, kFullQ), (unsigned)n_heads, (unsigned)n_seq);
-    full_block_kernel<<<grid, 128, smem, static_cast<cudaStream_t>(stream)>>>(p);
+    full_block_kernel<<<grid, 128, smem, st>>>(p);
     return cuda_status(cudaGetLastError());
 }
 

@@ -1,0 +1,284 @@
+// Full-sequence shared attention on the fifth-generation tensor cores (tcgen05, accumulators
+// in tensor memory), for sequences long enough to fill a 128-query tile.  Same operation as
+// full_block_kernel: S = Softmax(Q.K^T / 8) once per block (Eq. 1, Eq. 3), O_l = S.V_l for each
+// layer of the block (Eq. 2, Eq. 4).
+//
+// CTA = (128 queries, head, sequence), 128 threads; thread t owns query row t, which is lane t
+// of tensor memory, so every row statistic is thread-local (no shuffles).
+//   pass 0  for each chunk of 64 keys: stage the key rows in shared memory, one
+//           tcgen05.mma chain (M 128, N 64, K 64) writes the scores into tensor memory, each
+//           thread reads its row back and keeps a running (max, sum).
+//   pass 1  for each chunk again: scores once more (cheaper than keeping 128 x l floats),
+//           weights = exp2(z - max) / sum go out to S and, as a bf16 high part and a bf16
+//           remainder, into two shared-memory operand tiles; the value rows of every layer of
+//           the block are staged, and per layer two tcgen05.mma chains (M 128, N 64, K 64) add
+//           weights x values to that layer's accumulator, which stays in tensor memory
+//           (columns 64 + 64 l) until the last chunk.
+// Operand tiles are rows of 128 bytes with the 16-byte chunks XOR-swizzled by (row & 7), the
+// 128-byte swizzle the matrix descriptors name; queries, keys and weights are K-major, the
+// value rows (dims contiguous) are the MN-major B operand.  Every wait on the MMA barrier is
+// bounded; a CTA whose wait runs out stops issuing, frees its tensor memory and leaves its
+// outputs unwritten.
+#pragma once
+
+#include "san_full.cuh"
+#include "san_fused.cuh"
+
+namespace san {
+
+constexpr int kTcQ = 128;                 // queries per CTA = tensor-memory lanes
+constexpr int kTcChunk = 64;              // keys per MMA chain
+constexpr int kTcMaxLayers = 6;           // accumulators: 64 columns each after the 64 of the scores (512 columns in all)
+constexpr int kTcCols = 512;
+constexpr uint32_t kTcTileQ = kTcQ * 128, kTcTileK = kTcChunk * 128;      // bytes of a 128-row and of a 64-row operand tile
+
+// shared-memory matrix descriptor: 128-byte swizzle, 8-row groups 1024 bytes apart
+__device__ __forceinline__ uint64_t tc_desc(uint32_t smem_addr) {
+    return (uint64_t)((smem_addr >> 4) & 0x3fffu) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) |
+           ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+// instruction descriptor: float32 accumulator, bf16 operands, M 128, N 64; b_mn: B is MN-major
+__device__ __forceinline__ uint32_t tc_idesc(bool b_mn) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn ? (1u << 16) : 0u) | ((uint32_t)(64 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+}
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a, uint64_t b, uint32_t idesc, uint32_t accumulate) {
+    const uint32_t none = 0u;      // no output lane is disabled
+    asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n}"
+                 :: "r"(d_tmem), "l"(a), "l"(b), "r"(idesc), "r"(accumulate), "r"(none) : "memory");
+}
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, float (&v)[32]) {
+    uint32_t r[32];
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                 "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                   "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                   "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                 : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// rows [0, rows) of a [n][64] bf16 panel (row stride row_elems) into a swizzled 64-row operand
+// tile with 16-byte asynchronous copies (no registers held while they fly); the other rows are
+// zero-filled (a copy of source size 0).  Consecutive threads take consecutive pieces.
+__device__ __forceinline__ void tc_stage_async(uint32_t tile_s, const __nv_bfloat16* src, long long row_elems, int rows) {
+#pragma unroll
+    for (int i = 0; i < kTcChunk * 8 / kTcQ; ++i) {
+        const int u = (int)threadIdx.x + i * kTcQ, r = u >> 3, c = u & 7;
+        const uint32_t bytes = r < rows ? 16u : 0u;
+        const __nv_bfloat16* from = src + (long long)(r < rows ? r : 0) * row_elems + c * 8;
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;"
+                     :: "r"(tile_s + (uint32_t)(r * 128 + ((c ^ (r & 7)) << 4))), "l"(from), "r"(bytes) : "memory");
+    }
+}
+
+extern __shared__ __align__(1024) unsigned char tc_smem[];
+
+static __global__ void __launch_bounds__(kTcQ, 1) full_block_tc5_kernel(const FullParams p) {
+    const int seq = blockIdx.z, h = blockIdx.y, q0 = blockIdx.x * kTcQ;
+    const int len = min(p.lens[seq], p.max_len);
+    if (q0 >= len) return;                                   // uniform over the CTA, before anything is allocated
+    const int row = threadIdx.x, warp = threadIdx.x >> 5;
+    const int qrow = q0 + row;
+    const long long row_elems = (long long)p.H * kDh;
+    const long long seq_off = ((long long)seq * p.cap) * row_elems + (long long)h * kDh;
+    const int n_keys = p.causal ? min(len, q0 + kTcQ) : len;
+    const int n_chunks = (n_keys + kTcChunk - 1) / kTcChunk;
+
+    // shared memory (1024-byte aligned tiles): Q | weights high | weights remainder | two buffers of
+    // (K chunk, V chunk of each layer): the copies of the next chunk fly during this chunk's arithmetic
+    unsigned char* base = tc_smem + ((1024u - (smem_u32(tc_smem) & 1023u)) & 1023u);
+    unsigned char* sQ = base;
+    unsigned char* sPh = sQ + kTcTileQ;
+    unsigned char* sPl = sPh + kTcTileQ;
+    const uint32_t sKV = smem_u32(sPl + kTcTileQ);                     // buffer b: K at sKV + b * kBuf, V of layer l behind it
+    const uint32_t kBuf = (uint32_t)(1 + p.n_layers) * kTcTileK;
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int dead_s;
+
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        dead_s = 0;
+    }
+    __syncwarp();
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(smem_u32(&tmem_base_s)), "r"((uint32_t)kTcCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    // this thread's query row into the Q tile (zero beyond the sequence)
+    {
+        const __nv_bfloat16* qsrc = p.q + seq_off + (long long)qrow * row_elems;
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            const uint4 val = qrow < len ? ld16_stream(qsrc + c * 8) : make_uint4(0, 0, 0, 0);
+            *reinterpret_cast<uint4*>(sQ + row * 128 + ((c ^ (row & 7)) << 4)) = val;
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem = tmem_base_s;
+    const uint32_t t_lane = tmem + ((uint32_t)(warp * 32) << 16);         // this warp's 32 lanes
+    const uint32_t bar_s = smem_u32(&bar);
+    const uint64_t dQ = tc_desc(smem_u32(sQ)), dPh = tc_desc(smem_u32(sPh)), dPl = tc_desc(smem_u32(sPl));
+    const uint32_t idS = tc_idesc(false), idO = tc_idesc(true);
+    uint32_t phase = 0;
+    bool dead = false;
+
+    // waits for the MMAs committed last; false (for the whole CTA, after a barrier) if the wait ran out
+    auto mma_done = [&]() -> bool {
+        if (!mbar_try_wait(bar_s, phase) && !mbar_wait_slow(bar_s, phase)) dead_s = 1;
+        phase ^= 1u;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        return true;
+    };
+
+    // Chunk t of the run (pass 0: keys only; pass 1: keys and every layer's values) into buffer t & 1.
+    auto issue = [&](int t) {
+        if (t < 2 * n_chunks) {
+            const int pass = t >= n_chunks ? 1 : 0, k0 = (t - pass * n_chunks) * kTcChunk, rows = min(kTcChunk, len - k0);
+            const uint32_t buf = sKV + (uint32_t)(t & 1) * kBuf;
+            tc_stage_async(buf, p.k + seq_off + (long long)k0 * row_elems, row_elems, rows);
+            if (pass)
+                for (int l = 0; l < p.n_layers; ++l)
+                    tc_stage_async(buf + (uint32_t)(1 + l) * kTcTileK, p.v + (long long)l * p.layer_elems + seq_off + (long long)k0 * row_elems, row_elems, rows);
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    issue(0);
+    float m_run = -INFINITY, s_run = 0.f, inv = 0.f;
+    for (int pass = 0; pass < 2 && !dead; ++pass) {
+        if (pass == 1) inv = s_run > 0.f ? 1.0f / s_run : 0.f;
+        for (int kc = 0; kc < n_chunks && !dead; ++kc) {
+            const int k0 = kc * kTcChunk, t = pass * n_chunks + kc;
+            const uint32_t buf = sKV + (uint32_t)(t & 1) * kBuf;
+            const uint64_t dK = tc_desc(buf);
+            issue(t + 1);                           // its buffer was last read by the MMAs of chunk t - 1, which are complete
+            asm volatile("cp.async.wait_group 1;" ::: "memory");     // chunk t has landed (this thread's copies)
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncthreads();                        // chunk t staged by everyone; every thread has read the previous scores
+            if (threadIdx.x == 0) {
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks)      // 16 dims = 32 bytes along a row per step
+                    tc_mma(tmem, dQ + 2 * ks, dK + 2 * ks, idS, ks > 0 ? 1u : 0u);
+                tc_commit(bar_s);
+            }
+            mma_done();
+            __syncthreads();
+            if (dead_s) { dead = true; break; }
+            float z[kTcChunk];
+            {
+                float a[32], b[32];
+                tc_ld32(t_lane, a);
+                tc_ld32(t_lane + 32, b);
+#pragma unroll
+                for (int j = 0; j < 32; ++j) { z[j] = a[j]; z[32 + j] = b[j]; }
+            }
+            float m_chunk = -INFINITY;
+#pragma unroll
+            for (int j = 0; j < kTcChunk; ++j) {
+                const int key = k0 + j;
+                const bool ok = key < len && (!p.causal || key <= qrow);
+                z[j] = ok ? z[j] * p.scale_log2e : -INFINITY;
+                m_chunk = fmaxf(m_chunk, z[j]);
+            }
+            if (pass == 0) {
+                const float m_new = fmaxf(m_run, m_chunk);
+                if (m_new > -INFINITY) {
+                    float s = s_run * exp2f(m_run - m_new);
+#pragma unroll
+                    for (int j = 0; j < kTcChunk; ++j) s += exp2f(z[j] - m_new);
+                    s_run = s; m_run = m_new;
+                }
+                continue;
+            }
+            // ---- pass 1: weights of this chunk
+            float* Srow = (p.S && qrow < len) ? p.S + (((long long)seq * p.H + h) * p.cap + qrow) * p.ld_s + k0 : nullptr;
+            const float m_use = m_run > -INFINITY ? m_run : 0.f;
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {           // 8 keys = one 16-byte chunk of the operand rows
+                uint32_t hi[4], lo[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float w0 = exp2f(z[8 * c + 2 * e] - m_use) * inv, w1 = exp2f(z[8 * c + 2 * e + 1] - m_use) * inv;
+                    z[8 * c + 2 * e] = w0; z[8 * c + 2 * e + 1] = w1;
+                    hi[e] = full_pack(w0, w1);
+                    lo[e] = full_pack(w0 - __uint_as_float(hi[e] << 16), w1 - __uint_as_float(hi[e] & 0xffff0000u));
+                }
+                const int at = row * 128 + ((c ^ (row & 7)) << 4);
+                *reinterpret_cast<uint4*>(sPh + at) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+                *reinterpret_cast<uint4*>(sPl + at) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+            }
+            if (Srow) {
+#pragma unroll
+                for (int j = 0; j < kTcChunk; ++j)
+                    if (k0 + j < len) Srow[j] = z[j];              // keys a causal row does not see are stored as 0
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                for (int l = 0; l < p.n_layers; ++l) {
+                    const uint64_t dV = tc_desc(buf + (uint32_t)(1 + l) * kTcTileK);
+                    const uint32_t acc = tmem + 64u + 64u * (uint32_t)l;
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks) {        // 16 keys per step: 32 bytes along a weight row, two 8-row groups of values
+                        tc_mma(acc, dPh + 2 * ks, dV + 128 * ks, idO, (kc > 0 || ks > 0) ? 1u : 0u);
+                        tc_mma(acc, dPl + 2 * ks, dV + 128 * ks, idO, 1u);
+                    }
+                }
+                tc_commit(bar_s);
+            }
+            mma_done();                             // the operand tiles are free again
+            __syncthreads();
+            if (dead_s) { dead = true; break; }
+        }
+    }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    if (p.S && p.causal && qrow < len && !dead) {   // keys beyond the tile's last chunk: never seen by a causal row
+        float* Srow = p.S + (((long long)seq * p.H + h) * p.cap + qrow) * p.ld_s;
+        for (int j = n_chunks * kTcChunk; j < len; ++j) Srow[j] = 0.f;
+    }
+    // ---- outputs: this thread's row of every layer's accumulator
+    if (!dead) {
+        for (int l = 0; l < p.n_layers; ++l) {
+            float a[32], b[32];
+            tc_ld32(t_lane + 64u + 64u * (uint32_t)l, a);
+            tc_ld32(t_lane + 64u + 64u * (uint32_t)l + 32u, b);
+            if (qrow < len) {
+                uint4* dst = reinterpret_cast<uint4*>(p.out + (long long)l * p.layer_elems + seq_off + (long long)qrow * row_elems);
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    dst[c] = make_uint4(full_pack(a[8 * c], a[8 * c + 1]), full_pack(a[8 * c + 2], a[8 * c + 3]),
+                                        full_pack(a[8 * c + 4], a[8 * c + 5]), full_pack(a[8 * c + 6], a[8 * c + 7]));
+                    dst[4 + c] = make_uint4(full_pack(b[8 * c], b[8 * c + 1]), full_pack(b[8 * c + 2], b[8 * c + 3]),
+                                            full_pack(b[8 * c + 4], b[8 * c + 5]), full_pack(b[8 * c + 6], b[8 * c + 7]));
+                }
+            }
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 0)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem), "r"((uint32_t)kTcCols) : "memory");
+}
+
+// More than half of an SM's shared memory, so that CTAs never share an SM: each takes all 512
+// columns of tensor memory, and a second CTA would only sit in tcgen05.alloc until the first is done.
+constexpr size_t full_tc5_smem_bytes() {
+    constexpr size_t need = 1024 + 3 * (size_t)kTcTileQ + 2 * (size_t)(1 + kTcMaxLayers) * kTcTileK;
+    return need > 116 * 1024 ? need : 116 * 1024;
+}
+
+}  // namespace san

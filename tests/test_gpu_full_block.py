@@ -93,3 +93,16 @@ def test_argument_checks():
     assert f(B.SAN_BF16, 1, 1, 0, t, t, t, l, 1, 1024, 0, None, 0, t) == B.SAN_ERR_UNSUPPORTED
     assert f(B.SAN_BF16, 1, 1, 0, t, t, t, l, 1, 1, 2, None, 0, t) == B.SAN_ERR_SHAPE
     assert f(B.SAN_BF16, 1, 1, 0, t, t, t, l, 0, 1, 0, None, 0, t) == B.SAN_OK
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_tensor_memory_path_ragged_lengths(causal):
+    """A length bound of 128 or more selects the tcgen05 kernel (128-query tiles, accumulators in
+    tensor memory): lengths on both sides of the 64-key chunk and the 128-query tile, an empty
+    and a one-token sequence in the same batch."""
+    _run([1, 63, 64, 65, 127, 128, 129, 200, 0], cap=200, H=2, n_layers=3, causal=causal)
+
+
+def test_tensor_memory_path_one_and_six_layers():
+    _run([150, 333], cap=336, H=3, n_layers=1, causal=False)
+    _run([150, 333], cap=336, H=3, n_layers=6, causal=True, want_S=False)
