@@ -767,7 +767,7 @@ int32_t san_full_block(int32_t dtype, int32_t n_heads, int32_t n_layers, int32_t
         const size_t smem = full_tc5_smem_bytes();
         if (!opt_in((const void*)full_block_tc5_kernel, smem, set_tc5)) return SAN_ERR_CUDA;
         const dim3 grid((unsigned)ceil_div(max_len, kTcQ), (unsigned)n_heads, (unsigned)n_seq);
-        full_block_tc5_kernel<<<grid, kTcQ, smem, st>>>(p);
+        full_block_tc5_kernel<<<grid, kTcThreads, smem, st>>>(p);
         return cuda_status(cudaGetLastError());
     }
     static size_t set_mma[64] = {};

@@ -3,8 +3,10 @@
 // full_block_kernel: S = Softmax(Q.K^T / 8) once per block (Eq. 1, Eq. 3), O_l = S.V_l for each
 // layer of the block (Eq. 2, Eq. 4).
 //
-// CTA = (128 queries, head, sequence), 128 threads; thread t owns query row t, which is lane t
-// of tensor memory, so every row statistic is thread-local (no shuffles).
+// CTA = (128 queries, head, sequence), 256 threads; query row r is lane r of tensor memory and
+// belongs to threads r and r + 128, which take the lower and the upper 32 of a chunk's 64 score
+// columns (a warp reaches the 32 lanes of its rank modulo 4).  Row statistics are thread-local
+// and joined once, through shared memory, between the passes (no shuffles).
 //   pass 0  for each chunk of 64 keys: stage the key rows in shared memory, one
 //           tcgen05.mma chain (M 128, N 64, K 64) writes the scores into tensor memory, each
 //           thread reads its row back and keeps a running (max, sum).
@@ -28,6 +30,7 @@ namespace san {
 
 constexpr int kTcQ = 128;                 // queries per CTA = tensor-memory lanes
 constexpr int kTcChunk = 64;              // keys per MMA chain
+constexpr int kTcThreads = 256;
 constexpr int kTcMaxLayers = 6;           // accumulators: 64 columns each after the 64 of the scores (512 columns in all)
 constexpr int kTcCols = 512;
 constexpr uint32_t kTcTileQ = kTcQ * 128, kTcTileK = kTcChunk * 128;      // bytes of a 128-row and of a 64-row operand tile
@@ -69,8 +72,8 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, float (&v)[32]) {
 // zero-filled (a copy of source size 0).  Consecutive threads take consecutive pieces.
 __device__ __forceinline__ void tc_stage_async(uint32_t tile_s, const __nv_bfloat16* src, long long row_elems, int rows) {
 #pragma unroll
-    for (int i = 0; i < kTcChunk * 8 / kTcQ; ++i) {
-        const int u = (int)threadIdx.x + i * kTcQ, r = u >> 3, c = u & 7;
+    for (int i = 0; i < kTcChunk * 8 / kTcThreads; ++i) {
+        const int u = (int)threadIdx.x + i * kTcThreads, r = u >> 3, c = u & 7;
         const uint32_t bytes = r < rows ? 16u : 0u;
         const __nv_bfloat16* from = src + (long long)(r < rows ? r : 0) * row_elems + c * 8;
         asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;"
@@ -80,11 +83,11 @@ __device__ __forceinline__ void tc_stage_async(uint32_t tile_s, const __nv_bfloa
 
 extern __shared__ __align__(1024) unsigned char tc_smem[];
 
-static __global__ void __launch_bounds__(kTcQ, 1) full_block_tc5_kernel(const FullParams p) {
+static __global__ void __launch_bounds__(kTcThreads, 1) full_block_tc5_kernel(const FullParams p) {
     const int seq = blockIdx.z, h = blockIdx.y, q0 = blockIdx.x * kTcQ;
     const int len = min(p.lens[seq], p.max_len);
     if (q0 >= len) return;                                   // uniform over the CTA, before anything is allocated
-    const int row = threadIdx.x, warp = threadIdx.x >> 5;
+    const int row = threadIdx.x & (kTcQ - 1), half = threadIdx.x >> 7, warp = threadIdx.x >> 5;
     const int qrow = q0 + row;
     const long long row_elems = (long long)p.H * kDh;
     const long long seq_off = ((long long)seq * p.cap) * row_elems + (long long)h * kDh;
@@ -102,6 +105,7 @@ static __global__ void __launch_bounds__(kTcQ, 1) full_block_tc5_kernel(const Fu
     __shared__ __align__(8) uint64_t bar;
     __shared__ uint32_t tmem_base_s;
     __shared__ int dead_s;
+    __shared__ float2 stats_s[2][kTcQ];              // (max, sum) of each half of a row after pass 0
 
     if (threadIdx.x == 0) {
         mbar_init(&bar, 1);
@@ -117,7 +121,7 @@ static __global__ void __launch_bounds__(kTcQ, 1) full_block_tc5_kernel(const Fu
     {
         const __nv_bfloat16* qsrc = p.q + seq_off + (long long)qrow * row_elems;
 #pragma unroll
-        for (int c = 0; c < 8; ++c) {
+        for (int c = half * 4; c < half * 4 + 4; ++c) {
             const uint4 val = qrow < len ? ld16_stream(qsrc + c * 8) : make_uint4(0, 0, 0, 0);
             *reinterpret_cast<uint4*>(sQ + row * 128 + ((c ^ (row & 7)) << 4)) = val;
         }
@@ -126,7 +130,7 @@ static __global__ void __launch_bounds__(kTcQ, 1) full_block_tc5_kernel(const Fu
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem = tmem_base_s;
-    const uint32_t t_lane = tmem + ((uint32_t)(warp * 32) << 16);         // this warp's 32 lanes
+    const uint32_t t_lane = tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)half * 32u;   // this warp's 32 lanes, this thread's 32 columns of every 64
     const uint32_t bar_s = smem_u32(&bar);
     const uint64_t dQ = tc_desc(smem_u32(sQ)), dPh = tc_desc(smem_u32(sPh)), dPl = tc_desc(smem_u32(sPl));
     const uint32_t idS = tc_idesc(false), idO = tc_idesc(true);
@@ -156,7 +160,15 @@ static __global__ void __launch_bounds__(kTcQ, 1) full_block_tc5_kernel(const Fu
     issue(0);
     float m_run = -INFINITY, s_run = 0.f, inv = 0.f;
     for (int pass = 0; pass < 2 && !dead; ++pass) {
-        if (pass == 1) inv = s_run > 0.f ? 1.0f / s_run : 0.f;
+        if (pass == 1) {        // join the two halves of every row
+            stats_s[half][row] = make_float2(m_run, s_run);
+            __syncthreads();
+            const float2 o = stats_s[half ^ 1][row];
+            const float m_all = fmaxf(m_run, o.x);
+            if (m_all > -INFINITY) s_run = s_run * exp2f(m_run - m_all) + o.y * exp2f(o.x - m_all);
+            m_run = m_all;
+            inv = s_run > 0.f ? 1.0f / s_run : 0.f;
+        }
         for (int kc = 0; kc < n_chunks && !dead; ++kc) {
             const int k0 = kc * kTcChunk, t = pass * n_chunks + kc;
             const uint32_t buf = sKV + (uint32_t)(t & 1) * kBuf;
@@ -176,18 +188,13 @@ static __global__ void __launch_bounds__(kTcQ, 1) full_block_tc5_kernel(const Fu
             mma_done();
             __syncthreads();
             if (dead_s) { dead = true; break; }
-            float z[kTcChunk];
-            {
-                float a[32], b[32];
-                tc_ld32(t_lane, a);
-                tc_ld32(t_lane + 32, b);
-#pragma unroll
-                for (int j = 0; j < 32; ++j) { z[j] = a[j]; z[32 + j] = b[j]; }
-            }
+            float z[32];                            // this thread's half of the row's 64 scores
+            tc_ld32(t_lane, z);
+            const int kh = k0 + half * 32;          // first key of that half
             float m_chunk = -INFINITY;
 #pragma unroll
-            for (int j = 0; j < kTcChunk; ++j) {
-                const int key = k0 + j;
+            for (int j = 0; j < 32; ++j) {
+                const int key = kh + j;
                 const bool ok = key < len && (!p.causal || key <= qrow);
                 z[j] = ok ? z[j] * p.scale_log2e : -INFINITY;
                 m_chunk = fmaxf(m_chunk, z[j]);
@@ -197,16 +204,16 @@ static __global__ void __launch_bounds__(kTcQ, 1) full_block_tc5_kernel(const Fu
                 if (m_new > -INFINITY) {
                     float s = s_run * exp2f(m_run - m_new);
 #pragma unroll
-                    for (int j = 0; j < kTcChunk; ++j) s += exp2f(z[j] - m_new);
+                    for (int j = 0; j < 32; ++j) s += exp2f(z[j] - m_new);
                     s_run = s; m_run = m_new;
                 }
                 continue;
             }
             // ---- pass 1: weights of this chunk
-            float* Srow = (p.S && qrow < len) ? p.S + (((long long)seq * p.H + h) * p.cap + qrow) * p.ld_s + k0 : nullptr;
+            float* Srow = (p.S && qrow < len) ? p.S + (((long long)seq * p.H + h) * p.cap + qrow) * p.ld_s + kh : nullptr;
             const float m_use = m_run > -INFINITY ? m_run : 0.f;
 #pragma unroll
-            for (int c = 0; c < 8; ++c) {           // 8 keys = one 16-byte chunk of the operand rows
+            for (int c = 0; c < 4; ++c) {           // 8 keys = one 16-byte chunk of the operand rows; this half owns chunks 4 half ..
                 uint32_t hi[4], lo[4];
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
@@ -215,14 +222,14 @@ static __global__ void __launch_bounds__(kTcQ, 1) full_block_tc5_kernel(const Fu
                     hi[e] = full_pack(w0, w1);
                     lo[e] = full_pack(w0 - __uint_as_float(hi[e] << 16), w1 - __uint_as_float(hi[e] & 0xffff0000u));
                 }
-                const int at = row * 128 + ((c ^ (row & 7)) << 4);
+                const int at = row * 128 + (((half * 4 + c) ^ (row & 7)) << 4);
                 *reinterpret_cast<uint4*>(sPh + at) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
                 *reinterpret_cast<uint4*>(sPl + at) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
             }
             if (Srow) {
 #pragma unroll
-                for (int j = 0; j < kTcChunk; ++j)
-                    if (k0 + j < len) Srow[j] = z[j];              // keys a causal row does not see are stored as 0
+                for (int j = 0; j < 32; ++j)
+                    if (kh + j < len) Srow[j] = z[j];              // keys a causal row does not see are stored as 0
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -246,25 +253,21 @@ static __global__ void __launch_bounds__(kTcQ, 1) full_block_tc5_kernel(const Fu
         }
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
-    if (p.S && p.causal && qrow < len && !dead) {   // keys beyond the tile's last chunk: never seen by a causal row
+    if (p.S && p.causal && qrow < len && !dead && half == 0) {   // keys beyond the tile's last chunk: never seen by a causal row
         float* Srow = p.S + (((long long)seq * p.H + h) * p.cap + qrow) * p.ld_s;
         for (int j = n_chunks * kTcChunk; j < len; ++j) Srow[j] = 0.f;
     }
     // ---- outputs: this thread's row of every layer's accumulator
     if (!dead) {
-        for (int l = 0; l < p.n_layers; ++l) {
-            float a[32], b[32];
+        for (int l = 0; l < p.n_layers; ++l) {      // this thread's 32 dims of the row
+            float a[32];
             tc_ld32(t_lane + 64u + 64u * (uint32_t)l, a);
-            tc_ld32(t_lane + 64u + 64u * (uint32_t)l + 32u, b);
             if (qrow < len) {
-                uint4* dst = reinterpret_cast<uint4*>(p.out + (long long)l * p.layer_elems + seq_off + (long long)qrow * row_elems);
+                uint4* dst = reinterpret_cast<uint4*>(p.out + (long long)l * p.layer_elems + seq_off + (long long)qrow * row_elems + half * 32);
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
+                for (int c = 0; c < 4; ++c)
                     dst[c] = make_uint4(full_pack(a[8 * c], a[8 * c + 1]), full_pack(a[8 * c + 2], a[8 * c + 3]),
                                         full_pack(a[8 * c + 4], a[8 * c + 5]), full_pack(a[8 * c + 6], a[8 * c + 7]));
-                    dst[4 + c] = make_uint4(full_pack(b[8 * c], b[8 * c + 1]), full_pack(b[8 * c + 2], b[8 * c + 3]),
-                                            full_pack(b[8 * c + 4], b[8 * c + 5]), full_pack(b[8 * c + 6], b[8 * c + 7]));
-                }
             }
         }
     }
