@@ -423,9 +423,11 @@ def time_full_block(w, device, peak, reps=5):
     flops = float((2 + 2 * pi) * (src * src).sum() * H * 64)        # 2 l^2 d_h for the scores and per layer of S.V
     return {"call": "san_full_block", "layers_in_block": pi, "us_per_launch": secs * 1e6,
             "bytes_per_launch": nbytes, "achieved_gbs": nbytes / secs / 1e9, "frac_of_hbm_peak": nbytes / secs / 1e9 / peak,
-            "flops_per_launch": flops, "achieved_tflops": flops / secs / 1e12, "bound": "hbm",
-            "note": "sentences of 10-100 positions: Q, K and V are read once and the l x l products are small, "
-                    "so the launch is bound by HBM and latency, not by the tensor pipe"}
+            "flops_per_launch": flops, "achieved_tflops": flops / secs / 1e12,
+            "bound": "tensor" if cap >= 128 else "hbm",
+            "kernel": "full_block_tc5_kernel (tcgen05)" if cap >= 128 else "full_block_kernel (mma.sync)",
+            "note": "length bound >= 128: 128-query tcgen05 tiles, flops count each product once; "
+                    "below: sentences of 10-100 positions, bound by HBM and latency, not by the tensor pipe"}
 
 
 # ------------------------------------------------------------------------- the CPU oracle arm

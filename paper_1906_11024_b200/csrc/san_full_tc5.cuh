@@ -192,12 +192,21 @@ static __global__ void __launch_bounds__(kTcThreads, 1) full_block_tc5_kernel(co
             tc_ld32(t_lane, z);
             const int kh = k0 + half * 32;          // first key of that half
             float m_chunk = -INFINITY;
+            if (k0 + kTcChunk <= len && (!p.causal || k0 + kTcChunk - 1 <= q0)) {
+                // every row of the tile sees every key of the chunk (uniform over the CTA): no masks
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-                const int key = kh + j;
-                const bool ok = key < len && (!p.causal || key <= qrow);
-                z[j] = ok ? z[j] * p.scale_log2e : -INFINITY;
-                m_chunk = fmaxf(m_chunk, z[j]);
+                for (int j = 0; j < 32; ++j) {
+                    z[j] *= p.scale_log2e;
+                    m_chunk = fmaxf(m_chunk, z[j]);
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    const int key = kh + j;
+                    const bool ok = key < len && (!p.causal || key <= qrow);
+                    z[j] = ok ? z[j] * p.scale_log2e : -INFINITY;
+                    m_chunk = fmaxf(m_chunk, z[j]);
+                }
             }
             if (pass == 0) {
                 const float m_new = fmaxf(m_run, m_chunk);
