@@ -3,8 +3,8 @@
 // full_block_kernel: S = Softmax(Q.K^T / 8) once per block (Eq. 1, Eq. 3), O_l = S.V_l for each
 // layer of the block (Eq. 2, Eq. 4).
 //
-// CTA = (128 queries, head, sequence), 256 threads; query row r is lane r of tensor memory and
-// belongs to threads r and r + 128, which take the lower and the upper 32 of a chunk's 64 score
+// CTA = (128 queries, head, sequence), 512 threads; query row r is lane r of tensor memory and
+// belongs to threads r, r + 128, r + 256, r + 384, which take 16 each of a chunk's 64 score
 // columns (a warp reaches the 32 lanes of its rank modulo 4).  Row statistics are thread-local
 // and joined once, through shared memory, between the passes (no shuffles).
 //   pass 0  for each chunk of 64 keys: stage the key rows in shared memory, one
@@ -30,19 +30,23 @@ namespace san {
 
 constexpr int kTcQ = 128;                 // queries per CTA = tensor-memory lanes
 constexpr int kTcChunk = 64;              // keys per MMA chain
-constexpr int kTcThreads = 256;
+constexpr int kTcThreads = 512;
+constexpr int kTcSplit = kTcThreads / kTcQ;   // threads per query row; each takes 64 / kTcSplit score columns
+constexpr int kTcCols1 = kTcChunk / kTcSplit;  // score columns per thread
 constexpr int kTcMaxLayers = 6;           // accumulators: 64 columns each after the 64 of the scores (512 columns in all)
 constexpr int kTcCols = 512;
+constexpr uint32_t kTcScores1 = 448;       // second score buffer: the 64 columns behind the six accumulators
 constexpr uint32_t kTcTileQ = kTcQ * 128, kTcTileK = kTcChunk * 128;      // bytes of a 128-row and of a 64-row operand tile
 
-// shared-memory matrix descriptor: 128-byte swizzle, 8-row groups 1024 bytes apart
-__device__ __forceinline__ uint64_t tc_desc(uint32_t smem_addr) {
-    return (uint64_t)((smem_addr >> 4) & 0x3fffu) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) |
-           ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+// shared-memory matrix descriptor: 128-byte swizzle, 8-row groups 1024 bytes apart; lead_bytes =
+// distance between the 64-element column blocks of an MN-major operand wider than 64 (else unused)
+__device__ __forceinline__ uint64_t tc_desc(uint32_t smem_addr, uint32_t lead_bytes = 16) {
+    return (uint64_t)((smem_addr >> 4) & 0x3fffu) | ((uint64_t)((lead_bytes >> 4) & 0x3fffu) << 16) |
+           ((uint64_t)(1024 >> 4) << 32) | ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
 }
-// instruction descriptor: float32 accumulator, bf16 operands, M 128, N 64; b_mn: B is MN-major
-__device__ __forceinline__ uint32_t tc_idesc(bool b_mn) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn ? (1u << 16) : 0u) | ((uint32_t)(64 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+// instruction descriptor: float32 accumulator, bf16 operands, M 128, N n; b_mn: B is MN-major
+__device__ __forceinline__ uint32_t tc_idesc(bool b_mn, int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn ? (1u << 16) : 0u) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 }
 __device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a, uint64_t b, uint32_t idesc, uint32_t accumulate) {
     const uint32_t none = 0u;      // no output lane is disabled
@@ -67,6 +71,18 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, float (&v)[32]) {
     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, float (&v)[16]) {
+    uint32_t r[16];
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+                 "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+                 : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
 // rows [0, rows) of a [n][64] bf16 panel (row stride row_elems) into a swizzled 64-row operand
 // tile with 16-byte asynchronous copies (no registers held while they fly); the other rows are
 // zero-filled (a copy of source size 0).  Consecutive threads take consecutive pieces.
@@ -87,28 +103,29 @@ static __global__ void __launch_bounds__(kTcThreads, 1) full_block_tc5_kernel(co
     const int seq = blockIdx.z, h = blockIdx.y, q0 = blockIdx.x * kTcQ;
     const int len = min(p.lens[seq], p.max_len);
     if (q0 >= len) return;                                   // uniform over the CTA, before anything is allocated
-    const int row = threadIdx.x & (kTcQ - 1), half = threadIdx.x >> 7, warp = threadIdx.x >> 5;
+    const int row = threadIdx.x & (kTcQ - 1), part = threadIdx.x >> 7, warp = threadIdx.x >> 5;
     const int qrow = q0 + row;
     const long long row_elems = (long long)p.H * kDh;
     const long long seq_off = ((long long)seq * p.cap) * row_elems + (long long)h * kDh;
     const int n_keys = p.causal ? min(len, q0 + kTcQ) : len;
     const int n_chunks = (n_keys + kTcChunk - 1) / kTcChunk;
 
-    // shared memory (1024-byte aligned tiles): Q | weights high | weights remainder | two buffers of
-    // (K chunk, V chunk of each layer): the copies of the next chunk fly during this chunk's arithmetic
+    // shared memory (1024-byte aligned tiles): Q | weights high | weights remainder | three buffers of
+    // (K chunk, V chunk of each layer): copies run two steps ahead of the arithmetic
     unsigned char* base = tc_smem + ((1024u - (smem_u32(tc_smem) & 1023u)) & 1023u);
     unsigned char* sQ = base;
     unsigned char* sPh = sQ + kTcTileQ;
     unsigned char* sPl = sPh + kTcTileQ;
     const uint32_t sKV = smem_u32(sPl + kTcTileQ);                     // buffer b: K at sKV + b * kBuf, V of layer l behind it
     const uint32_t kBuf = (uint32_t)(1 + p.n_layers) * kTcTileK;
-    __shared__ __align__(8) uint64_t bar;
+    __shared__ __align__(8) uint64_t bar[2];         // completion of the score MMAs / of the output MMAs
     __shared__ uint32_t tmem_base_s;
     __shared__ int dead_s;
-    __shared__ float2 stats_s[2][kTcQ];              // (max, sum) of each half of a row after pass 0
+    __shared__ float2 stats_s[kTcSplit][kTcQ];       // (max, sum) of each part of a row after pass 0
 
     if (threadIdx.x == 0) {
-        mbar_init(&bar, 1);
+        mbar_init(&bar[0], 1);
+        mbar_init(&bar[1], 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         dead_s = 0;
     }
@@ -121,7 +138,7 @@ static __global__ void __launch_bounds__(kTcThreads, 1) full_block_tc5_kernel(co
     {
         const __nv_bfloat16* qsrc = p.q + seq_off + (long long)qrow * row_elems;
 #pragma unroll
-        for (int c = half * 4; c < half * 4 + 4; ++c) {
+        for (int c = part * (8 / kTcSplit); c < (part + 1) * (8 / kTcSplit); ++c) {
             const uint4 val = qrow < len ? ld16_stream(qsrc + c * 8) : make_uint4(0, 0, 0, 0);
             *reinterpret_cast<uint4*>(sQ + row * 128 + ((c ^ (row & 7)) << 4)) = val;
         }
@@ -130,26 +147,26 @@ static __global__ void __launch_bounds__(kTcThreads, 1) full_block_tc5_kernel(co
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem = tmem_base_s;
-    const uint32_t t_lane = tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)half * 32u;   // this warp's 32 lanes, this thread's 32 columns of every 64
-    const uint32_t bar_s = smem_u32(&bar);
+    const uint32_t t_lane = tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(part * kTcCols1);   // this warp's 32 lanes, this thread's columns of every 64
+    const uint32_t bar_s = smem_u32(&bar[0]), bar_o = smem_u32(&bar[1]);
     const uint64_t dQ = tc_desc(smem_u32(sQ)), dPh = tc_desc(smem_u32(sPh)), dPl = tc_desc(smem_u32(sPl));
-    const uint32_t idS = tc_idesc(false), idO = tc_idesc(true);
-    uint32_t phase = 0;
+    const uint32_t idS = tc_idesc(false, kTcChunk);
+    uint32_t phase_s = 0, phase_o = 0;
     bool dead = false;
+    const int n_steps = 2 * n_chunks;             // step t: pass t / n_chunks, chunk t % n_chunks
 
-    // waits for the MMAs committed last; false (for the whole CTA, after a barrier) if the wait ran out
-    auto mma_done = [&]() -> bool {
-        if (!mbar_try_wait(bar_s, phase) && !mbar_wait_slow(bar_s, phase)) dead_s = 1;
+    // Bounded wait on one of the two MMA barriers; a wait that runs out marks the CTA dead (seen by
+    // everyone after the next CTA barrier).
+    auto mma_wait = [&](uint32_t bar_addr, uint32_t& phase) {
+        if (!mbar_try_wait(bar_addr, phase) && !mbar_wait_slow(bar_addr, phase)) dead_s = 1;
         phase ^= 1u;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        return true;
     };
-
-    // Chunk t of the run (pass 0: keys only; pass 1: keys and every layer's values) into buffer t & 1.
+    // The copies of step t (pass 0: keys; pass 1: keys and every layer's values) into buffer t % 3.
     auto issue = [&](int t) {
-        if (t < 2 * n_chunks) {
+        if (t < n_steps) {
             const int pass = t >= n_chunks ? 1 : 0, k0 = (t - pass * n_chunks) * kTcChunk, rows = min(kTcChunk, len - k0);
-            const uint32_t buf = sKV + (uint32_t)(t & 1) * kBuf;
+            const uint32_t buf = sKV + (uint32_t)(t % 3) * kBuf;
             tc_stage_async(buf, p.k + seq_off + (long long)k0 * row_elems, row_elems, rows);
             if (pass)
                 for (int l = 0; l < p.n_layers; ++l)
@@ -157,124 +174,152 @@ static __global__ void __launch_bounds__(kTcThreads, 1) full_block_tc5_kernel(co
         }
         asm volatile("cp.async.commit_group;" ::: "memory");
     };
+    // Scores of step t: Q x (key chunk in buffer t % 3)^T into score buffer t & 1 of tensor memory.
+    auto issue_scores = [&](int t) {
+        const uint64_t dK = tc_desc(sKV + (uint32_t)(t % 3) * kBuf);
+        const uint32_t d = tmem + ((t & 1) ? kTcScores1 : 0u);
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks)            // 16 dims = 32 bytes along a row per step
+            tc_mma(d, dQ + 2 * ks, dK + 2 * ks, idS, ks > 0 ? 1u : 0u);
+        tc_commit(bar_s);
+    };
+
+    // The tensor pipe runs ahead of the threads: when the threads turn the scores of step t into
+    // statistics or weights, the scores of step t + 1 are being computed (second score buffer) and,
+    // in pass 1, so are the outputs of step t - 1; copies run two steps ahead (three buffers).
     issue(0);
+    issue(1);
+    asm volatile("cp.async.wait_group 1;" ::: "memory");             // step 0 has landed
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        issue_scores(0);
+    }
     float m_run = -INFINITY, s_run = 0.f, inv = 0.f;
-    for (int pass = 0; pass < 2 && !dead; ++pass) {
-        if (pass == 1) {        // join the two halves of every row
-            stats_s[half][row] = make_float2(m_run, s_run);
+    for (int t = 0; t < n_steps; ++t) {
+        const int pass = t >= n_chunks ? 1 : 0, kc = t - pass * n_chunks, k0 = kc * kTcChunk;
+        const uint32_t buf = sKV + (uint32_t)(t % 3) * kBuf;
+        mma_wait(bar_s, phase_s);                 // scores of step t (and everything issued before them) are complete
+        float z[kTcCols1];                        // this thread's part of the row's 64 scores
+        tc_ld16(t_lane + ((t & 1) ? kTcScores1 : 0u), z);
+        asm volatile("cp.async.wait_group 0;" ::: "memory");         // step t + 1 has landed (this thread's copies)
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncthreads();                          // ... everyone's; and everyone has read the scores of step t
+        if (dead_s) { dead = true; break; }
+        if (threadIdx.x == 0 && t + 1 < n_steps) {
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            issue_scores(t + 1);
+        }
+        if (pass == 0) issue(t + 2);              // buffer (t + 2) % 3 held step t - 1, whose scores are complete
+        if (t == n_chunks) {                      // between the passes: join the two halves of every row
+            stats_s[part][row] = make_float2(m_run, s_run);
             __syncthreads();
-            const float2 o = stats_s[half ^ 1][row];
-            const float m_all = fmaxf(m_run, o.x);
-            if (m_all > -INFINITY) s_run = s_run * exp2f(m_run - m_all) + o.y * exp2f(o.x - m_all);
-            m_run = m_all;
+            float m_all = -INFINITY, s_all = 0.f;
+#pragma unroll
+            for (int o = 0; o < kTcSplit; ++o) m_all = fmaxf(m_all, stats_s[o][row].x);
+            if (m_all > -INFINITY) {
+#pragma unroll
+                for (int o = 0; o < kTcSplit; ++o) s_all += stats_s[o][row].y * exp2f(stats_s[o][row].x - m_all);
+            }
+            m_run = m_all; s_run = s_all;
             inv = s_run > 0.f ? 1.0f / s_run : 0.f;
         }
-        for (int kc = 0; kc < n_chunks && !dead; ++kc) {
-            const int k0 = kc * kTcChunk, t = pass * n_chunks + kc;
-            const uint32_t buf = sKV + (uint32_t)(t & 1) * kBuf;
-            const uint64_t dK = tc_desc(buf);
-            issue(t + 1);                           // its buffer was last read by the MMAs of chunk t - 1, which are complete
-            asm volatile("cp.async.wait_group 1;" ::: "memory");     // chunk t has landed (this thread's copies)
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-            __syncthreads();                        // chunk t staged by everyone; every thread has read the previous scores
-            if (threadIdx.x == 0) {
-                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const int kh = k0 + part * kTcCols1;      // first key of this thread's part
+        float m_chunk = -INFINITY;
+        if (k0 + kTcChunk <= len && (!p.causal || k0 + kTcChunk - 1 <= q0)) {
+            // every row of the tile sees every key of the chunk (uniform over the CTA): no masks
 #pragma unroll
-                for (int ks = 0; ks < 4; ++ks)      // 16 dims = 32 bytes along a row per step
-                    tc_mma(tmem, dQ + 2 * ks, dK + 2 * ks, idS, ks > 0 ? 1u : 0u);
-                tc_commit(bar_s);
+            for (int j = 0; j < kTcCols1; ++j) {
+                z[j] *= p.scale_log2e;
+                m_chunk = fmaxf(m_chunk, z[j]);
             }
-            mma_done();
-            __syncthreads();
-            if (dead_s) { dead = true; break; }
-            float z[32];                            // this thread's half of the row's 64 scores
-            tc_ld32(t_lane, z);
-            const int kh = k0 + half * 32;          // first key of that half
-            float m_chunk = -INFINITY;
-            if (k0 + kTcChunk <= len && (!p.causal || k0 + kTcChunk - 1 <= q0)) {
-                // every row of the tile sees every key of the chunk (uniform over the CTA): no masks
+        } else {
 #pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    z[j] *= p.scale_log2e;
-                    m_chunk = fmaxf(m_chunk, z[j]);
+            for (int j = 0; j < kTcCols1; ++j) {
+                const int key = kh + j;
+                const bool ok = key < len && (!p.causal || key <= qrow);
+                z[j] = ok ? z[j] * p.scale_log2e : -INFINITY;
+                m_chunk = fmaxf(m_chunk, z[j]);
+            }
+        }
+        if (pass == 0) {
+            const float m_new = fmaxf(m_run, m_chunk);
+            if (m_new > -INFINITY) {
+                float s = s_run * exp2f(m_run - m_new);
+#pragma unroll
+                for (int j = 0; j < kTcCols1; ++j) s += exp2f(z[j] - m_new);
+                s_run = s; m_run = m_new;
+            }
+            continue;
+        }
+        // ---- pass 1: weights of this chunk, in registers first
+        float* Srow = (p.S && qrow < len) ? p.S + (((long long)seq * p.H + h) * p.cap + qrow) * p.ld_s + kh : nullptr;
+        const float m_use = m_run > -INFINITY ? m_run : 0.f;
+        uint32_t hi[kTcCols1 / 2], lo[kTcCols1 / 2];
+#pragma unroll
+        for (int e = 0; e < kTcCols1 / 2; ++e) {
+            const float w0 = exp2f(z[2 * e] - m_use) * inv, w1 = exp2f(z[2 * e + 1] - m_use) * inv;
+            z[2 * e] = w0; z[2 * e + 1] = w1;
+            hi[e] = full_pack(w0, w1);
+            lo[e] = full_pack(w0 - __uint_as_float(hi[e] << 16), w1 - __uint_as_float(hi[e] & 0xffff0000u));
+        }
+        if (Srow) {
+#pragma unroll
+            for (int j = 0; j < kTcCols1; ++j)
+                if (kh + j < len) Srow[j] = z[j];                  // keys a causal row does not see are stored as 0
+        }
+        if (kc > 0) mma_wait(bar_o, phase_o);     // outputs of step t - 1 complete: the weight tiles and its buffer are free
+        issue(t + 2);
+#pragma unroll
+        for (int c = 0; c < kTcCols1 / 8; ++c) {  // 8 keys = one 16-byte chunk of the operand rows; this part owns chunks part * kTcCols1 / 8 ..
+            const int at = row * 128 + (((part * (kTcCols1 / 8) + c) ^ (row & 7)) << 4);
+            *reinterpret_cast<uint4*>(sPh + at) = make_uint4(hi[4 * c], hi[4 * c + 1], hi[4 * c + 2], hi[4 * c + 3]);
+            *reinterpret_cast<uint4*>(sPl + at) = make_uint4(lo[4 * c], lo[4 * c + 1], lo[4 * c + 2], lo[4 * c + 3]);
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncthreads();
+        if (dead_s) { dead = true; break; }
+        if (threadIdx.x == 0) {
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            // Up to four layers per MMA: their value tiles lie one behind the other (8 KB apart) and
+            // form one MN-major B operand of 64 dims x layers columns; so do their accumulators.
+            for (int l0 = 0; l0 < p.n_layers; l0 += 4) {
+                const int nl = min(4, p.n_layers - l0);
+                const uint64_t dV = tc_desc(buf + (uint32_t)(1 + l0) * kTcTileK, kTcTileK);
+                const uint32_t idO = tc_idesc(true, nl * kDh);
+                const uint32_t acc = tmem + 64u + 64u * (uint32_t)l0;
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks) {  // 16 keys per step: 32 bytes along a weight row, two 8-row groups of values
+                    tc_mma(acc, dPh + 2 * ks, dV + 128 * ks, idO, (kc > 0 || ks > 0) ? 1u : 0u);
+                    tc_mma(acc, dPl + 2 * ks, dV + 128 * ks, idO, 1u);
                 }
-            } else {
-#pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    const int key = kh + j;
-                    const bool ok = key < len && (!p.causal || key <= qrow);
-                    z[j] = ok ? z[j] * p.scale_log2e : -INFINITY;
-                    m_chunk = fmaxf(m_chunk, z[j]);
-                }
             }
-            if (pass == 0) {
-                const float m_new = fmaxf(m_run, m_chunk);
-                if (m_new > -INFINITY) {
-                    float s = s_run * exp2f(m_run - m_new);
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) s += exp2f(z[j] - m_new);
-                    s_run = s; m_run = m_new;
-                }
-                continue;
-            }
-            // ---- pass 1: weights of this chunk
-            float* Srow = (p.S && qrow < len) ? p.S + (((long long)seq * p.H + h) * p.cap + qrow) * p.ld_s + kh : nullptr;
-            const float m_use = m_run > -INFINITY ? m_run : 0.f;
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {           // 8 keys = one 16-byte chunk of the operand rows; this half owns chunks 4 half ..
-                uint32_t hi[4], lo[4];
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const float w0 = exp2f(z[8 * c + 2 * e] - m_use) * inv, w1 = exp2f(z[8 * c + 2 * e + 1] - m_use) * inv;
-                    z[8 * c + 2 * e] = w0; z[8 * c + 2 * e + 1] = w1;
-                    hi[e] = full_pack(w0, w1);
-                    lo[e] = full_pack(w0 - __uint_as_float(hi[e] << 16), w1 - __uint_as_float(hi[e] & 0xffff0000u));
-                }
-                const int at = row * 128 + (((half * 4 + c) ^ (row & 7)) << 4);
-                *reinterpret_cast<uint4*>(sPh + at) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-                *reinterpret_cast<uint4*>(sPl + at) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
-            }
-            if (Srow) {
-#pragma unroll
-                for (int j = 0; j < 32; ++j)
-                    if (kh + j < len) Srow[j] = z[j];              // keys a causal row does not see are stored as 0
-            }
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-            __syncthreads();
-            if (threadIdx.x == 0) {
-                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                for (int l = 0; l < p.n_layers; ++l) {
-                    const uint64_t dV = tc_desc(buf + (uint32_t)(1 + l) * kTcTileK);
-                    const uint32_t acc = tmem + 64u + 64u * (uint32_t)l;
-#pragma unroll
-                    for (int ks = 0; ks < 4; ++ks) {        // 16 keys per step: 32 bytes along a weight row, two 8-row groups of values
-                        tc_mma(acc, dPh + 2 * ks, dV + 128 * ks, idO, (kc > 0 || ks > 0) ? 1u : 0u);
-                        tc_mma(acc, dPl + 2 * ks, dV + 128 * ks, idO, 1u);
-                    }
-                }
-                tc_commit(bar_s);
-            }
-            mma_done();                             // the operand tiles are free again
-            __syncthreads();
-            if (dead_s) { dead = true; break; }
+            tc_commit(bar_o);
         }
     }
+    if (!dead) {                                  // the outputs of the last step
+        mma_wait(bar_o, phase_o);
+        __syncthreads();
+        if (dead_s) dead = true;
+    }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
-    if (p.S && p.causal && qrow < len && !dead && half == 0) {   // keys beyond the tile's last chunk: never seen by a causal row
+    if (p.S && p.causal && qrow < len && !dead && part == 0) {   // keys beyond the tile's last chunk: never seen by a causal row
         float* Srow = p.S + (((long long)seq * p.H + h) * p.cap + qrow) * p.ld_s;
         for (int j = n_chunks * kTcChunk; j < len; ++j) Srow[j] = 0.f;
     }
     // ---- outputs: this thread's row of every layer's accumulator
     if (!dead) {
-        for (int l = 0; l < p.n_layers; ++l) {      // this thread's 32 dims of the row
-            float a[32];
-            tc_ld32(t_lane + 64u + 64u * (uint32_t)l, a);
+        for (int l = 0; l < p.n_layers; ++l) {      // this thread's 16 dims of the row
+            float a[kTcCols1];
+            tc_ld16(t_lane + 64u + 64u * (uint32_t)l, a);
             if (qrow < len) {
-                uint4* dst = reinterpret_cast<uint4*>(p.out + (long long)l * p.layer_elems + seq_off + (long long)qrow * row_elems + half * 32);
+                uint4* dst = reinterpret_cast<uint4*>(p.out + (long long)l * p.layer_elems + seq_off + (long long)qrow * row_elems + part * kTcCols1);
 #pragma unroll
-                for (int c = 0; c < 4; ++c)
+                for (int c = 0; c < kTcCols1 / 8; ++c)
                     dst[c] = make_uint4(full_pack(a[8 * c], a[8 * c + 1]), full_pack(a[8 * c + 2], a[8 * c + 3]),
                                         full_pack(a[8 * c + 4], a[8 * c + 5]), full_pack(a[8 * c + 6], a[8 * c + 7]));
             }
@@ -289,7 +334,7 @@ static __global__ void __launch_bounds__(kTcThreads, 1) full_block_tc5_kernel(co
 // More than half of an SM's shared memory, so that CTAs never share an SM: each takes all 512
 // columns of tensor memory, and a second CTA would only sit in tcgen05.alloc until the first is done.
 constexpr size_t full_tc5_smem_bytes() {
-    constexpr size_t need = 1024 + 3 * (size_t)kTcTileQ + 2 * (size_t)(1 + kTcMaxLayers) * kTcTileK;
+    constexpr size_t need = 1024 + 3 * (size_t)kTcTileQ + 3 * (size_t)(1 + kTcMaxLayers) * kTcTileK;
     return need > 116 * 1024 ? need : 116 * 1024;
 }
 
