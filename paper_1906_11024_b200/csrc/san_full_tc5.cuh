@@ -110,14 +110,16 @@ static __global__ void __launch_bounds__(kTcThreads, 1) full_block_tc5_kernel(co
     const int n_keys = p.causal ? min(len, q0 + kTcQ) : len;
     const int n_chunks = (n_keys + kTcChunk - 1) / kTcChunk;
 
-    // shared memory (1024-byte aligned tiles): Q | weights high | weights remainder | three buffers of
-    // (K chunk, V chunk of each layer): copies run two steps ahead of the arithmetic
+    // shared memory (1024-byte aligned tiles): Q | weights high | weights remainder | a ring of four
+    // K chunks | a ring of two (V chunk of each layer).  Keys are needed a step before the values of
+    // the same chunk (the scores run ahead), so they are copied three steps ahead, values one.
     unsigned char* base = tc_smem + ((1024u - (smem_u32(tc_smem) & 1023u)) & 1023u);
     unsigned char* sQ = base;
     unsigned char* sPh = sQ + kTcTileQ;
     unsigned char* sPl = sPh + kTcTileQ;
-    const uint32_t sKV = smem_u32(sPl + kTcTileQ);                     // buffer b: K at sKV + b * kBuf, V of layer l behind it
-    const uint32_t kBuf = (uint32_t)(1 + p.n_layers) * kTcTileK;
+    const uint32_t sKr = smem_u32(sPl + kTcTileQ);                     // K chunk of step t at sKr + (t % 4) * kTcTileK
+    const uint32_t sVr = sKr + 4 * kTcTileK;                            // V chunks of step t at sVr + (t % 2) * kVBuf, layer l at + l * kTcTileK
+    const uint32_t kVBuf = (uint32_t)p.n_layers * kTcTileK;
     __shared__ __align__(8) uint64_t bar[2];         // completion of the score MMAs / of the output MMAs
     __shared__ uint32_t tmem_base_s;
     __shared__ int dead_s;
@@ -162,21 +164,27 @@ static __global__ void __launch_bounds__(kTcThreads, 1) full_block_tc5_kernel(co
         phase ^= 1u;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     };
-    // The copies of step t (pass 0: keys; pass 1: keys and every layer's values) into buffer t % 3.
-    auto issue = [&](int t) {
+    // Copies of step t, each a group of its own (empty where the step has none): the key chunk, and in
+    // pass 1 the value chunk of every layer.
+    auto issue_keys = [&](int t) {
         if (t < n_steps) {
-            const int pass = t >= n_chunks ? 1 : 0, k0 = (t - pass * n_chunks) * kTcChunk, rows = min(kTcChunk, len - k0);
-            const uint32_t buf = sKV + (uint32_t)(t % 3) * kBuf;
-            tc_stage_async(buf, p.k + seq_off + (long long)k0 * row_elems, row_elems, rows);
-            if (pass)
-                for (int l = 0; l < p.n_layers; ++l)
-                    tc_stage_async(buf + (uint32_t)(1 + l) * kTcTileK, p.v + (long long)l * p.layer_elems + seq_off + (long long)k0 * row_elems, row_elems, rows);
+            const int k0 = (t >= n_chunks ? t - n_chunks : t) * kTcChunk;
+            tc_stage_async(sKr + (uint32_t)(t & 3) * kTcTileK, p.k + seq_off + (long long)k0 * row_elems, row_elems, min(kTcChunk, len - k0));
         }
         asm volatile("cp.async.commit_group;" ::: "memory");
     };
-    // Scores of step t: Q x (key chunk in buffer t % 3)^T into score buffer t & 1 of tensor memory.
+    auto issue_values = [&](int t) {
+        if (t >= n_chunks && t < n_steps) {
+            const int k0 = (t - n_chunks) * kTcChunk, rows = min(kTcChunk, len - k0);
+            for (int l = 0; l < p.n_layers; ++l)
+                tc_stage_async(sVr + (uint32_t)(t & 1) * kVBuf + (uint32_t)l * kTcTileK,
+                               p.v + (long long)l * p.layer_elems + seq_off + (long long)k0 * row_elems, row_elems, rows);
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    // Scores of step t: Q x (key chunk t)^T into score buffer t & 1 of tensor memory.
     auto issue_scores = [&](int t) {
-        const uint64_t dK = tc_desc(sKV + (uint32_t)(t % 3) * kBuf);
+        const uint64_t dK = tc_desc(sKr + (uint32_t)(t & 3) * kTcTileK);
         const uint32_t d = tmem + ((t & 1) ? kTcScores1 : 0u);
 #pragma unroll
         for (int ks = 0; ks < 4; ++ks)            // 16 dims = 32 bytes along a row per step
@@ -186,10 +194,12 @@ static __global__ void __launch_bounds__(kTcThreads, 1) full_block_tc5_kernel(co
 
     // The tensor pipe runs ahead of the threads: when the threads turn the scores of step t into
     // statistics or weights, the scores of step t + 1 are being computed (second score buffer) and,
-    // in pass 1, so are the outputs of step t - 1; copies run two steps ahead (three buffers).
-    issue(0);
-    issue(1);
-    asm volatile("cp.async.wait_group 1;" ::: "memory");             // step 0 has landed
+    // in pass 1, so are the outputs of step t - 1.  Every step commits two copy groups, keys of
+    // step t + 3 and values of step t + 1; the set-up commits what steps -3 .. -1 would have.
+    issue_keys(0); issue_values(-2);
+    issue_keys(1); issue_values(-1);
+    issue_keys(2); issue_values(0);
+    asm volatile("cp.async.wait_group 5;" ::: "memory");             // keys of step 0 have landed
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
@@ -200,11 +210,10 @@ static __global__ void __launch_bounds__(kTcThreads, 1) full_block_tc5_kernel(co
     float m_run = -INFINITY, s_run = 0.f, inv = 0.f;
     for (int t = 0; t < n_steps; ++t) {
         const int pass = t >= n_chunks ? 1 : 0, kc = t - pass * n_chunks, k0 = kc * kTcChunk;
-        const uint32_t buf = sKV + (uint32_t)(t % 3) * kBuf;
         mma_wait(bar_s, phase_s);                 // scores of step t (and everything issued before them) are complete
         float z[kTcCols1];                        // this thread's part of the row's 64 scores
         tc_ld16(t_lane + ((t & 1) ? kTcScores1 : 0u), z);
-        asm volatile("cp.async.wait_group 0;" ::: "memory");         // step t + 1 has landed (this thread's copies)
+        asm volatile("cp.async.wait_group 3;" ::: "memory");         // keys of step t + 1 have landed (this thread's copies)
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         __syncthreads();                          // ... everyone's; and everyone has read the scores of step t
@@ -213,7 +222,8 @@ static __global__ void __launch_bounds__(kTcThreads, 1) full_block_tc5_kernel(co
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             issue_scores(t + 1);
         }
-        if (pass == 0) issue(t + 2);              // buffer (t + 2) % 3 held step t - 1, whose scores are complete
+        issue_keys(t + 3);                        // into the slot of step t - 1, whose scores are complete
+        if (pass == 0) issue_values(t + 1);       // (a real copy only ahead of the first step of pass 1)
         if (t == n_chunks) {                      // between the passes: join the two halves of every row
             stats_s[part][row] = make_float2(m_run, s_run);
             __syncthreads();
@@ -272,13 +282,14 @@ static __global__ void __launch_bounds__(kTcThreads, 1) full_block_tc5_kernel(co
                 if (kh + j < len) Srow[j] = z[j];                  // keys a causal row does not see are stored as 0
         }
         if (kc > 0) mma_wait(bar_o, phase_o);     // outputs of step t - 1 complete: the weight tiles and its buffer are free
-        issue(t + 2);
+        issue_values(t + 1);                      // into the slot of step t - 1
 #pragma unroll
         for (int c = 0; c < kTcCols1 / 8; ++c) {  // 8 keys = one 16-byte chunk of the operand rows; this part owns chunks part * kTcCols1 / 8 ..
             const int at = row * 128 + (((part * (kTcCols1 / 8) + c) ^ (row & 7)) << 4);
             *reinterpret_cast<uint4*>(sPh + at) = make_uint4(hi[4 * c], hi[4 * c + 1], hi[4 * c + 2], hi[4 * c + 3]);
             *reinterpret_cast<uint4*>(sPl + at) = make_uint4(lo[4 * c], lo[4 * c + 1], lo[4 * c + 2], lo[4 * c + 3]);
         }
+        asm volatile("cp.async.wait_group 2;" ::: "memory");         // values of step t have landed
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         __syncthreads();
@@ -289,7 +300,7 @@ static __global__ void __launch_bounds__(kTcThreads, 1) full_block_tc5_kernel(co
             // form one MN-major B operand of 64 dims x layers columns; so do their accumulators.
             for (int l0 = 0; l0 < p.n_layers; l0 += 4) {
                 const int nl = min(4, p.n_layers - l0);
-                const uint64_t dV = tc_desc(buf + (uint32_t)(1 + l0) * kTcTileK, kTcTileK);
+                const uint64_t dV = tc_desc(sVr + (uint32_t)(t & 1) * kVBuf + (uint32_t)l0 * kTcTileK, kTcTileK);
                 const uint32_t idO = tc_idesc(true, nl * kDh);
                 const uint32_t acc = tmem + 64u + 64u * (uint32_t)l0;
 #pragma unroll
@@ -334,7 +345,7 @@ static __global__ void __launch_bounds__(kTcThreads, 1) full_block_tc5_kernel(co
 // More than half of an SM's shared memory, so that CTAs never share an SM: each takes all 512
 // columns of tensor memory, and a second CTA would only sit in tcgen05.alloc until the first is done.
 constexpr size_t full_tc5_smem_bytes() {
-    constexpr size_t need = 1024 + 3 * (size_t)kTcTileQ + 3 * (size_t)(1 + kTcMaxLayers) * kTcTileK;
+    constexpr size_t need = 1024 + 3 * (size_t)kTcTileQ + (4 + 2 * (size_t)kTcMaxLayers) * kTcTileK;
     return need > 116 * 1024 ? need : 116 * 1024;
 }
 
