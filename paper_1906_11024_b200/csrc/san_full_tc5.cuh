@@ -3,19 +3,21 @@
 // full_block_kernel: S = Softmax(Q.K^T / 8) once per block (Eq. 1, Eq. 3), O_l = S.V_l for each
 // layer of the block (Eq. 2, Eq. 4).
 //
-// CTA = (128 queries, head, sequence), 512 threads; query row r is lane r of tensor memory and
-// belongs to threads r, r + 128, r + 256, r + 384, which take 16 each of a chunk's 64 score
-// columns (a warp reaches the 32 lanes of its rank modulo 4).  Row statistics are thread-local
-// and joined once, through shared memory, between the passes (no shuffles).
-//   pass 0  for each chunk of 64 keys: stage the key rows in shared memory, one
-//           tcgen05.mma chain (M 128, N 64, K 64) writes the scores into tensor memory, each
-//           thread reads its row back and keeps a running (max, sum).
-//   pass 1  for each chunk again: scores once more (cheaper than keeping 128 x l floats),
-//           weights = exp2(z - max) / sum go out to S and, as a bf16 high part and a bf16
-//           remainder, into two shared-memory operand tiles; the value rows of every layer of
-//           the block are staged, and per layer two tcgen05.mma chains (M 128, N 64, K 64) add
-//           weights x values to that layer's accumulator, which stays in tensor memory
-//           (columns 64 + 64 l) until the last chunk.
+// CTA = (128 queries, head, sequence), kTcThreads threads; query row r is lane r of tensor
+// memory and belongs to threads r, r + 128, ..., which share a chunk's 64 score columns (a warp
+// reaches the 32 lanes of its rank modulo 4).  Row statistics are thread-local and joined once,
+// through shared memory, between the passes (no shuffles).  A run is 2 x chunks steps:
+//   pass 0  per chunk of 64 keys one tcgen05.mma chain (M 128, N 64, K 64) writes the scores
+//           into tensor memory; each thread reads its part of its row back and keeps a running
+//           (max, sum).
+//   pass 1  scores once more (cheaper than keeping 128 x l floats); weights =
+//           exp2(z - max) / sum go out to S and, as a bf16 high part and a bf16 remainder, into
+//           two shared-memory operand tiles; two MMA chains per group of up to four layers
+//           (N = 64 x layers) add weights x values to the layers' accumulators, which stay in
+//           tensor memory (columns 64 + 64 l) until the last chunk.
+// The tensor pipe runs ahead of the threads: the scores of step t + 1 go to a second score
+// buffer while the threads work on step t, and the outputs of step t - 1 are still being
+// accumulated; key chunks are copied (cp.async) three steps ahead, value chunks one.
 // Operand tiles are rows of 128 bytes with the 16-byte chunks XOR-swizzled by (row & 7), the
 // 128-byte swizzle the matrix descriptors name; queries, keys and weights are K-major, the
 // value rows (dims contiguous) are the MN-major B operand.  Every wait on the MMA barrier is
@@ -30,7 +32,7 @@ namespace san {
 
 constexpr int kTcQ = 128;                 // queries per CTA = tensor-memory lanes
 constexpr int kTcChunk = 64;              // keys per MMA chain
-constexpr int kTcThreads = 512;
+constexpr int kTcThreads = 256;
 constexpr int kTcSplit = kTcThreads / kTcQ;   // threads per query row; each takes 64 / kTcSplit score columns
 constexpr int kTcCols1 = kTcChunk / kTcSplit;  // score columns per thread
 constexpr int kTcMaxLayers = 6;           // accumulators: 64 columns each after the 64 of the scores (512 columns in all)
@@ -82,6 +84,9 @@ __device__ __forceinline__ void tc_ld16(uint32_t taddr, float (&v)[16]) {
 #pragma unroll
     for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
+
+__device__ __forceinline__ void tc_ld(uint32_t taddr, float (&v)[16]) { tc_ld16(taddr, v); }
+__device__ __forceinline__ void tc_ld(uint32_t taddr, float (&v)[32]) { tc_ld32(taddr, v); }
 
 // rows [0, rows) of a [n][64] bf16 panel (row stride row_elems) into a swizzled 64-row operand
 // tile with 16-byte asynchronous copies (no registers held while they fly); the other rows are
@@ -212,7 +217,7 @@ static __global__ void __launch_bounds__(kTcThreads, 1) full_block_tc5_kernel(co
         const int pass = t >= n_chunks ? 1 : 0, kc = t - pass * n_chunks, k0 = kc * kTcChunk;
         mma_wait(bar_s, phase_s);                 // scores of step t (and everything issued before them) are complete
         float z[kTcCols1];                        // this thread's part of the row's 64 scores
-        tc_ld16(t_lane + ((t & 1) ? kTcScores1 : 0u), z);
+        tc_ld(t_lane + ((t & 1) ? kTcScores1 : 0u), z);
         asm volatile("cp.async.wait_group 3;" ::: "memory");         // keys of step t + 1 have landed (this thread's copies)
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -326,7 +331,7 @@ static __global__ void __launch_bounds__(kTcThreads, 1) full_block_tc5_kernel(co
     if (!dead) {
         for (int l = 0; l < p.n_layers; ++l) {      // this thread's 16 dims of the row
             float a[kTcCols1];
-            tc_ld16(t_lane + 64u + 64u * (uint32_t)l, a);
+            tc_ld(t_lane + 64u + 64u * (uint32_t)l, a);
             if (qrow < len) {
                 uint4* dst = reinterpret_cast<uint4*>(p.out + (long long)l * p.layer_elems + seq_off + (long long)qrow * row_elems + part * kTcCols1);
 #pragma unroll
