@@ -17,7 +17,11 @@
 
 namespace san {
 
-constexpr int kReorderThreads = 256;      // one 16-byte piece per thread and beam: a tile is 4 KB of every beam
+// One 16-byte piece per thread and beam: a tile is 1 KB (8 bf16 rows) of every beam.  Small tiles
+// because rows are short (20-35 positions at sentence sizes): with 4 KB tiles a third of the
+// threads had no piece (measured: 256 threads 0.53, 128 threads 0.61, 64 threads 0.65 of the copy
+// bandwidth on 21-row panels; 0.98-1.0 on 256-row panels with any of them).
+constexpr int kReorderThreads = 64;
 
 // The tile is written later in the same kernel, so the read-only (non-coherent) path is not
 // allowed here: an ordinary load, kept out of L1 because every piece is read once.
@@ -43,7 +47,7 @@ struct ReorderParams {
 };
 
 // grid = (tiles_per_panel * n_heads * n_sent, n_planes).  Thread t of tile k owns piece
-// k * 256 + t of the (plane, sentence, head) panel in every beam: it loads the piece of each
+// k * kReorderThreads + t of the (plane, sentence, head) panel in every beam: it loads the piece of each
 // beam's parent, the CTA meets at a barrier, it stores.  The address arithmetic that does not
 // depend on the beam is done once per thread; the copy itself is a handful of instructions
 // per piece, so that the kernel is bound by HBM and not by instruction issue.
