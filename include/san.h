@@ -244,7 +244,10 @@ int32_t san_beam_reorder(san_ctx* ctx, const int32_t* d_sent_ids, const int32_t*
  *             to (causal) are written as 0, entries at or beyond d_lens[i] are not written
  * dtype must be SAN_BF16 (SAN_F32 is refused with SAN_ERR_UNSUPPORTED: tensor-core products
  * of float32 inputs would not meet the float32 tolerance).  max_len is a host bound on d_lens
- * (0 = cap_len); a longer length is cut to max_len; max_len above 512 is SAN_ERR_UNSUPPORTED. */
+ * (0 = cap_len); a longer length is cut to max_len.  It also selects the kernel: a bound of
+ * 128 or more with n_layers <= 6 runs 128-query tiles on the tcgen05 tensor cores with the
+ * accumulators in tensor memory (any length); otherwise 64-query tiles on mma.sync, for which
+ * max_len above 512 is SAN_ERR_UNSUPPORTED. */
 int32_t san_full_block(int32_t dtype, int32_t n_heads, int32_t n_layers, int32_t causal, const void* d_q,
                        const void* d_k, const void* d_v, const int32_t* d_lens, int32_t n_seq, int32_t cap_len,
                        int32_t max_len, float* d_S, int64_t ld_s, void* d_out, void* stream);

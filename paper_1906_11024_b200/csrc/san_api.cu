@@ -737,7 +737,8 @@ int32_t san_full_block(int32_t dtype, int32_t n_heads, int32_t n_layers, int32_t
     if (n_seq < 0 || n_seq > 65535 || cap_len < 1) return SAN_ERR_SHAPE;
     if (max_len == 0) max_len = cap_len;
     if (max_len < 1 || max_len > cap_len) return SAN_ERR_SHAPE;
-    if (max_len > kFullMaxLen) return SAN_ERR_UNSUPPORTED;
+    const bool tc5 = max_len >= kTcQ && n_layers <= kTcMaxLayers;      // sequences that fill a 128-query tile
+    if (!tc5 && max_len > kFullMaxLen) return SAN_ERR_UNSUPPORTED;      // the mma.sync kernel keeps a row of scores per query on chip
     if (d_S && ld_s < max_len) return SAN_ERR_SHAPE;
     if (n_seq == 0) return SAN_OK;
     FullParams p;
@@ -761,8 +762,8 @@ int32_t san_full_block(int32_t dtype, int32_t n_heads, int32_t n_layers, int32_t
         return true;
     };
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (max_len >= kTcQ && n_layers <= kTcMaxLayers) {
-        // sequences that fill a 128-query tile: tcgen05 path, accumulators in tensor memory
+    if (tc5) {
+        // tcgen05 path, accumulators in tensor memory; keys stream in chunks, so any length goes
         static size_t set_tc5[64] = {};
         const size_t smem = full_tc5_smem_bytes();
         if (!opt_in((const void*)full_block_tc5_kernel, smem, set_tc5)) return SAN_ERR_CUDA;

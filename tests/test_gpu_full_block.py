@@ -90,7 +90,7 @@ def test_argument_checks():
     f = B.san_full_block
     assert f(B.SAN_BF16, 1, 1, 0, None, t, t, l, 1, 1, 0, None, 0, t) == B.SAN_ERR_NULL
     assert f(B.SAN_F32, 1, 1, 0, t, t, t, l, 1, 1, 0, None, 0, t) == B.SAN_ERR_UNSUPPORTED
-    assert f(B.SAN_BF16, 1, 1, 0, t, t, t, l, 1, 1024, 0, None, 0, t) == B.SAN_ERR_UNSUPPORTED
+    assert f(B.SAN_BF16, 1, 7, 0, t, t, t, l, 1, 1024, 0, None, 0, t) == B.SAN_ERR_UNSUPPORTED   # 7 layers: mma.sync kernel, 512 at most
     assert f(B.SAN_BF16, 1, 1, 0, t, t, t, l, 1, 1, 2, None, 0, t) == B.SAN_ERR_SHAPE
     assert f(B.SAN_BF16, 1, 1, 0, t, t, t, l, 0, 1, 0, None, 0, t) == B.SAN_OK
 
@@ -101,6 +101,11 @@ def test_tensor_memory_path_ragged_lengths(causal):
     tensor memory): lengths on both sides of the 64-key chunk and the 128-query tile, an empty
     and a one-token sequence in the same batch."""
     _run([1, 63, 64, 65, 127, 128, 129, 200, 0], cap=200, H=2, n_layers=3, causal=causal)
+
+
+def test_tensor_memory_path_beyond_512_positions():
+    """The tcgen05 kernel streams the keys in chunks and has no length limit of its own."""
+    _run([700, 513], cap=704, H=1, n_layers=2, causal=True)
 
 
 def test_tensor_memory_path_one_and_six_layers():
