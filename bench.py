@@ -377,7 +377,8 @@ def time_js_matrix(w, dec, sb, pos, device, reps=50):
     nbytes = M * w.n_heads * int((pos.astype(np.int64) + 1).sum()) * 4
     return {"call": "san_js_matrix", "layers": M, "us_per_call": secs * 1e6, "bytes_per_call": nbytes,
             "achieved_gbs": nbytes / secs / 1e9,
-            "note": "three launches (clear, pairs, finish) over weights that fit in L2: launch-bound, not a roofline case"}
+            "note": "three launches (clear, pairs, finish) over weights that fit in L2; M(M-1)/2 pairs with two "
+                    "logarithms per position: launch-bound for few layers, logarithm-bound for many, never HBM-bound"}
 
 
 def time_full_block(w, device, peak, reps=5):
