@@ -12,7 +12,14 @@
  * (Eq. 3-4).  Hence only block-first layers keep a key cache (Section 3.2, memory note).
  *
  * General rules
- *  - Every function returns a status (SAN_OK = 0).  Nothing throws, traps or waits.
+ *  - Every function returns a status (SAN_OK = 0).  Nothing throws or traps, and no kernel
+ *    waits on another kernel, CTA or rank.  The only device-side waits are a CTA's waits for
+ *    its OWN asynchronous copies or tensor-core operations (mbarrier waits in the kernels
+ *    behind san_decode_step and san_full_block); each gives up after about a second, makes
+ *    the kernel stop early.  san_decode_step reports it as SAN_ERR_TIMEOUT through
+ *    san_device_status, which then also clears the context's split-row tickets so that later
+ *    steps start clean; san_full_block has no status word, and a tile whose wait ran out
+ *    leaves its output rows unwritten.
  *  - All `d_` pointers are DEVICE pointers owned by the caller; all others are HOST
  *    pointers.  The library allocates no device memory: the cache arena and the
  *    workspace are caller buffers handed to san_create.
@@ -64,7 +71,7 @@ enum {
     SAN_ERR_RANGE = 6,        /* layer/block/position outside what the policy or config allows */
     SAN_ERR_CUDA = 7,         /* a CUDA runtime call failed (launch configuration, bad stream...) */
     SAN_ERR_DEVICE_CHECK = 8, /* a kernel met an invalid id/length/position and skipped the item */
-    SAN_ERR_TIMEOUT = 9,      /* reserved for bounded device waits (the library has none) */
+    SAN_ERR_TIMEOUT = 9,      /* a kernel's bounded wait for its own copies ran out (see General rules) */
     SAN_ERR_UNSUPPORTED = 10
 };
 enum { SAN_F32 = 0, SAN_BF16 = 1 };
@@ -168,6 +175,15 @@ int32_t san_attn_apply(san_ctx* ctx, int32_t kind, int32_t block, int32_t layer_
 int32_t san_aan_step(san_ctx* ctx, int32_t layer_begin, int32_t layer_end, const void* d_x,
                      const int32_t* d_ids, const int32_t* d_t, int32_t n_items, void* d_out,
                      void* stream);
+
+/* Forget the history of the listed sequences under average attention (Table 6 pairing): the
+ * running sums of every layer are set to zero for each sequence d_seq_ids[i], i < n, so that
+ * a cache slot can be handed to another hypothesis or sentence at any point of its count.
+ * After the call the next san_aan_step at position t returns x / t for such a sequence, as
+ * if its earlier inputs had been zero; restarting the count at t = 1 needs no reset (that
+ * step overwrites the sum).  Only for contexts with self_is_aan (else SAN_ERR_UNSUPPORTED).
+ * An id outside 0 .. max_sent*beam-1 is skipped and reported through san_device_status. */
+int32_t san_seq_reset(san_ctx* ctx, const int32_t* d_seq_ids, int32_t n, void* stream);
 
 /* One whole decode step in ONE launch: for every block of both attention kinds, append
  * this step's rows (Section 4.1 cache), compute the block's weights at its lowest layer

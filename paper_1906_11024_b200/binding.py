@@ -27,7 +27,7 @@ SAN_MAX_LAYERS, SAN_MAX_BEAM = 64, 8
 EXPORTS = (
     "san_query_bytes", "san_create", "san_destroy",
     "san_policy_set_sizes", "san_policy_set_map", "san_policy_get_map",
-    "san_cache_append", "san_attn_weights", "san_attn_apply", "san_aan_step",
+    "san_cache_append", "san_attn_weights", "san_attn_apply", "san_aan_step", "san_seq_reset",
     "san_device_status", "san_status_string", "san_attn_weights_static", "san_decode_step",
     "san_decode_step_host", "san_full_block", "san_beam_reorder", "san_js_matrix", "san_block_similarity", "san_policy_search",
 )
@@ -81,6 +81,7 @@ def lib():
     L.san_attn_weights.argtypes = [vp, i32, i32, vp, vp, vp, i32, i32, vp, i64, vp]
     L.san_attn_apply.argtypes = [vp, i32, i32, i32, i32, vp, i64, vp, vp, vp, i32, i32, vp, i32, vp]
     L.san_aan_step.argtypes = [vp, i32, i32, vp, vp, vp, i32, vp, vp]
+    L.san_seq_reset.argtypes = [vp, vp, i32, vp]
     L.san_device_status.argtypes = [vp, _I32P, _I32P, vp]
     L.san_attn_weights_static.argtypes = [i32, i32, i32, vp, vp, i32, i32, vp, vp, i32, i32, vp, i64, vp, vp]
     L.san_decode_step.argtypes = [vp, C.POINTER(san_step_args), vp]
@@ -191,6 +192,11 @@ def san_attn_apply(ctx, kind, block, layer_begin, layer_end, d_S, ld_s, d_ids, d
 def san_aan_step(ctx, layer_begin, layer_end, d_x, d_ids, d_t, n_items, d_out, stream=None) -> int:
     return lib().san_aan_step(ctx, layer_begin, layer_end, _ptr(d_x), _ptr(d_ids), _ptr(d_t), n_items,
                               _ptr(d_out), _stream(stream))
+
+
+def san_seq_reset(ctx, d_seq_ids, n, stream=None) -> int:
+    """Zero the running sums of the listed sequences in every layer (average attention only)."""
+    return lib().san_seq_reset(ctx, _ptr(d_seq_ids), n, _stream(stream))
 
 
 def san_device_status(ctx, stream=None):

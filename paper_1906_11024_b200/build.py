@@ -9,14 +9,19 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsan_b200.so")
 SOURCES = ["san_api.cu", "san_static.cu", "san_policy.cpp"]
-HEADERS = ["san_kernels.cuh", "san_fused.cuh", "san_ctx.h", "san_policy.h", os.path.join("..", "..", "include", "san.h")]
+
+
+def _inputs():
+    """Everything the library is compiled from: every file under csrc/ and the public header."""
+    files = [os.path.join(CSRC, f) for f in sorted(os.listdir(CSRC)) if f.endswith((".cu", ".cuh", ".cpp", ".h"))]
+    return files + [os.path.join(HERE, "..", "include", "san.h")]
 
 
 def _stale() -> bool:
     if not os.path.exists(LIB):
         return True
     t = os.path.getmtime(LIB)
-    return any(os.path.getmtime(os.path.join(CSRC, f)) > t for f in SOURCES + HEADERS)
+    return any(os.path.getmtime(f) > t for f in _inputs())
 
 
 def build(force: bool = False, verbose: bool = False) -> str:

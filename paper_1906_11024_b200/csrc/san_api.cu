@@ -420,6 +420,23 @@ int32_t san_aan_step(san_ctx* ctx, int32_t layer_begin, int32_t layer_end, const
     return cuda_status(cudaGetLastError());
 }
 
+int32_t san_seq_reset(san_ctx* ctx, const int32_t* d_seq_ids, int32_t n, void* stream) {
+    if (!ctx || (n > 0 && !d_seq_ids)) return SAN_ERR_NULL;
+    const san_config& c = ctx->cfg;
+    if (!c.self_is_aan) return SAN_ERR_UNSUPPORTED;
+    if (n < 0 || n > ctx->n_seqs) return SAN_ERR_SHAPE;
+    if (n == 0) return SAN_OK;
+    ResetParams p;
+    p.sum = reinterpret_cast<float*>(ctx->cache + ctx->off_aan);
+    p.ids = d_seq_ids; p.n_items = n; p.d = c.n_heads * kDh; p.max_ids = ctx->n_seqs; p.n_layers = c.n_layers;
+    p.err = ctx->err;
+    const long long units = (long long)p.n_layers * n * (p.d / 4);
+    const long long grid = (units + 255) / 256;
+    if (grid > 0x7fffffffLL) return SAN_ERR_SHAPE;
+    aan_reset_kernel<<<(unsigned)grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(p);
+    return cuda_status(cudaGetLastError());
+}
+
 int32_t san_decode_step(san_ctx* ctx, const san_step_args* a, void* stream) {
     if (!ctx || !a) return SAN_ERR_NULL;
     const san_config& c = ctx->cfg;
@@ -530,8 +547,11 @@ int32_t san_decode_step(san_ctx* ctx, const san_step_args* a, void* stream) {
         }
         span_self = plan->span_self; lg_self = plan->lg_self; span_enc = plan->span_enc; lg_enc = plan->lg_enc;
     }
-    while (ceil_div(max_len, span_self) > kMaxSpans) span_self = std::min(kZFloats, span_self * 2);
-    while (ceil_div(max_src, span_enc) > kMaxSpans) span_enc = std::min(kZFloats / nqe, span_enc * 2);
+    // a row may be cut into at most kMaxSpans spans of at most what the score buffer holds
+    if (do_self && ceil_div(max_len, kZFloats) > kMaxSpans) return SAN_ERR_UNSUPPORTED;
+    if (do_enc && ceil_div(max_src, kZFloats / nqe) > kMaxSpans) return SAN_ERR_UNSUPPORTED;
+    while (do_self && ceil_div(max_len, span_self) > kMaxSpans && span_self < kZFloats) span_self = std::min(kZFloats, span_self * 2);
+    while (do_enc && ceil_div(max_src, span_enc) > kMaxSpans && span_enc < kZFloats / nqe) span_enc = std::min(kZFloats / nqe, span_enc * 2);
     const int nlg_self = ceil_div(pi_self, lg_self), nlg_enc = ceil_div(pi_enc, lg_enc);
     const long long rl_self = rows_self * nlg_self, rl_enc = rows_enc * nlg_enc;      // (row, layer group) pairs
     if ((size_t)(rl_self + rl_enc) > ctx->n_tickets) return SAN_ERR_CAPACITY;
@@ -824,7 +844,10 @@ int32_t san_device_status(san_ctx* ctx, int32_t* first_error, int32_t* detail, v
     cudaError_t e = cudaMemcpyAsync(words, ctx->err, sizeof(words), cudaMemcpyDeviceToHost, st);
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);
     if (e == cudaSuccess && words[0] != 0) {
-        e = cudaMemsetAsync(ctx->err, 0, sizeof(words), st);
+        // A step that stopped early (a wait ran out) may have left tickets of split rows part-way:
+        // clear them with the error words, or later rows would never see their last span arrive.
+        const size_t clear = words[0] == SAN_ERR_TIMEOUT ? ctx->ws_off_part : sizeof(words);
+        e = cudaMemsetAsync(ctx->err, 0, clear, st);
         if (e == cudaSuccess) e = cudaStreamSynchronize(st);
     }
     if (e != cudaSuccess) return SAN_ERR_CUDA;

@@ -23,7 +23,7 @@ constexpr int kDh = 64;          // d_head
 constexpr int kWarpsPerCta = 8;  // warps are independent; a CTA is only a scheduling unit
 constexpr int kSub = 128;        // cache positions staged on chip per pass of a warp
 
-enum KernelTag { TAG_APPEND = 1, TAG_WEIGHTS = 2, TAG_APPLY = 3, TAG_AAN = 4, TAG_REORDER = 5 };
+enum KernelTag { TAG_APPEND = 1, TAG_WEIGHTS = 2, TAG_APPLY = 3, TAG_AAN = 4, TAG_REORDER = 5, TAG_RESET = 7 };
 
 // Device error word: [0]=status, [1]=kernel tag, [2]=item, [3]=offending value, [4]=limit.
 __device__ __forceinline__ void record_error(int* err, int tag, int item, int value, int limit) {
@@ -489,6 +489,26 @@ __global__ void __launch_bounds__(256) aan_kernel(const AanParams p) {
     } else {
         *reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + io) = make_float4(o0, o1, o2, o3);
     }
+}
+
+// Zeroes the running sums of the listed sequences in every layer: one thread per 16 bytes.
+struct ResetParams {
+    float* sum;                    // [layer][max_ids][d]
+    const int* ids;
+    int n_items, d, max_ids, n_layers;
+    int* err;
+};
+
+static __global__ void __launch_bounds__(256) aan_reset_kernel(const ResetParams p) {
+    const int d4 = p.d >> 2;
+    long long u = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (u >= (long long)p.n_layers * p.n_items * d4) return;
+    const int c4 = (int)(u % d4); u /= d4;
+    const int item = (int)(u % p.n_items);
+    const int layer = (int)(u / p.n_items);
+    const int id = p.ids[item];
+    if (id < 0 || id >= p.max_ids) { if (c4 == 0 && layer == 0) record_error(p.err, TAG_RESET, item, id, p.max_ids); return; }
+    reinterpret_cast<float4*>(p.sum + ((long long)layer * p.max_ids + id) * p.d)[c4] = make_float4(0.f, 0.f, 0.f, 0.f);
 }
 
 }  // namespace san

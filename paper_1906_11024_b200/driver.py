@@ -22,14 +22,6 @@ from . import binding as B
 from . import synth
 
 
-def _first_layers(sizes) -> List[int]:
-    out, l = [], 0
-    for s in sizes:
-        out.append(l)
-        l += int(s)
-    return out
-
-
 def to_device(x_f32: np.ndarray, dtype: str, device) -> torch.Tensor:
     """float32 host values (already rounded to ``dtype``) -> device tensor of that dtype."""
     if dtype == synth.BF16:
@@ -79,8 +71,6 @@ class Decoder:
             self_is_aan=int(w.self_is_aan), encdec_shared_context=int(self.shared_ctx))
         self.self_sizes = list(w.self_blocks)
         self.enc_sizes = list(w.encdec_blocks)
-        self.self_first = _first_layers(self.self_sizes)
-        self.enc_first = _first_layers(self.enc_sizes)
         rc, cb, wb = B.san_query_bytes(self.cfg, len(self.self_sizes), len(self.enc_sizes))
         B.check(rc, "san_query_bytes")
         self.cache_bytes, self.ws_bytes = cb, wb
@@ -89,6 +79,11 @@ class Decoder:
             self.ws = torch.empty(wb, dtype=torch.uint8, device=self.device)
             rc, self.ctx = B.san_create(self.cfg, self.self_sizes, self.enc_sizes, self.cache, cb, self.ws, wb)
         B.check(rc, "san_create")
+        # the lowest layer of every block, as the library's own policy tables have it
+        rc, _, self.self_first = B.san_policy_get_map(self.ctx, B.SAN_SELF)
+        B.check(rc, "san_policy_get_map")
+        rc, _, self.enc_first = B.san_policy_get_map(self.ctx, B.SAN_ENCDEC)
+        B.check(rc, "san_policy_get_map")
         self.ld_t = (w.max_tgt_len() + 3) // 4 * 4
         self.ld_s = (w.max_src_len() + 3) // 4 * 4
 

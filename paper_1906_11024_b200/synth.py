@@ -127,14 +127,6 @@ class Workload:
         return (u % t.astype(np.int64)).astype(np.int32)      # uniform in [0, T_s)
 
 
-def block_map(sizes) -> List[int]:
-    """Layer -> block id for block sizes listed bottom-up (bookkeeping for callers/tests)."""
-    out: List[int] = []
-    for b, s in enumerate(sizes):
-        out += [b] * int(s)
-    return out
-
-
 WORKLOADS: Dict[str, Workload] = {
     # the five configurations, in order
     "tiny": Workload("tiny", F32, 6, 8, 64, 1, 4, (2, 2, 2), (3, 3), 16, 16, "fixed", 16, False, False, 0),

@@ -1,8 +1,8 @@
 """Parity of the one-launch decode step on rows of one length: every sequence sits at the same
 cache length (or every sentence has the same source length), for lengths on both sides of the
 tile boundaries (24 key rows beside the queries in an item's first tile, 32 rows per tile) and
-for blocks of 1, 2, 3 and 6 layers.  Also the shapes that the instruction counts in
-profiles/decode_step_instruction_costs.md were taken on."""
+for blocks of 1, 2, 3 and 6 layers.  One launch per test over rows of one shape, which also
+makes these the cases to count a kernel's instructions per row on."""
 import numpy as np
 import pytest
 import torch

@@ -315,6 +315,35 @@ def test_beam_reorder_is_a_gather_of_cached_rows():
             np.testing.assert_allclose(O[s], ref[:, 0].numpy(), rtol=1e-12, atol=1e-13)
 
 
+def test_beam_reorder_carries_the_running_average_of_the_parent():
+    """With average attention a hypothesis continues the prefix mean of the hypothesis it
+    extends: after a reorder, the next step's output is the mean of the PARENT's inputs at
+    positions 1..len plus the new input, written out here with cumsum/arange over the gathered
+    parent rows.  Parents differ per beam and one hypothesis keeps a shorter prefix."""
+    rng = np.random.default_rng(22)
+    M, n_sent, beam, H, dh, T = 2, 2, 3, 2, 64, 7
+    n, d = n_sent * beam, H * dh
+    o = so.Oracle(M, H, dh, n_sent, beam, T, 4, [1, 1], [2])
+    hist = 5
+    X = rng.standard_normal((M, hist, n, d)).astype(np.float32)
+    ids = np.arange(n)
+    for l in range(M):
+        for t in range(hist):
+            o.aan_step(l, ids, np.full(n, t + 1), X[l, t])
+    src = np.array([1, 2, 0, 5, 3, 3])            # every beam changes parent, two share one
+    lens = np.array([5, 5, 3, 5, 5, 5])           # sequence 2 keeps only 3 positions of its parent
+    o.beam_reorder(src, lens)
+    x_new = rng.standard_normal((M, n, d)).astype(np.float32)
+    for l in range(M):
+        got = o.aan_step(l, ids, lens + 1, x_new[l])
+        for s in range(n):
+            L = int(lens[s])
+            rows = np.concatenate([X[l, :L, src[s]], x_new[l, s][None]], 0).astype(np.float64)
+            ref = (np.cumsum(rows, 0) / np.arange(1, L + 2)[:, None])[-1]
+            np.testing.assert_allclose(got[s], ref, rtol=0, atol=1e-14)
+            assert np.abs(got[s] - (X[l, :L, s].astype(np.float64).sum(0) + x_new[l, s]) / (L + 1)).max() > 1e-3
+
+
 @pytest.mark.parametrize("causal", [False, True])
 def test_full_sequence_block_matches_library_attention(causal):
     """Encoder-side SAN (Table 5): S is l x l, computed once, applied to each layer's V."""
