@@ -219,6 +219,20 @@ typedef struct {
 } san_step_args;
 int32_t san_decode_step(san_ctx* ctx, const san_step_args* args, void* stream);
 
+/* Which kernel san_decode_step launches, and (for testing and tuning) how its rows are cut.
+ * The library has two implementations of the one-launch step (same arithmetic, Eq. 1-5):
+ *   which = 1  per-warp pipeline: every warp streams the tiles of its own row (float32 and bf16);
+ *   which = 2  team pipeline (bf16): four producer warps each stream bundles of four rows or row
+ *              spans to a team of four warps; SAN_ERR_UNSUPPORTED from the step if a shape does not fit;
+ *   which = 0  automatic (the default): the team pipeline where it applies, else the per-warp one.
+ * spans_log2 >= 0 overrides the automatic cut of the team pipeline: every row is dealt to
+ * 1 << spans_log2 warps (0..2), tiles hold tile_pos positions (a multiple of 16),
+ * layers_per_unit > 0 caps the layers one warp applies (the block's other layers go to
+ * further warps, which recompute S), grab_mult >= 1 makes the bundles shrink earlier towards
+ * the end of the launch.  spans_log2 < 0 restores the automatic cut. */
+int32_t san_step_kernel_select(san_ctx* ctx, int32_t which, int32_t spans_log2, int32_t tile_pos,
+                               int32_t layers_per_unit, int32_t grab_mult);
+
 /* san_decode_step for a caller whose step inputs and outputs live in HOST memory (pinned
  * memory if the copies are to overlap anything): the same step (Eq. 1-5, Section 4.1) with
  * the transfers issued by the library on `stream`, in order: every input array named in

@@ -29,7 +29,7 @@ EXPORTS = (
     "san_policy_set_sizes", "san_policy_set_map", "san_policy_get_map",
     "san_cache_append", "san_attn_weights", "san_attn_apply", "san_aan_step", "san_seq_reset",
     "san_device_status", "san_status_string", "san_attn_weights_static", "san_decode_step",
-    "san_decode_step_host", "san_full_block", "san_beam_reorder", "san_js_matrix", "san_block_similarity", "san_policy_search",
+    "san_decode_step_host", "san_step_kernel_select", "san_full_block", "san_beam_reorder", "san_js_matrix", "san_block_similarity", "san_policy_search",
 )
 
 
@@ -85,6 +85,7 @@ def lib():
     L.san_device_status.argtypes = [vp, _I32P, _I32P, vp]
     L.san_attn_weights_static.argtypes = [i32, i32, i32, vp, vp, i32, i32, vp, vp, i32, i32, vp, i64, vp, vp]
     L.san_decode_step.argtypes = [vp, C.POINTER(san_step_args), vp]
+    L.san_step_kernel_select.argtypes = [vp, i32, i32, i32, i32, i32]
     L.san_decode_step_host.argtypes = [vp, C.POINTER(san_step_args), C.POINTER(san_step_args), vp]
     L.san_full_block.argtypes = [i32, i32, i32, i32, vp, vp, vp, vp, i32, i32, i32, vp, i64, vp, vp]
     L.san_beam_reorder.argtypes = [vp, vp, vp, vp, i32, i32, vp]
@@ -225,6 +226,11 @@ def san_decode_step(ctx, *, d_q_self=None, d_k_new=None, d_v_new=None, d_seq_ids
                       _ptr(d_S_self), ld_t, _ptr(d_O_self), _ptr(d_q_enc), _ptr(d_sent_ids), _ptr(d_src_lens),
                       n_sent, max_src, _ptr(d_S_enc), ld_s, _ptr(d_O_enc), _ptr(d_x_aan), _ptr(d_t))
     return lib().san_decode_step(ctx, C.byref(a), _stream(stream))
+
+
+def san_step_kernel_select(ctx, which=0, spans_log2=-1, tile_pos=64, layers_per_unit=0, grab_mult=1) -> int:
+    """Choose the kernel behind san_decode_step (0 automatic, 1 per-warp, 2 team pipeline) and its cut."""
+    return lib().san_step_kernel_select(ctx, which, spans_log2, tile_pos, layers_per_unit, grab_mult)
 
 
 def san_beam_reorder(ctx, d_sent_ids, d_parent, d_lens, n_sent, max_len=0, stream=None) -> int:

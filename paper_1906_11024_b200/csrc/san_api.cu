@@ -12,6 +12,7 @@
 #include "san_ctx.h"
 #include "san_kernels.cuh"
 #include "san_fused.cuh"
+#include "san_step.cuh"
 #include "san_reorder.cuh"
 #include "san_learn.cuh"
 #include "san_full.cuh"
@@ -158,6 +159,168 @@ cudaError_t launch_apply(const ApplyParams& p, int nq_t, unsigned grid, cudaStre
         default: apply_kernel<T, 8><<<grid, block, 0, st>>>(p); break;
     }
     return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// The team-pipeline step kernel (san_step.cuh): how the rows are cut into units and how its
+// shared memory is laid out.  Returns SAN_ERR_UNSUPPORTED when the shape does not fit (the
+// caller then uses the per-warp kernel).
+constexpr size_t kStepSmemTotal = 232448;      // opt-in shared memory per CTA on sm_100
+
+struct TeamCut { int spr_log2, lg, tile_pos, zq; };
+
+int32_t launch_team_step(san_ctx* ctx, const san_step_args* a, int max_len, int max_src, cudaStream_t st) {
+    const san_config& c = ctx->cfg;
+    if (c.dtype != SAN_BF16) return SAN_ERR_UNSUPPORTED;
+    const bool aan = c.self_is_aan != 0;
+    const int n_seqs = a->n_seqs, n_sent = a->n_sent;
+    const bool do_self = n_seqs > 0 && !aan, do_enc = n_sent > 0, do_aan = aan && n_seqs > 0;
+    const int nqe = pick_nq_template(c.beam);
+    const int H = c.n_heads;
+    int pi_self = 1, pi_enc = 1;
+    for (int b = 0; b < ctx->self_pol.n_blocks; ++b) pi_self = std::max(pi_self, ctx->self_pol.size_of_block[b]);
+    for (int b = 0; b < ctx->enc_pol.n_blocks; ++b) pi_enc = std::max(pi_enc, ctx->enc_pol.size_of_block[b]);
+    if (c.encdec_shared_context) pi_enc = 1;
+    const long long rows_self = do_self ? (long long)ctx->self_pol.n_blocks * n_seqs * H : 0;
+    const long long rows_enc = do_enc ? (long long)ctx->enc_pol.n_blocks * n_sent * H : 0;
+    if (rows_self + rows_enc >= (1ll << 27)) return SAN_ERR_UNSUPPORTED;
+
+    // Units wanted: a few per consumer warp of the grid, so that the warps stay busy and the SMs
+    // finish together.  Long rows are cut into spans first (nothing is read twice), then a block's
+    // layers into groups (each group reads the block's keys again, mostly from L2).
+    constexpr int kZCapFloats = 1024;              // score slots a warp may hold
+    constexpr int kMaxSprLog2 = 2;                 // a row's spans are neighbouring warps of one team
+    const long long want_units = 3ll * ctx->sm_count * kStepConsumers;
+    auto span_of = [](int bound, int spr_log2) { return (int)align_up((size_t)ceil_div(bound, 1 << spr_log2), 16); };
+    auto cut = [&](long long rows, int bound, int pi, int nq_t, TeamCut* out) -> bool {
+        int s = 0, lg = pi;
+        while (s < kMaxSprLog2 && span_of(bound, s) * nq_t > kZCapFloats) ++s;
+        if (span_of(bound, s) * nq_t > kZCapFloats) return false;
+        while (s < kMaxSprLog2 && span_of(bound, s) > 64 && rows * (1ll << s) * ceil_div(pi, lg) < want_units) ++s;
+        while (lg > 2 && rows * (1ll << s) * ceil_div(pi, lg) < want_units &&
+               (long long)span_of(bound, s) * 128 * (1 + lg) > 48 * 1024) lg = std::max(2, ceil_div(lg, 2));
+        const int span = span_of(bound, s);
+        out->spr_log2 = s; out->lg = lg;
+        out->tile_pos = span <= 64 ? span : 32;
+        out->zq = span + 4;                         // + 4: the score rows of neighbouring queries start in different banks
+        return true;
+    };
+    TeamCut cs{0, 1, 16, 20}, ce{0, 1, 16, 20};
+    if (do_self && !cut(rows_self, max_len, pi_self, 1, &cs)) return SAN_ERR_UNSUPPORTED;
+    if (do_enc && !cut(rows_enc, max_src, pi_enc, nqe, &ce)) return SAN_ERR_UNSUPPORTED;
+    if (ctx->team_cut_override[0] >= 0) {           // testing and tuning: san_step_kernel_select
+        cs.spr_log2 = ce.spr_log2 = std::min(kMaxSprLog2, ctx->team_cut_override[0]);
+        if (span_of(max_len, cs.spr_log2) > kZCapFloats || span_of(max_src, ce.spr_log2) * nqe > kZCapFloats) return SAN_ERR_UNSUPPORTED;
+        cs.tile_pos = std::min(span_of(max_len, cs.spr_log2), std::max(16, ctx->team_cut_override[1]));
+        ce.tile_pos = std::min(span_of(max_src, ce.spr_log2), std::max(16, ctx->team_cut_override[1]));
+        cs.zq = span_of(max_len, cs.spr_log2) + 4; ce.zq = span_of(max_src, ce.spr_log2) + 4;
+        if (ctx->team_cut_override[2] > 0) { cs.lg = std::min(pi_self, ctx->team_cut_override[2]); ce.lg = std::min(pi_enc, ctx->team_cut_override[2]); }
+    }
+
+    TeamParams p;
+    std::memset(&p, 0, sizeof(p));
+    p.H = H;
+    p.err = ctx->err; p.queue = ctx->err + 16;
+    p.scale_log2e = (float)(1.4426950408889634 / std::sqrt((double)kDh));
+    auto fill = [&](TeamKind& k, const Policy& pol, const TeamCut& tc, int n_it, long long rows, int pi) {
+        k.spr_log2 = (unsigned)tc.spr_log2; k.lg_size = (unsigned)tc.lg; k.tile_pos = (unsigned)tc.tile_pos; k.zq = (unsigned)tc.zq;
+        const int n_lg = ceil_div(pi, tc.lg);
+        k.n_rowlg = (unsigned)(rows * n_lg);
+        k.n_units = (unsigned)align_up((size_t)k.n_rowlg << tc.spr_log2, kTeamWarps);
+        k.div_lg = make_fastdiv((unsigned)n_lg); k.div_rows = make_fastdiv((unsigned)std::max(1, n_it * H)); k.div_h = make_fastdiv((unsigned)H);
+        k.n_it = (unsigned)std::max(n_it, 1);
+        for (int b = 0; b < pol.n_blocks; ++b) {
+            k.first[b] = (unsigned char)pol.first_layer_of_block[b];
+            k.size[b] = (unsigned char)pol.size_of_block[b];
+        }
+    };
+    {   // decoder self-attention
+        TeamKind& k = p.k[0];
+        k.q = static_cast<const char*>(a->d_q_self); k.knew = static_cast<const char*>(a->d_k_new);
+        k.vnew = static_cast<const char*>(a->d_v_new);
+        k.K = ctx->cache + ctx->off_self_k; k.V = ctx->cache + ctx->off_self_v;
+        k.S = a->d_S_self; k.O = static_cast<char*>(a->d_O_self); k.ids = a->d_seq_ids; k.lens = a->d_pos;
+        k.plane_bytes = (long long)ctx->self_plane_bytes;
+        k.layer_bytes = (long long)n_seqs * H * 128;
+        k.S_ld = a->ld_t;
+        k.panel_bytes = (unsigned)c.max_tgt_len * 128u;
+        k.nq = 1; k.len_bias = 1; k.max_ids = (unsigned)ctx->n_seqs; k.bound = (unsigned)max_len;
+        k.q_first = 0; k.q_stride_items = 1; k.v_by_block = 0;
+        fill(k, ctx->self_pol, cs, n_seqs, rows_self, pi_self);
+    }
+    {   // encoder-decoder attention
+        TeamKind& k = p.k[1];
+        k.q = static_cast<const char*>(a->d_q_enc);
+        k.K = ctx->cache + ctx->off_mem_k; k.V = ctx->cache + ctx->off_mem_v;
+        k.S = a->d_S_enc; k.O = static_cast<char*>(a->d_O_enc); k.ids = a->d_sent_ids; k.lens = a->d_src_lens;
+        k.plane_bytes = (long long)ctx->mem_plane_bytes;
+        k.layer_bytes = (long long)n_sent * c.beam * H * 128;
+        k.S_ld = a->ld_s;
+        k.panel_bytes = (unsigned)c.max_src_len * 128u;
+        k.nq = (unsigned)c.beam; k.len_bias = 0; k.max_ids = (unsigned)c.max_sent; k.bound = (unsigned)max_src;
+        k.q_first = 0; k.q_stride_items = (unsigned)c.beam; k.v_by_block = c.encdec_shared_context ? 1 : 0;
+        fill(k, ctx->enc_pol, ce, n_sent, rows_enc, pi_enc);
+    }
+    if (!do_self) p.k[0].n_units = 0;
+    if (!do_enc) p.k[1].n_units = 0;
+    if (do_aan) {
+        const int d = H * kDh;
+        p.x_aan = static_cast<const char*>(a->d_x_aan); p.t_aan = a->d_t; p.aan_ids = a->d_seq_ids;
+        p.aan_sum = reinterpret_cast<float*>(ctx->cache + ctx->off_aan); p.aan_out = static_cast<char*>(a->d_O_self);
+        p.n_aan_layers = c.n_layers; p.n_aan_seqs = n_seqs; p.aan_max_seqs = ctx->n_seqs; p.aan_max_t = c.max_tgt_len;
+        p.aan_chunks_per_row = ceil_div(d, kAanChunk);
+        p.div_aan_chunks = make_fastdiv((unsigned)p.aan_chunks_per_row); p.div_aan_seqs = make_fastdiv((unsigned)n_seqs);
+        p.n_aan_units = (unsigned)align_up((size_t)c.n_layers * n_seqs * p.aan_chunks_per_row, kTeamWarps);
+    }
+    p.n_enc_units = p.k[1].n_units;
+    const long long n_units = (long long)p.n_aan_units + p.n_enc_units + p.k[0].n_units;
+    if (n_units > (1ll << 30)) return SAN_ERR_UNSUPPORTED;
+    p.n_units = (unsigned)n_units;
+    if (p.n_units == 0) return SAN_OK;
+
+    // shared memory: [ring | pad] per team, then per consumer warp its score slots and its scratch rows
+    // (queries, this step's key row and value rows), the exchange area of split rows, descriptors,
+    // barriers, a row of zeros
+    const bool split = (do_self && cs.spr_log2 > 0) || (do_enc && ce.spr_log2 > 0);
+    const int nq_x = std::max(do_self && cs.spr_log2 > 0 ? 1 : 0, do_enc && ce.spr_log2 > 0 ? nqe : 0);
+    const size_t zs_bytes = align_up((size_t)4 * std::max(do_self ? cs.zq : 0, do_enc ? ce.zq * nqe : 0), 16);
+    const size_t scr_bytes = (size_t)128 * std::max(do_self ? 2 + cs.lg : 0, do_enc ? nqe : 0);
+    p.xo_unit_floats = split ? (unsigned)(nq_x * kDh) : 0u;
+    const size_t xo_bytes = (size_t)kTeams * team_xch_bytes(p.xo_unit_floats);
+    const size_t tail = kStepConsumers * (zs_bytes + scr_bytes) + xo_bytes + kTeams * kTeamDescBytes + (kTeams * kTeamBarBytes + 16) + 128 + 256;
+    if (tail + kTeams * (16 * 1024 + kRingPad) > kStepSmemTotal) return SAN_ERR_UNSUPPORTED;
+    p.ring_bytes = (unsigned)(((kStepSmemTotal - tail) / kTeams - kRingPad) / 128 * 128);
+    p.ring_stride = p.ring_bytes + kRingPad;
+    const size_t slot_max = (size_t)kTeamWarps * 128 * std::max(do_self ? cs.tile_pos : 0, do_enc ? ce.tile_pos : 0);
+    if (slot_max > p.ring_bytes) return SAN_ERR_UNSUPPORTED;
+    p.zs_bytes = (unsigned)zs_bytes; p.scr_bytes = (unsigned)scr_bytes;
+    p.off_zs = kTeams * p.ring_stride;
+    p.off_scr = (unsigned)(p.off_zs + kStepConsumers * zs_bytes);
+    p.off_xo = (unsigned)align_up(p.off_scr + kStepConsumers * scr_bytes, 16);
+    p.off_desc = (unsigned)align_up(p.off_xo + xo_bytes, 16);
+    p.off_bars = (unsigned)align_up(p.off_desc + kTeams * kTeamDescBytes, 8);
+    p.off_zero = (unsigned)align_up(p.off_bars + kTeams * kTeamBarBytes + 16, 128);
+    const size_t smem = p.off_zero + 128;
+
+    const long long bundles = ((long long)p.n_units + kTeamWarps - 1) / kTeamWarps;
+    const long long ctas = std::max<long long>(1, std::min<long long>(ctx->sm_count, (bundles + kTeams - 1) / kTeams));
+    p.grab_teams = (unsigned)(ctas * kTeams) * (unsigned)std::max(1, ctx->team_grab_mult);
+
+    const void* fn = nqe == 1 ? (const void*)decode_step_team_kernel<1> : nqe == 2 ? (const void*)decode_step_team_kernel<2>
+                   : nqe == 4 ? (const void*)decode_step_team_kernel<4> : (const void*)decode_step_team_kernel<8>;
+    if (!ctx->team_attr_set) {
+        if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kStepSmemTotal) != cudaSuccess) return SAN_ERR_CUDA;
+        ctx->team_attr_set = true;
+    }
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)ctas); cfg.blockDim = dim3(kStepWarps * 32);
+    cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cfg.attrs = &attr; cfg.numAttrs = 1;
+    void* args[] = {&p};
+    return cuda_status(cudaLaunchKernelExC(&cfg, fn, args));
 }
 
 }  // namespace
@@ -456,6 +619,11 @@ int32_t san_decode_step(san_ctx* ctx, const san_step_args* a, void* stream) {
     if (n_seqs == 0 && n_sent == 0) return SAN_OK;
 
     const bool bf16 = c.dtype == SAN_BF16;
+    if (ctx->step_kernel != 1) {       // the team-pipeline kernel takes every bf16 shape that fits its shared memory
+        const int32_t rc = launch_team_step(ctx, a, max_len, max_src, static_cast<cudaStream_t>(stream));
+        if (rc != SAN_ERR_UNSUPPORTED) return rc;
+        if (ctx->step_kernel == 2) return rc;
+    }
     const int row_bytes = kDh * ctx->elem_bytes;
     const int TR = kStageBytes / row_bytes;
     const int nqe = pick_nq_template(c.beam);
@@ -652,6 +820,18 @@ int32_t san_decode_step(san_ctx* ctx, const san_step_args* a, void* stream) {
     void* args[] = {&p};
     cudaError_t e = cudaLaunchKernelExC(&cfg, fn, args);
     return cuda_status(e);
+}
+
+int32_t san_step_kernel_select(san_ctx* ctx, int32_t which, int32_t spans_log2, int32_t tile_pos, int32_t layers_per_unit,
+                               int32_t grab_mult) {
+    if (!ctx) return SAN_ERR_NULL;
+    if (which < 0 || which > 2 || spans_log2 > 2 || (spans_log2 >= 0 && (tile_pos < 16 || tile_pos % 16 != 0))) return SAN_ERR_RANGE;
+    ctx->step_kernel = which;
+    ctx->team_cut_override[0] = spans_log2 < 0 ? -1 : spans_log2;
+    ctx->team_cut_override[1] = tile_pos;
+    ctx->team_cut_override[2] = layers_per_unit;
+    ctx->team_grab_mult = grab_mult > 0 ? grab_mult : 1;
+    return SAN_OK;
 }
 
 int32_t san_decode_step_host(san_ctx* ctx, const san_step_args* h, const san_step_args* d, void* stream) {

@@ -28,6 +28,10 @@ struct san_ctx {
     int* tickets = nullptr;
     float* part = nullptr;
     bool fused_attr_set = false;   // shared-memory opt-in of the one-launch step kernel done
+    bool team_attr_set = false;    // the same for the team-pipeline step kernel
+    int step_kernel = 0;           // 0: automatic, 1: per-warp pipeline kernel, 2: team-pipeline kernel (san_step_kernel_select)
+    int team_cut_override[3] = {-1, 64, 0};   // spans per row (log2; -1: automatic), positions per tile, layers per unit (0: automatic)
+    int team_grab_mult = 1;
 
     // How the one-launch step cuts long rows (positions per item, layers per item), remembered
     // per launch shape: the search that balances the items over the warps costs more than a
