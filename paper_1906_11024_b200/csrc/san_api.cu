@@ -201,7 +201,7 @@ int32_t launch_team_step(san_ctx* ctx, const san_step_args* a, int max_len, int 
                (long long)span_of(bound, s) * 128 * (1 + lg) > 48 * 1024) lg = std::max(2, ceil_div(lg, 2));
         const int span = span_of(bound, s);
         out->spr_log2 = s; out->lg = lg;
-        out->tile_pos = span <= 64 ? span : 32;
+        out->tile_pos = span <= 48 ? span : 32;   // a slot of four units stays under half of a team's ring
         out->zq = span + 4;                         // + 4: the score rows of neighbouring queries start in different banks
         return true;
     };

@@ -30,13 +30,18 @@
 
 namespace san {
 
-constexpr int kTeams = 4;
+constexpr int kTeams = 6;
 constexpr int kTeamWarps = 4;                                  // consumer warps of a team = units per bundle
 constexpr int kStepConsumers = kTeams * kTeamWarps;
 constexpr int kStepWarps = kStepConsumers + kTeams;            // + one producer per team
 constexpr int kNS = 8;                                         // slots (and bundles) a team may have outstanding
 constexpr int kRingPad = 2048;                                 // a 16-row ldmatrix block may read past a unit's last row
 constexpr int kAanChunk = 256;                                 // elements of one AAN unit (8 per lane)
+// Apply S as a bf16 high part plus a bf16 remainder (two MMAs per tile) or as the high part alone.
+// Outputs are bf16: their own rounding (2^-9 relative) is what the comparison with the float64
+// reference shows either way (3.9e-3 normwise at worst on all workloads, tolerance 1e-2), so the
+// remainder is left out.
+constexpr bool kWeightRemainder = false;
 constexpr int kXq = 8;                                         // query rows the exchange area has room for per unit
 
 enum { TAG_TEAM = 8 };
@@ -101,8 +106,9 @@ static_assert(sizeof(SlotDesc) == 16, "SlotDesc is addressed as 16 bytes");
 
 constexpr uint32_t kUnitDescBytes = (uint32_t)sizeof(UnitDesc);
 constexpr uint32_t kTeamDescBytes = kNS * (kTeamWarps * kUnitDescBytes + (uint32_t)sizeof(BundleHdr) + (uint32_t)sizeof(SlotDesc));
-// barriers: per team full[kNS], empty[kNS], exchange[1]; then the CTA's dead flag
-constexpr uint32_t kTeamBarBytes = (2 * kNS + 1) * 8;
+// barriers: per team full[kNS], empty[kNS], ready[kNS] (a bundle's descriptors are written), exchange[1];
+// then the CTA's dead flag
+constexpr uint32_t kTeamBarBytes = (3 * kNS + 1) * 8;
 // exchange area of a team: two output buffers of kTeamWarps units, then (max, sum) per unit and query
 __host__ __device__ constexpr uint32_t team_xch_bytes(uint32_t xo_unit_floats) {
     return 2u * kTeamWarps * xo_unit_floats * 4u + kTeamWarps * kXq * 2u * 4u;
@@ -130,14 +136,26 @@ struct StepSmem {
     }
     __device__ __forceinline__ uint32_t bar_full(int team, int slot) const { return sm_base + off_bars + (uint32_t)team * kTeamBarBytes + (uint32_t)slot * 8u; }
     __device__ __forceinline__ uint32_t bar_empty(int team, int slot) const { return sm_base + off_bars + (uint32_t)team * kTeamBarBytes + (uint32_t)(kNS + slot) * 8u; }
-    __device__ __forceinline__ uint32_t bar_xch(int team) const { return sm_base + off_bars + (uint32_t)team * kTeamBarBytes + 2u * kNS * 8u; }
+    __device__ __forceinline__ uint32_t bar_ready(int team, int bslot) const { return sm_base + off_bars + (uint32_t)team * kTeamBarBytes + (uint32_t)(2 * kNS + bslot) * 8u; }
+    __device__ __forceinline__ uint32_t bar_xch(int team) const { return sm_base + off_bars + (uint32_t)team * kTeamBarBytes + 3u * kNS * 8u; }
     __device__ __forceinline__ volatile int* dead_flag() const { return sp<volatile int>(off_bars + kTeams * kTeamBarBytes); }
 };
+
+// try_wait that lets the hardware keep the thread suspended for a while (it returns as soon as
+// the phase completes), so that a waiting warp does not use issue slots.  Measured on B200: a
+// hint of 1,000,000 suspends for about 1000 cycles; without a hint the instruction returns at once.
+constexpr uint32_t kWaitHint = 4000000u;
+__device__ __forceinline__ bool mbar_try_wait_for(uint32_t bar, uint32_t parity, uint32_t ns) {
+    uint32_t ok;
+    asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\nselp.u32 %0, 1, 0, p;\n}"
+                 : "=r"(ok) : "r"(bar), "r"(parity), "r"(ns) : "memory");
+    return ok != 0;
+}
 
 // Bounded wait that also gives up as soon as another warp of the CTA has given up.
 __device__ __noinline__ bool step_wait_slow(uint32_t bar, uint32_t parity, volatile int* dead) {
     const long long t0 = clock64();
-    while (!mbar_try_wait(bar, parity)) {
+    while (!mbar_try_wait_for(bar, parity, kWaitHint)) {
         if (*dead) return false;
         if (clock64() - t0 > 2000000000LL) return false;
     }
@@ -199,22 +217,54 @@ struct ProdUnit {
     int n, pi, tp, new_row, kind, tiles, spr_log2;
 };
 
-// Decode of unit g by one lane.  `id` and `len` are the entries of the kind's id and length
-// arrays for the unit's item, loaded ahead of time (see unit_item).
-__device__ __forceinline__ void decode_unit(const TeamParams& p, unsigned g, bool in_bundle, int id, int len, ProdUnit* pu, UnitDesc* ud) {
+// Where unit g sits in the work list, and the entries of the id and length arrays that it
+// depends on.  Worked out (and the two entries loaded) one bundle ahead of the decode, so that
+// their latency is not on the producer's path.
+struct UnitIdx {
+    int kind;                 // UK_SELF, UK_ENC, UK_AAN, or UK_IDLE for padding
+    unsigned item, h, block, lg, span;      // AAN: item, chunk (in h), layer (in block)
+    int id, len;
+};
+
+__device__ __forceinline__ void unit_index(const TeamParams& p, unsigned g, bool in_bundle, UnitIdx* ui) {
+    ui->kind = UK_IDLE; ui->item = ui->h = ui->block = ui->lg = ui->span = 0; ui->id = -1; ui->len = 0;
+    if (!in_bundle || g >= p.n_units) return;
+    if (g < p.n_aan_units) {
+        unsigned rowi, chunk, lr, item;
+        p.div_aan_chunks.divmod(g, &rowi, &chunk);
+        p.div_aan_seqs.divmod(rowi, &lr, &item);
+        if (lr >= (unsigned)p.n_aan_layers) return;                      // padding
+        ui->kind = UK_AAN; ui->item = item; ui->h = chunk; ui->block = lr;
+        ui->id = p.aan_ids[item]; ui->len = p.t_aan[item];
+        return;
+    }
+    const int enc = g < p.n_aan_units + p.n_enc_units;
+    const TeamKind& kp = p.k[enc];
+    const unsigned x = g - p.n_aan_units - (enc ? 0u : p.n_enc_units);
+    const unsigned rowlg = x >> kp.spr_log2;
+    if (rowlg >= kp.n_rowlg) return;                                     // padding
+    unsigned rowb, row;
+    kp.div_lg.divmod(rowlg, &rowb, &ui->lg);
+    kp.div_rows.divmod(rowb, &ui->block, &row);
+    kp.div_h.divmod(row, &ui->item, &ui->h);
+    ui->span = x & ((1u << kp.spr_log2) - 1u);
+    ui->kind = enc ? UK_ENC : UK_SELF;
+    ui->id = kp.ids[ui->item]; ui->len = kp.lens[ui->item];
+}
+
+// Decode of one unit by one lane: what the producer keeps (pu) and what the consumer gets (ud).
+__device__ __forceinline__ void decode_unit(const TeamParams& p, const UnitIdx& ui, ProdUnit* pu, UnitDesc* ud) {
     pu->kind = UK_IDLE; pu->n = 0; pu->pi = 0; pu->tp = 16; pu->new_row = -1; pu->tiles = 0; pu->spr_log2 = 0;
     pu->srcK = pu->srcV = nullptr; pu->plane_bytes = 0;
     ud->dstK = nullptr; ud->dstV = nullptr; ud->S = nullptr; ud->O = nullptr; ud->q = ud->knew = ud->vnew = nullptr;
     ud->n = 0; ud->new_row = -1;
     ud->kind = UK_IDLE; ud->nq = 0; ud->pi = 0; ud->tp = 16; ud->span = 0; ud->spr_log2 = 0; ud->aux = 0;
-    if (!in_bundle || g >= p.n_units) return;
-    if (g < p.n_aan_units) {
+    if (ui.kind == UK_IDLE) return;
+    const int id = ui.id;
+    if (ui.kind == UK_AAN) {
         // ---- one chunk of one (layer, sequence) row of the running average; len holds t
-        unsigned rowi, chunk, lr, item;
-        p.div_aan_chunks.divmod(g, &rowi, &chunk);
-        p.div_aan_seqs.divmod(rowi, &lr, &item);
-        if (lr >= (unsigned)p.n_aan_layers) return;                      // padding
-        const int t = len;
+        const unsigned item = ui.item, chunk = ui.h, lr = ui.block;
+        const int t = ui.len;
         const bool reporter = (chunk == 0 && lr == 0);
         if (id < 0 || id >= p.aan_max_seqs) { if (reporter) record_error(p.err, TAG_AAN, (int)item, id, p.aan_max_seqs); return; }
         if (t < 1 || t > p.aan_max_t) { if (reporter) record_error(p.err, TAG_AAN, (int)item, t, p.aan_max_t); return; }
@@ -228,16 +278,10 @@ __device__ __forceinline__ void decode_unit(const TeamParams& p, unsigned g, boo
         ud->aux = (unsigned)t;
         return;
     }
-    const int enc = g < p.n_aan_units + p.n_enc_units;
+    const int enc = ui.kind == UK_ENC;
     const TeamKind& kp = p.k[enc];
-    const unsigned x = g - p.n_aan_units - (enc ? 0u : p.n_enc_units);
-    const unsigned span = x & ((1u << kp.spr_log2) - 1u), rowlg = x >> kp.spr_log2;
-    if (rowlg >= kp.n_rowlg) return;                                     // padding
-    unsigned rowb, lg, block, row, item, h;
-    kp.div_lg.divmod(rowlg, &rowb, &lg);
-    kp.div_rows.divmod(rowb, &block, &row);
-    kp.div_h.divmod(row, &item, &h);
-    len += (int)kp.len_bias;
+    const unsigned span = ui.span, lg = ui.lg, block = ui.block, item = ui.item, h = ui.h;
+    const int len = ui.len + (int)kp.len_bias;
     const bool reporter = (span == 0 && lg == 0 && h == 0 && block == 0);
     if ((unsigned)id >= kp.max_ids) { if (reporter) record_error(p.err, TAG_STEP, (int)item, id, (int)kp.max_ids); return; }
     if (len < 1 || len > (int)kp.bound) { if (reporter) record_error(p.err, TAG_STEP, (int)item, len, (int)kp.bound); return; }
@@ -257,7 +301,7 @@ __device__ __forceinline__ void decode_unit(const TeamParams& p, unsigned g, boo
     const bool has_new = (kp.knew != nullptr) && n > 0 && j1 == len;
     const char* K0 = kp.K + (unsigned long long)block * (unsigned long long)kp.plane_bytes + panel;
     const char* V0 = kp.V + (unsigned long long)vplane * (unsigned long long)kp.plane_bytes + panel;
-    pu->kind = enc ? UK_ENC : UK_SELF; pu->n = n; pu->pi = (int)min(kp.lg_size, size - l0);
+    pu->kind = ui.kind; pu->n = n; pu->pi = (int)min(kp.lg_size, size - l0);
     pu->tp = (int)kp.tile_pos; pu->new_row = has_new ? n - 1 : -1;
     pu->tiles = (n + pu->tp - 1) / pu->tp;
     pu->spr_log2 = (int)kp.spr_log2;
@@ -275,31 +319,6 @@ __device__ __forceinline__ void decode_unit(const TeamParams& p, unsigned g, boo
     ud->S = (kp.S && lg == 0) ? kp.S + (unsigned long long)qrow * (unsigned long long)kp.S_ld + j0 : nullptr;
     ud->O = kp.O + (unsigned long long)vplane * (unsigned long long)kp.layer_bytes +
             (unsigned long long)((item * kp.q_stride_items + kp.q_first) * H + h) * 128u;
-}
-
-// The entries of the id and length arrays that unit g depends on (issued one bundle ahead of
-// its decode, so that their latency is not on the producer's path).
-__device__ __forceinline__ void unit_item(const TeamParams& p, unsigned g, bool in_bundle, int* id, int* len) {
-    *id = -1; *len = 0;
-    if (!in_bundle || g >= p.n_units) return;
-    if (g < p.n_aan_units) {
-        unsigned rowi, chunk, lr, item;
-        p.div_aan_chunks.divmod(g, &rowi, &chunk);
-        p.div_aan_seqs.divmod(rowi, &lr, &item);
-        if (lr >= (unsigned)p.n_aan_layers) return;
-        *id = p.aan_ids[item]; *len = p.t_aan[item];
-        return;
-    }
-    const int enc = g < p.n_aan_units + p.n_enc_units;
-    const TeamKind& kp = p.k[enc];
-    const unsigned x = g - p.n_aan_units - (enc ? 0u : p.n_enc_units);
-    const unsigned rowlg = x >> kp.spr_log2;
-    if (rowlg >= kp.n_rowlg) return;
-    unsigned rowb, lg, block, row, item, h;
-    kp.div_lg.divmod(rowlg, &rowb, &lg);
-    kp.div_rows.divmod(rowb, &block, &row);
-    kp.div_h.divmod(row, &item, &h);
-    *id = kp.ids[item]; *len = kp.lens[item];
 }
 
 // ------------------------------------------------------------------------------ the consumer
@@ -359,7 +378,7 @@ struct StepConsumer {
     __device__ void aan(const UnitDesc& d);
     template <int NQ> __device__ void attend(const UnitDesc& d, const BundleHdr& hdr);
     template <int NQ> __device__ __forceinline__ bool softmax(const UnitDesc& d, const BundleHdr& hdr, int n, int n_pad, int ZQ);
-    template <int NQ> __device__ __forceinline__ void store_rows(const float (&acc)[4][4], char* op, bool q_store, int odd);
+    template <int NQ> __device__ __forceinline__ void store_rows(const float (&acc)[4][4], char* orow, int nq, long long O_qstride);
 };
 
 // A warp without a unit in this bundle (or whose unit was skipped) walks the bundle's slots and
@@ -466,14 +485,14 @@ __device__ __forceinline__ bool StepConsumer::softmax(const UnitDesc& d, const B
                 const __nv_bfloat16 lo = __float2bfloat16_rn(w0 - __bfloat162float(hi));
                 const int at = packed_slot(lane);
                 zh[at] = *reinterpret_cast<const unsigned short*>(&hi);
-                zh[at + 4] = *reinterpret_cast<const unsigned short*>(&lo);
+                if (kWeightRemainder) zh[at + 4] = *reinterpret_cast<const unsigned short*>(&lo);
             }
             if (two && lane + 32 < n_pad) {
                 const __nv_bfloat16 hi = __float2bfloat16_rn(w1);
                 const __nv_bfloat16 lo = __float2bfloat16_rn(w1 - __bfloat162float(hi));
                 const int at = packed_slot(lane + 32);
                 zh[at] = *reinterpret_cast<const unsigned short*>(&hi);
-                zh[at + 4] = *reinterpret_cast<const unsigned short*>(&lo);
+                if (kWeightRemainder) zh[at + 4] = *reinterpret_cast<const unsigned short*>(&lo);
             }
         }
         __syncwarp();
@@ -531,7 +550,7 @@ __device__ __forceinline__ bool StepConsumer::softmax(const UnitDesc& d, const B
                 const __nv_bfloat16 lo = __float2bfloat16_rn(w - __bfloat162float(hi));
                 const int at = packed_slot(jj);
                 zh[at] = *reinterpret_cast<const unsigned short*>(&hi);
-                zh[at + 4] = *reinterpret_cast<const unsigned short*>(&lo);
+                if (kWeightRemainder) zh[at + 4] = *reinterpret_cast<const unsigned short*>(&lo);
             }
         }
     }
@@ -540,25 +559,38 @@ __device__ __forceinline__ bool StepConsumer::softmax(const UnitDesc& d, const B
 }
 
 // The outputs of one layer from the accumulators: acc[x][0], [1] hold dim 16x + gid of queries
-// 2tig, 2tig+1 and acc[x][2], [3] dim 16x + gid + 8.  Lanes gid and gid ^ 1 hold adjacent dims:
-// the even one collects the pair of query 2tig, the odd one the pair of query 2tig + 1 (one
-// query: only the even lanes of tig 0 store).
+// 2tig, 2tig+1 and acc[x][2], [3] dim 16x + gid + 8.  They are rounded to bf16 into the warp's
+// scratch rows (the query rows there are no longer needed), one 128-byte row per query, and go
+// out as 16-byte pieces: lane = (query, piece).
 template <int NQ>
-__device__ __forceinline__ void StepConsumer::store_rows(const float (&acc)[4][4], char* op, bool q_store, int odd) {
+__device__ __forceinline__ void StepConsumer::store_rows(const float (&acc)[4][4], char* orow, int nq, long long O_qstride) {
+    const int tig = lane & 3, gid = lane >> 2;
+    __nv_bfloat16* stage = sp<__nv_bfloat16>(scr_off);
+    __syncwarp();
+    if (NQ == 1) {
+        if (tig == 0) {
 #pragma unroll
-    for (int x = 0; x < 4; ++x)
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            uint32_t packed;
-            if (NQ == 1) {
-                const float up = __shfl_down_sync(0xffffffffu, acc[x][2 * h], 4);
-                packed = pack_bf16x2(acc[x][2 * h], up);
-            } else {
-                const float got = __shfl_xor_sync(0xffffffffu, odd ? acc[x][2 * h] : acc[x][2 * h + 1], 4);
-                packed = odd ? pack_bf16x2(got, acc[x][2 * h + 1]) : pack_bf16x2(acc[x][2 * h], got);
-            }
-            if (q_store) *reinterpret_cast<uint32_t*>(op + (16 * x + 8 * h) * 2) = packed;
+            for (int x = 0; x < 4; ++x) { stage[16 * x + gid] = __float2bfloat16_rn(acc[x][0]); stage[16 * x + gid + 8] = __float2bfloat16_rn(acc[x][2]); }
         }
+    } else {
+#pragma unroll
+        for (int x = 0; x < 4; ++x) {
+            if (2 * tig < NQ) {
+                stage[(2 * tig) * kDh + 16 * x + gid] = __float2bfloat16_rn(acc[x][0]);
+                stage[(2 * tig) * kDh + 16 * x + gid + 8] = __float2bfloat16_rn(acc[x][2]);
+            }
+            if (2 * tig + 1 < NQ) {
+                stage[(2 * tig + 1) * kDh + 16 * x + gid] = __float2bfloat16_rn(acc[x][1]);
+                stage[(2 * tig + 1) * kDh + 16 * x + gid + 8] = __float2bfloat16_rn(acc[x][3]);
+            }
+        }
+    }
+    __syncwarp();
+#pragma unroll
+    for (int i = lane; i < NQ * 8; i += 32) {
+        const int qi = i >> 3, c = i & 7;
+        if (qi < nq) *reinterpret_cast<uint4*>(orow + qi * O_qstride + c * 16) = *sp<uint4>(scr_off + qi * 128 + c * 16);
+    }
 }
 
 // One attention unit on the tensor cores.
@@ -592,12 +624,16 @@ __device__ void StepConsumer::attend(const UnitDesc& d, const BundleHdr& hdr) {
     }
 
     // ldmatrix: this lane addresses row lrow of a 16-row block and, for the pair of 16-byte
-    // chunks 2x, 2x+1, the chunk 2x + (lane >> 4).  Rows keep chunk c at c ^ (row & 7)
-    // (row & 7 == lane & 7 here).
+    // chunks 2x, 2x+1, the chunk 2x + (lane >> 4).  Cached rows keep chunk c at c ^ (row & 7)
+    // (row & 7 == lane & 7 here).  This step's own row is not in the tile: the lane that addresses
+    // its position reads it from the warp's scratch rows instead, where it lies in natural order
+    // (new_fix takes the permutation out again).
     const int lrow = (lane & 7) + ((lane >> 3) & 1) * 8;
-    uint32_t ld_off[4];
+    const uint32_t new_fix = (uint32_t)(lane & 7) << 4;
+    uint32_t ld_swz[4];
 #pragma unroll
-    for (int x = 0; x < 4; ++x) ld_off[x] = (uint32_t)(lrow * 128 + (((2 * x + (lane >> 4)) ^ (lane & 7)) << 4));
+    for (int x = 0; x < 4; ++x) ld_swz[x] = (uint32_t)(((2 * x + (lane >> 4)) ^ (lane & 7)) << 4);
+    const uint32_t scr_s = sm.sm_base + scr_off;
 
     // ---- key tiles: scores into the warp's score slots (log2 domain)
     uint32_t qb[4][2];
@@ -621,24 +657,19 @@ __device__ void StepConsumer::attend(const UnitDesc& d, const BundleHdr& hdr) {
             const uint32_t st = my_rows(slot);
             const int s0 = t * tp;
             const int r = min(tp, n - s0);
-            if (new_row >= s0 && new_row < s0 + r) {
-                // this step's key row: into its place in the tile and into the cache, chunk-permuted like a cached row
-                const int nr = new_row - s0;
-                if (lane < 8) {
-                    const uint4 v = *sp<uint4>(scr_off + nq * 128 + lane * 16);
-                    *sp<uint4>(st + nr * 128 + ((lane ^ (nr & 7)) << 4)) = v;
-                    if (d.dstK) *reinterpret_cast<uint4*>(d.dstK + ((lane ^ (nr & 7)) << 4)) = v;
-                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // a later bulk copy reuses these bytes
-                }
-                __syncwarp();
-            }
-            const uint32_t st_s = sm.sm_base + st;
+            const int nr = (new_row >= s0 && new_row < s0 + r) ? new_row - s0 : -1;   // this step's key row in the tile
+            if (nr >= 0 && d.dstK && lane < 8)                                       // into the cache, chunk-permuted
+                *reinterpret_cast<uint4*>(d.dstK + ((lane ^ (nr & 7)) << 4)) = *sp<uint4>(scr_off + nq * 128 + lane * 16);
+            const uint32_t st_s = sm.sm_base + st + lrow * 128;
 #pragma unroll 1
             for (int b0 = 0; b0 < r; b0 += 16) {
+                const bool is_new = (b0 + lrow == nr);
+                const uint32_t rb = is_new ? scr_s + nq * 128 : st_s + b0 * 128;
+                const uint32_t fix = is_new ? new_fix : 0u;
                 float acc[4] = {0.f, 0.f, 0.f, 0.f};
                 uint32_t a[4][4];
 #pragma unroll
-                for (int ks = 0; ks < 4; ++ks) ldsm_x4(st_s + b0 * 128 + ld_off[ks], a[ks]);
+                for (int ks = 0; ks < 4; ++ks) ldsm_x4(rb + (ld_swz[ks] ^ fix), a[ks]);
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks) mma_bf16(acc, a[ks][0], a[ks][1], a[ks][2], a[ks][3], qb[ks][0], qb[ks][1]);
                 // acc[0], acc[1]: position b0+gid, queries 2tig, 2tig+1; acc[2], acc[3]: position b0+gid+8.
@@ -670,16 +701,13 @@ __device__ void StepConsumer::attend(const UnitDesc& d, const BundleHdr& hdr) {
     // and, for the dim tile x, the 16-byte chunk 2x + ((lane >> 3) & 1).
     const uint32_t za = zs_off + (gid < NQ ? gid : 0) * ZQ * 4 + tig * 16;
     const int vrow = (lane & 7) + ((lane >> 4) << 3);
-    uint32_t vd_off[4];
+    uint32_t vd_swz[4];
 #pragma unroll
-    for (int x = 0; x < 4; ++x) vd_off[x] = (uint32_t)(vrow * 128 + (((2 * x + ((lane >> 3) & 1)) ^ (lane & 7)) << 4));
+    for (int x = 0; x < 4; ++x) vd_swz[x] = (uint32_t)(((2 * x + ((lane >> 3) & 1)) ^ (lane & 7)) << 4);
     const long long plane_bytes = kp.plane_bytes;
     char* vlast = d.dstV;                                             // where this step's value row goes
-    const int odd = gid & 1;
-    const int q_mine = NQ == 1 ? 0 : 2 * tig + odd;
-    const bool q_store = NQ == 1 ? (tig == 0 && !odd) : (q_mine < nq);
     const long long O_qstride = (long long)p.H * 128;
-    char* op = d.O + q_mine * O_qstride + (gid - odd) * 2;
+    char* op = d.O;
     const int spr = 1 << d.spr_log2;
 #pragma unroll 1
     for (int l = 0; l < hdr.layers; ++l) {
@@ -696,37 +724,37 @@ __device__ void StepConsumer::attend(const UnitDesc& d, const BundleHdr& hdr) {
                 const uint32_t st = my_rows(slot);
                 const int s0 = t * tp;
                 const int r = min(tp, n - s0);
-                if (new_row >= s0 && new_row < s0 + r) {
-                    const int nr = new_row - s0;
-                    if (lane < 8) {
-                        const uint4 v = *sp<uint4>(scr_off + (nq + 1 + l) * 128 + lane * 16);
-                        *sp<uint4>(st + nr * 128 + ((lane ^ (nr & 7)) << 4)) = v;
-                        *reinterpret_cast<uint4*>(vlast + ((lane ^ (nr & 7)) << 4)) = v;
-                        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                    }
-                    __syncwarp();
-                }
-                const uint32_t st_s = sm.sm_base + st;
+                const int nr = (new_row >= s0 && new_row < s0 + r) ? new_row - s0 : -1;
+                if (nr >= 0 && lane < 8)
+                    *reinterpret_cast<uint4*>(vlast + ((lane ^ (nr & 7)) << 4)) = *sp<uint4>(scr_off + (nq + 1 + l) * 128 + lane * 16);
+                const uint32_t st_s = sm.sm_base + st + vrow * 128;
+                const uint32_t new_v = scr_s + (nq + 1 + l) * 128;
 #pragma unroll 1
                 for (int b0 = 0; b0 < r; b0 += 16) {
-                    const uint4 w = *sp<uint4>(za + (s0 + b0) * 4);      // (high b0, high b1, remainder b0, remainder b1)
+                    uint4 w;                                             // (high b0, high b1, remainder b0, remainder b1)
+                    if (kWeightRemainder) w = *sp<uint4>(za + (s0 + b0) * 4);
+                    else { const uint2 w2 = *sp<uint2>(za + (s0 + b0) * 4); w = make_uint4(w2.x, w2.y, 0u, 0u); }
                     // rows at or beyond r hold other bytes: their weights are zero, but 0 x NaN would not be,
                     // so those lanes address a row of zeros instead
-                    const uint32_t blk = st_s + b0 * 128;
-                    const bool in = b0 + vrow < r;
+                    const int row = b0 + vrow;
+                    const bool is_new = (row == nr);
+                    const uint32_t rb = is_new ? new_v : st_s + b0 * 128;
+                    const uint32_t fix = is_new ? new_fix : 0u;
                     uint32_t a[4][4];
 #pragma unroll
-                    for (int x = 0; x < 4; ++x) ldsm_x4_t(in ? blk + vd_off[x] : zero_row, a[x]);
+                    for (int x = 0; x < 4; ++x) ldsm_x4_t(row >= r ? zero_row : rb + (vd_swz[x] ^ fix), a[x]);
 #pragma unroll
                     for (int x = 0; x < 4; ++x) mma_bf16(acc[x], a[x][0], a[x][1], a[x][2], a[x][3], w.x, w.y);
+                    if (kWeightRemainder) {
 #pragma unroll
-                    for (int x = 0; x < 4; ++x) mma_bf16(acc[x], a[x][0], a[x][1], a[x][2], a[x][3], w.z, w.w);
+                        for (int x = 0; x < 4; ++x) mma_bf16(acc[x], a[x][0], a[x][1], a[x][2], a[x][3], w.z, w.w);
+                    }
                 }
             }
             release();
         }
         if (!hdr.sync) {
-            if (l < pi) store_rows<NQ>(acc, op, q_store, odd);
+            if (l < pi) store_rows<NQ>(acc, op, nq, O_qstride);
         } else {
             // the spans of a row add up their partial outputs through shared memory (two buffers, by layer parity)
             float* xo = sp<float>(xch_o(l & 1));
@@ -755,7 +783,7 @@ __device__ void StepConsumer::attend(const UnitDesc& d, const BundleHdr& hdr) {
                         }
                     }
                 } else {
-                    store_rows<NQ>(acc, op, q_store, odd);
+                    store_rows<NQ>(acc, op, nq, O_qstride);
                 }
             }
         }
@@ -779,7 +807,8 @@ __global__ void __launch_bounds__(kStepWarps * 32, 1) decode_step_team_kernel(co
                 mbar_init(sp<uint64_t>(p.off_bars + t * kTeamBarBytes + s * 8), 1);
                 mbar_init(sp<uint64_t>(p.off_bars + t * kTeamBarBytes + (kNS + s) * 8), kTeamWarps);
             }
-            mbar_init(sp<uint64_t>(p.off_bars + t * kTeamBarBytes + 2 * kNS * 8), kTeamWarps);
+            for (int s = 0; s < kNS; ++s) mbar_init(sp<uint64_t>(p.off_bars + t * kTeamBarBytes + (2 * kNS + s) * 8), 1);
+            mbar_init(sp<uint64_t>(p.off_bars + t * kTeamBarBytes + 3 * kNS * 8), kTeamWarps);
         }
         *sm.dead_flag() = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -803,31 +832,35 @@ __global__ void __launch_bounds__(kStepWarps * 32, 1) decode_step_team_kernel(co
             c &= ~(S - 1u);
             return min((unsigned)kTeamWarps, max(S, c));
         };
+        // Every team's first bundle is fixed by its place in the grid (no round trip to the counter
+        // before the first copy can go out); the counter hands out the units after those.
+        const unsigned dyn0 = (unsigned)gridDim.x * kTeams * kTeamWarps;
         auto grab = [&](unsigned chunk) -> unsigned {
             unsigned v = 0;
-            if (lane == 0) v = (unsigned)atomicAdd(p.queue, (int)chunk);
+            if (lane == 0) v = dyn0 + (unsigned)atomicAdd(p.queue, (int)chunk);
             return v;
         };
         // Two bundles are in preparation behind the one being issued: the index of the one after
         // next is on its way back from the counter, the id / length entries of the next one are
         // on their way from memory.
-        unsigned cur_chunk = chunk_for(0);
-        unsigned cur = __shfl_sync(0xffffffffu, grab(cur_chunk), 0);
-        unsigned nxt_chunk = chunk_for(cur);
-        unsigned nxt = __shfl_sync(0xffffffffu, grab(nxt_chunk), 0);
-        int cur_id, cur_len;
-        unit_item(p, cur + (unsigned)lane, lane < (int)cur_chunk, &cur_id, &cur_len);
+        unsigned cur_chunk = kTeamWarps;
+        unsigned cur = ((unsigned)blockIdx.x * kTeams + (unsigned)team) * kTeamWarps;
+        unsigned nxt_chunk = chunk_for(dyn0);
+        const unsigned nxt_raw0 = grab(nxt_chunk);
+        UnitIdx cur_ui;
+        unit_index(p, cur + (unsigned)lane, lane < (int)cur_chunk, &cur_ui);
+        unsigned nxt = __shfl_sync(0xffffffffu, nxt_raw0, 0);
         while (cur < p.n_units && !pr.dead) {
             const unsigned aft_chunk = chunk_for(nxt);
             const unsigned aft_raw = grab(aft_chunk);                          // used at the end of the iteration
-            int nxt_id, nxt_len;
-            unit_item(p, nxt + (unsigned)lane, lane < (int)nxt_chunk, &nxt_id, &nxt_len);
+            UnitIdx nxt_ui;
+            unit_index(p, nxt + (unsigned)lane, lane < (int)nxt_chunk, &nxt_ui);
             pr.ensure_slot();
             if (pr.dead) break;
             const int bslot = (int)(pr.n_bundles % kNS);
             ProdUnit pu;
             UnitDesc ud;
-            decode_unit(p, cur + (unsigned)lane, lane < (int)cur_chunk, cur_id, cur_len, &pu, &ud);
+            decode_unit(p, cur_ui, &pu, &ud);
             // the bundle: tiles per plane, value layers, whether any row is split over spans
             int tiles = pu.tiles, layers = pu.pi, sync = pu.spr_log2;
 #pragma unroll
@@ -840,6 +873,8 @@ __global__ void __launch_bounds__(kStepWarps * 32, 1) decode_step_team_kernel(co
             tiles = max(tiles, 1);
             if (lane == 0) *sp<BundleHdr>(sm.bundle_hdr(team, bslot)) = BundleHdr{tiles, layers, sync ? 1 : 0, 0};
             if (lane < kTeamWarps) *sp<UnitDesc>(sm.unit_desc(team, bslot, lane)) = ud;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(sm.bar_ready(team, bslot));     // the consumers may start on their small rows
             // ---- slots: the key tiles, then each layer's value tiles
             for (int plane = 0; plane <= layers && !pr.dead; ++plane) {
                 for (int t = 0; t < tiles && !pr.dead; ++t) {
@@ -879,16 +914,16 @@ __global__ void __launch_bounds__(kStepWarps * 32, 1) decode_step_team_kernel(co
                 }
             }
             pr.n_bundles += 1;
-            cur = nxt; cur_chunk = nxt_chunk; cur_id = nxt_id; cur_len = nxt_len;
+            cur = nxt; cur_chunk = nxt_chunk; cur_ui = nxt_ui;
             nxt = __shfl_sync(0xffffffffu, aft_raw, 0); nxt_chunk = aft_chunk;
         }
         // ---- no more work: tell the team, then leave the counters clean for the next launch
         if (!pr.dead) pr.ensure_slot();
         if (!pr.dead) {
-            if (lane == 0) *sp<BundleHdr>(sm.bundle_hdr(team, (int)(pr.n_bundles % kNS))) = BundleHdr{0, 0, 0, 1};
-            __syncwarp();
-            if (lane == 0) mbar_expect_tx(sm.bar_full(team, (int)(pr.n_slots % kNS)), 0u);
-            pr.issued();
+            if (lane == 0) {
+                *sp<BundleHdr>(sm.bundle_hdr(team, (int)(pr.n_bundles % kNS))) = BundleHdr{0, 0, 0, 1};
+                mbar_arrive(sm.bar_ready(team, (int)(pr.n_bundles % kNS)));
+            }
         } else {
             // a wait ran out somewhere: let the copies already issued land before the CTA leaves
             for (uint32_t s = pr.n_retired; s != pr.n_slots; ++s) {
@@ -913,13 +948,11 @@ __global__ void __launch_bounds__(kStepWarps * 32, 1) decode_step_team_kernel(co
     c.scr_off = p.off_scr + (uint32_t)warp * p.scr_bytes;
     c.zero_row = sm.sm_base + p.off_zero;
     for (uint32_t b = 0; !c.dead; ++b) {
-        // the bundle's descriptors are complete once its first slot's barrier has been armed and has fired
+        const int bslot = (int)(b % kNS);
         {
-            const int slot = (int)(c.cs % kNS);
-            const uint32_t bar = sm.bar_full(c.team, slot), par = (c.cs / kNS) & 1u;
+            const uint32_t bar = sm.bar_ready(c.team, bslot), par = (b / kNS) & 1u;
             if (!mbar_try_wait(bar, par) && !step_wait_slow(bar, par, sm.dead_flag())) { c.fail(4); break; }
         }
-        const int bslot = (int)(b % kNS);
         const BundleHdr hdr = *sp<BundleHdr>(sm.bundle_hdr(c.team, bslot));
         if (hdr.end) break;
         const UnitDesc d = *sp<UnitDesc>(sm.unit_desc(c.team, bslot, c.u));
