@@ -222,16 +222,24 @@ int32_t san_decode_step(san_ctx* ctx, const san_step_args* args, void* stream);
 /* Which kernel san_decode_step launches, and (for testing and tuning) how its rows are cut.
  * The library has two implementations of the one-launch step (same arithmetic, Eq. 1-5):
  *   which = 1  per-warp pipeline: every warp streams the tiles of its own row (float32 and bf16);
- *   which = 2  team pipeline (bf16): four producer warps each stream bundles of four rows or row
- *              spans to a team of four warps; SAN_ERR_UNSUPPORTED from the step if a shape does not fit;
+ *   which = 2  team pipeline (bf16): four producer warps each stream bundles of two units to a team
+ *              of two warps, a unit being up to four heads of one sequence or one of two spans of
+ *              a long row; SAN_ERR_UNSUPPORTED from the step if a shape does not fit;
  *   which = 0  automatic (the default): the team pipeline where it applies, else the per-warp one.
  * spans_log2 >= 0 overrides the automatic cut of the team pipeline: every row is dealt to
- * 1 << spans_log2 warps (0..2), tiles hold tile_pos positions (a multiple of 16),
+ * 1 << spans_log2 warps (0..1); with one span tile_pos / 16 (16, 32 or 64 -> 1, 2 or 4) heads
+ * go to a unit where the head count allows,
  * layers_per_unit > 0 caps the layers one warp applies (the block's other layers go to
  * further warps, which recompute S), grab_mult >= 1 makes the bundles shrink earlier towards
  * the end of the launch.  spans_log2 < 0 restores the automatic cut. */
 int32_t san_step_kernel_select(san_ctx* ctx, int32_t which, int32_t spans_log2, int32_t tile_pos,
                                int32_t layers_per_unit, int32_t grab_mult);
+
+/* Which kernel the last san_decode_step of this context launched (1 or 2 as above, 0 before the
+ * first step) and, for the team pipeline, how many heads of one sequence / sentence it gave
+ * to one warp: rows_per_unit[0] for self-attention, [1] for encoder-decoder attention (may
+ * be NULL).  For tests and benchmarks that must know what they measured. */
+int32_t san_step_kernel_used(const san_ctx* ctx, int32_t* which, int32_t* rows_per_unit);
 
 /* san_decode_step for a caller whose step inputs and outputs live in HOST memory (pinned
  * memory if the copies are to overlap anything): the same step (Eq. 1-5, Section 4.1) with

@@ -29,7 +29,7 @@ EXPORTS = (
     "san_policy_set_sizes", "san_policy_set_map", "san_policy_get_map",
     "san_cache_append", "san_attn_weights", "san_attn_apply", "san_aan_step", "san_seq_reset",
     "san_device_status", "san_status_string", "san_attn_weights_static", "san_decode_step",
-    "san_decode_step_host", "san_step_kernel_select", "san_full_block", "san_beam_reorder", "san_js_matrix", "san_block_similarity", "san_policy_search",
+    "san_decode_step_host", "san_step_kernel_select", "san_step_kernel_used", "san_full_block", "san_beam_reorder", "san_js_matrix", "san_block_similarity", "san_policy_search",
 )
 
 
@@ -86,6 +86,7 @@ def lib():
     L.san_attn_weights_static.argtypes = [i32, i32, i32, vp, vp, i32, i32, vp, vp, i32, i32, vp, i64, vp, vp]
     L.san_decode_step.argtypes = [vp, C.POINTER(san_step_args), vp]
     L.san_step_kernel_select.argtypes = [vp, i32, i32, i32, i32, i32]
+    L.san_step_kernel_used.argtypes = [vp, _I32P, _I32P]
     L.san_decode_step_host.argtypes = [vp, C.POINTER(san_step_args), C.POINTER(san_step_args), vp]
     L.san_full_block.argtypes = [i32, i32, i32, i32, vp, vp, vp, vp, i32, i32, i32, vp, i64, vp, vp]
     L.san_beam_reorder.argtypes = [vp, vp, vp, vp, i32, i32, vp]
@@ -231,6 +232,14 @@ def san_decode_step(ctx, *, d_q_self=None, d_k_new=None, d_v_new=None, d_seq_ids
 def san_step_kernel_select(ctx, which=0, spans_log2=-1, tile_pos=64, layers_per_unit=0, grab_mult=1) -> int:
     """Choose the kernel behind san_decode_step (0 automatic, 1 per-warp, 2 team pipeline) and its cut."""
     return lib().san_step_kernel_select(ctx, which, spans_log2, tile_pos, layers_per_unit, grab_mult)
+
+
+def san_step_kernel_used(ctx):
+    """Returns (status, kernel of the last san_decode_step: 0 none / 1 per-warp / 2 team, [heads per unit self, enc-dec])."""
+    which = C.c_int32(0)
+    rpu = (C.c_int32 * 2)()
+    rc = lib().san_step_kernel_used(ctx, C.byref(which), rpu)
+    return rc, which.value, list(rpu)
 
 
 def san_beam_reorder(ctx, d_sent_ids, d_parent, d_lens, n_sent, max_len=0, stream=None) -> int:

@@ -167,9 +167,9 @@ cudaError_t launch_apply(const ApplyParams& p, int nq_t, unsigned grid, cudaStre
 // caller then uses the per-warp kernel).
 constexpr size_t kStepSmemTotal = 232448;      // opt-in shared memory per CTA on sm_100
 
-struct TeamCut { int spr_log2, lg, tile_pos, zq; };
+struct TeamCut { int spr_log2, lg, tile_pos, zq, rpu; };
 
-int32_t launch_team_step(san_ctx* ctx, const san_step_args* a, int max_len, int max_src, cudaStream_t st) {
+int32_t launch_team_step(san_ctx* ctx, const san_step_args* a, int max_len, int max_src, cudaStream_t st, int* rows_per_unit) {
     const san_config& c = ctx->cfg;
     if (c.dtype != SAN_BF16) return SAN_ERR_UNSUPPORTED;
     const bool aan = c.self_is_aan != 0;
@@ -185,49 +185,91 @@ int32_t launch_team_step(san_ctx* ctx, const san_step_args* a, int max_len, int 
     const long long rows_enc = do_enc ? (long long)ctx->enc_pol.n_blocks * n_sent * H : 0;
     if (rows_self + rows_enc >= (1ll << 27)) return SAN_ERR_UNSUPPORTED;
 
-    // Units wanted: a few per consumer warp of the grid, so that the warps stay busy and the SMs
-    // finish together.  Long rows are cut into spans first (nothing is read twice), then a block's
-    // layers into groups (each group reads the block's keys again, mostly from L2).
-    constexpr int kZCapFloats = 1024;              // score slots a warp may hold
-    constexpr int kMaxSprLog2 = 2;                 // a row's spans are neighbouring warps of one team
-    const long long want_units = 3ll * ctx->sm_count * kStepConsumers;
+    // Long rows are cut into spans handled by the warps of a team (nothing is read twice); short
+    // rows are gathered, up to four heads of one sequence or sentence to a warp, so that the cost
+    // of a unit beside its arithmetic is shared.  A block's layers go to several units where a
+    // unit would otherwise be too fat for the SMs to finish together (each group reads the
+    // block's keys again, mostly from L2).
+    constexpr int kZCapFloats = 1024;              // score slots a warp may hold per head
+    constexpr int kMaxSprLog2 = 1;                 // a row's spans are the warps of one team
+    const long long want_units = 2ll * ctx->sm_count * kStepConsumers;
+    const int rpu_max = H % 4 == 0 ? 4 : H % 2 == 0 ? 2 : 1;
     auto span_of = [](int bound, int spr_log2) { return (int)align_up((size_t)ceil_div(bound, 1 << spr_log2), 16); };
     auto cut = [&](long long rows, int bound, int pi, int nq_t, TeamCut* out) -> bool {
         int s = 0, lg = pi;
         while (s < kMaxSprLog2 && span_of(bound, s) * nq_t > kZCapFloats) ++s;
         if (span_of(bound, s) * nq_t > kZCapFloats) return false;
-        while (s < kMaxSprLog2 && span_of(bound, s) > 64 && rows * (1ll << s) * ceil_div(pi, lg) < want_units) ++s;
-        while (lg > 2 && rows * (1ll << s) * ceil_div(pi, lg) < want_units &&
-               (long long)span_of(bound, s) * 128 * (1 + lg) > 48 * 1024) lg = std::max(2, ceil_div(lg, 2));
+        while (s < kMaxSprLog2 && span_of(bound, s) > 128 && rows * (1ll << s) * ceil_div(pi, lg) < want_units) ++s;
         const int span = span_of(bound, s);
-        out->spr_log2 = s; out->lg = lg;
-        out->tile_pos = span <= 48 ? span : 32;   // a slot of four units stays under half of a team's ring
+        out->spr_log2 = s;
+        out->rpu = s == 0 ? rpu_max : 1;
         out->zq = span + 4;                         // + 4: the score rows of neighbouring queries start in different banks
+        while (lg > 2 && rows / out->rpu * (1ll << s) * ceil_div(pi, lg) < want_units &&
+               (long long)out->rpu * span * 128 * (1 + lg) > 64 * 1024) lg = std::max(2, ceil_div(lg, 2));
+        out->lg = lg;
+        out->tile_pos = span;
         return true;
     };
-    TeamCut cs{0, 1, 16, 20}, ce{0, 1, 16, 20};
+    TeamCut cs{0, 1, 16, 20, 1}, ce{0, 1, 16, 20, 1};
     if (do_self && !cut(rows_self, max_len, pi_self, 1, &cs)) return SAN_ERR_UNSUPPORTED;
     if (do_enc && !cut(rows_enc, max_src, pi_enc, nqe, &ce)) return SAN_ERR_UNSUPPORTED;
     if (ctx->team_cut_override[0] >= 0) {           // testing and tuning: san_step_kernel_select
         cs.spr_log2 = ce.spr_log2 = std::min(kMaxSprLog2, ctx->team_cut_override[0]);
         if (span_of(max_len, cs.spr_log2) > kZCapFloats || span_of(max_src, ce.spr_log2) * nqe > kZCapFloats) return SAN_ERR_UNSUPPORTED;
-        cs.tile_pos = std::min(span_of(max_len, cs.spr_log2), std::max(16, ctx->team_cut_override[1]));
-        ce.tile_pos = std::min(span_of(max_src, ce.spr_log2), std::max(16, ctx->team_cut_override[1]));
-        cs.zq = span_of(max_len, cs.spr_log2) + 4; ce.zq = span_of(max_src, ce.spr_log2) + 4;
+        cs.tile_pos = span_of(max_len, cs.spr_log2); ce.tile_pos = span_of(max_src, ce.spr_log2);
+        cs.zq = cs.tile_pos + 4; ce.zq = ce.tile_pos + 4;
+        cs.rpu = ce.rpu = cs.spr_log2 == 0 ? std::min(rpu_max, std::max(1, ctx->team_cut_override[1] / 16)) : 1;   // tile_pos 16, 32, 64: 1, 2, 4 heads per unit
+        if (cs.rpu == 3) cs.rpu = ce.rpu = 2;
         if (ctx->team_cut_override[2] > 0) { cs.lg = std::min(pi_self, ctx->team_cut_override[2]); ce.lg = std::min(pi_enc, ctx->team_cut_override[2]); }
     }
 
     TeamParams p;
     std::memset(&p, 0, sizeof(p));
+    // Shared memory: [ring | pad] per team, then per consumer warp its score slots and its scratch
+    // rows (queries, this step's key and value rows), the exchange area of split rows, descriptors,
+    // barriers, a row of zeros.  Units of several heads need their whole span in one tile and the
+    // tile of every unit of a bundle in the ring: where that does not fit, fewer heads go to a unit;
+    // a lone head is cut into tiles of 32 positions.
+    size_t zs_bytes = 0, scr_bytes = 0, xo_bytes = 0;
+    const bool split = (do_self && cs.spr_log2 > 0) || (do_enc && ce.spr_log2 > 0);
+    const int nq_x = std::max(do_self && cs.spr_log2 > 0 ? 1 : 0, do_enc && ce.spr_log2 > 0 ? nqe : 0);
+    p.xo_unit_floats = split ? (unsigned)(nq_x * kDh) : 0u;
+    xo_bytes = (size_t)kTeams * team_xch_bytes(p.xo_unit_floats);
+    for (;;) {
+        zs_bytes = align_up((size_t)4 * std::max(do_self ? cs.rpu * cs.zq : 0, do_enc ? ce.rpu * ce.zq * nqe : 0), 16);
+        scr_bytes = (size_t)128 * std::max(do_self ? cs.rpu * (2 + cs.lg) : 0, do_enc ? ce.rpu * nqe : 0);
+        const size_t tail = kStepConsumers * (zs_bytes + scr_bytes) + xo_bytes + kTeams * kTeamDescBytes + (kTeams * kTeamBarBytes + 16) + 128 + 256;
+        if (tail + kTeams * (8 * 1024 + kRingPad) > kStepSmemTotal) return SAN_ERR_UNSUPPORTED;
+        p.ring_bytes = (unsigned)(((kStepSmemTotal - tail) / kTeams - kRingPad) / 128 * 128);
+        const size_t slot_self = do_self ? (size_t)kTeamWarps * cs.rpu * std::min(cs.tile_pos, max_len) * 128 : 0;   // no row is longer than its bound
+        const size_t slot_enc = do_enc ? (size_t)kTeamWarps * ce.rpu * std::min(ce.tile_pos, max_src) * 128 : 0;
+        if (slot_self <= p.ring_bytes && slot_enc <= p.ring_bytes) break;
+        TeamCut& big = slot_self >= slot_enc ? cs : ce;
+        if (big.rpu > 1) big.rpu /= 2;
+        else if (big.tile_pos > 32) big.tile_pos = 32;
+        else return SAN_ERR_UNSUPPORTED;
+    }
+    if (rows_per_unit) { rows_per_unit[0] = do_self ? cs.rpu : 0; rows_per_unit[1] = do_enc ? ce.rpu : 0; }
+    p.ring_stride = p.ring_bytes + kRingPad;
+    p.zs_bytes = (unsigned)zs_bytes; p.scr_bytes = (unsigned)scr_bytes;
+    p.off_zs = kTeams * p.ring_stride;
+    p.off_scr = (unsigned)(p.off_zs + kStepConsumers * zs_bytes);
+    p.off_xo = (unsigned)align_up(p.off_scr + kStepConsumers * scr_bytes, 16);
+    p.off_desc = (unsigned)align_up(p.off_xo + xo_bytes, 16);
+    p.off_bars = (unsigned)align_up(p.off_desc + kTeams * kTeamDescBytes, 8);
+    p.off_zero = (unsigned)align_up(p.off_bars + kTeams * kTeamBarBytes + 16, 128);
+    const size_t smem = p.off_zero + 128;
+
     p.H = H;
     p.err = ctx->err; p.queue = ctx->err + 16;
     p.scale_log2e = (float)(1.4426950408889634 / std::sqrt((double)kDh));
     auto fill = [&](TeamKind& k, const Policy& pol, const TeamCut& tc, int n_it, long long rows, int pi) {
         k.spr_log2 = (unsigned)tc.spr_log2; k.lg_size = (unsigned)tc.lg; k.tile_pos = (unsigned)tc.tile_pos; k.zq = (unsigned)tc.zq;
+        k.rpu = (unsigned)tc.rpu;
         const int n_lg = ceil_div(pi, tc.lg);
-        k.n_rowlg = (unsigned)(rows * n_lg);
+        k.n_rowlg = (unsigned)(rows / tc.rpu * n_lg);
         k.n_units = (unsigned)align_up((size_t)k.n_rowlg << tc.spr_log2, kTeamWarps);
-        k.div_lg = make_fastdiv((unsigned)n_lg); k.div_rows = make_fastdiv((unsigned)std::max(1, n_it * H)); k.div_h = make_fastdiv((unsigned)H);
+        k.div_lg = make_fastdiv((unsigned)n_lg); k.div_rows = make_fastdiv((unsigned)std::max(1, n_it * H / tc.rpu)); k.div_h = make_fastdiv((unsigned)H);
         k.n_it = (unsigned)std::max(n_it, 1);
         for (int b = 0; b < pol.n_blocks; ++b) {
             k.first[b] = (unsigned char)pol.first_layer_of_block[b];
@@ -277,30 +319,6 @@ int32_t launch_team_step(san_ctx* ctx, const san_step_args* a, int max_len, int 
     if (n_units > (1ll << 30)) return SAN_ERR_UNSUPPORTED;
     p.n_units = (unsigned)n_units;
     if (p.n_units == 0) return SAN_OK;
-
-    // shared memory: [ring | pad] per team, then per consumer warp its score slots and its scratch rows
-    // (queries, this step's key row and value rows), the exchange area of split rows, descriptors,
-    // barriers, a row of zeros
-    const bool split = (do_self && cs.spr_log2 > 0) || (do_enc && ce.spr_log2 > 0);
-    const int nq_x = std::max(do_self && cs.spr_log2 > 0 ? 1 : 0, do_enc && ce.spr_log2 > 0 ? nqe : 0);
-    const size_t zs_bytes = align_up((size_t)4 * std::max(do_self ? cs.zq : 0, do_enc ? ce.zq * nqe : 0), 16);
-    const size_t scr_bytes = (size_t)128 * std::max(do_self ? 2 + cs.lg : 0, do_enc ? nqe : 0);
-    p.xo_unit_floats = split ? (unsigned)(nq_x * kDh) : 0u;
-    const size_t xo_bytes = (size_t)kTeams * team_xch_bytes(p.xo_unit_floats);
-    const size_t tail = kStepConsumers * (zs_bytes + scr_bytes) + xo_bytes + kTeams * kTeamDescBytes + (kTeams * kTeamBarBytes + 16) + 128 + 256;
-    if (tail + kTeams * (16 * 1024 + kRingPad) > kStepSmemTotal) return SAN_ERR_UNSUPPORTED;
-    p.ring_bytes = (unsigned)(((kStepSmemTotal - tail) / kTeams - kRingPad) / 128 * 128);
-    p.ring_stride = p.ring_bytes + kRingPad;
-    const size_t slot_max = (size_t)kTeamWarps * 128 * std::max(do_self ? cs.tile_pos : 0, do_enc ? ce.tile_pos : 0);
-    if (slot_max > p.ring_bytes) return SAN_ERR_UNSUPPORTED;
-    p.zs_bytes = (unsigned)zs_bytes; p.scr_bytes = (unsigned)scr_bytes;
-    p.off_zs = kTeams * p.ring_stride;
-    p.off_scr = (unsigned)(p.off_zs + kStepConsumers * zs_bytes);
-    p.off_xo = (unsigned)align_up(p.off_scr + kStepConsumers * scr_bytes, 16);
-    p.off_desc = (unsigned)align_up(p.off_xo + xo_bytes, 16);
-    p.off_bars = (unsigned)align_up(p.off_desc + kTeams * kTeamDescBytes, 8);
-    p.off_zero = (unsigned)align_up(p.off_bars + kTeams * kTeamBarBytes + 16, 128);
-    const size_t smem = p.off_zero + 128;
 
     const long long bundles = ((long long)p.n_units + kTeamWarps - 1) / kTeamWarps;
     const long long ctas = std::max<long long>(1, std::min<long long>(ctx->sm_count, (bundles + kTeams - 1) / kTeams));
@@ -620,10 +638,11 @@ int32_t san_decode_step(san_ctx* ctx, const san_step_args* a, void* stream) {
 
     const bool bf16 = c.dtype == SAN_BF16;
     if (ctx->step_kernel != 1) {       // the team-pipeline kernel takes every bf16 shape that fits its shared memory
-        const int32_t rc = launch_team_step(ctx, a, max_len, max_src, static_cast<cudaStream_t>(stream));
-        if (rc != SAN_ERR_UNSUPPORTED) return rc;
+        const int32_t rc = launch_team_step(ctx, a, max_len, max_src, static_cast<cudaStream_t>(stream), ctx->last_rows_per_unit);
+        if (rc != SAN_ERR_UNSUPPORTED) { ctx->last_step_kernel = 2; return rc; }
         if (ctx->step_kernel == 2) return rc;
     }
+    ctx->last_step_kernel = 1;
     const int row_bytes = kDh * ctx->elem_bytes;
     const int TR = kStageBytes / row_bytes;
     const int nqe = pick_nq_template(c.beam);
@@ -825,12 +844,19 @@ int32_t san_decode_step(san_ctx* ctx, const san_step_args* a, void* stream) {
 int32_t san_step_kernel_select(san_ctx* ctx, int32_t which, int32_t spans_log2, int32_t tile_pos, int32_t layers_per_unit,
                                int32_t grab_mult) {
     if (!ctx) return SAN_ERR_NULL;
-    if (which < 0 || which > 2 || spans_log2 > 2 || (spans_log2 >= 0 && (tile_pos < 16 || tile_pos % 16 != 0))) return SAN_ERR_RANGE;
+    if (which < 0 || which > 2 || spans_log2 > 1 || (spans_log2 >= 0 && (tile_pos < 16 || tile_pos % 16 != 0))) return SAN_ERR_RANGE;
     ctx->step_kernel = which;
     ctx->team_cut_override[0] = spans_log2 < 0 ? -1 : spans_log2;
     ctx->team_cut_override[1] = tile_pos;
     ctx->team_cut_override[2] = layers_per_unit;
     ctx->team_grab_mult = grab_mult > 0 ? grab_mult : 1;
+    return SAN_OK;
+}
+
+int32_t san_step_kernel_used(const san_ctx* ctx, int32_t* which, int32_t* rows_per_unit) {
+    if (!ctx || !which) return SAN_ERR_NULL;
+    *which = ctx->last_step_kernel;
+    if (rows_per_unit) { rows_per_unit[0] = ctx->last_step_kernel == 2 ? ctx->last_rows_per_unit[0] : 0; rows_per_unit[1] = ctx->last_step_kernel == 2 ? ctx->last_rows_per_unit[1] : 0; }
     return SAN_OK;
 }
 

@@ -32,6 +32,8 @@ struct san_ctx {
     int step_kernel = 0;           // 0: automatic, 1: per-warp pipeline kernel, 2: team-pipeline kernel (san_step_kernel_select)
     int team_cut_override[3] = {-1, 64, 0};   // spans per row (log2; -1: automatic), positions per tile, layers per unit (0: automatic)
     int team_grab_mult = 1;
+    int last_step_kernel = 0;      // which kernel the last san_decode_step launched (0: none yet)
+    int last_rows_per_unit[2] = {0, 0};   // team pipeline: heads per unit for self / enc-dec attention in that launch
 
     // How the one-launch step cuts long rows (positions per item, layers per item), remembered
     // per launch shape: the search that balances the items over the warps costs more than a

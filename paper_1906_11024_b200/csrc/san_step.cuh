@@ -30,8 +30,9 @@
 
 namespace san {
 
-constexpr int kTeams = 6;
-constexpr int kTeamWarps = 4;                                  // consumer warps of a team = units per bundle
+constexpr int kTeams = 4;
+constexpr int kTeamWarps = 2;                                  // consumer warps of a team = units per bundle
+constexpr int kUnitRows = 4;                                   // a unit is up to four rows (heads) of one (block, id)
 constexpr int kStepConsumers = kTeams * kTeamWarps;
 constexpr int kStepWarps = kStepConsumers + kTeams;            // + one producer per team
 constexpr int kNS = 8;                                         // slots (and bundles) a team may have outstanding
@@ -60,7 +61,8 @@ struct TeamKind {
     unsigned q_first, q_stride_items;                  // first query row this launch covers; queries per item in q/S/O
     unsigned spr_log2;                                 // spans per row = 1 << spr_log2 (at most kTeamWarps)
     unsigned lg_size, v_by_block;
-    unsigned n_rowlg;                                  // (block, row, layer group) triples
+    unsigned rpu;                                      // rows (consecutive heads of one id) per unit: 1, 2 or 4; 1 when rows are split into spans
+    unsigned n_rowlg;                                  // (block, row group, layer group) triples
     unsigned tile_pos;                                 // positions per tile (multiple of 16)
     unsigned zq;                                       // floats between the score rows of two queries
     unsigned n_units;                                  // padded to a multiple of kTeamWarps
@@ -94,7 +96,7 @@ struct __align__(16) UnitDesc {
     const char* vnew;         // this step's value row of the unit's first layer
     int n;                    // positions in the span
     int new_row;              // index in the span of this step's row (not yet cached), or -1
-    unsigned char kind, nq, pi, tp, span, spr_log2, pad0, pad1;
+    unsigned char kind, nq, pi, tp, span, spr_log2, rows, pad1;
     unsigned int aux;         // AAN: target position t
     unsigned int pad[5];
 };
@@ -214,7 +216,8 @@ struct StepProducer {
 struct ProdUnit {
     const char* srcK; const char* srcV;
     long long plane_bytes;
-    int n, pi, tp, new_row, kind, tiles, spr_log2;
+    unsigned panel_bytes;
+    int n, pi, tp, new_row, kind, tiles, spr_log2, rows;
 };
 
 // Where unit g sits in the work list, and the entries of the id and length arrays that it
@@ -246,26 +249,26 @@ __device__ __forceinline__ void unit_index(const TeamParams& p, unsigned g, bool
     unsigned rowb, row;
     kp.div_lg.divmod(rowlg, &rowb, &ui->lg);
     kp.div_rows.divmod(rowb, &ui->block, &row);
-    kp.div_h.divmod(row, &ui->item, &ui->h);
+    kp.div_h.divmod(row * kp.rpu, &ui->item, &ui->h);           // row counts groups of rpu heads (rpu divides H)
     ui->span = x & ((1u << kp.spr_log2) - 1u);
     ui->kind = enc ? UK_ENC : UK_SELF;
     ui->id = kp.ids[ui->item]; ui->len = kp.lens[ui->item];
 }
 
 // Decode of one unit by one lane: what the producer keeps (pu) and what the consumer gets (ud).
-__device__ __forceinline__ void decode_unit(const TeamParams& p, const UnitIdx& ui, ProdUnit* pu, UnitDesc* ud) {
-    pu->kind = UK_IDLE; pu->n = 0; pu->pi = 0; pu->tp = 16; pu->new_row = -1; pu->tiles = 0; pu->spr_log2 = 0;
-    pu->srcK = pu->srcV = nullptr; pu->plane_bytes = 0;
+__device__ __forceinline__ void decode_unit(const TeamParams& p, const UnitIdx& ui, bool may_report, ProdUnit* pu, UnitDesc* ud) {
+    pu->kind = UK_IDLE; pu->n = 0; pu->pi = 0; pu->tp = 16; pu->new_row = -1; pu->tiles = 0; pu->spr_log2 = 0; pu->rows = 0;
+    pu->srcK = pu->srcV = nullptr; pu->plane_bytes = 0; pu->panel_bytes = 0;
     ud->dstK = nullptr; ud->dstV = nullptr; ud->S = nullptr; ud->O = nullptr; ud->q = ud->knew = ud->vnew = nullptr;
     ud->n = 0; ud->new_row = -1;
-    ud->kind = UK_IDLE; ud->nq = 0; ud->pi = 0; ud->tp = 16; ud->span = 0; ud->spr_log2 = 0; ud->aux = 0;
+    ud->kind = UK_IDLE; ud->nq = 0; ud->pi = 0; ud->tp = 16; ud->span = 0; ud->spr_log2 = 0; ud->rows = 0; ud->aux = 0;
     if (ui.kind == UK_IDLE) return;
     const int id = ui.id;
     if (ui.kind == UK_AAN) {
         // ---- one chunk of one (layer, sequence) row of the running average; len holds t
         const unsigned item = ui.item, chunk = ui.h, lr = ui.block;
         const int t = ui.len;
-        const bool reporter = (chunk == 0 && lr == 0);
+        const bool reporter = may_report && (chunk == 0 && lr == 0);
         if (id < 0 || id >= p.aan_max_seqs) { if (reporter) record_error(p.err, TAG_AAN, (int)item, id, p.aan_max_seqs); return; }
         if (t < 1 || t > p.aan_max_t) { if (reporter) record_error(p.err, TAG_AAN, (int)item, t, p.aan_max_t); return; }
         const int d = p.H * kDh;
@@ -282,7 +285,7 @@ __device__ __forceinline__ void decode_unit(const TeamParams& p, const UnitIdx& 
     const TeamKind& kp = p.k[enc];
     const unsigned span = ui.span, lg = ui.lg, block = ui.block, item = ui.item, h = ui.h;
     const int len = ui.len + (int)kp.len_bias;
-    const bool reporter = (span == 0 && lg == 0 && h == 0 && block == 0);
+    const bool reporter = may_report && (span == 0 && lg == 0 && h == 0 && block == 0);
     if ((unsigned)id >= kp.max_ids) { if (reporter) record_error(p.err, TAG_STEP, (int)item, id, (int)kp.max_ids); return; }
     if (len < 1 || len > (int)kp.bound) { if (reporter) record_error(p.err, TAG_STEP, (int)item, len, (int)kp.bound); return; }
     const unsigned size = kp.v_by_block ? 1u : kp.size[block];
@@ -304,7 +307,7 @@ __device__ __forceinline__ void decode_unit(const TeamParams& p, const UnitIdx& 
     pu->kind = ui.kind; pu->n = n; pu->pi = (int)min(kp.lg_size, size - l0);
     pu->tp = (int)kp.tile_pos; pu->new_row = has_new ? n - 1 : -1;
     pu->tiles = (n + pu->tp - 1) / pu->tp;
-    pu->spr_log2 = (int)kp.spr_log2;
+    pu->spr_log2 = (int)kp.spr_log2; pu->rows = (int)kp.rpu; pu->panel_bytes = kp.panel_bytes;
     pu->srcK = K0 + (unsigned)j0 * 128u; pu->srcV = V0 + (unsigned)j0 * 128u;
     pu->plane_bytes = kp.plane_bytes;
     const unsigned long long in_row = (unsigned long long)(item * H + h) * 128u;                 // self: one query per item
@@ -312,7 +315,7 @@ __device__ __forceinline__ void decode_unit(const TeamParams& p, const UnitIdx& 
     ud->knew = kp.knew ? kp.knew + (unsigned long long)block * (unsigned long long)kp.layer_bytes + in_row : nullptr;
     ud->vnew = kp.vnew ? kp.vnew + (unsigned long long)first * (unsigned long long)kp.layer_bytes + in_row : nullptr;
     ud->kind = (unsigned char)pu->kind; ud->nq = (unsigned char)kp.nq; ud->pi = (unsigned char)pu->pi; ud->tp = (unsigned char)pu->tp;
-    ud->span = (unsigned char)span; ud->spr_log2 = (unsigned char)kp.spr_log2;
+    ud->span = (unsigned char)span; ud->spr_log2 = (unsigned char)kp.spr_log2; ud->rows = (unsigned char)kp.rpu;
     ud->n = n; ud->new_row = pu->new_row;
     ud->dstK = (has_new && lg == 0) ? const_cast<char*>(K0) + (unsigned)(len - 1) * 128u : nullptr;   // the lead group stores the key row
     ud->dstV = has_new ? const_cast<char*>(V0) + (unsigned)(len - 1) * 128u : nullptr;
@@ -377,8 +380,10 @@ struct StepConsumer {
     __device__ void idle(const BundleHdr& hdr);
     __device__ void aan(const UnitDesc& d);
     template <int NQ> __device__ void attend(const UnitDesc& d, const BundleHdr& hdr);
-    template <int NQ> __device__ __forceinline__ bool softmax(const UnitDesc& d, const BundleHdr& hdr, int n, int n_pad, int ZQ);
-    template <int NQ> __device__ __forceinline__ void store_rows(const float (&acc)[4][4], char* orow, int nq, long long O_qstride);
+    template <int NQ> __device__ __forceinline__ bool softmax(const UnitDesc& d, const BundleHdr& hdr, int n, int n_pad, int ZQ,
+                                                              uint32_t zs_base, float* S_base, long long S_rstride, int nq);
+    template <int NQ> __device__ __forceinline__ void stage_rows(const float (&acc)[4][4], int nq, int R, int hh);
+    __device__ __forceinline__ void flush_rows(char* orow, int nq, int R, long long O_qstride);
 };
 
 // A warp without a unit in this bundle (or whose unit was skipped) walks the bundle's slots and
@@ -413,14 +418,16 @@ __device__ void StepConsumer::aan(const UnitDesc& d) {
     *reinterpret_cast<uint4*>(d.O + e0 * 2) = o;
 }
 
-// Softmax of the span's n scores (log2 domain) per query row, in place: the weights are left as
-// bf16 pairs (high part, remainder) in the order the apply MMAs read them (see packed_slot),
-// zero from n up to n_pad, and are written to S.  The spans of a split row first exchange their
-// (max, sum) through the team's shared memory, so every span normalises by the row's total.
+// Softmax of n scores (log2 domain) of NQ rows side by side, in place: row r has its scores at
+// zs_base + r * ZQ floats and its S row at S_base + r * S_rstride (rows at or beyond nq are
+// carried along and never stored).  The weights are left as bf16 words in the order the apply
+// MMAs read them (see packed_slot), zero from n up to n_pad, and are written to S.  The spans of
+// a split row first exchange their (max, sum) through the team's shared memory, so every span
+// normalises by the row's total.
 template <int NQ>
-__device__ __forceinline__ bool StepConsumer::softmax(const UnitDesc& d, const BundleHdr& hdr, int n, int n_pad, int ZQ) {
-    const int nq = d.nq;
-    const long long S_qstride = (long long)p.H * p.k[d.kind].S_ld;
+__device__ __forceinline__ bool StepConsumer::softmax(const UnitDesc& d, const BundleHdr& hdr, int n, int n_pad, int ZQ,
+                                                      uint32_t zs_base, float* S_base, long long S_rstride, int nq) {
+    const long long S_qstride = S_rstride;
     const int spr = 1 << d.spr_log2;
     float* ms = sp<float>(xch_ms());     // (max, sum) of every unit of the team and query: [unit][8][2] floats
     if (n <= 64) {
@@ -429,7 +436,7 @@ __device__ __forceinline__ bool StepConsumer::softmax(const UnitDesc& d, const B
         float z0[NQ], z1[NQ], m[NQ], sum[NQ];
 #pragma unroll
         for (int qi = 0; qi < NQ; ++qi) {
-            const float* zq = sp<float>(zs_off + qi * ZQ * 4);
+            const float* zq = sp<float>(zs_base + qi * ZQ * 4);
             z0[qi] = in0 ? zq[lane] : -INFINITY;
             z1[qi] = (two && in1) ? zq[lane + 32] : -INFINITY;
             m[qi] = fmaxf(z0[qi], z1[qi]);
@@ -472,11 +479,11 @@ __device__ __forceinline__ bool StepConsumer::softmax(const UnitDesc& d, const B
         __syncwarp();                                   // every lane has read its scores: the words may be reused
 #pragma unroll
         for (int qi = 0; qi < NQ; ++qi) {
-            float* zq = sp<float>(zs_off + qi * ZQ * 4);
+            float* zq = sp<float>(zs_base + qi * ZQ * 4);
             unsigned short* zh = reinterpret_cast<unsigned short*>(zq);
             const float w0 = z0[qi] * inv[qi], w1 = z1[qi] * inv[qi];
-            if (d.S && qi < nq) {
-                float* Srow = d.S + qi * S_qstride;
+            if (S_base && qi < nq) {
+                float* Srow = S_base + qi * S_qstride;
                 if (in0) Srow[lane] = w0;
                 if (two && in1) Srow[lane + 32] = w1;
             }
@@ -502,7 +509,7 @@ __device__ __forceinline__ bool StepConsumer::softmax(const UnitDesc& d, const B
     float mq[NQ], sq[NQ];
 #pragma unroll
     for (int qi = 0; qi < NQ; ++qi) {
-        float* zq = sp<float>(zs_off + qi * ZQ * 4);
+        float* zq = sp<float>(zs_base + qi * ZQ * 4);
         float m = -INFINITY;
 #pragma unroll 1
         for (int jj = lane; jj < n; jj += 32) m = fmaxf(m, zq[jj]);
@@ -535,9 +542,9 @@ __device__ __forceinline__ bool StepConsumer::softmax(const UnitDesc& d, const B
     __syncwarp();
 #pragma unroll
     for (int qi = 0; qi < NQ; ++qi) {
-        float* zq = sp<float>(zs_off + qi * ZQ * 4);
+        float* zq = sp<float>(zs_base + qi * ZQ * 4);
         unsigned short* zh = reinterpret_cast<unsigned short*>(zq);
-        float* Srow = (d.S && qi < nq) ? d.S + qi * S_qstride : nullptr;
+        float* Srow = (S_base && qi < nq) ? S_base + qi * S_qstride : nullptr;
         const float inv = sq[qi];
 #pragma unroll 1
         for (int j0 = 0; j0 < n_pad; j0 += 32) {      // warp-uniform trip count
@@ -558,66 +565,77 @@ __device__ __forceinline__ bool StepConsumer::softmax(const UnitDesc& d, const B
     return true;
 }
 
-// The outputs of one layer from the accumulators: acc[x][0], [1] hold dim 16x + gid of queries
-// 2tig, 2tig+1 and acc[x][2], [3] dim 16x + gid + 8.  They are rounded to bf16 into the warp's
-// scratch rows (the query rows there are no longer needed), one 128-byte row per query, and go
-// out as 16-byte pieces: lane = (query, piece).
+// The outputs of one layer and one head from the accumulators: acc[x][0], [1] hold dim 16x + gid
+// of queries 2tig, 2tig+1 and acc[x][2], [3] dim 16x + gid + 8.  They are rounded to bf16 into
+// the warp's scratch rows (the query rows there are no longer needed), row = query * R + head, so
+// that the heads of one query lie side by side as they do in the output.
 template <int NQ>
-__device__ __forceinline__ void StepConsumer::store_rows(const float (&acc)[4][4], char* orow, int nq, long long O_qstride) {
+__device__ __forceinline__ void StepConsumer::stage_rows(const float (&acc)[4][4], int nq, int R, int hh) {
     const int tig = lane & 3, gid = lane >> 2;
     __nv_bfloat16* stage = sp<__nv_bfloat16>(scr_off);
-    __syncwarp();
     if (NQ == 1) {
         if (tig == 0) {
 #pragma unroll
-            for (int x = 0; x < 4; ++x) { stage[16 * x + gid] = __float2bfloat16_rn(acc[x][0]); stage[16 * x + gid + 8] = __float2bfloat16_rn(acc[x][2]); }
+            for (int x = 0; x < 4; ++x) { stage[hh * kDh + 16 * x + gid] = __float2bfloat16_rn(acc[x][0]); stage[hh * kDh + 16 * x + gid + 8] = __float2bfloat16_rn(acc[x][2]); }
         }
     } else {
 #pragma unroll
         for (int x = 0; x < 4; ++x) {
-            if (2 * tig < NQ) {
-                stage[(2 * tig) * kDh + 16 * x + gid] = __float2bfloat16_rn(acc[x][0]);
-                stage[(2 * tig) * kDh + 16 * x + gid + 8] = __float2bfloat16_rn(acc[x][2]);
+            if (2 * tig < nq) {
+                stage[((2 * tig) * R + hh) * kDh + 16 * x + gid] = __float2bfloat16_rn(acc[x][0]);
+                stage[((2 * tig) * R + hh) * kDh + 16 * x + gid + 8] = __float2bfloat16_rn(acc[x][2]);
             }
-            if (2 * tig + 1 < NQ) {
-                stage[(2 * tig + 1) * kDh + 16 * x + gid] = __float2bfloat16_rn(acc[x][1]);
-                stage[(2 * tig + 1) * kDh + 16 * x + gid + 8] = __float2bfloat16_rn(acc[x][3]);
+            if (2 * tig + 1 < nq) {
+                stage[((2 * tig + 1) * R + hh) * kDh + 16 * x + gid] = __float2bfloat16_rn(acc[x][1]);
+                stage[((2 * tig + 1) * R + hh) * kDh + 16 * x + gid + 8] = __float2bfloat16_rn(acc[x][3]);
             }
         }
     }
+}
+// The staged rows of a layer to the output, 16 bytes per lane: piece i = (query, head, chunk).
+__device__ __forceinline__ void StepConsumer::flush_rows(char* orow, int nq, int R, long long O_qstride) {
     __syncwarp();
-#pragma unroll
-    for (int i = lane; i < NQ * 8; i += 32) {
-        const int qi = i >> 3, c = i & 7;
-        if (qi < nq) *reinterpret_cast<uint4*>(orow + qi * O_qstride + c * 16) = *sp<uint4>(scr_off + qi * 128 + c * 16);
+    const int pieces = nq * R * 8;
+    for (int i = lane; i < pieces; i += 32) {
+        const int row = i >> 3, c = i & 7;
+        const int qi = R == 4 ? row >> 2 : R == 2 ? row >> 1 : row, hh = row - qi * R;
+        *reinterpret_cast<uint4*>(orow + qi * O_qstride + hh * 128 + c * 16) = *sp<uint4>(scr_off + row * 128 + c * 16);
     }
+    __syncwarp();
 }
 
-// One attention unit on the tensor cores.
+// One attention unit on the tensor cores: up to four rows (heads) of one (block, id), one after
+// the other inside each phase, so that what a unit costs beside its arithmetic (descriptors,
+// barrier waits, address set-up, output stores) is paid once for all of them.
 //   scores:  D[16 positions x 8 queries] = K_tile[16 x 64] . q^T              (queries padded to 8)
 //   apply:   D[16 dims x 8 queries]     += V_tile^T[16 x 16 positions] . S^T   (four dim tiles)
-// S is used as a bf16 high part plus a bf16 remainder (two MMAs), so that the weights keep about
-// 16 bits; products and sums are float32.  Columns of D that belong to padding queries are
-// computed from whatever the padding lanes load and are never stored.
+// S is applied as bf16; products and sums are float32.  Columns of D that belong to padding
+// queries are computed from whatever the padding lanes load and are never stored.
 template <int NQ>
 __device__ void StepConsumer::attend(const UnitDesc& d, const BundleHdr& hdr) {
     const TeamKind& kp = p.k[d.kind];
     const int ZQ = (int)kp.zq;
-    const int n = d.n, nq = d.nq, pi = d.pi, tp = d.tp, new_row = d.new_row;
+    const int n = d.n, nq = d.nq, pi = d.pi, tp = d.tp, new_row = d.new_row, R = d.rows;
     const int my_tiles = (n + tp - 1) / tp;
     const int tig = lane & 3, gid = lane >> 2;                 // mma fragment coordinates
     const long long layer_bytes = kp.layer_bytes;
+    const unsigned panel_bytes = kp.panel_bytes;
+    const uint32_t zs_head = (uint32_t)(NQ * ZQ * 4);          // bytes between the score rows of two heads
 
     // ---- this unit's small rows, fetched by the warp itself while the producer's copies are in
-    // flight: scratch rows [0, nq) = queries, [nq] = this step's key row, [nq + 1 + l] = this
-    // step's value row of layer l (the last two only when the span ends in the new position)
+    // flight.  Scratch rows: [qi * R + hh] = query qi of head hh; then R rows = this step's key
+    // rows; then [l * R + hh] = this step's value rows of layer l (the last two groups only when
+    // the span ends in the new position).
+    const int scr_k = nq * R, scr_v = scr_k + R;
     {
-        const int rows = nq + (new_row >= 0 ? 1 + pi : 0);
+        const int rows = scr_k + (new_row >= 0 ? R * (1 + pi) : 0);
         const unsigned q_stride = (unsigned)p.H * 128u;
         for (int i = lane; i < rows * 8; i += 32) {
             const int row = i >> 3, c = i & 7;
-            const char* src = row < nq ? d.q + (unsigned long long)row * q_stride
-                            : row == nq ? d.knew : d.vnew + (long long)(row - nq - 1) * layer_bytes;
+            const char* src;
+            if (row < scr_k) { const int qi = R == 4 ? row >> 2 : R == 2 ? row >> 1 : row; src = d.q + (unsigned long long)qi * q_stride + (row - qi * R) * 128; }
+            else if (row < scr_v) src = d.knew + (row - scr_k) * 128;
+            else { const int lr = row - scr_v, l = R == 4 ? lr >> 2 : R == 2 ? lr >> 1 : lr; src = d.vnew + (long long)l * layer_bytes + (lr - l * R) * 128; }
             cp_async16(sm.sm_base + scr_off + row * 128 + c * 16, src + c * 16);
         }
         asm volatile("cp.async.commit_group;" ::: "memory");
@@ -636,7 +654,6 @@ __device__ void StepConsumer::attend(const UnitDesc& d, const BundleHdr& hdr) {
     const uint32_t scr_s = sm.sm_base + scr_off;
 
     // ---- key tiles: scores into the warp's score slots (log2 domain)
-    uint32_t qb[4][2];
     const float sc = p.scale_log2e;
     const uint32_t zk = zs_off + ((2 * tig) * ZQ + gid) * 4;   // queries 2tig, 2tig+1; positions gid, gid+8
     for (int t = 0; t < hdr.tiles; ++t) {
@@ -645,45 +662,52 @@ __device__ void StepConsumer::attend(const UnitDesc& d, const BundleHdr& hdr) {
         if (t == 0) {
             asm volatile("cp.async.wait_group 0;" ::: "memory");
             __syncwarp();
-            // the query rows (natural chunk order) as B fragments (k = dims, n = query)
-            const uint32_t qrow = scr_off + (uint32_t)(gid < nq ? gid : 0) * 128u + 4u * tig;
-#pragma unroll
-            for (int ks = 0; ks < 4; ++ks) {
-                qb[ks][0] = *sp<uint32_t>(qrow + 32 * ks);
-                qb[ks][1] = *sp<uint32_t>(qrow + 32 * ks + 16);
-            }
         }
         if (t < my_tiles) {
-            const uint32_t st = my_rows(slot);
+            const uint32_t st0 = my_rows(slot);
             const int s0 = t * tp;
             const int r = min(tp, n - s0);
             const int nr = (new_row >= s0 && new_row < s0 + r) ? new_row - s0 : -1;   // this step's key row in the tile
-            if (nr >= 0 && d.dstK && lane < 8)                                       // into the cache, chunk-permuted
-                *reinterpret_cast<uint4*>(d.dstK + ((lane ^ (nr & 7)) << 4)) = *sp<uint4>(scr_off + nq * 128 + lane * 16);
-            const uint32_t st_s = sm.sm_base + st + lrow * 128;
 #pragma unroll 1
-            for (int b0 = 0; b0 < r; b0 += 16) {
-                const bool is_new = (b0 + lrow == nr);
-                const uint32_t rb = is_new ? scr_s + nq * 128 : st_s + b0 * 128;
-                const uint32_t fix = is_new ? new_fix : 0u;
-                float acc[4] = {0.f, 0.f, 0.f, 0.f};
-                uint32_t a[4][4];
+            for (int hh = 0; hh < R; ++hh) {
+                // the head's query rows (natural chunk order) as B fragments (k = dims, n = query)
+                uint32_t qb[4][2];
+                const uint32_t qrow = scr_off + (uint32_t)((gid < nq ? gid : 0) * R + hh) * 128u + 4u * tig;
 #pragma unroll
-                for (int ks = 0; ks < 4; ++ks) ldsm_x4(rb + (ld_swz[ks] ^ fix), a[ks]);
-#pragma unroll
-                for (int ks = 0; ks < 4; ++ks) mma_bf16(acc, a[ks][0], a[ks][1], a[ks][2], a[ks][3], qb[ks][0], qb[ks][1]);
-                // acc[0], acc[1]: position b0+gid, queries 2tig, 2tig+1; acc[2], acc[3]: position b0+gid+8.
-                // Rows of the block at or beyond r (another unit's rows, stale bytes) give scores that
-                // are never stored.
-                const int pos = s0 + b0 + gid;
-                float* z = sp<float>(zk + (s0 + b0) * 4);
-                if (2 * tig < NQ) {
-                    if (pos < n) z[0] = acc[0] * sc;
-                    if (pos + 8 < n) z[8] = acc[2] * sc;
+                for (int ks = 0; ks < 4; ++ks) {
+                    qb[ks][0] = *sp<uint32_t>(qrow + 32 * ks);
+                    qb[ks][1] = *sp<uint32_t>(qrow + 32 * ks + 16);
                 }
-                if (2 * tig + 1 < NQ) {
-                    if (pos < n) z[ZQ] = acc[1] * sc;
-                    if (pos + 8 < n) z[ZQ + 8] = acc[3] * sc;
+                if (nr >= 0 && d.dstK && lane < 8)                                   // into the cache, chunk-permuted
+                    *reinterpret_cast<uint4*>(d.dstK + (unsigned long long)hh * panel_bytes + ((lane ^ (nr & 7)) << 4)) =
+                        *sp<uint4>(scr_off + (scr_k + hh) * 128 + lane * 16);
+                const uint32_t st_s = sm.sm_base + st0 + (uint32_t)(hh * r + lrow) * 128u;
+                const uint32_t new_k = scr_s + (scr_k + hh) * 128;
+                const uint32_t zh = zk + hh * zs_head;
+#pragma unroll 1
+                for (int b0 = 0; b0 < r; b0 += 16) {
+                    const bool is_new = (b0 + lrow == nr);
+                    const uint32_t rb = is_new ? new_k : st_s + b0 * 128;
+                    const uint32_t fix = is_new ? new_fix : 0u;
+                    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+                    uint32_t a[4][4];
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks) ldsm_x4(rb + (ld_swz[ks] ^ fix), a[ks]);
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks) mma_bf16(acc, a[ks][0], a[ks][1], a[ks][2], a[ks][3], qb[ks][0], qb[ks][1]);
+                    // acc[0], acc[1]: position b0+gid, queries 2tig, 2tig+1; acc[2], acc[3]: position b0+gid+8.
+                    // Rows of the block at or beyond r (another head's or unit's rows, stale bytes) give
+                    // scores that are never stored.
+                    const int pos = s0 + b0 + gid;
+                    float* z = sp<float>(zh + (s0 + b0) * 4);
+                    if (2 * tig < NQ) {
+                        if (pos < n) z[0] = acc[0] * sc;
+                        if (pos + 8 < n) z[8] = acc[2] * sc;
+                    }
+                    if (2 * tig + 1 < NQ) {
+                        if (pos < n) z[ZQ] = acc[1] * sc;
+                        if (pos + 8 < n) z[ZQ + 8] = acc[3] * sc;
+                    }
                 }
             }
         }
@@ -692,11 +716,19 @@ __device__ void StepConsumer::attend(const UnitDesc& d, const BundleHdr& hdr) {
     __syncwarp();
 
     const int n_pad = (n + 15) & ~15;
-    if (!softmax<NQ>(d, hdr, n, n_pad, ZQ)) return;
+    const long long S_qstride = (long long)p.H * kp.S_ld;
+    if (NQ == 1 && R == 4) {
+        // one query per head: the four heads' rows go through the softmax side by side
+        if (!softmax<4>(d, hdr, n, n_pad, ZQ, zs_off, d.S, kp.S_ld, 4)) return;
+    } else {
+#pragma unroll 1
+        for (int hh = 0; hh < R; ++hh)
+            if (!softmax<NQ>(d, hdr, n, n_pad, ZQ, zs_off + hh * zs_head, d.S ? d.S + (long long)hh * kp.S_ld : nullptr, S_qstride, nq)) return;
+    }
 
     // ---- value tiles, layer by layer
     // B fragments: the weights of query gid at positions b0 + {2tig, 2tig+1} and b0 + {2tig+8, 2tig+9},
-    // high parts and remainders, one 16-byte load per block straight from the packed words.
+    // one load per block straight from the packed words.
     // A fragments: the tile transposed by ldmatrix; this lane addresses position vrow of a block
     // and, for the dim tile x, the 16-byte chunk 2x + ((lane >> 3) & 1).
     const uint32_t za = zs_off + (gid < NQ ? gid : 0) * ZQ * 4 + tig * 16;
@@ -712,49 +744,66 @@ __device__ void StepConsumer::attend(const UnitDesc& d, const BundleHdr& hdr) {
 #pragma unroll 1
     for (int l = 0; l < hdr.layers; ++l) {
         float acc[4][4];
+        if (R == 1) {
 #pragma unroll
-        for (int x = 0; x < 4; ++x)
+            for (int x = 0; x < 4; ++x)
 #pragma unroll
-            for (int e = 0; e < 4; ++e) acc[x][e] = 0.f;
+                for (int e = 0; e < 4; ++e) acc[x][e] = 0.f;
+        }
 #pragma unroll 1
         for (int t = 0; t < hdr.tiles; ++t) {
             const int slot = acquire();
             if (slot < 0) return;
             if (l < pi && t < my_tiles) {
-                const uint32_t st = my_rows(slot);
+                const uint32_t st0 = my_rows(slot);
                 const int s0 = t * tp;
                 const int r = min(tp, n - s0);
                 const int nr = (new_row >= s0 && new_row < s0 + r) ? new_row - s0 : -1;
-                if (nr >= 0 && lane < 8)
-                    *reinterpret_cast<uint4*>(vlast + ((lane ^ (nr & 7)) << 4)) = *sp<uint4>(scr_off + (nq + 1 + l) * 128 + lane * 16);
-                const uint32_t st_s = sm.sm_base + st + vrow * 128;
-                const uint32_t new_v = scr_s + (nq + 1 + l) * 128;
 #pragma unroll 1
-                for (int b0 = 0; b0 < r; b0 += 16) {
-                    uint4 w;                                             // (high b0, high b1, remainder b0, remainder b1)
-                    if (kWeightRemainder) w = *sp<uint4>(za + (s0 + b0) * 4);
-                    else { const uint2 w2 = *sp<uint2>(za + (s0 + b0) * 4); w = make_uint4(w2.x, w2.y, 0u, 0u); }
-                    // rows at or beyond r hold other bytes: their weights are zero, but 0 x NaN would not be,
-                    // so those lanes address a row of zeros instead
-                    const int row = b0 + vrow;
-                    const bool is_new = (row == nr);
-                    const uint32_t rb = is_new ? new_v : st_s + b0 * 128;
-                    const uint32_t fix = is_new ? new_fix : 0u;
-                    uint32_t a[4][4];
+                for (int hh = 0; hh < R; ++hh) {
+                    if (R > 1) {          // several heads: each is one tile (the host cuts them so); a lone head keeps its sums across tiles
 #pragma unroll
-                    for (int x = 0; x < 4; ++x) ldsm_x4_t(row >= r ? zero_row : rb + (vd_swz[x] ^ fix), a[x]);
+                        for (int x = 0; x < 4; ++x)
 #pragma unroll
-                    for (int x = 0; x < 4; ++x) mma_bf16(acc[x], a[x][0], a[x][1], a[x][2], a[x][3], w.x, w.y);
-                    if (kWeightRemainder) {
-#pragma unroll
-                        for (int x = 0; x < 4; ++x) mma_bf16(acc[x], a[x][0], a[x][1], a[x][2], a[x][3], w.z, w.w);
+                            for (int e = 0; e < 4; ++e) acc[x][e] = 0.f;
                     }
+                    const uint32_t new_v = scr_s + (scr_v + l * R + hh) * 128;
+                    if (nr >= 0 && lane < 8)
+                        *reinterpret_cast<uint4*>(vlast + (unsigned long long)hh * panel_bytes + ((lane ^ (nr & 7)) << 4)) =
+                            *sp<uint4>(scr_off + (scr_v + l * R + hh) * 128 + lane * 16);
+                    const uint32_t st_s = sm.sm_base + st0 + (uint32_t)(hh * r + vrow) * 128u;
+                    const uint32_t zb = za + hh * zs_head;
+#pragma unroll 1
+                    for (int b0 = 0; b0 < r; b0 += 16) {
+                        uint4 w;                                             // (high b0, high b1, remainder b0, remainder b1)
+                        if (kWeightRemainder) w = *sp<uint4>(zb + (s0 + b0) * 4);
+                        else { const uint2 w2 = *sp<uint2>(zb + (s0 + b0) * 4); w = make_uint4(w2.x, w2.y, 0u, 0u); }
+                        // rows at or beyond r hold other bytes: their weights are zero, but 0 x NaN would not be,
+                        // so those lanes address a row of zeros instead
+                        const int row = b0 + vrow;
+                        const bool is_new = (row == nr);
+                        const uint32_t rb = is_new ? new_v : st_s + b0 * 128;
+                        const uint32_t fix = is_new ? new_fix : 0u;
+                        uint32_t a[4][4];
+#pragma unroll
+                        for (int x = 0; x < 4; ++x) ldsm_x4_t(row >= r ? zero_row : rb + (vd_swz[x] ^ fix), a[x]);
+#pragma unroll
+                        for (int x = 0; x < 4; ++x) mma_bf16(acc[x], a[x][0], a[x][1], a[x][2], a[x][3], w.x, w.y);
+                        if (kWeightRemainder) {
+#pragma unroll
+                            for (int x = 0; x < 4; ++x) mma_bf16(acc[x], a[x][0], a[x][1], a[x][2], a[x][3], w.z, w.w);
+                        }
+                    }
+                    if (R > 1) stage_rows<NQ>(acc, nq, R, hh);
                 }
             }
             release();
         }
         if (!hdr.sync) {
-            if (l < pi) store_rows<NQ>(acc, op, nq, O_qstride);
+            if (l < pi) {
+                if (R == 1) stage_rows<NQ>(acc, nq, 1, 0);
+                flush_rows(op, nq, R, O_qstride);
+            }
         } else {
             // the spans of a row add up their partial outputs through shared memory (two buffers, by layer parity)
             float* xo = sp<float>(xch_o(l & 1));
@@ -772,7 +821,7 @@ __device__ void StepConsumer::attend(const UnitDesc& d, const BundleHdr& hdr) {
             if (l < pi) {
                 if (spr > 1) {
                     if (d.span == 0) {
-                        char* orow = d.O + (long long)l * layer_bytes + lane * 4;
+                        char* orow = op + lane * 4;
                         for (int qi = 0; qi < nq; ++qi) {
                             float2 s2 = make_float2(0.f, 0.f);
                             for (int s = 0; s < spr; ++s) {
@@ -783,7 +832,8 @@ __device__ void StepConsumer::attend(const UnitDesc& d, const BundleHdr& hdr) {
                         }
                     }
                 } else {
-                    store_rows<NQ>(acc, op, nq, O_qstride);
+                    if (R == 1) stage_rows<NQ>(acc, nq, 1, 0);
+                    flush_rows(op, nq, R, O_qstride);
                 }
             }
         }
@@ -847,47 +897,51 @@ __global__ void __launch_bounds__(kStepWarps * 32, 1) decode_step_team_kernel(co
         unsigned cur = ((unsigned)blockIdx.x * kTeams + (unsigned)team) * kTeamWarps;
         unsigned nxt_chunk = chunk_for(dyn0);
         const unsigned nxt_raw0 = grab(nxt_chunk);
+        // Lane u * kUnitRows + hh works for head hh of the bundle's unit u: the lanes of a unit decode
+        // it alike, each issues the copy of its own head's rows.
+        constexpr int kCopyLanes = kTeamWarps * kUnitRows;
+        const int lu = lane / kUnitRows, hh = lane % kUnitRows;
         UnitIdx cur_ui;
-        unit_index(p, cur + (unsigned)lane, lane < (int)cur_chunk, &cur_ui);
+        unit_index(p, cur + (unsigned)lu, lu < (int)cur_chunk, &cur_ui);
         unsigned nxt = __shfl_sync(0xffffffffu, nxt_raw0, 0);
         while (cur < p.n_units && !pr.dead) {
             const unsigned aft_chunk = chunk_for(nxt);
             const unsigned aft_raw = grab(aft_chunk);                          // used at the end of the iteration
             UnitIdx nxt_ui;
-            unit_index(p, nxt + (unsigned)lane, lane < (int)nxt_chunk, &nxt_ui);
+            unit_index(p, nxt + (unsigned)lu, lu < (int)nxt_chunk, &nxt_ui);
             pr.ensure_slot();
             if (pr.dead) break;
             const int bslot = (int)(pr.n_bundles % kNS);
             ProdUnit pu;
             UnitDesc ud;
-            decode_unit(p, cur_ui, &pu, &ud);
+            decode_unit(p, cur_ui, hh == 0, &pu, &ud);
             // the bundle: tiles per plane, value layers, whether any row is split over spans
             int tiles = pu.tiles, layers = pu.pi, sync = pu.spr_log2;
 #pragma unroll
-            for (int o = kTeamWarps / 2; o > 0; o >>= 1) {
+            for (int o = 16; o > 0; o >>= 1) {
                 tiles = max(tiles, __shfl_xor_sync(0xffffffffu, tiles, o));
                 layers = max(layers, __shfl_xor_sync(0xffffffffu, layers, o));
                 sync = max(sync, __shfl_xor_sync(0xffffffffu, sync, o));
             }
-            tiles = __shfl_sync(0xffffffffu, tiles, 0); layers = __shfl_sync(0xffffffffu, layers, 0); sync = __shfl_sync(0xffffffffu, sync, 0);
             tiles = max(tiles, 1);
             if (lane == 0) *sp<BundleHdr>(sm.bundle_hdr(team, bslot)) = BundleHdr{tiles, layers, sync ? 1 : 0, 0};
-            if (lane < kTeamWarps) *sp<UnitDesc>(sm.unit_desc(team, bslot, lane)) = ud;
+            if (hh == 0 && lu < kTeamWarps) *sp<UnitDesc>(sm.unit_desc(team, bslot, lu)) = ud;
             __syncwarp();
             if (lane == 0) mbar_arrive(sm.bar_ready(team, bslot));     // the consumers may start on their small rows
             // ---- slots: the key tiles, then each layer's value tiles
+            const bool attn = lane < kCopyLanes && (pu.kind == UK_SELF || pu.kind == UK_ENC);
             for (int plane = 0; plane <= layers && !pr.dead; ++plane) {
                 for (int t = 0; t < tiles && !pr.dead; ++t) {
-                    const bool attn = lane < kTeamWarps && (pu.kind == UK_SELF || pu.kind == UK_ENC);
-                    const int r = (attn && plane <= pu.pi && t < pu.tiles) ? min(pu.tp, pu.n - t * pu.tp) : 0;
-                    int off = r;                                               // prefix sum over the unit lanes
+                    const int r = (attn && plane <= pu.pi && t < pu.tiles) ? min(pu.tp, pu.n - t * pu.tp) : 0;   // rows of one head
+                    // rows of the units before this one (a unit's lanes agree; only lanes hh == 0 are added up)
+                    int off = (hh == 0) ? r * pu.rows : 0;
 #pragma unroll
-                    for (int o = 1; o < kTeamWarps; o <<= 1) {
+                    for (int o = kUnitRows; o < kCopyLanes; o <<= 1) {
                         const int a = __shfl_up_sync(0xffffffffu, off, o);
-                        if ((lane & (kTeamWarps - 1)) >= o) off += a;
+                        if (lane >= o) off += a;
                     }
-                    const int tot = __shfl_sync(0xffffffffu, off, kTeamWarps - 1);
-                    off -= r;
+                    const int tot = __shfl_sync(0xffffffffu, off, kCopyLanes - kUnitRows);
+                    off = __shfl_sync(0xffffffffu, off, lu * kUnitRows) - r * pu.rows;
                     const uint32_t bytes = (uint32_t)tot * 128u;
                     pr.ensure_slot();
                     const uint32_t base = pr.alloc(bytes);
@@ -895,20 +949,21 @@ __global__ void __launch_bounds__(kStepWarps * 32, 1) decode_step_team_kernel(co
                     const int slot = (int)(pr.n_slots % kNS);
                     const uint32_t sd = sm.slot_desc(team, slot);
                     if (lane == 0) *sp<uint32_t>(sd) = base;
-                    if (lane < kTeamWarps) *sp<uint16_t>(sd + 4 + 2 * lane) = (uint16_t)off;
-                    // this step's row is not cached yet: its place in the tile is left for the consumer to fill
-                    const bool with_new = r > 0 && pu.new_row >= t * pu.tp && pu.new_row < t * pu.tp + r;
-                    const uint32_t cached = (uint32_t)(r - (with_new ? 1 : 0)) * 128u;
+                    if (hh == 0 && lu < kTeamWarps) *sp<uint16_t>(sd + 4 + 2 * lu) = (uint16_t)off;
+                    // this step's row is not cached yet: the consumer reads it from its own scratch rows
+                    const bool copies = r > 0 && hh < pu.rows;
+                    const bool with_new = copies && pu.new_row >= t * pu.tp && pu.new_row < t * pu.tp + r;
+                    const uint32_t cached = copies ? (uint32_t)(r - (with_new ? 1 : 0)) * 128u : 0u;
                     uint32_t tx = cached;
 #pragma unroll
-                    for (int o = kTeamWarps / 2; o > 0; o >>= 1) tx += __shfl_xor_sync(0xffffffffu, tx, o);
-                    tx = __shfl_sync(0xffffffffu, tx, 0);
+                    for (int o = 16; o > 0; o >>= 1) tx += __shfl_xor_sync(0xffffffffu, tx, o);
                     __syncwarp();
                     const uint32_t bar = sm.bar_full(team, slot);
                     if (lane == 0) mbar_expect_tx(bar, tx);
                     if (cached) {
-                        const char* src = (plane == 0 ? pu.srcK : pu.srcV + (long long)(plane - 1) * pu.plane_bytes) + (unsigned)(t * pu.tp) * 128u;
-                        bulk_g2s(sm.sm_base + base + (uint32_t)off * 128u, src, cached, bar);
+                        const char* src = (plane == 0 ? pu.srcK : pu.srcV + (long long)(plane - 1) * pu.plane_bytes) +
+                                          (unsigned long long)hh * pu.panel_bytes + (unsigned)(t * pu.tp) * 128u;
+                        bulk_g2s(sm.sm_base + base + (uint32_t)(off + hh * r) * 128u, src, cached, bar);
                     }
                     pr.issued();
                 }
