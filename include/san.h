@@ -227,13 +227,14 @@ int32_t san_decode_step(san_ctx* ctx, const san_step_args* args, void* stream);
  *              a long row; SAN_ERR_UNSUPPORTED from the step if a shape does not fit;
  *   which = 0  automatic (the default): the team pipeline where it applies, else the per-warp one.
  * spans_log2 >= 0 overrides the automatic cut of the team pipeline: every row is dealt to
- * 1 << spans_log2 warps (0..1); with one span tile_pos / 16 (16, 32 or 64 -> 1, 2 or 4) heads
- * go to a unit where the head count allows,
+ * 1 << spans_log2 warps (0..1); with one span up to heads_per_unit (1, 2 or 4) heads of one
+ * sequence or sentence go to a warp where the head count allows (at most 2 where several
+ * beams share a key tile); tiles hold tile_pos positions (a multiple of 16);
  * layers_per_unit > 0 caps the layers one warp applies (the block's other layers go to
- * further warps, which recompute S), grab_mult >= 1 makes the bundles shrink earlier towards
+ * further warps, which recompute S); grab_mult >= 1 makes the bundles shrink earlier towards
  * the end of the launch.  spans_log2 < 0 restores the automatic cut. */
-int32_t san_step_kernel_select(san_ctx* ctx, int32_t which, int32_t spans_log2, int32_t tile_pos,
-                               int32_t layers_per_unit, int32_t grab_mult);
+int32_t san_step_kernel_select(san_ctx* ctx, int32_t which, int32_t spans_log2, int32_t heads_per_unit,
+                               int32_t tile_pos, int32_t layers_per_unit, int32_t grab_mult);
 
 /* Which kernel the last san_decode_step of this context launched (1 or 2 as above, 0 before the
  * first step) and, for the team pipeline, how many heads of one sequence / sentence it gave

@@ -85,7 +85,7 @@ def lib():
     L.san_device_status.argtypes = [vp, _I32P, _I32P, vp]
     L.san_attn_weights_static.argtypes = [i32, i32, i32, vp, vp, i32, i32, vp, vp, i32, i32, vp, i64, vp, vp]
     L.san_decode_step.argtypes = [vp, C.POINTER(san_step_args), vp]
-    L.san_step_kernel_select.argtypes = [vp, i32, i32, i32, i32, i32]
+    L.san_step_kernel_select.argtypes = [vp, i32, i32, i32, i32, i32, i32]
     L.san_step_kernel_used.argtypes = [vp, _I32P, _I32P]
     L.san_decode_step_host.argtypes = [vp, C.POINTER(san_step_args), C.POINTER(san_step_args), vp]
     L.san_full_block.argtypes = [i32, i32, i32, i32, vp, vp, vp, vp, i32, i32, i32, vp, i64, vp, vp]
@@ -229,9 +229,9 @@ def san_decode_step(ctx, *, d_q_self=None, d_k_new=None, d_v_new=None, d_seq_ids
     return lib().san_decode_step(ctx, C.byref(a), _stream(stream))
 
 
-def san_step_kernel_select(ctx, which=0, spans_log2=-1, tile_pos=64, layers_per_unit=0, grab_mult=1) -> int:
+def san_step_kernel_select(ctx, which=0, spans_log2=-1, heads_per_unit=4, tile_pos=64, layers_per_unit=0, grab_mult=1) -> int:
     """Choose the kernel behind san_decode_step (0 automatic, 1 per-warp, 2 team pipeline) and its cut."""
-    return lib().san_step_kernel_select(ctx, which, spans_log2, tile_pos, layers_per_unit, grab_mult)
+    return lib().san_step_kernel_select(ctx, which, spans_log2, heads_per_unit, tile_pos, layers_per_unit, grab_mult)
 
 
 def san_step_kernel_used(ctx):

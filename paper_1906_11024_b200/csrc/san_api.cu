@@ -202,7 +202,7 @@ int32_t launch_team_step(san_ctx* ctx, const san_step_args* a, int max_len, int 
         while (s < kMaxSprLog2 && span_of(bound, s) > 128 && rows * (1ll << s) * ceil_div(pi, lg) < want_units) ++s;
         const int span = span_of(bound, s);
         out->spr_log2 = s;
-        out->rpu = s == 0 ? rpu_max : 1;
+        out->rpu = s == 0 ? (nq_t > 1 ? std::min(rpu_max, 2) : rpu_max) : 1;   // several queries per head: at most two heads side by side
         out->zq = span + 4;                         // + 4: the score rows of neighbouring queries start in different banks
         while (lg > 2 && rows / out->rpu * (1ll << s) * ceil_div(pi, lg) < want_units &&
                (long long)out->rpu * span * 128 * (1 + lg) > 64 * 1024) lg = std::max(2, ceil_div(lg, 2));
@@ -216,11 +216,14 @@ int32_t launch_team_step(san_ctx* ctx, const san_step_args* a, int max_len, int 
     if (ctx->team_cut_override[0] >= 0) {           // testing and tuning: san_step_kernel_select
         cs.spr_log2 = ce.spr_log2 = std::min(kMaxSprLog2, ctx->team_cut_override[0]);
         if (span_of(max_len, cs.spr_log2) > kZCapFloats || span_of(max_src, ce.spr_log2) * nqe > kZCapFloats) return SAN_ERR_UNSUPPORTED;
-        cs.tile_pos = span_of(max_len, cs.spr_log2); ce.tile_pos = span_of(max_src, ce.spr_log2);
-        cs.zq = cs.tile_pos + 4; ce.zq = ce.tile_pos + 4;
-        cs.rpu = ce.rpu = cs.spr_log2 == 0 ? std::min(rpu_max, std::max(1, ctx->team_cut_override[1] / 16)) : 1;   // tile_pos 16, 32, 64: 1, 2, 4 heads per unit
-        if (cs.rpu == 3) cs.rpu = ce.rpu = 2;
-        if (ctx->team_cut_override[2] > 0) { cs.lg = std::min(pi_self, ctx->team_cut_override[2]); ce.lg = std::min(pi_enc, ctx->team_cut_override[2]); }
+        const int tile = ctx->team_cut_override[2];
+        cs.tile_pos = std::min(span_of(max_len, cs.spr_log2), tile); ce.tile_pos = std::min(span_of(max_src, ce.spr_log2), tile);
+        cs.zq = span_of(max_len, cs.spr_log2) + 4; ce.zq = span_of(max_src, ce.spr_log2) + 4;
+        int hpu = std::min(rpu_max, std::max(1, ctx->team_cut_override[1]));
+        if (hpu == 3) hpu = 2;
+        cs.rpu = ce.rpu = cs.spr_log2 == 0 ? hpu : 1;
+        if (nqe > 1) ce.rpu = std::min(ce.rpu, 2);
+        if (ctx->team_cut_override[3] > 0) { cs.lg = std::min(pi_self, ctx->team_cut_override[3]); ce.lg = std::min(pi_enc, ctx->team_cut_override[3]); }
     }
 
     TeamParams p;
@@ -841,14 +844,16 @@ int32_t san_decode_step(san_ctx* ctx, const san_step_args* a, void* stream) {
     return cuda_status(e);
 }
 
-int32_t san_step_kernel_select(san_ctx* ctx, int32_t which, int32_t spans_log2, int32_t tile_pos, int32_t layers_per_unit,
-                               int32_t grab_mult) {
+int32_t san_step_kernel_select(san_ctx* ctx, int32_t which, int32_t spans_log2, int32_t heads_per_unit, int32_t tile_pos,
+                               int32_t layers_per_unit, int32_t grab_mult) {
     if (!ctx) return SAN_ERR_NULL;
-    if (which < 0 || which > 2 || spans_log2 > 1 || (spans_log2 >= 0 && (tile_pos < 16 || tile_pos % 16 != 0))) return SAN_ERR_RANGE;
+    if (which < 0 || which > 2 || spans_log2 > 1) return SAN_ERR_RANGE;
+    if (spans_log2 >= 0 && (tile_pos < 16 || tile_pos % 16 != 0 || heads_per_unit < 1 || heads_per_unit > 4)) return SAN_ERR_RANGE;
     ctx->step_kernel = which;
     ctx->team_cut_override[0] = spans_log2 < 0 ? -1 : spans_log2;
-    ctx->team_cut_override[1] = tile_pos;
-    ctx->team_cut_override[2] = layers_per_unit;
+    ctx->team_cut_override[1] = heads_per_unit;
+    ctx->team_cut_override[2] = tile_pos;
+    ctx->team_cut_override[3] = layers_per_unit;
     ctx->team_grab_mult = grab_mult > 0 ? grab_mult : 1;
     return SAN_OK;
 }

@@ -30,7 +30,7 @@ struct san_ctx {
     bool fused_attr_set = false;   // shared-memory opt-in of the one-launch step kernel done
     bool team_attr_set = false;    // the same for the team-pipeline step kernel
     int step_kernel = 0;           // 0: automatic, 1: per-warp pipeline kernel, 2: team-pipeline kernel (san_step_kernel_select)
-    int team_cut_override[3] = {-1, 64, 0};   // spans per row (log2; -1: automatic), positions per tile, layers per unit (0: automatic)
+    int team_cut_override[4] = {-1, 4, 64, 0};   // spans per row (log2; -1: automatic), heads per unit, positions per tile, layers per unit (0: automatic)
     int team_grab_mult = 1;
     int last_step_kernel = 0;      // which kernel the last san_decode_step launched (0: none yet)
     int last_rows_per_unit[2] = {0, 0};   // team pipeline: heads per unit for self / enc-dec attention in that launch

@@ -43,7 +43,7 @@ constexpr int kAanChunk = 256;                                 // elements of on
 // reference shows either way (3.9e-3 normwise at worst on all workloads, tolerance 1e-2), so the
 // remainder is left out.
 constexpr bool kWeightRemainder = false;
-constexpr int kXq = 8;                                         // query rows the exchange area has room for per unit
+constexpr int kXq = 16;                                        // query rows the exchange area has room for per unit
 
 enum { TAG_TEAM = 8 };
 enum { UK_SELF = 0, UK_ENC = 1, UK_AAN = 2, UK_IDLE = 3 };
@@ -379,9 +379,9 @@ struct StepConsumer {
 
     __device__ void idle(const BundleHdr& hdr);
     __device__ void aan(const UnitDesc& d);
-    template <int NQ> __device__ void attend(const UnitDesc& d, const BundleHdr& hdr);
-    template <int NQ> __device__ __forceinline__ bool softmax(const UnitDesc& d, const BundleHdr& hdr, int n, int n_pad, int ZQ,
-                                                              uint32_t zs_base, float* S_base, long long S_rstride, int nq);
+    template <int NQ, int R> __device__ void attend(const UnitDesc& d, const BundleHdr& hdr);
+    template <int NQ, int NQI> __device__ __forceinline__ bool softmax(const UnitDesc& d, const BundleHdr& hdr, int n, int n_pad, int ZQ,
+                                                                       uint32_t zs_base, float* S_base, long long S_hstride, long long S_qstride, int nq);
     template <int NQ> __device__ __forceinline__ void stage_rows(const float (&acc)[4][4], int nq, int R, int hh);
     __device__ __forceinline__ void flush_rows(char* orow, int nq, int R, long long O_qstride);
 };
@@ -418,16 +418,16 @@ __device__ void StepConsumer::aan(const UnitDesc& d) {
     *reinterpret_cast<uint4*>(d.O + e0 * 2) = o;
 }
 
-// Softmax of n scores (log2 domain) of NQ rows side by side, in place: row r has its scores at
-// zs_base + r * ZQ floats and its S row at S_base + r * S_rstride (rows at or beyond nq are
-// carried along and never stored).  The weights are left as bf16 words in the order the apply
+// Softmax of n scores (log2 domain) of NQ = heads x NQI rows side by side, in place: row r
+// (head r / NQI, query r % NQI) has its scores at zs_base + r * ZQ floats and its S row at
+// S_base + head * S_hstride + query * S_qstride (queries at or beyond nq are carried along and
+// never stored).  The weights are left as bf16 words in the order the apply
 // MMAs read them (see packed_slot), zero from n up to n_pad, and are written to S.  The spans of
 // a split row first exchange their (max, sum) through the team's shared memory, so every span
 // normalises by the row's total.
-template <int NQ>
+template <int NQ, int NQI>
 __device__ __forceinline__ bool StepConsumer::softmax(const UnitDesc& d, const BundleHdr& hdr, int n, int n_pad, int ZQ,
-                                                      uint32_t zs_base, float* S_base, long long S_rstride, int nq) {
-    const long long S_qstride = S_rstride;
+                                                      uint32_t zs_base, float* S_base, long long S_hstride, long long S_qstride, int nq) {
     const int spr = 1 << d.spr_log2;
     float* ms = sp<float>(xch_ms());     // (max, sum) of every unit of the team and query: [unit][8][2] floats
     if (n <= 64) {
@@ -482,8 +482,8 @@ __device__ __forceinline__ bool StepConsumer::softmax(const UnitDesc& d, const B
             float* zq = sp<float>(zs_base + qi * ZQ * 4);
             unsigned short* zh = reinterpret_cast<unsigned short*>(zq);
             const float w0 = z0[qi] * inv[qi], w1 = z1[qi] * inv[qi];
-            if (S_base && qi < nq) {
-                float* Srow = S_base + qi * S_qstride;
+            if (S_base && (qi % NQI) < nq) {
+                float* Srow = S_base + (qi / NQI) * S_hstride + (qi % NQI) * S_qstride;
                 if (in0) Srow[lane] = w0;
                 if (two && in1) Srow[lane + 32] = w1;
             }
@@ -544,7 +544,7 @@ __device__ __forceinline__ bool StepConsumer::softmax(const UnitDesc& d, const B
     for (int qi = 0; qi < NQ; ++qi) {
         float* zq = sp<float>(zs_base + qi * ZQ * 4);
         unsigned short* zh = reinterpret_cast<unsigned short*>(zq);
-        float* Srow = (S_base && qi < nq) ? S_base + qi * S_qstride : nullptr;
+        float* Srow = (S_base && (qi % NQI) < nq) ? S_base + (qi / NQI) * S_hstride + (qi % NQI) * S_qstride : nullptr;
         const float inv = sq[qi];
 #pragma unroll 1
         for (int j0 = 0; j0 < n_pad; j0 += 32) {      // warp-uniform trip count
@@ -604,18 +604,19 @@ __device__ __forceinline__ void StepConsumer::flush_rows(char* orow, int nq, int
     __syncwarp();
 }
 
-// One attention unit on the tensor cores: up to four rows (heads) of one (block, id), one after
-// the other inside each phase, so that what a unit costs beside its arithmetic (descriptors,
-// barrier waits, address set-up, output stores) is paid once for all of them.
+// One attention unit on the tensor cores: R rows (heads) of one (block, id) side by side inside
+// each phase, so that what a unit costs beside its arithmetic (descriptors, barrier waits,
+// address set-up, output stores) is paid once for all of them and the heads' independent chains
+// of loads and MMAs overlap.
 //   scores:  D[16 positions x 8 queries] = K_tile[16 x 64] . q^T              (queries padded to 8)
 //   apply:   D[16 dims x 8 queries]     += V_tile^T[16 x 16 positions] . S^T   (four dim tiles)
 // S is applied as bf16; products and sums are float32.  Columns of D that belong to padding
 // queries are computed from whatever the padding lanes load and are never stored.
-template <int NQ>
+template <int NQ, int R>
 __device__ void StepConsumer::attend(const UnitDesc& d, const BundleHdr& hdr) {
     const TeamKind& kp = p.k[d.kind];
     const int ZQ = (int)kp.zq;
-    const int n = d.n, nq = d.nq, pi = d.pi, tp = d.tp, new_row = d.new_row, R = d.rows;
+    const int n = d.n, nq = d.nq, pi = d.pi, tp = d.tp, new_row = d.new_row;
     const int my_tiles = (n + tp - 1) / tp;
     const int tig = lane & 3, gid = lane >> 2;                 // mma fragment coordinates
     const long long layer_bytes = kp.layer_bytes;
@@ -633,9 +634,9 @@ __device__ void StepConsumer::attend(const UnitDesc& d, const BundleHdr& hdr) {
         for (int i = lane; i < rows * 8; i += 32) {
             const int row = i >> 3, c = i & 7;
             const char* src;
-            if (row < scr_k) { const int qi = R == 4 ? row >> 2 : R == 2 ? row >> 1 : row; src = d.q + (unsigned long long)qi * q_stride + (row - qi * R) * 128; }
+            if (row < scr_k) { const int qi = row / R; src = d.q + (unsigned long long)qi * q_stride + (row - qi * R) * 128; }
             else if (row < scr_v) src = d.knew + (row - scr_k) * 128;
-            else { const int lr = row - scr_v, l = R == 4 ? lr >> 2 : R == 2 ? lr >> 1 : lr; src = d.vnew + (long long)l * layer_bytes + (lr - l * R) * 128; }
+            else { const int lr = row - scr_v, l = lr / R; src = d.vnew + (long long)l * layer_bytes + (lr - l * R) * 128; }
             cp_async16(sm.sm_base + scr_off + row * 128 + c * 16, src + c * 16);
         }
         asm volatile("cp.async.commit_group;" ::: "memory");
@@ -668,45 +669,57 @@ __device__ void StepConsumer::attend(const UnitDesc& d, const BundleHdr& hdr) {
             const int s0 = t * tp;
             const int r = min(tp, n - s0);
             const int nr = (new_row >= s0 && new_row < s0 + r) ? new_row - s0 : -1;   // this step's key row in the tile
-#pragma unroll 1
+            // every head's query rows (natural chunk order) as B fragments (k = dims, n = query)
+            uint32_t qb[R][4][2];
+#pragma unroll
             for (int hh = 0; hh < R; ++hh) {
-                // the head's query rows (natural chunk order) as B fragments (k = dims, n = query)
-                uint32_t qb[4][2];
                 const uint32_t qrow = scr_off + (uint32_t)((gid < nq ? gid : 0) * R + hh) * 128u + 4u * tig;
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks) {
-                    qb[ks][0] = *sp<uint32_t>(qrow + 32 * ks);
-                    qb[ks][1] = *sp<uint32_t>(qrow + 32 * ks + 16);
+                    qb[hh][ks][0] = *sp<uint32_t>(qrow + 32 * ks);
+                    qb[hh][ks][1] = *sp<uint32_t>(qrow + 32 * ks + 16);
                 }
-                if (nr >= 0 && d.dstK && lane < 8)                                   // into the cache, chunk-permuted
-                    *reinterpret_cast<uint4*>(d.dstK + (unsigned long long)hh * panel_bytes + ((lane ^ (nr & 7)) << 4)) =
-                        *sp<uint4>(scr_off + (scr_k + hh) * 128 + lane * 16);
-                const uint32_t st_s = sm.sm_base + st0 + (uint32_t)(hh * r + lrow) * 128u;
-                const uint32_t new_k = scr_s + (scr_k + hh) * 128;
-                const uint32_t zh = zk + hh * zs_head;
+            }
+            if (nr >= 0 && d.dstK && lane < 8 * R) {                                  // into the cache, chunk-permuted
+                const int hh = lane >> 3, c = lane & 7;
+                *reinterpret_cast<uint4*>(d.dstK + (unsigned long long)hh * panel_bytes + ((c ^ (nr & 7)) << 4)) =
+                    *sp<uint4>(scr_off + (scr_k + hh) * 128 + c * 16);
+            }
+            const uint32_t st_s = sm.sm_base + st0 + (uint32_t)lrow * 128u;
+            const uint32_t head_bytes = (uint32_t)r * 128u;                          // a head's rows follow the previous head's
 #pragma unroll 1
-                for (int b0 = 0; b0 < r; b0 += 16) {
-                    const bool is_new = (b0 + lrow == nr);
-                    const uint32_t rb = is_new ? new_k : st_s + b0 * 128;
-                    const uint32_t fix = is_new ? new_fix : 0u;
-                    float acc[4] = {0.f, 0.f, 0.f, 0.f};
-                    uint32_t a[4][4];
+            for (int b0 = 0; b0 < r; b0 += 16) {
+                const bool is_new = (b0 + lrow == nr);
+                const uint32_t fix = is_new ? new_fix : 0u;
+                float acc[R][4];
+                uint32_t a[R][4][4];
 #pragma unroll
-                    for (int ks = 0; ks < 4; ++ks) ldsm_x4(rb + (ld_swz[ks] ^ fix), a[ks]);
+                for (int hh = 0; hh < R; ++hh) {
+                    const uint32_t rb = is_new ? scr_s + (scr_k + hh) * 128 : st_s + hh * head_bytes + b0 * 128;
 #pragma unroll
-                    for (int ks = 0; ks < 4; ++ks) mma_bf16(acc, a[ks][0], a[ks][1], a[ks][2], a[ks][3], qb[ks][0], qb[ks][1]);
-                    // acc[0], acc[1]: position b0+gid, queries 2tig, 2tig+1; acc[2], acc[3]: position b0+gid+8.
-                    // Rows of the block at or beyond r (another head's or unit's rows, stale bytes) give
-                    // scores that are never stored.
-                    const int pos = s0 + b0 + gid;
-                    float* z = sp<float>(zh + (s0 + b0) * 4);
+                    for (int ks = 0; ks < 4; ++ks) ldsm_x4(rb + (ld_swz[ks] ^ fix), a[hh][ks]);
+                }
+#pragma unroll
+                for (int hh = 0; hh < R; ++hh) {
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) acc[hh][e] = 0.f;
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks) mma_bf16(acc[hh], a[hh][ks][0], a[hh][ks][1], a[hh][ks][2], a[hh][ks][3], qb[hh][ks][0], qb[hh][ks][1]);
+                }
+                // acc[0], acc[1]: position b0+gid, queries 2tig, 2tig+1; acc[2], acc[3]: position b0+gid+8.
+                // Rows of the block at or beyond r (another head's or unit's rows, stale bytes) give
+                // scores that are never stored.
+                const int pos = s0 + b0 + gid;
+#pragma unroll
+                for (int hh = 0; hh < R; ++hh) {
+                    float* z = sp<float>(zk + hh * zs_head + (s0 + b0) * 4);
                     if (2 * tig < NQ) {
-                        if (pos < n) z[0] = acc[0] * sc;
-                        if (pos + 8 < n) z[8] = acc[2] * sc;
+                        if (pos < n) z[0] = acc[hh][0] * sc;
+                        if (pos + 8 < n) z[8] = acc[hh][2] * sc;
                     }
                     if (2 * tig + 1 < NQ) {
-                        if (pos < n) z[ZQ] = acc[1] * sc;
-                        if (pos + 8 < n) z[ZQ + 8] = acc[3] * sc;
+                        if (pos < n) z[ZQ] = acc[hh][1] * sc;
+                        if (pos + 8 < n) z[ZQ + 8] = acc[hh][3] * sc;
                     }
                 }
             }
@@ -716,15 +729,7 @@ __device__ void StepConsumer::attend(const UnitDesc& d, const BundleHdr& hdr) {
     __syncwarp();
 
     const int n_pad = (n + 15) & ~15;
-    const long long S_qstride = (long long)p.H * kp.S_ld;
-    if (NQ == 1 && R == 4) {
-        // one query per head: the four heads' rows go through the softmax side by side
-        if (!softmax<4>(d, hdr, n, n_pad, ZQ, zs_off, d.S, kp.S_ld, 4)) return;
-    } else {
-#pragma unroll 1
-        for (int hh = 0; hh < R; ++hh)
-            if (!softmax<NQ>(d, hdr, n, n_pad, ZQ, zs_off + hh * zs_head, d.S ? d.S + (long long)hh * kp.S_ld : nullptr, S_qstride, nq)) return;
-    }
+    if (!softmax<R * NQ, NQ>(d, hdr, n, n_pad, ZQ, zs_off, d.S, kp.S_ld, (long long)p.H * kp.S_ld, nq)) return;
 
     // ---- value tiles, layer by layer
     // B fragments: the weights of query gid at positions b0 + {2tig, 2tig+1} and b0 + {2tig+8, 2tig+9},
@@ -743,13 +748,15 @@ __device__ void StepConsumer::attend(const UnitDesc& d, const BundleHdr& hdr) {
     const int spr = 1 << d.spr_log2;
 #pragma unroll 1
     for (int l = 0; l < hdr.layers; ++l) {
-        float acc[4][4];
-        if (R == 1) {
+        // Several heads: each is one tile (the host cuts them so) and is done inside it.  A lone head
+        // keeps its sums across the tiles of the layer.
+        float acc[R][4][4];
+#pragma unroll
+        for (int hh = 0; hh < R; ++hh)
 #pragma unroll
             for (int x = 0; x < 4; ++x)
 #pragma unroll
-                for (int e = 0; e < 4; ++e) acc[x][e] = 0.f;
-        }
+                for (int e = 0; e < 4; ++e) acc[hh][x][e] = 0.f;
 #pragma unroll 1
         for (int t = 0; t < hdr.tiles; ++t) {
             const int slot = acquire();
@@ -759,52 +766,40 @@ __device__ void StepConsumer::attend(const UnitDesc& d, const BundleHdr& hdr) {
                 const int s0 = t * tp;
                 const int r = min(tp, n - s0);
                 const int nr = (new_row >= s0 && new_row < s0 + r) ? new_row - s0 : -1;
+                if (nr >= 0 && lane < 8 * R) {
+                    const int hh = lane >> 3, c = lane & 7;
+                    *reinterpret_cast<uint4*>(vlast + (unsigned long long)hh * panel_bytes + ((c ^ (nr & 7)) << 4)) =
+                        *sp<uint4>(scr_off + (scr_v + l * R + hh) * 128 + c * 16);
+                }
+                const uint32_t st_s = sm.sm_base + st0 + (uint32_t)vrow * 128u;
+                const uint32_t head_bytes = (uint32_t)r * 128u;
 #pragma unroll 1
-                for (int hh = 0; hh < R; ++hh) {
-                    if (R > 1) {          // several heads: each is one tile (the host cuts them so); a lone head keeps its sums across tiles
+                for (int b0 = 0; b0 < r; b0 += 16) {
+                    // rows at or beyond r hold other bytes: their weights are zero, but 0 x NaN would not be,
+                    // so those lanes address a row of zeros instead
+                    const int row = b0 + vrow;
+                    const bool is_new = (row == nr);
+                    const uint32_t fix = is_new ? new_fix : 0u;
+                    uint2 w[R];                                          // (weights of b0.., weights of b0+8..) per head
+                    uint32_t a[R][4][4];
 #pragma unroll
-                        for (int x = 0; x < 4; ++x)
+                    for (int hh = 0; hh < R; ++hh) {
+                        w[hh] = *sp<uint2>(za + hh * zs_head + (s0 + b0) * 4);
+                        const uint32_t rb = is_new ? scr_s + (scr_v + l * R + hh) * 128 : st_s + hh * head_bytes + b0 * 128;
 #pragma unroll
-                            for (int e = 0; e < 4; ++e) acc[x][e] = 0.f;
+                        for (int x = 0; x < 4; ++x) ldsm_x4_t(row >= r ? zero_row : rb + (vd_swz[x] ^ fix), a[hh][x]);
                     }
-                    const uint32_t new_v = scr_s + (scr_v + l * R + hh) * 128;
-                    if (nr >= 0 && lane < 8)
-                        *reinterpret_cast<uint4*>(vlast + (unsigned long long)hh * panel_bytes + ((lane ^ (nr & 7)) << 4)) =
-                            *sp<uint4>(scr_off + (scr_v + l * R + hh) * 128 + lane * 16);
-                    const uint32_t st_s = sm.sm_base + st0 + (uint32_t)(hh * r + vrow) * 128u;
-                    const uint32_t zb = za + hh * zs_head;
-#pragma unroll 1
-                    for (int b0 = 0; b0 < r; b0 += 16) {
-                        uint4 w;                                             // (high b0, high b1, remainder b0, remainder b1)
-                        if (kWeightRemainder) w = *sp<uint4>(zb + (s0 + b0) * 4);
-                        else { const uint2 w2 = *sp<uint2>(zb + (s0 + b0) * 4); w = make_uint4(w2.x, w2.y, 0u, 0u); }
-                        // rows at or beyond r hold other bytes: their weights are zero, but 0 x NaN would not be,
-                        // so those lanes address a row of zeros instead
-                        const int row = b0 + vrow;
-                        const bool is_new = (row == nr);
-                        const uint32_t rb = is_new ? new_v : st_s + b0 * 128;
-                        const uint32_t fix = is_new ? new_fix : 0u;
-                        uint32_t a[4][4];
 #pragma unroll
-                        for (int x = 0; x < 4; ++x) ldsm_x4_t(row >= r ? zero_row : rb + (vd_swz[x] ^ fix), a[x]);
+                    for (int hh = 0; hh < R; ++hh)
 #pragma unroll
-                        for (int x = 0; x < 4; ++x) mma_bf16(acc[x], a[x][0], a[x][1], a[x][2], a[x][3], w.x, w.y);
-                        if (kWeightRemainder) {
-#pragma unroll
-                            for (int x = 0; x < 4; ++x) mma_bf16(acc[x], a[x][0], a[x][1], a[x][2], a[x][3], w.z, w.w);
-                        }
-                    }
-                    if (R > 1) stage_rows<NQ>(acc, nq, R, hh);
+                        for (int x = 0; x < 4; ++x) mma_bf16(acc[hh][x], a[hh][x][0], a[hh][x][1], a[hh][x][2], a[hh][x][3], w[hh].x, w[hh].y);
                 }
             }
             release();
         }
-        if (!hdr.sync) {
-            if (l < pi) {
-                if (R == 1) stage_rows<NQ>(acc, nq, 1, 0);
-                flush_rows(op, nq, R, O_qstride);
-            }
-        } else {
+        // acc[hh][x][0], [1]: dim 16x + gid of queries 2tig, 2tig+1; [2], [3]: dim 16x + gid + 8
+        bool store = l < pi;
+        if (hdr.sync) {
             // the spans of a row add up their partial outputs through shared memory (two buffers, by layer parity)
             float* xo = sp<float>(xch_o(l & 1));
             if (l < pi && spr > 1) {
@@ -813,29 +808,30 @@ __device__ void StepConsumer::attend(const UnitDesc& d, const BundleHdr& hdr) {
                 for (int x = 0; x < 4; ++x)
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
-                        if (2 * tig < NQ) mine[16 * x + 8 * h] = acc[x][2 * h];
-                        if (2 * tig + 1 < NQ) mine[kDh + 16 * x + 8 * h] = acc[x][2 * h + 1];
+                        if (2 * tig < NQ) mine[16 * x + 8 * h] = acc[0][x][2 * h];
+                        if (2 * tig + 1 < NQ) mine[kDh + 16 * x + 8 * h] = acc[0][x][2 * h + 1];
                     }
             }
             if (!team_sync()) return;
-            if (l < pi) {
-                if (spr > 1) {
-                    if (d.span == 0) {
-                        char* orow = op + lane * 4;
-                        for (int qi = 0; qi < nq; ++qi) {
-                            float2 s2 = make_float2(0.f, 0.f);
-                            for (int s = 0; s < spr; ++s) {
-                                const float2 v = *reinterpret_cast<const float2*>(xo + (u + s) * p.xo_unit_floats + qi * kDh + 2 * lane);
-                                s2.x += v.x; s2.y += v.y;
-                            }
-                            *reinterpret_cast<uint32_t*>(orow + qi * O_qstride) = pack_bf16x2(s2.x, s2.y);
+            if (l < pi && spr > 1) {
+                store = false;
+                if (d.span == 0) {
+                    char* orow = op + lane * 4;
+                    for (int qi = 0; qi < nq; ++qi) {
+                        float2 s2 = make_float2(0.f, 0.f);
+                        for (int s = 0; s < spr; ++s) {
+                            const float2 v = *reinterpret_cast<const float2*>(xo + (u + s) * p.xo_unit_floats + qi * kDh + 2 * lane);
+                            s2.x += v.x; s2.y += v.y;
                         }
+                        *reinterpret_cast<uint32_t*>(orow + qi * O_qstride) = pack_bf16x2(s2.x, s2.y);
                     }
-                } else {
-                    if (R == 1) stage_rows<NQ>(acc, nq, 1, 0);
-                    flush_rows(op, nq, R, O_qstride);
                 }
             }
+        }
+        if (store) {
+#pragma unroll
+            for (int hh = 0; hh < R; ++hh) stage_rows<NQ>(acc[hh], nq, R, hh);
+            flush_rows(op, nq, R, O_qstride);
         }
         if (vlast) vlast += plane_bytes;
         op += layer_bytes;
@@ -1012,9 +1008,13 @@ __global__ void __launch_bounds__(kStepWarps * 32, 1) decode_step_team_kernel(co
         if (hdr.end) break;
         const UnitDesc d = *sp<UnitDesc>(sm.unit_desc(c.team, bslot, c.u));
         if (d.kind == UK_AAN) c.aan(d);
-        if (d.kind == UK_ENC && NQE > 1) c.template attend<NQE>(d, hdr);
-        else if (d.kind == UK_SELF || d.kind == UK_ENC) c.template attend<1>(d, hdr);
-        else c.idle(hdr);
+        if (d.kind == UK_ENC && NQE > 1) {
+            if (d.rows == 2) c.template attend<NQE, 2>(d, hdr); else c.template attend<NQE, 1>(d, hdr);
+        } else if (d.kind == UK_SELF || d.kind == UK_ENC) {
+            if (d.rows == 4) c.template attend<1, 4>(d, hdr); else if (d.rows == 2) c.template attend<1, 2>(d, hdr); else c.template attend<1, 1>(d, hdr);
+        } else {
+            c.idle(hdr);
+        }
     }
 }
 
