@@ -225,7 +225,8 @@ int32_t san_decode_step(san_ctx* ctx, const san_step_args* args, void* stream);
  *   which = 2  team pipeline (bf16): four producer warps each stream bundles of two units to a team
  *              of two warps, a unit being up to four heads of one sequence or one of two spans of
  *              a long row; SAN_ERR_UNSUPPORTED from the step if a shape does not fit;
- *   which = 0  automatic (the default): the team pipeline where it applies, else the per-warp one.
+ *   which = 0  automatic (the default): the team pipeline for steps whose rows are long enough to be
+ *              split over the warps of a team (where it measured faster), else the per-warp one.
  * spans_log2 >= 0 overrides the automatic cut of the team pipeline: every row is dealt to
  * 1 << spans_log2 warps (0..1); with one span up to heads_per_unit (1, 2 or 4) heads of one
  * sequence or sentence go to a warp where the head count allows (at most 2 where several

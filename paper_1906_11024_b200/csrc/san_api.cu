@@ -169,7 +169,8 @@ constexpr size_t kStepSmemTotal = 232448;      // opt-in shared memory per CTA o
 
 struct TeamCut { int spr_log2, lg, tile_pos, zq, rpu; };
 
-int32_t launch_team_step(san_ctx* ctx, const san_step_args* a, int max_len, int max_src, cudaStream_t st, int* rows_per_unit) {
+int32_t launch_team_step(san_ctx* ctx, const san_step_args* a, int max_len, int max_src, cudaStream_t st, int* rows_per_unit,
+                         bool only_if_split) {
     const san_config& c = ctx->cfg;
     if (c.dtype != SAN_BF16) return SAN_ERR_UNSUPPORTED;
     const bool aan = c.self_is_aan != 0;
@@ -214,17 +215,30 @@ int32_t launch_team_step(san_ctx* ctx, const san_step_args* a, int max_len, int 
     if (do_self && !cut(rows_self, max_len, pi_self, 1, &cs)) return SAN_ERR_UNSUPPORTED;
     if (do_enc && !cut(rows_enc, max_src, pi_enc, nqe, &ce)) return SAN_ERR_UNSUPPORTED;
     if (ctx->team_cut_override[0] >= 0) {           // testing and tuning: san_step_kernel_select
-        cs.spr_log2 = ce.spr_log2 = std::min(kMaxSprLog2, ctx->team_cut_override[0]);
-        if (span_of(max_len, cs.spr_log2) > kZCapFloats || span_of(max_src, ce.spr_log2) * nqe > kZCapFloats) return SAN_ERR_UNSUPPORTED;
-        const int tile = ctx->team_cut_override[2];
-        cs.tile_pos = std::min(span_of(max_len, cs.spr_log2), tile); ce.tile_pos = std::min(span_of(max_src, ce.spr_log2), tile);
-        cs.zq = span_of(max_len, cs.spr_log2) + 4; ce.zq = span_of(max_src, ce.spr_log2) + 4;
-        int hpu = std::min(rpu_max, std::max(1, ctx->team_cut_override[1]));
-        if (hpu == 3) hpu = 2;
-        cs.rpu = ce.rpu = cs.spr_log2 == 0 ? hpu : 1;
-        if (nqe > 1) ce.rpu = std::min(ce.rpu, 2);
-        if (ctx->team_cut_override[3] > 0) { cs.lg = std::min(pi_self, ctx->team_cut_override[3]); ce.lg = std::min(pi_enc, ctx->team_cut_override[3]); }
+        // each value may carry a second one for encoder-decoder attention in its bits 8 and up (absent: the same)
+        auto pick = [](int v, bool enc) { return enc && (v >> 8) > 0 ? (v >> 8) - 1 : (v & 255); };
+        auto apply = [&](TeamCut& tc, bool enc, int bound, int pi, int nq_t) -> bool {
+            tc.spr_log2 = std::min(kMaxSprLog2, pick(ctx->team_cut_override[0], enc));
+            const int span = span_of(bound, tc.spr_log2);
+            if (span * nq_t > kZCapFloats) return false;
+            tc.tile_pos = std::min(span, std::max(16, pick(ctx->team_cut_override[2], enc)));
+            tc.zq = span + 4;
+            int hpu = std::min(rpu_max, std::max(1, pick(ctx->team_cut_override[1], enc)));
+            if (hpu == 3) hpu = 2;
+            tc.rpu = tc.spr_log2 == 0 ? hpu : 1;
+            if (nq_t > 1) tc.rpu = std::min(tc.rpu, 2);
+            const int lg = pick(ctx->team_cut_override[3], enc);
+            if (lg > 0) tc.lg = std::min(pi, lg);
+            return true;
+        };
+        if (!apply(cs, false, max_len, pi_self, 1) || !apply(ce, true, max_src, pi_enc, nqe)) return SAN_ERR_UNSUPPORTED;
     }
+
+    // Measured on B200 (bench.py, all five workloads): where no row is long enough to be split over
+    // the warps of a team, the per-warp kernel is as fast or faster (its 16 warps per SM each
+    // carry one row; here 8 consumer warps carry up to four), so the automatic choice keeps
+    // this kernel for steps with split rows.
+    if (only_if_split && !((do_self && cs.spr_log2 > 0) || (do_enc && ce.spr_log2 > 0))) return SAN_ERR_UNSUPPORTED;
 
     TeamParams p;
     std::memset(&p, 0, sizeof(p));
@@ -640,8 +654,9 @@ int32_t san_decode_step(san_ctx* ctx, const san_step_args* a, void* stream) {
     if (n_seqs == 0 && n_sent == 0) return SAN_OK;
 
     const bool bf16 = c.dtype == SAN_BF16;
-    if (ctx->step_kernel != 1) {       // the team-pipeline kernel takes every bf16 shape that fits its shared memory
-        const int32_t rc = launch_team_step(ctx, a, max_len, max_src, static_cast<cudaStream_t>(stream), ctx->last_rows_per_unit);
+    if (ctx->step_kernel != 1) {       // automatic: the team-pipeline kernel for steps with rows long enough to be split over a team
+        const int32_t rc = launch_team_step(ctx, a, max_len, max_src, static_cast<cudaStream_t>(stream), ctx->last_rows_per_unit,
+                                            ctx->step_kernel == 0 && ctx->team_cut_override[0] < 0);
         if (rc != SAN_ERR_UNSUPPORTED) { ctx->last_step_kernel = 2; return rc; }
         if (ctx->step_kernel == 2) return rc;
     }
@@ -847,8 +862,8 @@ int32_t san_decode_step(san_ctx* ctx, const san_step_args* a, void* stream) {
 int32_t san_step_kernel_select(san_ctx* ctx, int32_t which, int32_t spans_log2, int32_t heads_per_unit, int32_t tile_pos,
                                int32_t layers_per_unit, int32_t grab_mult) {
     if (!ctx) return SAN_ERR_NULL;
-    if (which < 0 || which > 2 || spans_log2 > 1) return SAN_ERR_RANGE;
-    if (spans_log2 >= 0 && (tile_pos < 16 || tile_pos % 16 != 0 || heads_per_unit < 1 || heads_per_unit > 4)) return SAN_ERR_RANGE;
+    if (which < 0 || which > 2) return SAN_ERR_RANGE;
+    if (spans_log2 >= 0 && ((tile_pos & 255) < 16 || heads_per_unit < 1)) return SAN_ERR_RANGE;
     ctx->step_kernel = which;
     ctx->team_cut_override[0] = spans_log2 < 0 ? -1 : spans_log2;
     ctx->team_cut_override[1] = heads_per_unit;

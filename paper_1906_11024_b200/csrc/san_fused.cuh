@@ -113,10 +113,19 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
                  : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
+// try_wait that lets the hardware keep the thread suspended for a while (it returns as soon as
+// the phase completes), so that a waiting warp does not use issue slots.  Measured on B200: a
+// hint of 1,000,000 suspends for about 1000 cycles; without a hint the instruction returns at once.
+__device__ __forceinline__ bool mbar_try_wait_hint(uint32_t bar, uint32_t parity, uint32_t hint) {
+    uint32_t ok;
+    asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\nselp.u32 %0, 1, 0, p;\n}"
+                 : "=r"(ok) : "r"(bar), "r"(parity), "r"(hint) : "memory");
+    return ok != 0;
+}
 // Bounded wait: gives up after about a second and reports it; never spins for ever.
 __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity) {
     const long long t0 = clock64();
-    while (!mbar_try_wait(bar, parity)) {
+    while (!mbar_try_wait_hint(bar, parity, 2000000u)) {
         if (clock64() - t0 > 2000000000LL) return false;
     }
     return true;

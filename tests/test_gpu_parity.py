@@ -51,11 +51,16 @@ def _compare(w, dec, sb, ref, n, lens, src_lens_per_seq, tag):
     assert err <= tol, (tag, "O_enc", err)
 
 
+STEP_KERNEL = [0]        # which kernel san_decode_step is told to launch (see san_step_kernel_select); tests set it
+
+
 def _run(w, check_steps=None, max_steps=None, shared_context=False, jumps=None, fused=False):
     """Decode the workload on both sides.  Sequences start at their prefix length, advance in
     lock-step and drop out when their sentence is done.  ``jumps`` = list of (start_pos, n_steps)
     segments for long runs: the caches are re-prefilled to start_pos before each segment."""
     dec = Decoder(w, encdec_shared_context=shared_context)
+    if STEP_KERNEL[0]:
+        B.check(B.san_step_kernel_select(dec.ctx, STEP_KERNEL[0]), "san_step_kernel_select")
     orc = OracleRun(w, shared_context)
     dec.load_encoder_memory()
     T = np.repeat(w.tgt_lens(), w.beam)
@@ -203,10 +208,43 @@ def test_one_launch_step_matches_oracle(case):
     FUSED_CASES[case]()
 
 
+TEAM_CASES = [c for c in sorted(FUSED_CASES) if not c.startswith(("tiny", "fp32"))]      # the team pipeline is bf16 only
+
+
+@pytest.mark.parametrize("case", TEAM_CASES)
+def test_one_launch_step_team_pipeline_matches_oracle(case):
+    """The same cases with the team-pipeline kernel forced (automatically it only takes steps with split rows)."""
+    STEP_KERNEL[0] = 2
+    try:
+        FUSED_CASES[case]()
+    finally:
+        STEP_KERNEL[0] = 0
+
+
+@pytest.mark.parametrize("kernel", [0, 2])
 @pytest.mark.parametrize("beam", [1, 2, 3, 5, 8])
-def test_one_launch_step_other_beam_sizes(beam):
+def test_one_launch_step_other_beam_sizes(beam, kernel):
     w = dataclasses.replace(synth.scaled(synth.WORKLOADS["base"], 3), beam=beam, name=f"beam{beam}")
-    _run(w, max_steps=5, fused=True)
+    STEP_KERNEL[0] = kernel
+    try:
+        _run(w, max_steps=5, fused=True)
+    finally:
+        STEP_KERNEL[0] = 0
+
+
+def test_automatic_kernel_choice():
+    """Rows long enough to be split over a team go to the team pipeline, sentence-sized rows to the per-warp kernel."""
+    for name, want in (("base", 1), ("long", 2)):
+        w = synth.scaled(synth.WORKLOADS[name], 2)
+        dec = Decoder(w)
+        dec.load_encoder_memory()
+        sb = dec.new_step_buffers()
+        dec.fill_step_inputs(sb, 0, np.arange(w.n_seqs, dtype=np.int32), np.zeros(w.n_seqs, np.int32))
+        dec.step_fused(sb)
+        rc, which, rpu = B.san_step_kernel_used(dec.ctx)
+        assert rc == 0 and which == want, (name, which, rpu)
+        assert dec.device_status()[0] == 0
+        dec.close()
 
 
 def test_one_launch_step_writes_the_cache_like_append():

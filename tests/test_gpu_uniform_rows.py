@@ -22,6 +22,17 @@ def _built():
     B.lib()
 
 
+# which kernel runs the step and how it cuts the rows (san_step_kernel_select): the automatic choice, the team
+# pipeline with its own cut (up to four heads to a warp), and the team pipeline with one head
+# to a warp in tiles of 16 positions
+CUTS = {"auto": None, "team": (2,), "team-1head-tile16": (2, 0, 1, 16, 0, 1)}
+
+
+def _select(dec, cut):
+    if CUTS[cut] is not None:
+        B.check(B.san_step_kernel_select(dec.ctx, *CUTS[cut]), "san_step_kernel_select")
+
+
 def _wl(pi_self, pi_enc, src, T, n_sent=16):
     return synth.Workload(name=f"uniform-{pi_self}-{pi_enc}-{src}-{T}", dtype=synth.BF16, n_layers=6, n_heads=8, d_head=64,
                           n_sent=n_sent, beam=4, self_blocks=(pi_self,) * (6 // pi_self),
@@ -29,12 +40,14 @@ def _wl(pi_self, pi_enc, src, T, n_sent=16):
                           tgt_fixed=T, ragged_prefix=False, self_is_aan=False, seed=5)
 
 
+@pytest.mark.parametrize("cut", sorted(CUTS))
 @pytest.mark.parametrize("L", [8, 21, 24, 25, 40, 56, 88])
 @pytest.mark.parametrize("pi", [1, 2, 3])
-def test_self_attention_rows_of_one_length(L, pi):
+def test_self_attention_rows_of_one_length(L, pi, cut):
     """Self-attention only (no sentence in the step): prefill L-1 rows, decode the L-th."""
     w = _wl(pi, 1, 8, L)
     dec, orc = Decoder(w), OracleRun(w)
+    _select(dec, cut)
     n = w.n_seqs
     ids = np.arange(n, dtype=np.int32)
     if L > 1:
@@ -70,12 +83,14 @@ def test_self_attention_rows_of_one_length(L, pi):
     dec.close()
 
 
+@pytest.mark.parametrize("cut", sorted(CUTS))
 @pytest.mark.parametrize("Ls", [16, 24, 38, 60])
 @pytest.mark.parametrize("pi", [1, 3, 6])
-def test_encoder_memory_rows_of_one_length(Ls, pi):
+def test_encoder_memory_rows_of_one_length(Ls, pi, cut):
     """Encoder-decoder attention only (no sequence in the step's self-attention part)."""
     w = _wl(1, pi, Ls, 8)
     dec, orc = Decoder(w), OracleRun(w)
+    _select(dec, cut)
     dec.load_encoder_memory()
     ids = np.arange(w.n_seqs, dtype=np.int32)
     full = dec.new_step_buffers()
