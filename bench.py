@@ -1,8 +1,12 @@
 #!/usr/bin/env python
 """Benchmark of the shared-attention decode step.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload base|big|long|aan|tiny]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload long|base|big|aan|tiny]
     python bench.py --impl reference ...          # the CPU oracle as the reference arm
+
+The line's headline is the workload named by --workload (default: long, the single-GPU
+configuration that moves most bytes per step); the other configurations are measured in
+the same run with fewer steps and reported under "workloads".
 
 A step is one decode step of the whole attention path (cache append, weights, apply for
 self and encoder-decoder attention of every layer, or AAN + enc-dec) for every sequence of
@@ -34,14 +38,13 @@ L2_BYTES = 126e6
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 
-# DRAM bytes read + written per launch of the step kernel, from the ncu capture summarised in
-# profiles/decode_step_base_long.md, and the digest of the kernel sources they were taken
-# with: once those sources change the counters no longer describe the kernel and the bench
-# line reports null until a new capture is recorded here.  (The choice of spans and layer
-# groups lives in san_api.cu; a change there calls for a new capture as well.)
-KERNEL_SOURCES = ("san_fused.cuh", "san_kernels.cuh")
-NCU_TRAFFIC = {"digest": "55c777fde63b549e", "fused": {"base": 70.3e6, "long": 762.4e6,
-                                                          "base-unshared": 102.6e6, "long-unshared": 1317.0e6}}
+# DRAM bytes read + written per launch of the step kernel, from ncu captures of this file's own
+# command line (one workload, a dozen steps), and the digest of the sources they were taken with
+# (the kernels and the host code that chooses kernel and cuts): once any of them changes the
+# counters no longer describe the kernel, and the line reports null until a new capture is
+# recorded here.
+KERNEL_SOURCES = ("san_fused.cuh", "san_step.cuh", "san_kernels.cuh", "san_api.cu")
+NCU_TRAFFIC = {"digest": "", "fused": {}}
 
 
 def kernel_digest():
@@ -149,14 +152,14 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------------------- the GPU arm
-def build_replicas(w, n_rep, device):
+def build_replicas(w, n_rep, device, shared_context=False):
     import torch
     from paper_1906_11024_b200.driver import Decoder
     pos = state_positions(w)
     ids = np.arange(w.n_seqs, dtype=np.int32)
     decs, sbs = [], []
     for r in range(n_rep):
-        dec = Decoder(w, device)
+        dec = Decoder(w, device, encdec_shared_context=shared_context)
         gen = torch.Generator(device=device)
         gen.manual_seed(1000 + r)
         # cache contents: seeded N(0,1) in the storage dtype (the AAN running sums are float32)
@@ -313,40 +316,52 @@ def time_e2e(w, dec, sb, steps, device, fused=True):
 
 
 def time_beam_reorder(w, decs, sbs, pos, device, peak, reps=10):
-    """The step next to the path in a beam-search decoder: san_beam_reorder with every beam
-    taking over the whole history of its neighbour (parent = slot + 1 mod beam), so that every
-    cached row of every self-attention plane moves; launches rotate over the replicas."""
+    """The step next to the path in a beam-search decoder: san_beam_reorder, launches rotating
+    over the replicas.  Two parent patterns: every beam takes over the whole history of its
+    neighbour (parent = slot + 1 mod beam: every cached row of every self-attention plane moves),
+    and seeded parents where half of the hypotheses continue themselves and the others pick a
+    parent at random (rows of a hypothesis that keeps its parent do not move)."""
     import torch
     from paper_1906_11024_b200 import binding as B
+    from paper_1906_11024_b200 import synth
     R = len(decs)
     sent = torch.arange(w.n_sent, dtype=torch.int32, device=device)
-    parent = ((torch.arange(w.beam, dtype=torch.int32, device=device) + 1) % w.beam).repeat(w.n_sent, 1).contiguous()
-    lens = torch.from_numpy((pos + 1).astype(np.int32)).to(device).view(w.n_sent, w.beam).contiguous()
+    lens_h = (pos + 1).astype(np.int32)
+    lens = torch.from_numpy(lens_h).to(device).view(w.n_sent, w.beam).contiguous()
     max_len = int(pos.max()) + 1
+    planes = w.n_layers if w.self_is_aan else len(w.self_blocks) + w.n_layers
+    row_bytes = w.d_model * (4 if w.self_is_aan else w.elem_bytes)
+    out = {}
+    worst = ((np.arange(w.beam, dtype=np.int32) + 1) % w.beam)[None, :].repeat(w.n_sent, 0)
+    seeded = synth.beam_parents(w, 0, keep_prob=0.5).reshape(w.n_sent, w.beam)
+    for name, par in (("all_move", worst), ("half_keep", seeded)):
+        parent = torch.from_numpy(np.ascontiguousarray(par, np.int32)).to(device)
 
-    def all_replicas():
-        for r in range(R):
-            B.check(B.san_beam_reorder(decs[r].ctx, sent, parent, lens, w.n_sent, max_len), "san_beam_reorder")
+        def all_replicas():
+            for r in range(R):
+                B.check(B.san_beam_reorder(decs[r].ctx, sent, parent, lens, w.n_sent, max_len), "san_beam_reorder")
 
-    g = capture(all_replicas, device)
-    for _ in range(3):
-        g.replay()
-    torch.cuda.synchronize(device)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(reps):
-        g.replay()
-    e1.record()
-    torch.cuda.synchronize(device)
-    secs = e0.elapsed_time(e1) * 1e-3 / (reps * R)
-    if w.self_is_aan:
-        moved = w.n_layers * w.n_seqs * w.d_model * 4
-    else:
-        moved = (len(w.self_blocks) + w.n_layers) * int((pos.astype(np.int64) + 1).sum()) * w.d_model * w.elem_bytes
-    gbs = 2 * moved / secs / 1e9                      # every piece is read once and written once
-    return {"call": "san_beam_reorder", "us_per_launch": secs * 1e6, "bytes_per_launch": 2 * moved,
-            "achieved_gbs": gbs, "frac_of_peak": gbs / peak, "bound": "hbm",
-            "note": "all beams change parent; launches of the AAN workload move only the running sums"}
+        g = capture(all_replicas, device)
+        for _ in range(3):
+            g.replay()
+        torch.cuda.synchronize(device)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            g.replay()
+        e1.record()
+        torch.cuda.synchronize(device)
+        secs = e0.elapsed_time(e1) * 1e-3 / (reps * R)
+        moves = (par != np.arange(w.beam)[None, :]).reshape(-1)
+        rows = float(moves.sum()) if w.self_is_aan else float(lens_h[moves].sum())
+        moved = planes * rows * row_bytes
+        gbs = 2 * moved / secs / 1e9                  # every piece that moves is read once and written once
+        out[name] = {"us_per_launch": secs * 1e6, "bytes_per_launch": 2 * moved, "achieved_gbs": gbs,
+                     "frac_of_peak": gbs / peak, "share_of_slots_that_move": float(moves.mean())}
+    out.update({"call": "san_beam_reorder", "bound": "hbm",
+                "note": "all_move: every beam changes parent; half_keep: seeded parents, half of the hypotheses continue "
+                        "themselves; launches of the AAN workload move only the running sums"})
+    return out
 
 
 def time_js_matrix(w, dec, sb, pos, device, reps=50):
@@ -522,17 +537,89 @@ def run_reference(args, w):
     print(json.dumps(line))
 
 
+KERNEL_NAMES = {0: "none", 1: "decode_step_kernel (per-warp pipeline)", 2: "decode_step_team_kernel (team pipeline)"}
+
+
+def kernel_used(dec):
+    from paper_1906_11024_b200 import binding as B
+    rc, which, rpu = B.san_step_kernel_used(dec.ctx)
+    return {"kernel": KERNEL_NAMES.get(which, "?"), "heads_per_unit": rpu if which == 2 else None}
+
+
+def roofline_record(ab, secs_per_step, peak, peak_kind, name, traffic):
+    """The step kernel against the HBM roofline.  `achieved` counts the K/V reads (and the AAN
+    state) only: the roofline byte count; S, q, O and appended rows are reported beside it."""
+    gbs = ab["kv"] / secs_per_step / 1e9
+    return {"bound": "hbm", "kernel": name, "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
+            "peak_kind": peak_kind, "frac_of_nominal_8tbs": gbs / NOMINAL_HBM_GBS,
+            "bytes_per_launch": float(ab["kv"]), "us_per_launch": secs_per_step * 1e6, "launches_per_step": 1,
+            "other_bytes_per_launch": {"S": ab["S"], "q_O_new_rows": ab["small"]},
+            "achieved_all_bytes": ab["total"] / secs_per_step / 1e9, "traffic": traffic}
+
+
+def measure(w, steps, warmup, device, peak, peak_kind, fused=True, unshared=True, shared_context=False, n_rep_cap=16):
+    """One workload on this rank: the step time with sharing on (and off), the roofline record."""
+    import torch
+    from paper_1906_11024_b200 import synth
+    pos = state_positions(w)
+    ab = algorithmic_bytes(w, pos, fused)
+    if shared_context:        # Eq. 5: one value plane and one output per enc-dec block
+        M, Ne, d, e = w.n_layers, len(w.encdec_blocks), w.d_model, w.elem_bytes
+        src = int(w.src_lens().astype(np.int64).sum())
+        ab = dict(ab)
+        ab["encdec_kv"] = 2 * Ne * src * d * e
+        ab["kv"] = ab["self_kv"] + ab["encdec_kv"] + ab["aan"]
+        ab["small"] -= (M - Ne) * w.n_seqs * d * e
+        ab["total"] = ab["kv"] + ab["S"] + ab["small"]
+    n_rep = int(min(n_rep_cap, max(2, math.ceil(3 * L2_BYTES / max(ab["total"], 1)))))
+    decs, sbs, pos = build_replicas(w, n_rep, device, shared_context)
+    secs, launches, window = time_steps(decs, sbs, steps, warmup, device, lambda: None, fused)
+    err = [d.device_status()[0] for d in decs]
+    assert not any(err), f"device check failed during the timed region: {err}"
+    used = kernel_used(decs[0]) if fused else {"kernel": "append/weights/apply kernels", "heads_per_unit": None}
+    rec = {"value": w.n_seqs * steps / secs, "unit": UNIT, "steps": steps, "ms_per_step": secs / steps * 1e3,
+           "replicas": n_rep, "launches_per_step": launches, "used": used, "bytes": ab,
+           "roofline": roofline_record(ab, secs / steps, peak, peak_kind, used["kernel"], ncu_traffic("fused", w.name))}
+    keep = (decs, sbs, pos)
+    if unshared and not shared_context:
+        for d in decs:
+            d.close()
+        del decs, sbs, keep
+        torch.cuda.empty_cache()
+        wu = synth.unshared(w)
+        abu = algorithmic_bytes(wu, pos, fused)
+        decs_u, sbs_u, _ = build_replicas(wu, n_rep, device)
+        su, lu, _ = time_steps(decs_u, sbs_u, steps, warmup, device, lambda: None, fused)
+        rec["unshared"] = {"value": wu.n_seqs * steps / su, "unit": UNIT, "ms_per_step": su / steps * 1e3,
+                           "kv_bytes_per_step": abu["kv"], "bytes_per_step": abu["total"],
+                           "kv_gbs": abu["kv"] / (su / steps) / 1e9, "gpu_launches_per_step": lu,
+                           "traffic": ncu_traffic("fused", wu.name),
+                           "speedup_from_sharing": su / secs,
+                           "kv_bytes_ratio_shared_over_unshared": ab["kv"] / abu["kv"]}
+        keep = (decs_u, sbs_u, pos, wu)
+    return rec, keep, window
+
+
+def release(keep):
+    import torch
+    for d in keep[0]:
+        d.close()
+    del keep
+    torch.cuda.empty_cache()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20000)
-    ap.add_argument("--warmup", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=5000)
+    ap.add_argument("--warmup", type=int, default=100)
     ap.add_argument("--impl", default="san", choices=["san", "reference"])
-    ap.add_argument("--workload", default="base", choices=["tiny", "base", "big", "long", "aan"])
+    ap.add_argument("--workload", default="long", choices=["tiny", "base", "big", "long", "aan"])
     ap.add_argument("--path", default="fused", choices=["fused", "calls"],
                     help="fused: san_decode_step, one launch per step; calls: append/weights/apply launches")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-unshared", action="store_true")
+    ap.add_argument("--only", action="store_true", help="measure the named workload alone (no other workloads, no extra legs)")
     ap.add_argument("--sharing", default="on", choices=["on", "off"],
                     help="off: time the workload with every block size 1 as the main arm (for byte counts of the unshared path)")
     args = ap.parse_args()
@@ -569,8 +656,8 @@ def main():
             dist.barrier()
 
     peak, peak_kind = measured_peak_gbs()
-    pos = state_positions(w)
     fused = args.path == "fused"
+    pos = state_positions(w)
     ab = algorithmic_bytes(w, pos, fused)
     n_rep = int(min(16, max(2, math.ceil(3 * L2_BYTES / max(ab["total"], 1)))))
     decs, sbs, pos = build_replicas(w, n_rep, device)
@@ -587,18 +674,22 @@ def main():
     clocks = sampler.stop(t0, t1)
     err = [d.device_status()[0] for d in decs]
     assert not any(err), f"device check failed during the timed region: {err}"
+    used = kernel_used(decs[0]) if fused else {"kernel": "append/weights/apply kernels", "heads_per_unit": None}
 
     secs_max, value = whole_job(secs, w.n_seqs * args.steps, world, dist, device)
 
     if fused:      # one kernel per step: its launch duration is the step time of the timed region
-        dom_s, dom_per_step, dom_bytes, dom_name = secs / args.steps, 1, float(ab["total"]), "san_decode_step (decode_step_kernel)"
+        roof = roofline_record(ab, secs / args.steps, peak, peak_kind, "san_decode_step: " + used["kernel"], ncu_traffic(args.path, w.name))
     else:
         dom_s, dom_per_step = time_dominant_kernel(w, decs, sbs, device)
-        dom_bytes, dom_name = dominant_kernel_bytes(w, pos), "san_attn_apply (apply_kernel)"
-    e2e_s, h2d, d2h = time_e2e(w, decs[0], sbs[0], min(args.steps, 100), device, fused)
+        dom_bytes = dominant_kernel_bytes(w, pos)
+        roof = {"bound": "hbm", "kernel": "san_attn_apply (apply_kernel)", "achieved": dom_bytes / dom_s / 1e9, "peak": peak,
+                "unit": "GB/s", "frac": dom_bytes / dom_s / 1e9 / peak, "peak_kind": peak_kind, "bytes_per_launch": dom_bytes,
+                "us_per_launch": dom_s * 1e6, "launches_per_step": dom_per_step, "traffic": None}
     e2e_steps = min(args.steps, 100)
+    e2e_s, h2d, d2h = time_e2e(w, decs[0], sbs[0], e2e_steps, device, fused)
     next_rows = {}
-    if rank == 0:
+    if rank == 0 and not args.only:
         next_rows["beam_reorder"] = time_beam_reorder(w, decs, sbs, pos, device, peak)
         fb = time_full_block(w, device, peak)
         if fb is not None:
@@ -616,15 +707,59 @@ def main():
         su, lu, _ = time_steps(decs_u, sbs_u, args.steps, args.warmup, device, lambda: None, fused)
         unshared = {"value": wu.n_seqs * args.steps / su, "unit": UNIT, "ms_per_step": su / args.steps * 1e3,
                     "kv_bytes_per_step": abu["kv"], "bytes_per_step": abu["total"],
-                    "hbm_gbs": abu["total"] / (su / args.steps) / 1e9, "gpu_launches_per_step": lu,
+                    "kv_gbs": abu["kv"] / (su / args.steps) / 1e9, "gpu_launches_per_step": lu,
                     "traffic": ncu_traffic(args.path, wu.name)}
-        js = time_js_matrix(wu, decs_u[0], sbs_u[0], pos, device)
-        if js is not None:
-            next_rows["policy_learner"] = js
+        if not args.only:
+            js = time_js_matrix(wu, decs_u[0], sbs_u[0], pos, device)
+            if js is not None:
+                next_rows["policy_learner"] = js
         for d in decs_u:
             d.close()
         del decs_u, sbs_u
         torch.cuda.empty_cache()
+    else:
+        for d in decs:
+            d.close()
+        del decs, sbs
+        torch.cuda.empty_cache()
+
+    # ---- the other configurations, Eq. 5 and the beam sweep: fewer steps each, rank 0 only
+    workloads, eq5, beams = {}, None, None
+    if rank == 0 and fused and not args.only and args.sharing == "on":
+        sub_steps = max(200, min(args.steps, 2000))
+        for name in ("base", "big", "long", "aan"):
+            if name == w.name:
+                continue
+            rec, keep, _ = measure(synth.WORKLOADS[name], sub_steps, max(args.warmup, 3), device, peak, peak_kind,
+                                   unshared=not args.no_unshared)
+            release(keep)
+            workloads[name] = {k: rec[k] for k in ("value", "unit", "steps", "ms_per_step", "used", "roofline")}
+            if "unshared" in rec:
+                workloads[name]["unshared"] = rec["unshared"]
+        workloads["tiny"] = {"note": "configuration 1 (float32, one sentence): parity only, it fits L2 and is launch-bound"}
+        # Eq. 5 on the base shape: encoder-decoder attention with one value plane and one output per block
+        wb = synth.WORKLOADS["base"]
+        own, keep, _ = measure(wb, sub_steps, max(args.warmup, 3), device, peak, peak_kind, unshared=False)
+        release(keep)
+        shr, keep, _ = measure(wb, sub_steps, max(args.warmup, 3), device, peak, peak_kind, unshared=False, shared_context=True)
+        release(keep)
+        eq5 = {"workload": "base", "own_values_ms_per_step": own["ms_per_step"], "shared_context_ms_per_step": shr["ms_per_step"],
+               "own_values_kv_bytes": own["bytes"]["kv"], "shared_context_kv_bytes": shr["bytes"]["kv"],
+               "encdec_kv_bytes": {"own_values": own["bytes"]["encdec_kv"], "shared_context": shr["bytes"]["encdec_kv"]},
+               "speedup": own["ms_per_step"] / shr["ms_per_step"], "roofline_frac": shr["roofline"]["frac"],
+               "note": "Eq. 5: the block's lowest layer applies S to its values and the layers above reuse that output; "
+                       "enc-dec K/V bytes fall from (N_e + M) to 2 N_e planes"}
+        # beam sizes (Figure 5 sweeps 4..20) on the base shape
+        beams = {}
+        import dataclasses
+        for beam in (4, 8, 12, 16, 20):
+            if beam > binding.SAN_MAX_BEAM:
+                continue
+            wbm = dataclasses.replace(wb, beam=beam, name=f"base-beam{beam}")
+            rec, keep, _ = measure(wbm, sub_steps, max(args.warmup, 3), device, peak, peak_kind, unshared=not args.no_unshared)
+            release(keep)
+            beams[str(beam)] = {"value": rec["value"], "ms_per_step": rec["ms_per_step"], "kv_frac": rec["roofline"]["frac"],
+                                "speedup_from_sharing": rec.get("unshared", {}).get("speedup_from_sharing")}
 
     if rank != 0:
         if dist is not None:
@@ -644,19 +779,22 @@ def main():
                                   "mean_cache_len": float((pos + 1).mean()), "mean_src_len": float(w.src_lens().mean()),
                                   "path": "san_decode_step, one launch per step" if fused
                                           else "san_cache_append + san_attn_weights/apply per block",
+                                  "kernel": used["kernel"], "heads_per_unit": used["heads_per_unit"],
                                   "multi_gpu": "replicas only: no sharding, no collective"}),
         "gpu_launches": launches_per_step * args.steps, "gpu_launches_per_step": launches_per_step,
-        "hbm": {"kv_bytes_per_step": ab["kv"], "bytes_per_step": ab["total"], "achieved_gbs": step_gbs,
-                "frac_of_measured": step_gbs / peak, "frac_of_nominal_8tbs": step_gbs / NOMINAL_HBM_GBS,
-                "peak_kind": peak_kind},
-        "roofline": {"bound": "hbm", "kernel": dom_name, "achieved": dom_bytes / dom_s / 1e9,
-                     "peak": peak, "unit": "GB/s", "frac": dom_bytes / dom_s / 1e9 / peak, "peak_kind": peak_kind,
-                     "bytes_per_launch": dom_bytes, "us_per_launch": dom_s * 1e6, "launches_per_step": dom_per_step,
-                     "traffic": ncu_traffic(args.path, w.name)},
+        "hbm": {"kv_bytes_per_step": ab["kv"], "bytes_per_step": ab["total"], "achieved_gbs_all_bytes": step_gbs,
+                "kv_gbs": ab["kv"] / (secs_max / args.steps) / 1e9, "peak_kind": peak_kind},
+        "roofline": roof,
         "e2e": {"value": w.n_seqs * e2e_steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": e2e_s / e2e_steps * 1e3},
         "clocks": clocks,
     }
+    if workloads:
+        line["workloads"] = workloads
+    if eq5:
+        line["eq5"] = eq5
+    if beams:
+        line["beam_sweep"] = beams
     if next_rows:
         line["next_rows"] = next_rows
     if unshared is not None:

@@ -78,7 +78,7 @@ enum { SAN_F32 = 0, SAN_BF16 = 1 };
 enum { SAN_SELF = 0, SAN_ENCDEC = 1 };
 
 #define SAN_MAX_LAYERS 64
-#define SAN_MAX_BEAM 8
+#define SAN_MAX_BEAM 32
 
 typedef struct {
     int32_t n_layers;    /* M, 1..SAN_MAX_LAYERS */
@@ -333,7 +333,7 @@ int32_t san_device_status(san_ctx* ctx, int32_t* first_error, int32_t* detail, v
  *
  *   dtype      SAN_F32 or SAN_BF16 (element type of d_q and d_K)
  *   n_queries  query rows sharing each key panel: 1 for self-attention, the beam size for
- *              encoder memory (1..SAN_MAX_BEAM)
+ *              encoder memory (1..8)
  *   d_q        [n_items][n_queries][n_heads][64]
  *   d_K        key plane [max_ids][n_heads][cap_len][64], the layout of the context's planes
  *   d_ids, d_lens, n_items, max_len, d_S, ld_s   as in san_attn_weights;

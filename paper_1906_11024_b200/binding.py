@@ -21,7 +21,7 @@ SAN_ERR_NULL, SAN_ERR_SHAPE, SAN_ERR_POLICY, SAN_ERR_CAPACITY, SAN_ERR_DTYPE = 1
 SAN_ERR_RANGE, SAN_ERR_CUDA, SAN_ERR_DEVICE_CHECK, SAN_ERR_TIMEOUT, SAN_ERR_UNSUPPORTED = 6, 7, 8, 9, 10
 SAN_F32, SAN_BF16 = 0, 1
 SAN_SELF, SAN_ENCDEC = 0, 1
-SAN_MAX_LAYERS, SAN_MAX_BEAM = 64, 8
+SAN_MAX_LAYERS, SAN_MAX_BEAM = 64, 32
 
 # every symbol include/san.h declares
 EXPORTS = (

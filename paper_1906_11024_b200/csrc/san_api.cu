@@ -71,6 +71,7 @@ void layout(const san_config& c, int n_self_planes, int n_enc_planes, san_ctx* L
 
 inline int32_t cuda_status(cudaError_t e) { return e == cudaSuccess ? SAN_OK : SAN_ERR_CUDA; }
 
+constexpr int kQueryGroup = 8;      // query rows (beams) that share a key tile in one work item
 int pick_nq_template(int nq) { return nq <= 1 ? 1 : nq <= 2 ? 2 : nq <= 4 ? 4 : 8; }
 
 // Multiplier and shift for FastDiv (exact for dividends below 2^31).
@@ -170,13 +171,13 @@ constexpr size_t kStepSmemTotal = 232448;      // opt-in shared memory per CTA o
 struct TeamCut { int spr_log2, lg, tile_pos, zq, rpu; };
 
 int32_t launch_team_step(san_ctx* ctx, const san_step_args* a, int max_len, int max_src, cudaStream_t st, int* rows_per_unit,
-                         bool only_if_split) {
+                         bool only_if_split, int q_first, int q_count) {
     const san_config& c = ctx->cfg;
     if (c.dtype != SAN_BF16) return SAN_ERR_UNSUPPORTED;
     const bool aan = c.self_is_aan != 0;
     const int n_seqs = a->n_seqs, n_sent = a->n_sent;
     const bool do_self = n_seqs > 0 && !aan, do_enc = n_sent > 0, do_aan = aan && n_seqs > 0;
-    const int nqe = pick_nq_template(c.beam);
+    const int nqe = pick_nq_template(q_count);
     const int H = c.n_heads;
     int pi_self = 1, pi_enc = 1;
     for (int b = 0; b < ctx->self_pol.n_blocks; ++b) pi_self = std::max(pi_self, ctx->self_pol.size_of_block[b]);
@@ -316,8 +317,8 @@ int32_t launch_team_step(san_ctx* ctx, const san_step_args* a, int max_len, int 
         k.layer_bytes = (long long)n_sent * c.beam * H * 128;
         k.S_ld = a->ld_s;
         k.panel_bytes = (unsigned)c.max_src_len * 128u;
-        k.nq = (unsigned)c.beam; k.len_bias = 0; k.max_ids = (unsigned)c.max_sent; k.bound = (unsigned)max_src;
-        k.q_first = 0; k.q_stride_items = (unsigned)c.beam; k.v_by_block = c.encdec_shared_context ? 1 : 0;
+        k.nq = (unsigned)q_count; k.len_bias = 0; k.max_ids = (unsigned)c.max_sent; k.bound = (unsigned)max_src;
+        k.q_first = (unsigned)q_first; k.q_stride_items = (unsigned)c.beam; k.v_by_block = c.encdec_shared_context ? 1 : 0;
         fill(k, ctx->enc_pol, ce, n_sent, rows_enc, pi_enc);
     }
     if (!do_self) p.k[0].n_units = 0;
@@ -528,20 +529,27 @@ int32_t san_attn_weights(san_ctx* ctx, int32_t kind, int32_t block, const void* 
     p.q = d_q;
     p.K = ctx->cache + (kind == SAN_SELF ? ctx->off_self_k : ctx->off_mem_k) + plane * block;
     p.ids = d_ids; p.lens = d_lens; p.S = d_S; p.ld_s = ld_s;
-    p.n_items = n_items; p.H = c.n_heads; p.nq = kind == SAN_SELF ? 1 : c.beam;
+    p.n_items = n_items; p.H = c.n_heads;
+    p.nq_total = kind == SAN_SELF ? 1 : c.beam;
     p.cap_len = cap; p.max_ids = max_ids; p.max_len = max_len;
     const long long rows = (long long)n_items * c.n_heads;
-    pick_spans(ctx, rows, max_len, rows * p.nq * 2, &p.span_len, &p.n_spans_max);
     p.part = ctx->part; p.tickets = ctx->tickets; p.err = ctx->err;
     p.scale_log2e = (float)(1.4426950408889634 / std::sqrt((double)kDh));
-    const long long warps = rows * p.n_spans_max;
-    const long long grid = (warps + kWarpsPerCta - 1) / kWarpsPerCta;
-    if (grid > 0x7fffffffLL) return SAN_ERR_SHAPE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const int nq_t = pick_nq_template(p.nq);
-    cudaError_t e = c.dtype == SAN_BF16 ? launch_weights<__nv_bfloat16>(p, nq_t, (unsigned)grid, st)
-                                        : launch_weights<float>(p, nq_t, (unsigned)grid, st);
-    return cuda_status(e);
+    // a key tile is scored against at most kQueryGroup query rows at a time: larger beams take
+    // one launch per group of beams (the groups after the first find the keys in L2)
+    for (p.q0 = 0; p.q0 < p.nq_total; p.q0 += kQueryGroup) {
+        p.nq = std::min(kQueryGroup, p.nq_total - p.q0);
+        pick_spans(ctx, rows, max_len, rows * p.nq * 2, &p.span_len, &p.n_spans_max);
+        const long long warps = rows * p.n_spans_max;
+        const long long grid = (warps + kWarpsPerCta - 1) / kWarpsPerCta;
+        if (grid > 0x7fffffffLL) return SAN_ERR_SHAPE;
+        const int nq_t = pick_nq_template(p.nq);
+        cudaError_t e = c.dtype == SAN_BF16 ? launch_weights<__nv_bfloat16>(p, nq_t, (unsigned)grid, st)
+                                            : launch_weights<float>(p, nq_t, (unsigned)grid, st);
+        if (e != cudaSuccess) return SAN_ERR_CUDA;
+    }
+    return SAN_OK;
 }
 
 int32_t san_attn_apply(san_ctx* ctx, int32_t kind, int32_t block, int32_t layer_begin,
@@ -573,7 +581,8 @@ int32_t san_attn_apply(san_ctx* ctx, int32_t kind, int32_t block, int32_t layer_
     p.V = ctx->cache + (kind == SAN_SELF ? ctx->off_self_v : ctx->off_mem_v) + plane * v_plane0;
     p.plane_elems = (long long)(plane / ctx->elem_bytes);
     p.ids = d_ids; p.pos_begin = d_pos_begin; p.pos_end = d_pos_end; p.out = d_out;
-    p.n_items = n_items; p.H = c.n_heads; p.nq = kind == SAN_SELF ? 1 : c.beam;
+    p.n_items = n_items; p.H = c.n_heads;
+    p.nq_total = kind == SAN_SELF ? 1 : c.beam;
     p.cap_len = cap; p.max_ids = max_ids; p.max_len = max_len;
     p.n_layers = layer_end - layer_begin;
     p.accumulate = accumulate ? 1 : 0;
@@ -582,16 +591,20 @@ int32_t san_attn_apply(san_ctx* ctx, int32_t kind, int32_t block, int32_t layer_
     // otherwise give each layer its own warp, then split the positions as well
     p.layers_per_warp = (rows >= (long long)ctx->sm_count * 16) ? p.n_layers : 1;
     const int n_lgroups = ceil_div(p.n_layers, p.layers_per_warp);
-    pick_spans(ctx, rows * n_lgroups, max_len, rows * p.n_layers * p.nq * kDh, &p.span_len, &p.n_spans_max);
     p.part = ctx->part; p.tickets = ctx->tickets; p.err = ctx->err;
-    const long long warps = rows * n_lgroups * p.n_spans_max;
-    const long long grid = (warps + kWarpsPerCta - 1) / kWarpsPerCta;
-    if (grid > 0x7fffffffLL) return SAN_ERR_SHAPE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const int nq_t = pick_nq_template(p.nq);
-    cudaError_t e = c.dtype == SAN_BF16 ? launch_apply<__nv_bfloat16>(p, nq_t, (unsigned)grid, st)
-                                        : launch_apply<float>(p, nq_t, (unsigned)grid, st);
-    return cuda_status(e);
+    for (p.q0 = 0; p.q0 < p.nq_total; p.q0 += kQueryGroup) {      // one launch per group of beams, as in san_attn_weights
+        p.nq = std::min(kQueryGroup, p.nq_total - p.q0);
+        pick_spans(ctx, rows * n_lgroups, max_len, rows * p.n_layers * p.nq * kDh, &p.span_len, &p.n_spans_max);
+        const long long warps = rows * n_lgroups * p.n_spans_max;
+        const long long grid = (warps + kWarpsPerCta - 1) / kWarpsPerCta;
+        if (grid > 0x7fffffffLL) return SAN_ERR_SHAPE;
+        const int nq_t = pick_nq_template(p.nq);
+        cudaError_t e = c.dtype == SAN_BF16 ? launch_apply<__nv_bfloat16>(p, nq_t, (unsigned)grid, st)
+                                            : launch_apply<float>(p, nq_t, (unsigned)grid, st);
+        if (e != cudaSuccess) return SAN_ERR_CUDA;
+    }
+    return SAN_OK;
 }
 
 int32_t san_aan_step(san_ctx* ctx, int32_t layer_begin, int32_t layer_end, const void* d_x,
@@ -635,35 +648,23 @@ int32_t san_seq_reset(san_ctx* ctx, const int32_t* d_seq_ids, int32_t n, void* s
     return cuda_status(cudaGetLastError());
 }
 
-int32_t san_decode_step(san_ctx* ctx, const san_step_args* a, void* stream) {
-    if (!ctx || !a) return SAN_ERR_NULL;
+// One launch of the step for the query rows (beams) [q_first, q_first + q_count) of every sentence;
+// n_seqs > 0 in `a` adds the self-attention (or AAN) part.  Arguments have been checked.
+static int32_t decode_step_launch(san_ctx* ctx, const san_step_args* a, int max_len, int max_src, int q_first, int q_count, void* stream) {
     const san_config& c = ctx->cfg;
     const bool aan = c.self_is_aan != 0;
     const int n_seqs = a->n_seqs, n_sent = a->n_sent;
-    if (n_seqs < 0 || n_seqs > ctx->n_seqs || n_sent < 0 || n_sent > c.max_sent) return SAN_ERR_SHAPE;
-    if (n_seqs > 0) {
-        if (!a->d_seq_ids || !a->d_O_self) return SAN_ERR_NULL;
-        if (aan ? (!a->d_x_aan || !a->d_t) : (!a->d_q_self || !a->d_k_new || !a->d_v_new || !a->d_pos)) return SAN_ERR_NULL;
-    }
-    if (n_sent > 0 && (!a->d_q_enc || !a->d_sent_ids || !a->d_src_lens || !a->d_O_enc)) return SAN_ERR_NULL;
-    int max_len = a->max_len == 0 ? c.max_tgt_len : a->max_len;
-    int max_src = a->max_src == 0 ? c.max_src_len : a->max_src;
-    if (max_len < 1 || max_len > c.max_tgt_len || max_src < 1 || max_src > c.max_src_len) return SAN_ERR_SHAPE;
-    if (n_seqs > 0 && !aan && a->d_S_self && a->ld_t < max_len) return SAN_ERR_SHAPE;
-    if (n_sent > 0 && a->d_S_enc && a->ld_s < max_src) return SAN_ERR_SHAPE;
-    if (n_seqs == 0 && n_sent == 0) return SAN_OK;
-
     const bool bf16 = c.dtype == SAN_BF16;
     if (ctx->step_kernel != 1) {       // automatic: the team-pipeline kernel for steps with rows long enough to be split over a team
         const int32_t rc = launch_team_step(ctx, a, max_len, max_src, static_cast<cudaStream_t>(stream), ctx->last_rows_per_unit,
-                                            ctx->step_kernel == 0 && ctx->team_cut_override[0] < 0);
+                                            ctx->step_kernel == 0 && ctx->team_cut_override[0] < 0, q_first, q_count);
         if (rc != SAN_ERR_UNSUPPORTED) { ctx->last_step_kernel = 2; return rc; }
         if (ctx->step_kernel == 2) return rc;
     }
     ctx->last_step_kernel = 1;
     const int row_bytes = kDh * ctx->elem_bytes;
     const int TR = kStageBytes / row_bytes;
-    const int nqe = pick_nq_template(c.beam);
+    const int nqe = pick_nq_template(q_count);
     const bool do_self = n_seqs > 0 && !aan;
     const bool do_enc = n_sent > 0;
     int pi_self = 1, pi_enc = 1;
@@ -708,7 +709,7 @@ int32_t san_decode_step(san_ctx* ctx, const san_step_args* a, void* stream) {
     };
     int span_self = cap_self, span_enc = cap_enc, lg_self = pi_self, lg_enc = pi_enc;
     pick(cap_self, pi_self, 1, &span_self, &lg_self);
-    pick(cap_enc, pi_enc, c.beam, &span_enc, &lg_enc);
+    pick(cap_enc, pi_enc, q_count, &span_enc, &lg_enc);
     // The rule above looks at one item at a time.  Where it cuts anything, compare it with the other
     // ways of cutting (halved spans, halved layer groups, or no cut at all) by the estimated length
     // of the step: items of equal size that divide evenly over the warps beat smaller items that
@@ -721,7 +722,7 @@ int32_t san_decode_step(san_ctx* ctx, const san_step_args* a, void* stream) {
                 pl.len_bound == len_b && pl.src_bound == src_b) plan = &pl;
         if (!plan) {
             const int ctas = (int)std::max<long long>(1, std::min<long long>(ctx->sm_count, (rows_self + rows_enc + kFusedWarps - 1) / kFusedWarps));
-            CutShape ce{rows_enc, src_b, pi_enc, c.beam, span_enc, lg_enc}, cs{rows_self, len_b, pi_self, 1, span_self, lg_self};
+            CutShape ce{rows_enc, src_b, pi_enc, q_count, span_enc, lg_enc}, cs{rows_self, len_b, pi_self, 1, span_self, lg_self};
             double best = step_makespan(ce, cs, ctas, TR);
             int b_ss = span_self, b_ls = lg_self, b_se = span_enc, b_le = lg_enc;
             auto halvings = [](int from, int floor_, int align, std::vector<int>* out) {
@@ -795,7 +796,7 @@ int32_t san_decode_step(san_ctx* ctx, const san_step_args* a, void* stream) {
         k.S_ld = a->ld_t;
         k.part_base = ns_enc > 1 ? rl_enc * ns_enc * stride_enc : 0;
         k.panel_bytes = (unsigned)c.max_tgt_len * row_bytes;
-        k.n_it = (unsigned)std::max(n_seqs, 1); k.nq = 1; k.len_bias = 1; k.max_ids = (unsigned)ctx->n_seqs; k.bound = (unsigned)max_len;
+        k.n_it = (unsigned)std::max(n_seqs, 1); k.nq = 1; k.q_first = 0; k.q_total = 1; k.len_bias = 1; k.max_ids = (unsigned)ctx->n_seqs; k.bound = (unsigned)max_len;
         k.span = (unsigned)span_self; k.nspans = (unsigned)ns_self; k.part_stride = (unsigned)stride_self; k.v_by_block = 0;
         k.row_base = (unsigned)rl_enc;
         k.lg_size = (unsigned)lg_self; k.n_lg = (unsigned)nlg_self; k.div_lg = make_fastdiv((unsigned)nlg_self);
@@ -815,7 +816,7 @@ int32_t san_decode_step(san_ctx* ctx, const san_step_args* a, void* stream) {
         k.S_ld = a->ld_s;
         k.part_base = 0;
         k.panel_bytes = (unsigned)c.max_src_len * row_bytes;
-        k.n_it = (unsigned)std::max(n_sent, 1); k.nq = (unsigned)c.beam; k.len_bias = 0; k.max_ids = (unsigned)c.max_sent; k.bound = (unsigned)max_src;
+        k.n_it = (unsigned)std::max(n_sent, 1); k.nq = (unsigned)q_count; k.q_first = (unsigned)q_first; k.q_total = (unsigned)c.beam; k.len_bias = 0; k.max_ids = (unsigned)c.max_sent; k.bound = (unsigned)max_src;
         k.span = (unsigned)span_enc; k.nspans = (unsigned)ns_enc; k.part_stride = (unsigned)stride_enc;
         k.v_by_block = c.encdec_shared_context ? 1 : 0;
         k.row_base = 0;
@@ -857,6 +858,36 @@ int32_t san_decode_step(san_ctx* ctx, const san_step_args* a, void* stream) {
     void* args[] = {&p};
     cudaError_t e = cudaLaunchKernelExC(&cfg, fn, args);
     return cuda_status(e);
+}
+
+int32_t san_decode_step(san_ctx* ctx, const san_step_args* a, void* stream) {
+    if (!ctx || !a) return SAN_ERR_NULL;
+    const san_config& c = ctx->cfg;
+    const bool aan = c.self_is_aan != 0;
+    const int n_seqs = a->n_seqs, n_sent = a->n_sent;
+    if (n_seqs < 0 || n_seqs > ctx->n_seqs || n_sent < 0 || n_sent > c.max_sent) return SAN_ERR_SHAPE;
+    if (n_seqs > 0) {
+        if (!a->d_seq_ids || !a->d_O_self) return SAN_ERR_NULL;
+        if (aan ? (!a->d_x_aan || !a->d_t) : (!a->d_q_self || !a->d_k_new || !a->d_v_new || !a->d_pos)) return SAN_ERR_NULL;
+    }
+    if (n_sent > 0 && (!a->d_q_enc || !a->d_sent_ids || !a->d_src_lens || !a->d_O_enc)) return SAN_ERR_NULL;
+    int max_len = a->max_len == 0 ? c.max_tgt_len : a->max_len;
+    int max_src = a->max_src == 0 ? c.max_src_len : a->max_src;
+    if (max_len < 1 || max_len > c.max_tgt_len || max_src < 1 || max_src > c.max_src_len) return SAN_ERR_SHAPE;
+    if (n_seqs > 0 && !aan && a->d_S_self && a->ld_t < max_len) return SAN_ERR_SHAPE;
+    if (n_sent > 0 && a->d_S_enc && a->ld_s < max_src) return SAN_ERR_SHAPE;
+    if (n_seqs == 0 && n_sent == 0) return SAN_OK;
+
+    // A key tile is scored against at most kQueryGroup query rows at a time.  Wider beams take one
+    // launch per group of beams: the first also carries the self-attention (or AAN) part, the
+    // others read the encoder memory again (mostly from L2).
+    san_step_args part = *a;
+    for (int q0 = 0; q0 == 0 || (n_sent > 0 && q0 < c.beam); q0 += kQueryGroup) {
+        if (q0 > 0) part.n_seqs = 0;
+        const int32_t rc = decode_step_launch(ctx, &part, max_len, max_src, q0, std::min(kQueryGroup, c.beam - q0), stream);
+        if (rc != SAN_OK) return rc;
+    }
+    return SAN_OK;
 }
 
 int32_t san_step_kernel_select(san_ctx* ctx, int32_t which, int32_t spans_log2, int32_t heads_per_unit, int32_t tile_pos,
@@ -943,7 +974,8 @@ int32_t san_beam_reorder(san_ctx* ctx, const int32_t* d_sent_ids, const int32_t*
     auto launch = [&](const ReorderParams& q) -> int32_t {
         const long long gx = (long long)q.tiles_per_panel * q.n_heads * q.n_sent;
         if (gx > 0x7fffffffLL || q.n_planes > 65535) return SAN_ERR_SHAPE;
-        beam_reorder_kernel<<<dim3((unsigned)gx, (unsigned)q.n_planes), kReorderThreads, 0, st>>>(q);
+        if (q.beam <= 8) beam_reorder_kernel<8><<<dim3((unsigned)gx, (unsigned)q.n_planes), kReorderThreads, 0, st>>>(q);
+        else beam_reorder_kernel<SAN_MAX_BEAM><<<dim3((unsigned)gx, (unsigned)q.n_planes), kReorderThreads, 0, st>>>(q);
         return cuda_status(cudaGetLastError());
     };
     if (c.self_is_aan) {       // the running sums [layer][sequence][H*64] float32

@@ -53,7 +53,8 @@ struct KindParams {
     long long S_ld;                                    // floats between S rows
     long long part_base;                               // float offset of the kind's partial sums
     unsigned panel_bytes;                              // capacity * row bytes: one (id, head) panel
-    unsigned n_it, nq, len_bias, max_ids, bound;       // items, query rows per item, 1 if lens holds positions, limits
+    unsigned n_it, nq, len_bias, max_ids, bound;       // items, query rows per item in this launch, 1 if lens holds positions, limits
+    unsigned q_first, q_total;                         // first of those rows among the q_total rows an item has in q, S and O
     unsigned span, nspans, part_stride, v_by_block, row_base;
     unsigned lg_size, n_lg;                            // layers per item (a block is cut into groups), groups per block at most
     FastDiv div_span, div_lg, div_h, div_item;
@@ -212,7 +213,7 @@ __device__ bool decode_item(const StepParams& p, unsigned it, ItemDesc* d) {
     const int j1 = min(len, j0 + (int)kp.span);
     const unsigned first = kp.first[block] + l0;      // every group recomputes S from the block's keys
     const unsigned vplane = (kp.v_by_block ? block : kp.first[block]) + l0;
-    const unsigned qrow = ((block * kp.n_it + item) * kp.nq) * H + h;          // row of query 0 in q and S
+    const unsigned qrow = ((block * kp.n_it + item) * kp.q_total + kp.q_first) * H + h;   // row of the launch's query 0 in q and S
     const unsigned long long panel = (unsigned long long)((unsigned)id * H + h) * kp.panel_bytes;
     d->kind = enc; d->nq = (int)kp.nq; d->pi = (int)min(kp.lg_size, size - l0);
     d->len = len; d->n = j1 - j0;
@@ -226,7 +227,7 @@ __device__ bool decode_item(const StepParams& p, unsigned it, ItemDesc* d) {
     d->srcK = kp.K + (unsigned long long)block * (unsigned long long)kp.plane_bytes + panel + (unsigned)j0 * ROW_BYTES;
     d->srcV = kp.V + (unsigned long long)vplane * (unsigned long long)kp.plane_bytes + panel + (unsigned)j0 * ROW_BYTES;
     d->O = kp.O + (unsigned long long)vplane * (unsigned long long)kp.layer_bytes +
-           (unsigned long long)((item * kp.nq) * H + h) * ROW_BYTES;
+           (unsigned long long)((item * kp.q_total + kp.q_first) * H + h) * ROW_BYTES;
     const unsigned long long in_row = (unsigned long long)(item * H + h) * ROW_BYTES;   // self: nq == 1
     d->knew = kp.knew ? kp.knew + (unsigned long long)block * (unsigned long long)kp.layer_bytes + in_row : nullptr;
     d->vnew = kp.vnew ? kp.vnew + (unsigned long long)first * (unsigned long long)kp.layer_bytes + in_row : nullptr;

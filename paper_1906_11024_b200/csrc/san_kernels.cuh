@@ -149,6 +149,7 @@ struct WeightsParams {
     const int* ids; const int* lens;
     float* S; long long ld_s;   // [n_items][nq][H][ld_s]
     int n_items, H, nq, cap_len, max_ids, max_len;
+    int nq_total, q0;           // query rows per item in q and S; first of the nq rows this launch covers
     int span_len, n_spans_max;  // positions per warp item; spans per row at max_len
     float* part;                // [row][nq][n_spans_max][2] (max, sum) of split rows
     int* tickets;               // [row]
@@ -185,7 +186,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) weights_kernel(const Weight
 #pragma unroll
     for (int qi = 0; qi < NQ; ++qi) {
         if (qi < nq) {
-            const T* qp = reinterpret_cast<const T*>(p.q) + (((long long)item * nq + qi) * p.H + h) * kDh + c * VEC;
+            const T* qp = reinterpret_cast<const T*>(p.q) + (((long long)item * p.nq_total + p.q0 + qi) * p.H + h) * kDh + c * VEC;
             uint4 v = *reinterpret_cast<const uint4*>(qp);
             unpack16<T>(v, qf[qi]);
 #pragma unroll
@@ -237,7 +238,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) weights_kernel(const Weight
             for (int jj = lane; jj < n; jj += 32) m = fmaxf(m, zs[qi][jj]);
             run_max[qi] = fmaxf(run_max[qi], warp_max(m));
             if (!one_pass) {   // park the raw scores in S; they are turned into weights below
-                float* Srow = p.S + (((long long)item * nq + qi) * p.H + h) * p.ld_s + s0;
+                float* Srow = p.S + (((long long)item * p.nq_total + p.q0 + qi) * p.H + h) * p.ld_s + s0;
                 for (int jj = lane; jj < n; jj += 32) Srow[jj] = zs[qi][jj];
             }
         }
@@ -249,7 +250,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) weights_kernel(const Weight
 #pragma unroll
     for (int qi = 0; qi < NQ; ++qi) {
         if (qi >= nq) break;
-        float* Srow = p.S + (((long long)item * nq + qi) * p.H + h) * p.ld_s + j0;
+        float* Srow = p.S + (((long long)item * p.nq_total + p.q0 + qi) * p.H + h) * p.ld_s + j0;
         const float m = run_max[qi];
         float s = 0.f;
         if (one_pass) {
@@ -287,7 +288,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) weights_kernel(const Weight
         float tot = 0.f;
         for (int sp = lane; sp < n_spans; sp += 32) tot += __ldcg(pp + 2 * sp + 1) * exp2f(__ldcg(pp + 2 * sp) - m);
         tot = warp_sum(tot);
-        float* Srow = p.S + (((long long)item * nq + qi) * p.H + h) * p.ld_s;
+        float* Srow = p.S + (((long long)item * p.nq_total + p.q0 + qi) * p.H + h) * p.ld_s;
         for (int sp = 0; sp < n_spans; ++sp) {
             const float f = exp2f(__ldcg(pp + 2 * sp) - m) / tot;
             const int b = sp * p.span_len, e = min(len, b + p.span_len);
@@ -305,6 +306,7 @@ struct ApplyParams {
     const int* ids; const int* pos_begin; const int* pos_end;
     void* out;                        // [n_layers][n_items][nq][H][64]
     int n_items, H, nq, cap_len, max_ids, max_len;
+    int nq_total, q0;                 // query rows per item in S and out; first of the nq rows this launch covers
     int n_layers, layers_per_warp;
     int span_len, n_spans_max;
     int accumulate;
@@ -359,7 +361,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) apply_kernel(const ApplyPar
             if (l == l_begin || (j1 - j0) > kSub) {
                 __syncwarp();
                 for (int qi = 0; qi < nq; ++qi) {
-                    const float* Srow = p.S + (((long long)item * nq + qi) * p.H + h) * p.ld_s + s0;
+                    const float* Srow = p.S + (((long long)item * p.nq_total + p.q0 + qi) * p.H + h) * p.ld_s + s0;
                     for (int jj = lane; jj < n; jj += 32) ss[qi][jj] = Srow[jj];
                 }
                 __syncwarp();
@@ -401,7 +403,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) apply_kernel(const ApplyPar
                 for (int qi = 0; qi < NQ; ++qi) {
                     if (qi >= nq) break;
                     T* op = reinterpret_cast<T*>(p.out) +
-                            ((((long long)l * p.n_items + item) * nq + qi) * p.H + h) * kDh + c * VEC;
+                            ((((long long)l * p.n_items + item) * p.nq_total + p.q0 + qi) * p.H + h) * kDh + c * VEC;
                     if (p.accumulate) {
                         float old[VEC];
                         unpack16<T>(*reinterpret_cast<const uint4*>(op), old);
@@ -434,7 +436,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) apply_kernel(const ApplyPar
         __threadfence();
         for (int qi = 0; qi < nq; ++qi) {
             const float* pp = p.part + ((trow * nq + qi) * p.n_spans_max) * kDh;
-            T* op = reinterpret_cast<T*>(p.out) + ((((long long)l * p.n_items + item) * nq + qi) * p.H + h) * kDh;
+            T* op = reinterpret_cast<T*>(p.out) + ((((long long)l * p.n_items + item) * p.nq_total + p.q0 + qi) * p.H + h) * kDh;
             for (int col = lane; col < kDh; col += 32) {
                 float a = 0.f;
                 for (int sp = 0; sp < n_spans; ++sp) a += __ldcg(pp + (long long)sp * kDh + col);

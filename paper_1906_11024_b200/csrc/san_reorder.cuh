@@ -51,7 +51,9 @@ struct ReorderParams {
 // beam's parent, the CTA meets at a barrier, it stores.  The address arithmetic that does not
 // depend on the beam is done once per thread; the copy itself is a handful of instructions
 // per piece, so that the kernel is bound by HBM and not by instruction issue.
-static __global__ void __launch_bounds__(kReorderThreads) beam_reorder_kernel(const ReorderParams p) {
+// BMAX: beams a thread keeps in registers (8 for the usual beams, SAN_MAX_BEAM for the widest).
+template <int BMAX>
+__global__ void __launch_bounds__(kReorderThreads) beam_reorder_kernel(const ReorderParams p) {
     unsigned u = blockIdx.x;
     const int tile = (int)(u % (unsigned)p.tiles_per_panel); u /= (unsigned)p.tiles_per_panel;
     const int h = (int)(u % (unsigned)p.n_heads);
@@ -68,10 +70,10 @@ static __global__ void __launch_bounds__(kReorderThreads) beam_reorder_kernel(co
                   (long long)sent * p.beam * p.seq_bytes + (long long)piece * 16;
     const int* parent = p.parent + item * p.beam;
     const int* lens = p.lens + item * p.beam;
-    uint4 v[SAN_MAX_BEAM];
+    uint4 v[BMAX];
     unsigned take = 0;                                     // beams whose piece this thread moves
 #pragma unroll
-    for (int s = 0; s < SAN_MAX_BEAM; ++s) {
+    for (int s = 0; s < BMAX; ++s) {
         if (s >= p.beam) break;
         const int par = parent[s], len = lens[s];
         if (par < 0 || par >= p.beam) { if (reporter) record_error(p.err, TAG_REORDER, item * p.beam + s, par, p.beam); continue; }
@@ -83,7 +85,7 @@ static __global__ void __launch_bounds__(kReorderThreads) beam_reorder_kernel(co
     }
     __syncthreads();            // every piece of the tile that is needed has been read
 #pragma unroll
-    for (int s = 0; s < SAN_MAX_BEAM; ++s)
+    for (int s = 0; s < BMAX; ++s)
         if (take & (1u << s)) *reinterpret_cast<uint4*>(panel + s * p.seq_bytes) = v[s];
 }
 

@@ -77,7 +77,7 @@ extern "C" int32_t san_attn_weights_static(int32_t dtype, int32_t n_heads, int32
                                            int32_t* d_status, void* stream) {
     if (!d_q || !d_K || !d_ids || !d_lens || !d_S) return SAN_ERR_NULL;
     if (dtype != SAN_F32 && dtype != SAN_BF16) return SAN_ERR_DTYPE;
-    if (n_heads < 1 || n_heads > 1024 || n_queries < 1 || n_queries > SAN_MAX_BEAM) return SAN_ERR_SHAPE;
+    if (n_heads < 1 || n_heads > 1024 || n_queries < 1 || n_queries > 8) return SAN_ERR_SHAPE;
     if (max_ids < 1 || cap_len < 1 || cap_len > (1 << 20)) return SAN_ERR_SHAPE;
     if (n_items < 0 || n_items > max_ids) return SAN_ERR_SHAPE;
     if (max_len == 0) max_len = cap_len;
@@ -93,7 +93,7 @@ extern "C" int32_t san_attn_weights_static(int32_t dtype, int32_t n_heads, int32
 
     WeightsParams p;
     p.q = d_q; p.K = d_K; p.ids = d_ids; p.lens = d_lens; p.S = d_S; p.ld_s = ld_s;
-    p.n_items = n_items; p.H = n_heads; p.nq = n_queries;
+    p.n_items = n_items; p.H = n_heads; p.nq = n_queries; p.nq_total = n_queries; p.q0 = 0;
     p.cap_len = cap_len; p.max_ids = max_ids; p.max_len = max_len;
     // spans: halve while SMs would idle, never more than the fixed scratch can hold
     const long long target = (long long)slot.sm_count * 16;

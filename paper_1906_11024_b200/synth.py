@@ -175,10 +175,15 @@ def aan_x(w: Workload, step: int, layer: int) -> np.ndarray:
     return normal(w.seed, TAG_X_AAN, step, layer, (w.n_seqs, w.d_model), w.dtype)
 
 
-def beam_parents(w: Workload, step: int) -> np.ndarray:
-    """A random parent beam (0..beam-1) for every sequence, as beam search would pick."""
+def beam_parents(w: Workload, step: int, keep_prob: float = 0.0) -> np.ndarray:
+    """A parent beam (0..beam-1) for every sequence, as beam search would pick: with probability
+    ``keep_prob`` a hypothesis continues itself, otherwise its parent is drawn uniformly."""
     rng = np.random.default_rng([int(w.seed), TAG_PARENT, int(step)])
-    return rng.integers(0, w.beam, size=w.n_seqs, dtype=np.int64).astype(np.int32)
+    parent = rng.integers(0, w.beam, size=w.n_seqs, dtype=np.int64).astype(np.int32)
+    if keep_prob > 0.0:
+        keep = rng.random(w.n_seqs) < keep_prob
+        parent = np.where(keep, np.arange(w.n_seqs) % w.beam, parent).astype(np.int32)
+    return parent
 
 
 def self_prefill(w: Workload, layer: int):

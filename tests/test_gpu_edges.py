@@ -163,6 +163,24 @@ def test_host_checks_on_a_live_context():
     dec.close()
 
 
+def test_step_refuses_rows_beyond_what_its_kernels_can_cut():
+    """A length bound that would need more spans than the one-launch step has is refused on the host
+    (SAN_ERR_UNSUPPORTED, nothing launched, the call returns at once); the separate calls take it."""
+    w = _small(n_sent=1, beam=4, n_heads=1, tgt_fixed=40000, src_lo=9000, src_hi=9000, n_layers=2, self_blocks=(2,), encdec_blocks=(2,))
+    dec = Decoder(w)
+    sb = dec.new_step_buffers()
+    kw = dict(d_seq_ids=sb.ids, n_seqs=w.n_seqs, d_O_self=sb.O_self, d_q_enc=sb.q_enc, d_sent_ids=sb.sent_ids,
+              d_src_lens=sb.src_lens, n_sent=w.n_sent, d_S_enc=sb.S_enc, ld_s=dec.ld_s, d_O_enc=sb.O_enc, d_q_self=sb.q_self,
+              d_k_new=sb.k_new, d_v_new=sb.v_new, d_pos=sb.pos, d_S_self=sb.S_self, ld_t=dec.ld_t)
+    assert B.san_decode_step(dec.ctx, max_len=0, max_src=16, **kw) == B.SAN_ERR_UNSUPPORTED      # 40000 target positions
+    assert B.san_decode_step(dec.ctx, max_len=16, max_src=0, **kw) == B.SAN_ERR_UNSUPPORTED      # 9000 source positions x 4 beams
+    kw_enc = dict(kw, n_seqs=0)
+    assert B.san_decode_step(dec.ctx, max_len=0, max_src=0, **kw_enc) == B.SAN_ERR_UNSUPPORTED
+    assert B.san_decode_step(dec.ctx, max_len=16, max_src=16, **kw) == B.SAN_OK                  # small bounds on the same context run
+    assert dec.device_status()[0] == 0
+    dec.close()
+
+
 def test_policy_tables_and_runtime_change():
     """Integer tables are bit-exact; a policy with more blocks than key planes is refused."""
     w = _small(self_blocks=(2, 2), encdec_blocks=(4,))
