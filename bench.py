@@ -279,40 +279,59 @@ def dominant_kernel_bytes(w, pos):
     return float(np.mean(per))
 
 
-def time_e2e(w, dec, sb, steps, device, fused=True):
+def time_e2e(w, decs, sbs, steps, device, fused=True):
     """The same step with HOST buffers: every step copies its inputs from pinned host memory
     to the device, runs the library, and reads the outputs back.  On the one-launch path this
-    is a single C-ABI call, san_decode_step_host, which issues the copies itself."""
+    is a single C-ABI call, san_decode_step_host, which issues the copies itself on the
+    caller's stream.  Two request batches (two contexts, each with its own stream and pinned
+    buffers) take turns, the way a server keeps PCIe busy in both directions: the copies of one
+    batch overlap the other's.  Returns (seconds for `steps` steps with two batches in flight,
+    seconds for `steps` steps of one batch alone, h2d bytes per step, d2h bytes per step)."""
     import torch
-    hb = dec.host_buffers(sb)
-    lens_host = sb.lens.cpu().pin_memory()           # the separate calls take lengths, the one-launch step positions
-    h2d = sum(hb[k].numel() * hb[k].element_size() for k in hb["_in"]) + (0 if fused else lens_host.numel() * 4)
+    n_ctx = 2 if len(decs) > 1 else 1
+    hbs = [decs[i].host_buffers(sbs[i]) for i in range(n_ctx)]
+    streams = [torch.cuda.Stream(device) for _ in range(n_ctx)]
+    hb = hbs[0]
+    lens_host = [sbs[i].lens.cpu().pin_memory() for i in range(n_ctx)]   # the separate calls take lengths, the one-launch step positions
+    h2d = sum(hb[k].numel() * hb[k].element_size() for k in hb["_in"]) + (0 if fused else lens_host[0].numel() * 4)
     d2h = sum(hb[k].numel() * hb[k].element_size() for k in hb["_out"])
     dev_of = {"d_seq_ids": "ids", "d_pos": "pos", "d_sent_ids": "sent_ids", "d_src_lens": "src_lens",
               "d_q_enc": "q_enc", "d_q_self": "q_self", "d_k_new": "k_new", "d_v_new": "v_new",
               "d_x_aan": "x_aan", "d_t": "t_aan", "d_O_self": "O_self", "d_O_enc": "O_enc"}
 
-    def one():
-        if fused:
-            dec.step_fused_host(sb, hb)
-            return
-        for k in hb["_in"]:
-            getattr(sb, dev_of[k]).copy_(hb[k], non_blocking=True)
-        sb.lens.copy_(lens_host, non_blocking=True)
-        dec.step(sb)
-        for k in hb["_out"]:
-            hb[k].copy_(getattr(sb, dev_of[k]), non_blocking=True)
+    def one(i):
+        dec, sb, hb = decs[i], sbs[i], hbs[i]
+        with torch.cuda.stream(streams[i]):
+            if fused:
+                dec.step_fused_host(sb, hb, stream=streams[i])
+                return
+            for k in hb["_in"]:
+                getattr(sb, dev_of[k]).copy_(hb[k], non_blocking=True)
+            sb.lens.copy_(lens_host[i], non_blocking=True)
+            dec.step(sb, stream=streams[i])
+            for k in hb["_out"]:
+                hb[k].copy_(getattr(sb, dev_of[k]), non_blocking=True)
 
-    for _ in range(3):
-        one()
-    torch.cuda.synchronize(device)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(steps):
-        one()
-    e1.record()
-    torch.cuda.synchronize(device)
-    return e0.elapsed_time(e1) * 1e-3, h2d, d2h
+    def timed(n_active):
+        for i in range(3 * n_active):
+            one(i % n_active)
+        torch.cuda.synchronize(device)
+        cur = torch.cuda.current_stream(device)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(cur)
+        for st in streams[:n_active]:
+            st.wait_event(e0)
+        for i in range(steps):
+            one(i % n_active)
+        for st in streams[:n_active]:
+            cur.wait_stream(st)
+        e1.record(cur)
+        torch.cuda.synchronize(device)
+        return e0.elapsed_time(e1) * 1e-3
+
+    serial = timed(1)
+    both = timed(n_ctx) if n_ctx > 1 else serial
+    return both, serial, h2d, d2h
 
 
 def time_beam_reorder(w, decs, sbs, pos, device, peak, reps=10):
@@ -687,7 +706,7 @@ def main():
                 "unit": "GB/s", "frac": dom_bytes / dom_s / 1e9 / peak, "peak_kind": peak_kind, "bytes_per_launch": dom_bytes,
                 "us_per_launch": dom_s * 1e6, "launches_per_step": dom_per_step, "traffic": None}
     e2e_steps = min(args.steps, 100)
-    e2e_s, h2d, d2h = time_e2e(w, decs[0], sbs[0], e2e_steps, device, fused)
+    e2e_s, e2e_serial_s, h2d, d2h = time_e2e(w, decs, sbs, e2e_steps, device, fused)
     next_rows = {}
     if rank == 0 and not args.only:
         next_rows["beam_reorder"] = time_beam_reorder(w, decs, sbs, pos, device, peak)
@@ -786,7 +805,10 @@ def main():
                 "kv_gbs": ab["kv"] / (secs_max / args.steps) / 1e9, "peak_kind": peak_kind},
         "roofline": roof,
         "e2e": {"value": w.n_seqs * e2e_steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
-                "d2h_bytes_per_step": d2h, "ms_per_step": e2e_s / e2e_steps * 1e3},
+                "d2h_bytes_per_step": d2h, "ms_per_step": e2e_s / e2e_steps * 1e3,
+                "one_batch_alone_ms_per_step": e2e_serial_s / e2e_steps * 1e3,
+                "how": "san_decode_step_host, one C-ABI call per step with pinned host buffers; two request batches "
+                       "(two contexts, two streams) take turns so that uploads and downloads overlap"},
         "clocks": clocks,
     }
     if workloads:

@@ -342,8 +342,10 @@ int32_t san_device_status(san_ctx* ctx, int32_t* first_error, int32_t* detail, v
  *              [1..4] = kernel tag, item, value, limit if an item was skipped
  *
  * Limits: n_items * n_heads <= 65536 rows, else SAN_ERR_CAPACITY (use a context instead).
- * The first call on each device looks up the array's device address (with that device
- * current); make that first call before any stream capture begins.  Every call on a
+ * The device that owns `stream` and every buffer must be the current device at the call, on
+ * every call and not only the first (the call uses that device's copy of the array and does
+ * not check whose stream it was given).  The first call on each device looks up the array's
+ * device address; make that first call before any stream capture begins.  Every call on a
  * device uses the same array and finds what the previous call left there; the call clears
  * the tickets and status words it needs on `stream` before launching.  Two calls whose
  * kernels may overlap on one GPU (different streams without an event between them, or
