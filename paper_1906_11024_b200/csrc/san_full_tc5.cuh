@@ -35,6 +35,10 @@ constexpr int kTcChunk = 64;              // keys per MMA chain
 constexpr int kTcThreads = 256;
 constexpr int kTcSplit = kTcThreads / kTcQ;   // threads per query row; each takes 64 / kTcSplit score columns
 constexpr int kTcCols1 = kTcChunk / kTcSplit;  // score columns per thread
+// Apply the weights as a bf16 high part plus a bf16 remainder (two MMAs per key step) or as the high
+// part alone.  The outputs are bf16: their own rounding (2^-9) is what shows against the float64
+// reference either way (tolerance 1e-2), so the remainder is left out.
+constexpr bool kTcRemainder = false;
 constexpr int kTcMaxLayers = 6;           // accumulators: 64 columns each after the 64 of the scores (512 columns in all)
 constexpr int kTcCols = 512;
 constexpr uint32_t kTcScores1 = 448;       // second score buffer: the 64 columns behind the six accumulators
@@ -250,28 +254,29 @@ static __global__ void __launch_bounds__(kTcThreads, 1) full_block_tc5_kernel(co
         }
         const int kh = k0 + part * kTcCols1;      // first key of this thread's part
         float m_chunk = -INFINITY;
+        // z stays unscaled: the scale (positive, so it commutes with the maximum) is folded into the
+        // exponent's argument, ex2(z * scale - m), one multiply-add per score
+        const float sc = p.scale_log2e;
         if (k0 + kTcChunk <= len && (!p.causal || k0 + kTcChunk - 1 <= q0)) {
             // every row of the tile sees every key of the chunk (uniform over the CTA): no masks
 #pragma unroll
-            for (int j = 0; j < kTcCols1; ++j) {
-                z[j] *= p.scale_log2e;
-                m_chunk = fmaxf(m_chunk, z[j]);
-            }
+            for (int j = 0; j < kTcCols1; ++j) m_chunk = fmaxf(m_chunk, z[j]);
         } else {
 #pragma unroll
             for (int j = 0; j < kTcCols1; ++j) {
                 const int key = kh + j;
                 const bool ok = key < len && (!p.causal || key <= qrow);
-                z[j] = ok ? z[j] * p.scale_log2e : -INFINITY;
+                z[j] = ok ? z[j] : -INFINITY;
                 m_chunk = fmaxf(m_chunk, z[j]);
             }
         }
+        m_chunk *= sc;
         if (pass == 0) {
             const float m_new = fmaxf(m_run, m_chunk);
             if (m_new > -INFINITY) {
                 float s = s_run * exp2f(m_run - m_new);
 #pragma unroll
-                for (int j = 0; j < kTcCols1; ++j) s += tc_ex2(z[j] - m_new);
+                for (int j = 0; j < kTcCols1; ++j) s += tc_ex2(fmaf(z[j], sc, -m_new));
                 s_run = s; m_run = m_new;
             }
             continue;
@@ -282,10 +287,10 @@ static __global__ void __launch_bounds__(kTcThreads, 1) full_block_tc5_kernel(co
         uint32_t hi[kTcCols1 / 2], lo[kTcCols1 / 2];
 #pragma unroll
         for (int e = 0; e < kTcCols1 / 2; ++e) {
-            const float w0 = tc_ex2(z[2 * e] - m_use) * inv, w1 = tc_ex2(z[2 * e + 1] - m_use) * inv;
+            const float w0 = tc_ex2(fmaf(z[2 * e], sc, -m_use)) * inv, w1 = tc_ex2(fmaf(z[2 * e + 1], sc, -m_use)) * inv;
             z[2 * e] = w0; z[2 * e + 1] = w1;
             hi[e] = full_pack(w0, w1);
-            lo[e] = full_pack(w0 - __uint_as_float(hi[e] << 16), w1 - __uint_as_float(hi[e] & 0xffff0000u));
+            if (kTcRemainder) lo[e] = full_pack(w0 - __uint_as_float(hi[e] << 16), w1 - __uint_as_float(hi[e] & 0xffff0000u));
         }
         if (Srow) {
 #pragma unroll
@@ -298,7 +303,7 @@ static __global__ void __launch_bounds__(kTcThreads, 1) full_block_tc5_kernel(co
         for (int c = 0; c < kTcCols1 / 8; ++c) {  // 8 keys = one 16-byte chunk of the operand rows; this part owns chunks part * kTcCols1 / 8 ..
             const int at = row * 128 + (((part * (kTcCols1 / 8) + c) ^ (row & 7)) << 4);
             *reinterpret_cast<uint4*>(sPh + at) = make_uint4(hi[4 * c], hi[4 * c + 1], hi[4 * c + 2], hi[4 * c + 3]);
-            *reinterpret_cast<uint4*>(sPl + at) = make_uint4(lo[4 * c], lo[4 * c + 1], lo[4 * c + 2], lo[4 * c + 3]);
+            if (kTcRemainder) *reinterpret_cast<uint4*>(sPl + at) = make_uint4(lo[4 * c], lo[4 * c + 1], lo[4 * c + 2], lo[4 * c + 3]);
         }
         asm volatile("cp.async.wait_group 2;" ::: "memory");         // values of step t have landed
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -317,7 +322,7 @@ static __global__ void __launch_bounds__(kTcThreads, 1) full_block_tc5_kernel(co
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks) {  // 16 keys per step: 32 bytes along a weight row, two 8-row groups of values
                     tc_mma(acc, dPh + 2 * ks, dV + 128 * ks, idO, (kc > 0 || ks > 0) ? 1u : 0u);
-                    tc_mma(acc, dPl + 2 * ks, dV + 128 * ks, idO, 1u);
+                    if (kTcRemainder) tc_mma(acc, dPl + 2 * ks, dV + 128 * ks, idO, 1u);
                 }
             }
             tc_commit(bar_o);
