@@ -44,7 +44,9 @@ FALLBACK_HBM_GBS = 6650.0
 # counters no longer describe the kernel, and the line reports null until a new capture is
 # recorded here.
 KERNEL_SOURCES = ("san_fused.cuh", "san_step.cuh", "san_kernels.cuh", "san_api.cu")
-NCU_TRAFFIC = {"digest": "", "fused": {}}
+NCU_TRAFFIC = {"digest": "42838876b574e926",
+               "fused": {"long": 735.4e6, "base": 70.2e6, "big": 426.7e6, "aan": 25.4e6,
+                         "long-unshared": 1256.6e6, "base-unshared": 104.8e6}}
 
 
 def kernel_digest():
