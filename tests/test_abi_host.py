@@ -62,7 +62,7 @@ def test_query_bytes_counts_key_planes_only_for_block_first_layers(lib):
     (dict(d_head=32), B.SAN_ERR_UNSUPPORTED),
     (dict(n_layers=0), B.SAN_ERR_SHAPE),
     (dict(n_layers=65), B.SAN_ERR_SHAPE),
-    (dict(beam=9), B.SAN_ERR_SHAPE),
+    (dict(beam=B.SAN_MAX_BEAM + 1), B.SAN_ERR_SHAPE),
     (dict(beam=0), B.SAN_ERR_SHAPE),
     (dict(max_tgt_len=0), B.SAN_ERR_SHAPE),
     (dict(dtype=7), B.SAN_ERR_DTYPE),
