@@ -917,11 +917,25 @@ __global__ void __launch_bounds__(kFusedWarps * 32, 1) decode_step_kernel(const 
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
 
-    // ---- AAN running average (Table 6 pairing): element-wise, every thread of the grid
-    if (p.x_aan) {
+    // ---- AAN running average (Table 6 pairing): element-wise.  The CTA's share is cut into chunks of
+    // 32 lanes x 4 columns that its warps take from a shared counter once they have no attention
+    // item left (or never had one), so that the averages run beside the attention items' chains
+    // and not ahead of them.
+    __shared__ unsigned aan_next;
+    if (threadIdx.x == 0) aan_next = 0u;
+    auto aan_part = [&]() {
+        if (!p.x_aan) return;
         const int d = p.H * kDh, d4 = d >> 2;
         const long long total = (long long)p.n_aan_layers * p.n_aan_seqs * d4;
-        for (long long u = (long long)blockIdx.x * blockDim.x + threadIdx.x; u < total; u += (long long)gridDim.x * blockDim.x) {
+        const long long n_chunks = (total + 31) / 32;
+        for (;;) {
+            unsigned j = 0;
+            if (lane == 0) j = atomicAdd(&aan_next, 1u);
+            j = __shfl_sync(0xffffffffu, j, 0);
+            const long long ck = (long long)blockIdx.x + (long long)j * gridDim.x;
+            if (ck >= n_chunks) break;
+            const long long u = ck * 32 + lane;
+            if (u >= total) continue;
             const int c4 = (int)(u % d4);
             const int item = (int)((u / d4) % p.n_aan_seqs);
             const int lr = (int)(u / ((long long)d4 * p.n_aan_seqs));
@@ -952,8 +966,8 @@ __global__ void __launch_bounds__(kFusedWarps * 32, 1) decode_step_kernel(const 
                 *reinterpret_cast<float4*>(p.aan_out + io * 4) = make_float4(o[0], o[1], o[2], o[3]);
             }
         }
-    }
-    if (p.n_items == 0) return;
+    };
+    if (p.n_items == 0) { __syncthreads(); aan_part(); return; }
 
     // ---- attention items.  CTA b owns list slots b, b + G, b + 2G, ...  It takes them in rounds
     // of kCtaItems slots: every thread decodes one slot, the survivors are packed in list order
@@ -971,6 +985,7 @@ __global__ void __launch_bounds__(kFusedWarps * 32, 1) decode_step_kernel(const 
     w.p_stage = 0; w.c_stage = 0; w.c_par = 0; w.dead = false; w.p_active = false;
 
     const unsigned long long my_slots = (p.n_items > blockIdx.x) ? ((unsigned long long)p.n_items - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+    if (my_slots == 0) { __syncthreads(); aan_part(); }     // a CTA without attention items still has its share of the averages
     for (unsigned long long k0 = 0; k0 < my_slots; k0 += kCtaItems) {
         // -- decode: thread t takes slot k0 + t; survivors keep their order
         ItemDesc mine;
@@ -1008,6 +1023,7 @@ __global__ void __launch_bounds__(kFusedWarps * 32, 1) decode_step_kernel(const 
                 if (NQE > 1 && d.kind) w.template process<NQE>(d); else w.template process<1>(d);
             }
         }
+        if (k0 == 0) aan_part();      // warps that are out of attention items (or never had one) take the averages
         // a warp whose wait ran out stops working but keeps meeting the CTA at the barriers above
     }
 }
