@@ -13,6 +13,7 @@
 #include "san_kernels.cuh"
 #include "san_fused.cuh"
 #include "san_step.cuh"
+#include "san_rows.cuh"
 #include "san_reorder.cuh"
 #include "san_learn.cuh"
 #include "san_full.cuh"
@@ -655,7 +656,7 @@ static int32_t decode_step_launch(san_ctx* ctx, const san_step_args* a, int max_
     const bool aan = c.self_is_aan != 0;
     const int n_seqs = a->n_seqs, n_sent = a->n_sent;
     const bool bf16 = c.dtype == SAN_BF16;
-    if (ctx->step_kernel != 1) {       // automatic: the team-pipeline kernel for steps with rows long enough to be split over a team
+    if (ctx->step_kernel == 0 || ctx->step_kernel == 2) {       // automatic: the team-pipeline kernel for steps with rows long enough to be split over a team
         const int32_t rc = launch_team_step(ctx, a, max_len, max_src, static_cast<cudaStream_t>(stream), ctx->last_rows_per_unit,
                                             ctx->step_kernel == 0 && ctx->team_cut_override[0] < 0, q_first, q_count);
         if (rc != SAN_ERR_UNSUPPORTED) { ctx->last_step_kernel = 2; return rc; }
@@ -667,6 +668,12 @@ static int32_t decode_step_launch(san_ctx* ctx, const san_step_args* a, int max_
     const int nqe = pick_nq_template(q_count);
     const bool do_self = n_seqs > 0 && !aan;
     const bool do_enc = n_sent > 0;
+    // Sentence-sized rows (every row a handful of 16-position blocks): the kernel that takes a whole
+    // plane per copy and keeps the scores in registers.
+    const bool rows_fit = bf16 && (!do_self || (max_len <= kRowsMaxPos && (max_len + 1) * 128 <= kRowsRing)) &&
+                          (!do_enc || (max_src <= kRowsMaxPos && (max_src + nqe) * 128 <= kRowsRing));
+    if (ctx->step_kernel == 3 && !rows_fit) return SAN_ERR_UNSUPPORTED;
+    const bool use_rows = rows_fit && (ctx->step_kernel == 3 || (ctx->step_kernel == 0 && kRowsKernelByDefault));
     int pi_self = 1, pi_enc = 1;
     for (int b = 0; b < ctx->self_pol.n_blocks; ++b) pi_self = std::max(pi_self, ctx->self_pol.size_of_block[b]);
     for (int b = 0; b < ctx->enc_pol.n_blocks; ++b) pi_enc = std::max(pi_enc, ctx->enc_pol.size_of_block[b]);
@@ -714,7 +721,13 @@ static int32_t decode_step_launch(san_ctx* ctx, const san_step_args* a, int max_
     // ways of cutting (halved spans, halved layer groups, or no cut at all) by the estimated length
     // of the step: items of equal size that divide evenly over the warps beat smaller items that
     // leave a warp with one more than its neighbours.  The choice is remembered per launch shape.
-    if (span_self < cap_self || lg_self < pi_self || span_enc < cap_enc || lg_enc < pi_enc) {
+    if (use_rows) {      // whole rows; layers per item as above unless told otherwise
+        span_self = cap_self; span_enc = cap_enc;
+        const int o = ctx->team_cut_override[3];
+        const int o_enc = (o >> 8) > 0 ? (o >> 8) - 1 : (o & 255);     // as in san_step_kernel_select
+        if (ctx->step_kernel == 3 && (o & 255) > 0) lg_self = std::min(pi_self, o & 255);
+        if (ctx->step_kernel == 3 && o_enc > 0) lg_enc = std::min(pi_enc, o_enc);
+    } else if (span_self < cap_self || lg_self < pi_self || span_enc < cap_enc || lg_enc < pi_enc) {
         const int len_b = std::min(c.max_tgt_len, (int)align_up((size_t)max_len, TR)), src_b = std::min(c.max_src_len, (int)align_up((size_t)max_src, TR));
         san_ctx::StepPlan* plan = nullptr;
         for (auto& pl : ctx->plans)
@@ -833,6 +846,27 @@ static int32_t decode_step_launch(san_ctx* ctx, const san_step_args* a, int max_
         p.n_aan_layers = c.n_layers; p.n_aan_seqs = n_seqs; p.aan_max_seqs = ctx->n_seqs; p.aan_max_t = c.max_tgt_len;
     }
 
+    if (use_rows) {
+        ctx->last_step_kernel = 3;
+        const void* rfn = (const void*)decode_step_rows_kernel;
+        const size_t rsmem = rows_smem_bytes();
+        if (!ctx->rows_attr_set) {
+            if (cudaFuncSetAttribute(rfn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rsmem) != cudaSuccess) return SAN_ERR_CUDA;
+            ctx->rows_attr_set = true;
+        }
+        long long rctas = std::min<long long>(ctx->sm_count, (p.n_items + kRowsWarps - 1) / kRowsWarps);
+        if (p.x_aan) rctas = ctx->sm_count;
+        if (rctas < 1) rctas = 1;
+        cudaLaunchAttribute rattr;
+        rattr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        rattr.val.programmaticStreamSerializationAllowed = 1;
+        cudaLaunchConfig_t rcfg = {};
+        rcfg.gridDim = dim3((unsigned)rctas); rcfg.blockDim = dim3(kRowsWarps * 32);
+        rcfg.dynamicSmemBytes = rsmem; rcfg.stream = static_cast<cudaStream_t>(stream);
+        rcfg.attrs = &rattr; rcfg.numAttrs = 1;
+        void* rargs[] = {&p};
+        return cuda_status(cudaLaunchKernelExC(&rcfg, rfn, rargs));
+    }
     const void* fn = nullptr;
     if (bf16) fn = nqe == 1 ? (const void*)decode_step_kernel<__nv_bfloat16, 1> : nqe == 2 ? (const void*)decode_step_kernel<__nv_bfloat16, 2>
                    : nqe == 4 ? (const void*)decode_step_kernel<__nv_bfloat16, 4> : (const void*)decode_step_kernel<__nv_bfloat16, 8>;
@@ -893,7 +927,7 @@ int32_t san_decode_step(san_ctx* ctx, const san_step_args* a, void* stream) {
 int32_t san_step_kernel_select(san_ctx* ctx, int32_t which, int32_t spans_log2, int32_t heads_per_unit, int32_t tile_pos,
                                int32_t layers_per_unit, int32_t grab_mult) {
     if (!ctx) return SAN_ERR_NULL;
-    if (which < 0 || which > 2) return SAN_ERR_RANGE;
+    if (which < 0 || which > 3) return SAN_ERR_RANGE;
     if (spans_log2 >= 0 && ((tile_pos & 255) < 16 || heads_per_unit < 1)) return SAN_ERR_RANGE;
     ctx->step_kernel = which;
     ctx->team_cut_override[0] = spans_log2 < 0 ? -1 : spans_log2;

@@ -29,7 +29,8 @@ struct san_ctx {
     float* part = nullptr;
     bool fused_attr_set = false;   // shared-memory opt-in of the one-launch step kernel done
     bool team_attr_set = false;    // the same for the team-pipeline step kernel
-    int step_kernel = 0;           // 0: automatic, 1: per-warp pipeline kernel, 2: team-pipeline kernel (san_step_kernel_select)
+    bool rows_attr_set = false;    // and for the short-rows step kernel
+    int step_kernel = 0;           // 0: automatic, 1: per-warp pipeline kernel, 2: team-pipeline kernel, 3: short-rows kernel (san_step_kernel_select)
     int team_cut_override[4] = {-1, 4, 64, 0};   // spans per row (log2; -1: automatic), heads per unit, positions per tile, layers per unit (0: automatic)
     int team_grab_mult = 1;
     int last_step_kernel = 0;      // which kernel the last san_decode_step launched (0: none yet)

@@ -123,13 +123,36 @@ __device__ __forceinline__ bool mbar_try_wait_hint(uint32_t bar, uint32_t parity
                  : "=r"(ok) : "r"(bar), "r"(parity), "r"(hint) : "memory");
     return ok != 0;
 }
+// Polls the barrier up to `tries` times, each try suspending the thread for a while; true once the
+// phase is complete.  A suspended thread is woken whenever any barrier of the CTA completes, far more
+// often than its own does, so the loop is kept to four instructions a turn.
+__device__ __forceinline__ bool mbar_poll(uint32_t bar, uint32_t parity, uint32_t hint, uint32_t tries) {
+    uint32_t ok;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        ".reg .u32 n;\n"
+        "mov.u32 n, %4;\n"
+        "POLL:\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n"
+        "@p bra DONE;\n"
+        "sub.u32 n, n, 1;\n"
+        "setp.ne.u32 p, n, 0;\n"
+        "@p bra POLL;\n"
+        "setp.ne.u32 p, n, 0;\n"
+        "DONE:\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(ok) : "r"(bar), "r"(parity), "r"(hint), "r"(tries) : "memory");
+    return ok != 0;
+}
 // Bounded wait: gives up after about a second and reports it; never spins for ever.
 __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity) {
     const long long t0 = clock64();
-    while (!mbar_try_wait_hint(bar, parity, 2000000u)) {
-        if (clock64() - t0 > 2000000000LL) return false;
-    }
-    return true;
+    do {
+        if (mbar_poll(bar, parity, 2000000u, 4096u)) return true;
+    } while (clock64() - t0 < 2000000000LL);
+    return false;
 }
 
 // Four 8x8 b16 matrices from shared memory, one row address per lane (plain / transposed).
@@ -888,6 +911,56 @@ __device__ __noinline__ void combine_spans(const StepParams& p, const ItemDesc& 
     if (lane == 0) p.tickets[d.row_id] = 0;
 }
 
+// AAN running average (Table 6 pairing): element-wise.  A CTA's share is cut into chunks of
+// 32 lanes x 4 columns that its warps take from a counter in shared memory once they have no
+// attention item left (or never had one), so that the averages run beside the attention items'
+// chains and not ahead of them.  Called by whole warps; *aan_next starts at zero.
+template <typename T>
+__device__ __forceinline__ void aan_chunks(const StepParams& p, int lane, unsigned* aan_next) {
+    if (!p.x_aan) return;
+    const int d = p.H * kDh, d4 = d >> 2;
+    const long long total = (long long)p.n_aan_layers * p.n_aan_seqs * d4;
+    const long long n_chunks = (total + 31) / 32;
+    for (;;) {
+        unsigned j = 0;
+        if (lane == 0) j = atomicAdd(aan_next, 1u);
+        j = __shfl_sync(0xffffffffu, j, 0);
+        const long long ck = (long long)blockIdx.x + (long long)j * gridDim.x;
+        if (ck >= n_chunks) break;
+        const long long u = ck * 32 + lane;
+        if (u >= total) continue;
+        const int c4 = (int)(u % d4);
+        const int item = (int)((u / d4) % p.n_aan_seqs);
+        const int lr = (int)(u / ((long long)d4 * p.n_aan_seqs));
+        const int id = p.aan_ids[item], t = p.t_aan[item];
+        if (id < 0 || id >= p.aan_max_seqs) { if (c4 == 0 && lr == 0) record_error(p.err, TAG_AAN, item, id, p.aan_max_seqs); continue; }
+        if (t < 1 || t > p.aan_max_t) { if (c4 == 0 && lr == 0) record_error(p.err, TAG_AAN, item, t, p.aan_max_t); continue; }
+        const long long io = ((long long)lr * p.n_aan_seqs + item) * d + c4 * 4;
+        float xv[4];
+        if (sizeof(T) == 2) {
+            const uint2 raw = *reinterpret_cast<const uint2*>(p.x_aan + io * 2);
+            xv[0] = __uint_as_float(raw.x << 16); xv[1] = __uint_as_float(raw.x & 0xffff0000u);
+            xv[2] = __uint_as_float(raw.y << 16); xv[3] = __uint_as_float(raw.y & 0xffff0000u);
+        } else {
+            const float4 raw = *reinterpret_cast<const float4*>(p.x_aan + io * 4);
+            xv[0] = raw.x; xv[1] = raw.y; xv[2] = raw.z; xv[3] = raw.w;
+        }
+        float4* sum = reinterpret_cast<float4*>(p.aan_sum + ((long long)lr * p.aan_max_seqs + id) * d + c4 * 4);
+        float4 s = (t == 1) ? make_float4(0.f, 0.f, 0.f, 0.f) : *sum;
+        s.x += xv[0]; s.y += xv[1]; s.z += xv[2]; s.w += xv[3];
+        *sum = s;
+        const float ft = (float)t;
+        const float o[4] = {s.x / ft, s.y / ft, s.z / ft, s.w / ft};
+        if (sizeof(T) == 2) {
+            __nv_bfloat162 a = __floats2bfloat162_rn(o[0], o[1]), b = __floats2bfloat162_rn(o[2], o[3]);
+            uint2 r; r.x = *reinterpret_cast<uint32_t*>(&a); r.y = *reinterpret_cast<uint32_t*>(&b);
+            *reinterpret_cast<uint2*>(p.aan_out + io * 2) = r;
+        } else {
+            *reinterpret_cast<float4*>(p.aan_out + io * 4) = make_float4(o[0], o[1], o[2], o[3]);
+        }
+    }
+}
+
 constexpr int kCtaItems = 144;      // decoded items a CTA holds at a time (at most 255: the warps queue them by byte)
 constexpr size_t fused_smem_bytes() {
     return (size_t)kFusedWarps * (kFusedStages * kStageBytes + kZFloats * sizeof(float) + kFusedStages * sizeof(uint64_t)) +
@@ -917,56 +990,10 @@ __global__ void __launch_bounds__(kFusedWarps * 32, 1) decode_step_kernel(const 
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
 
-    // ---- AAN running average (Table 6 pairing): element-wise.  The CTA's share is cut into chunks of
-    // 32 lanes x 4 columns that its warps take from a shared counter once they have no attention
-    // item left (or never had one), so that the averages run beside the attention items' chains
-    // and not ahead of them.
+    // ---- AAN running average: see aan_chunks
     __shared__ unsigned aan_next;
     if (threadIdx.x == 0) aan_next = 0u;
-    auto aan_part = [&]() {
-        if (!p.x_aan) return;
-        const int d = p.H * kDh, d4 = d >> 2;
-        const long long total = (long long)p.n_aan_layers * p.n_aan_seqs * d4;
-        const long long n_chunks = (total + 31) / 32;
-        for (;;) {
-            unsigned j = 0;
-            if (lane == 0) j = atomicAdd(&aan_next, 1u);
-            j = __shfl_sync(0xffffffffu, j, 0);
-            const long long ck = (long long)blockIdx.x + (long long)j * gridDim.x;
-            if (ck >= n_chunks) break;
-            const long long u = ck * 32 + lane;
-            if (u >= total) continue;
-            const int c4 = (int)(u % d4);
-            const int item = (int)((u / d4) % p.n_aan_seqs);
-            const int lr = (int)(u / ((long long)d4 * p.n_aan_seqs));
-            const int id = p.aan_ids[item], t = p.t_aan[item];
-            if (id < 0 || id >= p.aan_max_seqs) { if (c4 == 0 && lr == 0) record_error(p.err, TAG_AAN, item, id, p.aan_max_seqs); continue; }
-            if (t < 1 || t > p.aan_max_t) { if (c4 == 0 && lr == 0) record_error(p.err, TAG_AAN, item, t, p.aan_max_t); continue; }
-            const long long io = ((long long)lr * p.n_aan_seqs + item) * d + c4 * 4;
-            float xv[4];
-            if (sizeof(T) == 2) {
-                const uint2 raw = *reinterpret_cast<const uint2*>(p.x_aan + io * 2);
-                xv[0] = __uint_as_float(raw.x << 16); xv[1] = __uint_as_float(raw.x & 0xffff0000u);
-                xv[2] = __uint_as_float(raw.y << 16); xv[3] = __uint_as_float(raw.y & 0xffff0000u);
-            } else {
-                const float4 raw = *reinterpret_cast<const float4*>(p.x_aan + io * 4);
-                xv[0] = raw.x; xv[1] = raw.y; xv[2] = raw.z; xv[3] = raw.w;
-            }
-            float4* sum = reinterpret_cast<float4*>(p.aan_sum + ((long long)lr * p.aan_max_seqs + id) * d + c4 * 4);
-            float4 s = (t == 1) ? make_float4(0.f, 0.f, 0.f, 0.f) : *sum;
-            s.x += xv[0]; s.y += xv[1]; s.z += xv[2]; s.w += xv[3];
-            *sum = s;
-            const float ft = (float)t;
-            const float o[4] = {s.x / ft, s.y / ft, s.z / ft, s.w / ft};
-            if (sizeof(T) == 2) {
-                __nv_bfloat162 a = __floats2bfloat162_rn(o[0], o[1]), b = __floats2bfloat162_rn(o[2], o[3]);
-                uint2 r; r.x = *reinterpret_cast<uint32_t*>(&a); r.y = *reinterpret_cast<uint32_t*>(&b);
-                *reinterpret_cast<uint2*>(p.aan_out + io * 2) = r;
-            } else {
-                *reinterpret_cast<float4*>(p.aan_out + io * 4) = make_float4(o[0], o[1], o[2], o[3]);
-            }
-        }
-    };
+    auto aan_part = [&]() { aan_chunks<T>(p, lane, &aan_next); };
     if (p.n_items == 0) { __syncthreads(); aan_part(); return; }
 
     // ---- attention items.  CTA b owns list slots b, b + G, b + 2G, ...  It takes them in rounds

@@ -157,11 +157,11 @@ __device__ __forceinline__ bool mbar_try_wait_for(uint32_t bar, uint32_t parity,
 // Bounded wait that also gives up as soon as another warp of the CTA has given up.
 __device__ __noinline__ bool step_wait_slow(uint32_t bar, uint32_t parity, volatile int* dead) {
     const long long t0 = clock64();
-    while (!mbar_try_wait_for(bar, parity, kWaitHint)) {
+    do {
+        if (mbar_poll(bar, parity, kWaitHint, 1024u)) return true;
         if (*dead) return false;
-        if (clock64() - t0 > 2000000000LL) return false;
-    }
-    return true;
+    } while (clock64() - t0 < 2000000000LL);
+    return false;
 }
 
 // ------------------------------------------------------------------------------ the producer

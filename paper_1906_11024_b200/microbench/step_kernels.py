@@ -29,6 +29,7 @@ def main():
     ap.add_argument("--n-seqs", default="")
     ap.add_argument("--replicas", type=int, default=6)
     ap.add_argument("--reps", type=int, default=300)
+    ap.add_argument("--unshared", action="store_true", help="every block one layer (sharing off)")
     args = ap.parse_args()
 
     import torch
@@ -40,6 +41,8 @@ def main():
     B.lib()
     dev = torch.device("cuda:0")
     w = synth.WORKLOADS[args.workload]
+    if args.unshared:
+        w = synth.unshared(w)
     decs, sbs, _ = bench.build_replicas(w, args.replicas, dev)
     R = len(decs)
 

@@ -82,6 +82,8 @@ def _run(w, check_steps=None, max_steps=None, shared_context=False, jumps=None, 
             step_id = g if start is None else 100000 + start + g
             host = dec.fill_step_inputs(sb, step_id, active, pos[active], sent)
             (dec.step_fused if fused else dec.step)(sb)
+            if fused and STEP_KERNEL[0]:
+                assert B.san_step_kernel_used(dec.ctx)[1] == STEP_KERNEL[0]      # the forced kernel is the one that ran
             do_check = check_steps is None or g in check_steps
             ref = orc.step(host, active, pos[active], want_S=do_check)
             if do_check:
@@ -222,7 +224,31 @@ def test_one_launch_step_team_pipeline_matches_oracle(case):
         STEP_KERNEL[0] = 0
 
 
-@pytest.mark.parametrize("kernel", [0, 2])
+ROWS_CASES = [c for c in TEAM_CASES if c.startswith(("base", "aan", "learned", "eq5"))]   # rows of at most 96 positions
+
+
+@pytest.mark.parametrize("case", ROWS_CASES)
+def test_one_launch_step_short_rows_kernel_matches_oracle(case):
+    """The same cases with the short-rows kernel forced (whole planes per copy, scores in registers)."""
+    STEP_KERNEL[0] = 3
+    try:
+        FUSED_CASES[case]()
+    finally:
+        STEP_KERNEL[0] = 0
+
+
+def test_short_rows_kernel_every_length_up_to_its_limit():
+    """One sentence per source length 1..96, decoded for 96 steps: every block count and every ragged tail."""
+    w = dataclasses.replace(synth.WORKLOADS["base"], name="rows-all-lengths", n_sent=12, src_lo=1, src_hi=96,
+                            tgt_rule="fixed", tgt_fixed=96, self_blocks=(1, 2, 3), encdec_blocks=(5, 1))
+    STEP_KERNEL[0] = 3
+    try:
+        _run(w, fused=True)
+    finally:
+        STEP_KERNEL[0] = 0
+
+
+@pytest.mark.parametrize("kernel", [0, 2, 3])
 @pytest.mark.parametrize("beam", [1, 2, 3, 5, 8, 12, 20])
 def test_one_launch_step_other_beam_sizes(beam, kernel):
     w = dataclasses.replace(synth.scaled(synth.WORKLOADS["base"], 3), beam=beam, name=f"beam{beam}")
