@@ -669,17 +669,40 @@ static int32_t decode_step_launch(san_ctx* ctx, const san_step_args* a, int max_
     const bool do_self = n_seqs > 0 && !aan;
     const bool do_enc = n_sent > 0;
     // Sentence-sized rows (every row a handful of 16-position blocks): the kernel that takes a whole
-    // plane per copy and keeps the scores in registers.
-    const bool rows_fit = bf16 && (!do_self || (max_len <= kRowsMaxPos && (max_len + 1) * 128 <= kRowsRing)) &&
-                          (!do_enc || (max_src <= kRowsMaxPos && (max_src + nqe) * 128 <= kRowsRing));
-    if (ctx->step_kernel == 3 && !rows_fit) return SAN_ERR_UNSUPPORTED;
-    const bool use_rows = rows_fit && (ctx->step_kernel == 3 || (ctx->step_kernel == 0 && kRowsKernelByDefault));
+    // plane per copy and keeps the scores in registers.  An item is 1, 2 or 4 heads of a (block,
+    // sequence): as many as the head count divides by, the warp's ring holds as one plane, and the
+    // registers hold the weights of.
+    auto rows_heads = [&](int bound, int nq, int want) {
+        for (int r = 4; r >= 1; r >>= 1) {
+            if (r > want || c.n_heads % r) continue;
+            if (r * (bound + nq) > kRowsRingRows || r * nq > 8) continue;
+            if (ceil_div(bound, 16) > rows_max_blocks(r)) continue;
+            return r;
+        }
+        return 0;
+    };
+    int hpi_self = 1, hpi_enc = 1;
+    bool use_rows = false;
+    // Measured on B200 (sentence-sized workload, microbench/step_kernels.py): a launch with encoder-decoder
+    // attention alone takes 9.3 us with this kernel (one head per item) against 19.7 us with the per-warp
+    // kernel; with self-attention in the launch the two are level (23.3 against 23.1 us), and beside the
+    // running averages the per-warp kernel is ahead (13.4 against 14.3 us).  So automatically it takes the
+    // launches without a self-attention part: the query groups of a wide beam after the first.
+    const bool rows_auto = ctx->step_kernel == 0 && n_seqs == 0 && do_enc;
+    if (bf16 && (ctx->step_kernel == 3 || rows_auto)) {
+        const int o = ctx->team_cut_override[1];       // heads per item wanted: as in san_step_kernel_select
+        const int want_self = ctx->step_kernel == 3 && (o & 255) > 0 ? (o & 255) : 2;
+        const int want_enc = ctx->step_kernel == 3 ? ((o >> 8) > 0 ? (o >> 8) - 1 : (o & 255) > 0 ? (o & 255) : 1) : 1;
+        const int rs = do_self ? rows_heads(max_len, 1, want_self) : 1, re = do_enc ? rows_heads(max_src, nqe, want_enc) : 1;
+        if (rs > 0 && re > 0) { use_rows = true; hpi_self = rs; hpi_enc = re; }
+    }
+    if (ctx->step_kernel == 3 && !use_rows) return SAN_ERR_UNSUPPORTED;
     int pi_self = 1, pi_enc = 1;
     for (int b = 0; b < ctx->self_pol.n_blocks; ++b) pi_self = std::max(pi_self, ctx->self_pol.size_of_block[b]);
     for (int b = 0; b < ctx->enc_pol.n_blocks; ++b) pi_enc = std::max(pi_enc, ctx->enc_pol.size_of_block[b]);
     if (c.encdec_shared_context) pi_enc = 1;
-    const long long rows_self = do_self ? (long long)ctx->self_pol.n_blocks * n_seqs * c.n_heads : 0;
-    const long long rows_enc = do_enc ? (long long)ctx->enc_pol.n_blocks * n_sent * c.n_heads : 0;
+    const long long rows_self = do_self ? (long long)ctx->self_pol.n_blocks * n_seqs * (c.n_heads / hpi_self) : 0;
+    const long long rows_enc = do_enc ? (long long)ctx->enc_pol.n_blocks * n_sent * (c.n_heads / hpi_enc) : 0;
     if ((size_t)(rows_self + rows_enc) > ctx->n_tickets) return SAN_ERR_CAPACITY;
 
     // positions per item: what the on-chip score buffer holds, then smaller while items are
@@ -813,7 +836,8 @@ static int32_t decode_step_launch(san_ctx* ctx, const san_step_args* a, int max_
         k.span = (unsigned)span_self; k.nspans = (unsigned)ns_self; k.part_stride = (unsigned)stride_self; k.v_by_block = 0;
         k.row_base = (unsigned)rl_enc;
         k.lg_size = (unsigned)lg_self; k.n_lg = (unsigned)nlg_self; k.div_lg = make_fastdiv((unsigned)nlg_self);
-        k.div_span = make_fastdiv((unsigned)ns_self); k.div_h = make_fastdiv((unsigned)c.n_heads); k.div_item = make_fastdiv(k.n_it);
+        k.hpi = (unsigned)hpi_self;
+        k.div_span = make_fastdiv((unsigned)ns_self); k.div_h = make_fastdiv((unsigned)(c.n_heads / hpi_self)); k.div_item = make_fastdiv(k.n_it);
         for (int b = 0; b < ctx->self_pol.n_blocks; ++b) {
             k.first[b] = (unsigned char)ctx->self_pol.first_layer_of_block[b];
             k.size[b] = (unsigned char)ctx->self_pol.size_of_block[b];
@@ -834,7 +858,8 @@ static int32_t decode_step_launch(san_ctx* ctx, const san_step_args* a, int max_
         k.v_by_block = c.encdec_shared_context ? 1 : 0;
         k.row_base = 0;
         k.lg_size = (unsigned)lg_enc; k.n_lg = (unsigned)nlg_enc; k.div_lg = make_fastdiv((unsigned)nlg_enc);
-        k.div_span = make_fastdiv((unsigned)ns_enc); k.div_h = make_fastdiv((unsigned)c.n_heads); k.div_item = make_fastdiv(k.n_it);
+        k.hpi = (unsigned)hpi_enc;
+        k.div_span = make_fastdiv((unsigned)ns_enc); k.div_h = make_fastdiv((unsigned)(c.n_heads / hpi_enc)); k.div_item = make_fastdiv(k.n_it);
         for (int b = 0; b < ctx->enc_pol.n_blocks; ++b) {
             k.first[b] = (unsigned char)ctx->enc_pol.first_layer_of_block[b];
             k.size[b] = (unsigned char)ctx->enc_pol.size_of_block[b];
@@ -848,6 +873,7 @@ static int32_t decode_step_launch(san_ctx* ctx, const san_step_args* a, int max_
 
     if (use_rows) {
         ctx->last_step_kernel = 3;
+        ctx->last_rows_per_unit[0] = hpi_self; ctx->last_rows_per_unit[1] = hpi_enc;
         const void* rfn = (const void*)decode_step_rows_kernel;
         const size_t rsmem = rows_smem_bytes();
         if (!ctx->rows_attr_set) {
@@ -941,7 +967,7 @@ int32_t san_step_kernel_select(san_ctx* ctx, int32_t which, int32_t spans_log2, 
 int32_t san_step_kernel_used(const san_ctx* ctx, int32_t* which, int32_t* rows_per_unit) {
     if (!ctx || !which) return SAN_ERR_NULL;
     *which = ctx->last_step_kernel;
-    if (rows_per_unit) { rows_per_unit[0] = ctx->last_step_kernel == 2 ? ctx->last_rows_per_unit[0] : 0; rows_per_unit[1] = ctx->last_step_kernel == 2 ? ctx->last_rows_per_unit[1] : 0; }
+    if (rows_per_unit) { rows_per_unit[0] = ctx->last_step_kernel >= 2 ? ctx->last_rows_per_unit[0] : 0; rows_per_unit[1] = ctx->last_step_kernel >= 2 ? ctx->last_rows_per_unit[1] : 0; }
     return SAN_OK;
 }
 

@@ -57,6 +57,7 @@ struct KindParams {
     unsigned q_first, q_total;                         // first of those rows among the q_total rows an item has in q, S and O
     unsigned span, nspans, part_stride, v_by_block, row_base;
     unsigned lg_size, n_lg;                            // layers per item (a block is cut into groups), groups per block at most
+    unsigned hpi;                                      // heads per item (1 unless the short-rows kernel takes several side by side); div_h divides by H / hpi
     FastDiv div_span, div_lg, div_h, div_item;
     unsigned char first[SAN_MAX_LAYERS], size[SAN_MAX_LAYERS];   // per block
 };
@@ -87,6 +88,7 @@ struct ItemDesc {
     int kind, nq, pi, n_spans, span;
     int has_new;                              // the span's last position is this step's row, not yet in the cache
     int lead;                                 // this item also stores the key row of the step
+    int heads;                                // heads it covers, from the one its pointers name
 };
 
 // The kernel's dynamic shared memory.  Everything a warp keeps there is addressed by a 32-bit
@@ -222,6 +224,7 @@ __device__ bool decode_item(const StepParams& p, unsigned it, ItemDesc* d) {
     kp.div_span.divmod(enc ? it : it - p.n_enc_items, &rl, &span);    // rl = (row, layer group)
     kp.div_lg.divmod(rl, &row, &lg);
     kp.div_h.divmod(row, &bi, &h);
+    h *= kp.hpi;
     kp.div_item.divmod(bi, &block, &item);
     const int id = kp.ids[item], len = kp.lens[item] + (int)kp.len_bias;
     const bool reporter = (span == 0 && lg == 0 && h == 0 && block == 0);
@@ -242,6 +245,7 @@ __device__ bool decode_item(const StepParams& p, unsigned it, ItemDesc* d) {
     d->len = len; d->n = j1 - j0;
     d->n_spans = (len + (int)kp.span - 1) / (int)kp.span; d->span = (int)span;
     d->has_new = (kp.knew != nullptr && j1 == len) ? 1 : 0;
+    d->heads = (int)kp.hpi;
     d->lead = (lg == 0) ? 1 : 0;                      // the group that also stores S and this step's key row
     d->row_id = kp.row_base + rl;
     d->part = p.part + kp.part_base + (unsigned long long)(rl * kp.nspans + span) * kp.part_stride;

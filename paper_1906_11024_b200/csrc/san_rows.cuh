@@ -6,15 +6,17 @@
 // decode_step_kernel.  What differs is how a warp works through an item, because with rows this
 // short a step is as long as the chain of dependent instructions and memory round trips of the
 // items one warp takes one after the other:
-//   * a whole plane of an item (its key rows, or the value rows of one layer) is one copy and one
-//     barrier, and the planes of the next items are requested while the warp still computes on
-//     this one: each warp owns a ring of kRowsRing bytes that holds planes of any size back to
-//     back.  All planes that fit are requested by ONE copy instruction, lane j issuing the j-th
-//     of them (a bulk copy costs its warp about 400 cycles to issue whatever its size, 55 more
-//     for each further lane);
-//   * the query rows and this step's own key / value rows (not yet in the cache) are fetched in
-//     16-byte pieces (cp.async) into the plane's slot, the latter already chunk-permuted like a
-//     cached row, so that the arithmetic sees one uniform tile;
+//   * an item is R heads (1, 2 or 4) of one (block, sequence), so that what an item costs beside
+//     its arithmetic is paid once for all of them and their independent chains overlap;
+//   * a whole plane of an item (its key rows, or the value rows of one layer, of all its heads) is
+//     one slot of the warp's ring, which holds planes of any size back to back, and the planes of
+//     the next items are requested while the warp still computes on this one.  The warp fetches
+//     them itself in 16-byte pieces (cp.async, one group per plane): a bulk copy costs its warp
+//     some 400 cycles to issue however small it is, and more when all warps of an SM issue at once
+//     (measured: a third of a warp's time went into issuing them), while a plane of 20 rows is five
+//     cp.async instructions.  This step's own key / value row (not yet in the cache) and the query
+//     rows come the same way, the former already chunk-permuted like a cached row, so that the
+//     arithmetic sees one uniform tile;
 //   * the queries are the M side of the tensor-core products (16 rows, 1 to 8 of them real):
 //       scores:  D[16 queries x 8 positions] = q[16 x 64] . K_tile^T
 //       apply:   D[16 queries x 8 dims]     += S[16 x 16 positions] . V_tile
@@ -28,34 +30,42 @@
 
 namespace san {
 
-constexpr int kRowsWarps = 16;
-constexpr int kRowsRing = 13312;        // bytes per warp: 104 rows
-constexpr int kRowsSlots = 8;           // planes in flight per warp at most (one barrier each)
+constexpr int kRowsWarps = 12;
+constexpr int kRowsRing = 17792;        // bytes per warp: 139 rows
+constexpr int kRowsRingRows = kRowsRing / 128;
+constexpr int kRowsSlots = 8;           // planes in flight per warp at most (one cp.async group each)
 constexpr int kRowsMaxBlocks = 6;
-constexpr int kRowsMaxPos = 16 * kRowsMaxBlocks;   // positions per row at most; a key plane with 8 query rows still fits the ring
-static_assert((kRowsMaxPos + 8) * 128 <= kRowsRing, "a key plane and its query rows fit the ring");
+constexpr int kRowsMaxPos = 16 * kRowsMaxBlocks;   // positions per row at most
+constexpr int kRowsMaxWeights = 24;     // bf16 pairs of weights an item keeps in registers: heads x 2 x blocks
 
 enum { TAG_ROWS = 9 };
-constexpr bool kRowsKernelByDefault = false;
+
+// Blocks of 16 positions an item of `heads` heads may have (its weights stay in registers).
+__host__ __device__ constexpr int rows_max_blocks(int heads) { return heads == 4 ? 3 : heads == 2 ? 5 : kRowsMaxBlocks; }
 
 constexpr size_t rows_smem_bytes() {
-    return (size_t)kRowsWarps * (kRowsRing + kRowsSlots * sizeof(uint64_t)) + 128 /* a row of zeros */ + (size_t)kCtaItems * sizeof(ItemDesc);
+    return (size_t)kRowsWarps * kRowsRing + 128 /* a row of zeros */ + (size_t)kCtaItems * sizeof(ItemDesc);
 }
 
-__device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
-}
 // D(16x8) += A(16x16) * B(16x8) where rows 8..15 of A are zero.  d[2], d[3] (rows 8..15 of D) stay
 // zero; they are carried along because the instruction takes its accumulator as four registers in a row.
 __device__ __forceinline__ void mma_bf16_top(float (&d)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
     asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%5}, {%7,%8}, {%0,%1,%2,%3};"
         : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3]) : "r"(a0), "r"(0u), "r"(a2), "r"(b0), "r"(b1));
 }
+__device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ float ex2_fast(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
 
 struct RowWarp {
     const StepParams& p;
     uint32_t sm_base;             // shared-space address of san_smem
-    uint32_t ring, bars;          // offsets of this warp's ring and of its barriers
+    uint32_t ring;                // offset of this warp's ring
     uint32_t descs_off;           // offset of the CTA's decoded items
     uint32_t zero_row;            // shared-space address of 128 zero bytes
     unsigned* q_next;             // shared counter: next item to hand out
@@ -67,9 +77,7 @@ struct RowWarp {
     int p_plane;                  // 0 = keys, l + 1 = values of the item's layer l
     uint32_t head_v, tail_v, head_p;   // ring: virtual byte counters of what was requested / given back, physical write offset
     uint32_t n_slots, n_ret;      // planes requested / given back
-    uint32_t rec_base, rec_end;   // lane i: offset of the plane with sequence number i (mod kRowsSlots), head_v behind it,
-    uint32_t rec_grp;             //         and the cp.async group its small rows went out with
-    uint32_t n_groups;            // cp.async groups committed so far (one per top_up that requested anything)
+    uint32_t rec_base, rec_end;   // lane i < kRowsSlots: offset of the plane with sequence number i (mod kRowsSlots), head_v behind it
     unsigned long long fifo;      // items whose planes are (being) requested and whose arithmetic is still to do
     int fifo_n;
     bool dead;                    // a wait ran out: leave
@@ -98,96 +106,77 @@ struct RowWarp {
         dead = true;
     }
 
-    // Requests, in order, as many of the planes still to come as the ring and its barriers have room
-    // for: ONE copy instruction, lane j issuing the j-th of them.  The planes of an item lie back to
-    // back (key rows, query rows, then each layer's value rows), so every lane works out its own
-    // plane's place without a loop over planes.
+    // Requests, in order, as many of the planes still to come as the ring has room for (at most
+    // kRowsSlots at a time).  A plane of an item with R heads is R runs of cached rows (the heads'
+    // panels lie apart in the cache and side by side in the slot), this step's own row of every head
+    // where it closes the plane, and, behind the key plane, the query rows.  One cp.async group each.
     __device__ __forceinline__ void top_up() {
-        uint32_t my_dst = 0, my_bytes = 0, my_bar = 0;
-        const char* my_src = nullptr;
-        int k = 0;                                   // planes requested so far in this call (lanes 0 .. k-1)
-        while (p_active) {
-            const int room = kRowsSlots - (int)(n_slots - n_ret);
-            if (room == 0) break;
+        while (p_active && n_slots - n_ret < (uint32_t)kRowsSlots) {
             const ItemDesc& d = desc(p_idx);
-            const int n = d.n, has_new = d.has_new, nq = d.nq, pi = d.pi;
-            const uint32_t S = (uint32_t)n * 128u, Q = p_plane == 0 ? (uint32_t)nq * 128u : 0u;
-            const int want = min(pi + 1 - p_plane, room);
-            // how many of them fit in one piece: behind head_p, else from the start of the ring
+            const int n = d.n, has_new = d.has_new, R = d.heads, pi = d.pi;
+            const int nqr = p_plane == 0 ? R * d.nq : 0;               // the query rows ride behind the key rows
+            const uint32_t bytes = (uint32_t)(R * n + nqr) * 128u;
             uint32_t hv = head_v, hp = head_p;
-            const uint32_t free_all = (uint32_t)kRowsRing - (hv - tail_v), run = (uint32_t)kRowsRing - hp;
-            const uint32_t need_me = Q + (uint32_t)(lane + 1) * S;      // bytes of the first lane + 1 planes
-            int m = __popc(__ballot_sync(0xffffffffu, lane < want && need_me <= min(run, free_all)));
-            if (m == 0) {
-                if (free_all <= run) break;
-                m = __popc(__ballot_sync(0xffffffffu, lane < want && need_me <= free_all - run));
-                if (m == 0) break;
-                hv += run; hp = 0;
-            }
+            if (hp + bytes > (uint32_t)kRowsRing) { hv += (uint32_t)kRowsRing - hp; hp = 0; }     // a plane is contiguous
+            if (hv + bytes - tail_v > (uint32_t)kRowsRing) break;
             const uint32_t base = ring + hp;
+            head_v = hv + bytes; head_p = hp + bytes;
+            if ((uint32_t)lane == n_slots % kRowsSlots) { rec_base = base; rec_end = head_v; }
             const KindParams& kp = p.k[d.kind];
-            const int j = lane - k;
-            if (j >= 0 && j < m) {
-                const int pl = p_plane + j;
-                my_dst = sm_base + base + (uint32_t)j * S + (j > 0 ? Q : 0u);
-                my_src = pl == 0 ? d.srcK : d.srcV + (long long)(pl - 1) * kp.plane_bytes;
-                my_bytes = (uint32_t)(n - has_new) * 128u;
-                my_bar = sm_base + bars + ((n_slots + (uint32_t)j) % kRowsSlots) * 8u;
+            const char* src = p_plane == 0 ? d.srcK : d.srcV + (long long)(p_plane - 1) * kp.plane_bytes;
+            const uint32_t dst = sm_base + base + (uint32_t)lane * 16u;
+            const int cached = (n - has_new) * 8;                        // 16-byte pieces of a head's cached rows
+            src += lane * 16;
+            for (int hh = 0; hh < R; ++hh) {
+                const char* sh = src + (unsigned long long)hh * kp.panel_bytes;
+                const uint32_t dh = dst + (uint32_t)(hh * n) * 128u;
+#pragma unroll 4
+                for (int i = 0; i < cached; i += 32)
+                    if (i + lane < cached) cp_async_16(dh + i * 16, sh + i * 16);
             }
-            {   // lane L < kRowsSlots keeps the record of the plane with sequence number L (mod kRowsSlots)
-                const uint32_t jj = ((uint32_t)lane - n_slots) % kRowsSlots;
-                if (lane < kRowsSlots && jj < (uint32_t)m) {
-                    rec_base = base + jj * S + (jj > 0 ? Q : 0u);
-                    rec_end = hv + Q + (jj + 1) * S;
-                    rec_grp = n_groups;
-                }
+            if (has_new) {      // this step's row of every head, chunk-permuted like a cached row: piece (head, chunk) per lane
+                const char* nw = p_plane == 0 ? d.knew : d.vnew + (long long)(p_plane - 1) * kp.layer_bytes;
+                const int hh = lane >> 3, c = lane & 7;
+                if (hh < R) cp_async_16(sm_base + base + (uint32_t)(hh * n + n - 1) * 128u + (uint32_t)((c ^ ((n - 1) & 7)) << 4), nw + hh * 128 + c * 16);
             }
-            if (has_new) {      // this step's row closes every plane, chunk-permuted like a cached row: 8 lanes per plane
-                const int c = lane & 7;
-                for (int j2 = lane >> 3; j2 < m; j2 += 4) {
-                    const int pl = p_plane + j2;
-                    const char* nw = pl == 0 ? d.knew : d.vnew + (long long)(pl - 1) * kp.layer_bytes;
-                    cp_async_16(sm_base + base + (uint32_t)j2 * S + (j2 > 0 ? Q : 0u) + (uint32_t)(n - 1) * 128u + (uint32_t)((c ^ ((n - 1) & 7)) << 4), nw + c * 16);
-                }
-            }
-            if (p_plane == 0) {             // the query rows ride behind the key rows: chunk c of row r at c ^ r
+            if (nqr) {          // query row hh * nq + qi: chunk c at c ^ (row & 7)
+                const int nq = d.nq;
                 const unsigned q_stride = (unsigned)p.H * 128u;
-                for (int i = lane; i < nq * 8; i += 32) {
+                for (int i = lane; i < nqr * 8; i += 32) {
                     const int r = i >> 3, c = i & 7;
-                    cp_async_16(sm_base + base + S + (uint32_t)r * 128u + (uint32_t)((c ^ r) << 4), d.q + (unsigned long long)r * q_stride + c * 16);
+                    int hh = 0;
+                    if (r >= nq) hh = 1;
+                    if (r >= 2 * nq) hh = 2;
+                    if (r >= 3 * nq) hh = 3;
+                    cp_async_16(sm_base + base + (uint32_t)(R * n + r) * 128u + (uint32_t)((c ^ (r & 7)) << 4),
+                                d.q + hh * 128 + (unsigned long long)(r - hh * nq) * q_stride + c * 16);
                 }
             }
-            const uint32_t tot = Q + (uint32_t)m * S;
-            head_v = hv + tot; head_p = hp + tot;
-            n_slots += (uint32_t)m; k += m;
-            p_plane += m;
-            if (p_plane > pi) next_item(); else break;      // no room for the rest of this item yet
-        }
-        if (k == 0) return;
-        asm volatile("cp.async.commit_group;" ::: "memory");
-        n_groups += 1;
-        if (lane < k) {
-            mbar_expect_tx(my_bar, my_bytes);
-            if (my_bytes) bulk_g2s(my_dst, my_src, my_bytes, my_bar);
+            asm volatile("cp.async.commit_group;" ::: "memory");
+            n_slots += 1;
+            if (p_plane == pi) next_item(); else p_plane += 1;
         }
     }
 
-    // Waits for the next plane in order; returns the offset of its rows, or kNoPlane after a timeout.
+    // Waits for the next plane in order; returns the offset of its rows, or kNoPlane if it was never requested.
     static constexpr uint32_t kNoPlane = 0xffffffffu;
     __device__ __forceinline__ uint32_t acquire() {
         if (n_ret == n_slots) { fail(100); return kNoPlane; }      // top_up always finds room in an empty ring
-        const uint32_t seq = n_ret;
-        const uint32_t bar = sm_base + bars + (seq % kRowsSlots) * 8u, par = (seq / kRowsSlots) & 1u;
-        if (!mbar_try_wait(bar, par) && !mbar_wait_slow(bar, par)) { fail((int)(seq % kRowsSlots)); return kNoPlane; }
-        // The plane's small rows: groups complete in order, and all but the latest have had an item's
-        // worth of arithmetic to arrive, so only a plane requested by the latest top_up waits for that one too.
-        const uint32_t grp = __shfl_sync(0xffffffffu, rec_grp, (int)(seq % kRowsSlots));
-        if (grp + 1 == n_groups) asm volatile("cp.async.wait_group 0;" ::: "memory");
-        else asm volatile("cp.async.wait_group 1;" ::: "memory");
+        // groups complete in order: all but the planes requested after this one
+        switch (n_slots - n_ret - 1u) {
+            case 0: asm volatile("cp.async.wait_group 0;" ::: "memory"); break;
+            case 1: asm volatile("cp.async.wait_group 1;" ::: "memory"); break;
+            case 2: asm volatile("cp.async.wait_group 2;" ::: "memory"); break;
+            case 3: asm volatile("cp.async.wait_group 3;" ::: "memory"); break;
+            case 4: asm volatile("cp.async.wait_group 4;" ::: "memory"); break;
+            case 5: asm volatile("cp.async.wait_group 5;" ::: "memory"); break;
+            case 6: asm volatile("cp.async.wait_group 6;" ::: "memory"); break;
+            default: asm volatile("cp.async.wait_group 7;" ::: "memory"); break;
+        }
         __syncwarp();
-        return __shfl_sync(0xffffffffu, rec_base, (int)(seq % kRowsSlots));
+        return __shfl_sync(0xffffffffu, rec_base, (int)(n_ret % kRowsSlots));
     }
-    // Every lane is done with the plane: its bytes and its barrier are free again.
+    // Every lane is done with the plane: its bytes are free again.
     __device__ __forceinline__ void release() {
         __syncwarp();
         tail_v = __shfl_sync(0xffffffffu, rec_end, (int)(n_ret % kRowsSlots));
@@ -195,47 +184,51 @@ struct RowWarp {
         if (n_ret == n_slots) { tail_v = head_v; head_p = 0; }      // nothing outstanding: the next plane starts the ring afresh
     }
 
-    template <int NB> __device__ __forceinline__ void scores(const ItemDesc& d, uint32_t st, uint32_t (&pw)[2 * kRowsMaxBlocks]);
-    template <int NB> __device__ __forceinline__ void apply(const ItemDesc& d, uint32_t st, const uint32_t (&pw)[2 * kRowsMaxBlocks], int l);
+    template <int NB, int NBLO, int R> __device__ __forceinline__ void scores(const ItemDesc& d, uint32_t st, uint32_t (&pw)[kRowsMaxWeights]);
+    template <int NB, int NBLO, int R> __device__ __forceinline__ void apply(const ItemDesc& d, uint32_t st, const uint32_t (&pw)[kRowsMaxWeights], int l);
 };
 
-__device__ __forceinline__ float ex2_fast(float x) {
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-
-// The key plane of an item of at most NB blocks of 16 positions (at st, with the query rows behind
-// the key rows): this step's key row to the cache, scores, softmax in registers, S to the caller;
-// leaves the weights as bf16 pairs in pw, the A fragments of the apply products.
-template <int NB>
-__device__ __forceinline__ void RowWarp::scores(const ItemDesc& d, uint32_t st, uint32_t (&pw)[2 * kRowsMaxBlocks]) {
-    const int n = d.n, nq = d.nq;
+// The key plane of an item of R heads with more than NBLO and at most NB blocks of 16 positions (at
+// st: the heads' key rows one head after the other, then their query rows): this step's key row to
+// the cache, scores, softmax in registers, S to the caller; leaves the weights as bf16 pairs in pw
+// (head hh at pw[hh * 2 NB ..]), the A fragments of the apply products.  Cached rows keep chunk c
+// at c ^ (position & 7), and so does this step's own row in the slot; query row r keeps chunk c at c ^ (r & 7).
+template <int NB, int NBLO, int R>
+__device__ __forceinline__ void RowWarp::scores(const ItemDesc& d, uint32_t st, uint32_t (&pw)[kRowsMaxWeights]) {
+    static_assert(R * 2 * NB <= kRowsMaxWeights, "the weights of all heads stay in registers");
+    const int n = d.n, nq = d.nq, has_new = d.has_new;
     const int tig = lane & 3, gid = lane >> 2;                 // mma fragment coordinates
     const int r8 = lane & 7, m4 = lane >> 3;                   // ldmatrix: this lane addresses row r8 of matrix m4
     const uint32_t st_s = sm_base + st;
-    if (d.has_new && d.lead && lane < 8)                        // this step's key row into the cache (already permuted)
-        *reinterpret_cast<uint4*>(const_cast<char*>(d.srcK) + (n - 1) * 128 + lane * 16) = *sp<uint4>(st + (uint32_t)(n - 1) * 128u + lane * 16);
-    // A fragments of the queries: matrix m4 = rows 0..7, 16-byte chunk 4 kp + m4; registers (a0, a2) of
-    // k-steps 2 kp and 2 kp + 1.  Rows 8..15 are zero and never loaded; rows at or beyond nq read zeros.
-    uint32_t qa[4][2];
-    {
-        const uint32_t a = (r8 < nq) ? st_s + (uint32_t)(n + r8) * 128u + (uint32_t)((m4 ^ r8) << 4) : zero_row;
-        const uint32_t flip = (r8 < nq) ? 64u : 0u;
-        uint32_t r[4];
-        ldsm_x4(a, r);        qa[0][0] = r[0]; qa[0][1] = r[1]; qa[1][0] = r[2]; qa[1][1] = r[3];
-        ldsm_x4(a ^ flip, r); qa[2][0] = r[0]; qa[2][1] = r[1]; qa[3][0] = r[2]; qa[3][1] = r[3];
-    }
-    // B fragments of 8 positions: matrix m4 = positions 8 j + r8, chunk 4 kp + m4 (cached rows keep
-    // chunk c at c ^ (position & 7)); registers (b0, b1) of k-steps 2 kp and 2 kp + 1.
-    float sc[2 * NB][2];
-    {
-        const uint32_t ka = st_s + (uint32_t)r8 * 128u + (uint32_t)((m4 ^ r8) << 4);
+    const KindParams& kp = p.k[d.kind];
+    const float scl = p.scale_log2e;
+    const int lim = n - 2 * tig;                               // position 8 j + 2 tig + e is in the row iff 8 j + e < lim
+#pragma unroll
+    for (int hh = 0; hh < R; ++hh) {
+        if (has_new && d.lead && lane < 8)                      // this step's key row into the cache (already permuted)
+            *reinterpret_cast<uint4*>(const_cast<char*>(d.srcK) + (unsigned long long)hh * kp.panel_bytes + (n - 1) * 128 + lane * 16) =
+                *sp<uint4>(st + (uint32_t)(hh * n + n - 1) * 128u + lane * 16);
+        // A fragments of the queries: matrix m4 = rows 0..7, 16-byte chunk 4 kp + m4; registers (a0, a2) of
+        // k-steps 2 kp and 2 kp + 1.  Rows 8..15 are zero and never loaded; rows at or beyond nq read zeros.
+        uint32_t qa[4][2];
+        {
+            const uint32_t qr = (uint32_t)(hh * nq + r8);
+            const uint32_t a = (r8 < nq) ? st_s + ((uint32_t)(R * n) + qr) * 128u + (((uint32_t)m4 ^ (qr & 7u)) << 4) : zero_row;
+            const uint32_t flip = (r8 < nq) ? 64u : 0u;
+            uint32_t r[4];
+            ldsm_x4(a, r);        qa[0][0] = r[0]; qa[0][1] = r[1]; qa[1][0] = r[2]; qa[1][1] = r[3];
+            ldsm_x4(a ^ flip, r); qa[2][0] = r[0]; qa[2][1] = r[1]; qa[3][0] = r[2]; qa[3][1] = r[3];
+        }
+        // B fragments of 8 positions: matrix m4 = positions 8 j + r8, chunk 4 kp + m4; registers (b0, b1)
+        // of k-steps 2 kp and 2 kp + 1.
+        float sc[2 * NB][2];
+        const uint32_t ka = st_s + (uint32_t)(hh * n + r8) * 128u + (uint32_t)((m4 ^ r8) << 4);
 #pragma unroll
         for (int j = 0; j < 2 * NB; ++j) {
+            const uint32_t kj = ka + j * 1024;
             uint32_t b0[4], b1[4];
-            ldsm_x4(ka + j * 1024, b0);
-            ldsm_x4((ka ^ 64u) + j * 1024, b1);
+            ldsm_x4(kj, b0);
+            ldsm_x4(kj ^ 64u, b1);
             float c[4] = {0.f, 0.f, 0.f, 0.f};
             mma_bf16_top(c, qa[0][0], qa[0][1], b0[0], b0[1]);
             mma_bf16_top(c, qa[1][0], qa[1][1], b0[2], b0[3]);
@@ -243,39 +236,37 @@ __device__ __forceinline__ void RowWarp::scores(const ItemDesc& d, uint32_t st, 
             mma_bf16_top(c, qa[3][0], qa[3][1], b1[2], b1[3]);
             sc[j][0] = c[0]; sc[j][1] = c[1];
         }
-    }
-    // Softmax in registers: sc[j][e] is query gid, position 8 j + 2 tig + e (log2 domain after scaling).
-    // Positions at or beyond n (the query rows, stale bytes) are masked out.
-    const float scl = p.scale_log2e;
-    const int lim = n - 2 * tig;                     // position 8 j + 2 tig + e is in the row iff 8 j + e < lim
-    float mx = -INFINITY;
+        // Softmax in registers: sc[j][e] is query gid, position 8 j + 2 tig + e (log2 domain after scaling).
+        // Positions at or beyond n (the next head's rows, the query rows, stale bytes) are masked out.
+        float mx = -INFINITY;
 #pragma unroll
-    for (int j = 0; j < 2 * NB; ++j)
+        for (int j = 0; j < 2 * NB; ++j)
 #pragma unroll
-        for (int e = 0; e < 2; ++e) {
-            const float v = (8 * j + e < lim) ? sc[j][e] * scl : -INFINITY;
-            sc[j][e] = v;
-            mx = fmaxf(mx, v);
+            for (int e = 0; e < 2; ++e) {
+                const float v = (j < 2 * NBLO || 8 * j + e < lim) ? sc[j][e] * scl : -INFINITY;
+                sc[j][e] = v;
+                mx = fmaxf(mx, v);
+            }
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+        float sum = 0.f;
+#pragma unroll
+        for (int j = 0; j < 2 * NB; ++j)
+#pragma unroll
+            for (int e = 0; e < 2; ++e) { sc[j][e] = ex2_fast(sc[j][e] - mx); sum += sc[j][e]; }
+        sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+        sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+        const float inv = 1.0f / sum;
+        float* Srow = (d.S && gid < nq) ? d.S + (long long)hh * kp.S_ld + (long long)gid * ((long long)p.H * kp.S_ld) + 2 * tig : nullptr;
+#pragma unroll
+        for (int j = 0; j < 2 * NB; ++j) {
+            const float w0 = sc[j][0] * inv, w1 = sc[j][1] * inv;
+            if (Srow) {
+                if (j < 2 * NBLO || 8 * j < lim) Srow[8 * j] = w0;
+                if (j < 2 * NBLO || 8 * j + 1 < lim) Srow[8 * j + 1] = w1;
+            }
+            pw[hh * 2 * NB + j] = pack_bf16x2(w0, w1);
         }
-    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-    float sum = 0.f;
-#pragma unroll
-    for (int j = 0; j < 2 * NB; ++j)
-#pragma unroll
-        for (int e = 0; e < 2; ++e) { sc[j][e] = ex2_fast(sc[j][e] - mx); sum += sc[j][e]; }
-    sum += __shfl_xor_sync(0xffffffffu, sum, 1);
-    sum += __shfl_xor_sync(0xffffffffu, sum, 2);
-    const float inv = 1.0f / sum;
-    float* Srow = (d.S && gid < nq) ? d.S + (long long)gid * ((long long)p.H * p.k[d.kind].S_ld) + 2 * tig : nullptr;
-#pragma unroll
-    for (int j = 0; j < 2 * NB; ++j) {
-        const float w0 = sc[j][0] * inv, w1 = sc[j][1] * inv;
-        if (Srow) {
-            if (8 * j < lim) Srow[8 * j] = w0;
-            if (8 * j + 1 < lim) Srow[8 * j + 1] = w1;
-        }
-        pw[j] = pack_bf16x2(w0, w1);
     }
 }
 
@@ -283,38 +274,43 @@ __device__ __forceinline__ void RowWarp::scores(const ItemDesc& d, uint32_t st, 
 // B fragments through ldmatrix.trans: matrix m4 = positions 16 kk + 8 (m4 & 1) + r8, chunk
 // 2 jp + (m4 >> 1); registers (b0, b1) of dim tiles 2 jp and 2 jp + 1.  Rows at or beyond n hold other
 // bytes: their weights are zero, but 0 x NaN would not be, so those lanes address a row of zeros.
-template <int NB>
-__device__ __forceinline__ void RowWarp::apply(const ItemDesc& d, uint32_t st, const uint32_t (&pw)[2 * kRowsMaxBlocks], int l) {
-    const int n = d.n;
+template <int NB, int NBLO, int R>
+__device__ __forceinline__ void RowWarp::apply(const ItemDesc& d, uint32_t st, const uint32_t (&pw)[kRowsMaxWeights], int l) {
+    const int n = d.n, has_new = d.has_new;
     const int tig = lane & 3, gid = lane >> 2;
     const int r8 = lane & 7, m4 = lane >> 3;
     const KindParams& kp = p.k[d.kind];
     const uint32_t st_s = sm_base + st;
-    if (d.has_new && lane < 8)
-        *reinterpret_cast<uint4*>(const_cast<char*>(d.srcV) + (long long)l * kp.plane_bytes + (n - 1) * 128 + lane * 16) =
-            *sp<uint4>(st + (uint32_t)(n - 1) * 128u + lane * 16);
     const int vpos = 8 * (m4 & 1) + r8;
-    const uint32_t va = st_s + (uint32_t)vpos * 128u + (uint32_t)(((m4 >> 1) ^ r8) << 4);
-    float acc[8][4];
+    const bool writes = gid < d.nq;
+    char* op = d.O + (long long)l * kp.layer_bytes + (long long)gid * ((long long)p.H * 128) + tig * 4;
+    char* vdst = const_cast<char*>(d.srcV) + (long long)l * kp.plane_bytes + (n - 1) * 128 + lane * 16;
 #pragma unroll
-    for (int x = 0; x < 8; ++x) { acc[x][0] = 0.f; acc[x][1] = 0.f; acc[x][2] = 0.f; acc[x][3] = 0.f; }
+    for (int hh = 0; hh < R; ++hh) {
+        if (has_new && lane < 8)
+            *reinterpret_cast<uint4*>(vdst + (unsigned long long)hh * kp.panel_bytes) = *sp<uint4>(st + (uint32_t)(hh * n + n - 1) * 128u + lane * 16);
+        const uint32_t va = st_s + (uint32_t)(hh * n + vpos) * 128u + (uint32_t)(((m4 >> 1) ^ r8) << 4);
+        float acc[8][4];
 #pragma unroll
-    for (int kk = 0; kk < NB; ++kk) {
-        const bool in_row = 16 * kk + vpos < n;
-        uint32_t b[4][4];
+        for (int x = 0; x < 8; ++x) { acc[x][0] = 0.f; acc[x][1] = 0.f; acc[x][2] = 0.f; acc[x][3] = 0.f; }
 #pragma unroll
-        for (int jp = 0; jp < 4; ++jp) ldsm_x4_t(in_row ? (va + kk * 2048) ^ (uint32_t)(jp << 5) : zero_row, b[jp]);
+        for (int kk = 0; kk < NB; ++kk) {
+            const uint32_t vk = va + kk * 2048;
+            const bool in_row = kk < NBLO || 16 * kk + vpos < n;
+            uint32_t b[4][4];
 #pragma unroll
-        for (int jp = 0; jp < 4; ++jp) {
-            mma_bf16_top(acc[2 * jp], pw[2 * kk], pw[2 * kk + 1], b[jp][0], b[jp][1]);
-            mma_bf16_top(acc[2 * jp + 1], pw[2 * kk], pw[2 * kk + 1], b[jp][2], b[jp][3]);
+            for (int jp = 0; jp < 4; ++jp) ldsm_x4_t(in_row ? vk ^ (uint32_t)(jp << 5) : zero_row, b[jp]);
+#pragma unroll
+            for (int jp = 0; jp < 4; ++jp) {
+                mma_bf16_top(acc[2 * jp], pw[hh * 2 * NB + 2 * kk], pw[hh * 2 * NB + 2 * kk + 1], b[jp][0], b[jp][1]);
+                mma_bf16_top(acc[2 * jp + 1], pw[hh * 2 * NB + 2 * kk], pw[hh * 2 * NB + 2 * kk + 1], b[jp][2], b[jp][3]);
+            }
         }
-    }
-    // acc[x][0], [1]: query gid, dims 8 x + 2 tig, + 1
-    if (gid < d.nq) {
-        char* op = d.O + (long long)l * kp.layer_bytes + (long long)gid * ((long long)p.H * 128) + tig * 4;
+        // acc[x][0], [1]: query gid, dims 8 x + 2 tig, + 1
+        if (writes) {
 #pragma unroll
-        for (int x = 0; x < 8; ++x) *reinterpret_cast<uint32_t*>(op + x * 16) = pack_bf16x2(acc[x][0], acc[x][1]);
+            for (int x = 0; x < 8; ++x) *reinterpret_cast<uint32_t*>(op + hh * 128 + x * 16) = pack_bf16x2(acc[x][0], acc[x][1]);
+        }
     }
 }
 
@@ -323,15 +319,9 @@ __global__ void __launch_bounds__(kRowsWarps * 32, 1) decode_step_rows_kernel(co
     // Programmatic stream serialization as in decode_step_kernel: only the set-up of shared memory
     // runs ahead of the preceding kernel's completion.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    constexpr uint32_t kBarsAll = kRowsWarps * kRowsRing;
-    constexpr uint32_t kZeroRow = kBarsAll + kRowsWarps * kRowsSlots * (uint32_t)sizeof(uint64_t);
+    constexpr uint32_t kZeroRow = kRowsWarps * kRowsRing;
     constexpr uint32_t kDescsAll = kZeroRow + 128;
     if (threadIdx.x < 32) *sp<uint32_t>(kZeroRow + threadIdx.x * 4) = 0u;
-    if (lane == 0) {
-        for (int s = 0; s < kRowsSlots; ++s) mbar_init(sp<uint64_t>(kBarsAll + ((uint32_t)warp * kRowsSlots + s) * 8), 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
 
     __shared__ unsigned aan_next;
@@ -344,10 +334,9 @@ __global__ void __launch_bounds__(kRowsWarps * 32, 1) decode_step_rows_kernel(co
     RowWarp w(p);
     w.sm_base = smem_u32(san_smem);
     w.ring = (uint32_t)warp * kRowsRing;
-    w.bars = kBarsAll + (uint32_t)warp * kRowsSlots * 8;
     w.descs_off = kDescsAll; w.q_next = &q_next; w.zero_row = w.sm_base + kZeroRow;
     w.lane = lane;
-    w.head_v = w.tail_v = w.head_p = 0; w.n_slots = w.n_ret = 0; w.rec_base = w.rec_end = w.rec_grp = 0; w.n_groups = 0;
+    w.head_v = w.tail_v = w.head_p = 0; w.n_slots = w.n_ret = 0; w.rec_base = w.rec_end = 0;
     w.dead = false; w.p_active = false; w.p_plane = 0; w.p_idx = 0;
 
     const unsigned long long my_slots = (p.n_items > blockIdx.x) ? ((unsigned long long)p.n_items - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
@@ -380,7 +369,7 @@ __global__ void __launch_bounds__(kRowsWarps * 32, 1) decode_step_rows_kernel(co
         // One plane per turn: the item in hand is `c_idx`, its next plane `c_plane` (0 = keys, l + 1 = the
         // values of its layer l).  More planes are requested when an item starts (what the item before
         // gave back goes to the items behind this one) and while a fat item's own planes are not all out.
-        uint32_t pw[2 * kRowsMaxBlocks];
+        uint32_t pw[kRowsMaxWeights];
         unsigned c_idx = 0;
         int c_plane = 0;
         bool have = false;
@@ -395,12 +384,16 @@ __global__ void __launch_bounds__(kRowsWarps * 32, 1) decode_step_rows_kernel(co
             const ItemDesc& d = w.desc(c_idx);
             const uint32_t st = w.acquire();
             if (st == RowWarp::kNoPlane) break;
-            const int nb = (d.n + 15) >> 4;
-            if (c_plane == 0) {
-                if (nb <= 2) w.scores<2>(d, st, pw); else if (nb <= 4) w.scores<4>(d, st, pw); else w.scores<6>(d, st, pw);
+            const int nb = (d.n + 15) >> 4, R = d.heads, l = c_plane - 1;
+#define SAN_ROWS_PLANE(NB, NBLO, RR) do { if (c_plane == 0) w.scores<NB, NBLO, RR>(d, st, pw); else w.apply<NB, NBLO, RR>(d, st, pw, l); } while (0)
+            if (R == 1) {
+                if (nb <= 2) SAN_ROWS_PLANE(2, 0, 1); else if (nb <= 4) SAN_ROWS_PLANE(4, 2, 1); else SAN_ROWS_PLANE(6, 4, 1);
+            } else if (R == 2) {
+                if (nb <= 2) SAN_ROWS_PLANE(2, 0, 2); else if (nb == 3) SAN_ROWS_PLANE(3, 2, 2); else if (nb == 4) SAN_ROWS_PLANE(4, 3, 2); else SAN_ROWS_PLANE(5, 4, 2);
             } else {
-                if (nb <= 2) w.apply<2>(d, st, pw, c_plane - 1); else if (nb <= 4) w.apply<4>(d, st, pw, c_plane - 1); else w.apply<6>(d, st, pw, c_plane - 1);
+                if (nb <= 2) SAN_ROWS_PLANE(2, 0, 4); else SAN_ROWS_PLANE(3, 2, 4);
             }
+#undef SAN_ROWS_PLANE
             w.release();
             if (c_plane == d.pi) have = false; else c_plane += 1;
         }

@@ -268,6 +268,9 @@ class Decoder:
         sb.lens.copy_(torch.from_numpy(pos + 1))
         sb.sent_ids.copy_(torch.from_numpy(sent_ids))
         sb.src_lens.copy_(torch.from_numpy(src[sent_ids]))
+        # the host knows where every hypothesis stands: the bounds of this step, not of the whole run
+        sb.max_len = int(pos.max()) + 1 if len(pos) else 1
+        sb.max_src = int(src[sent_ids].max()) if len(sent_ids) else 1
         if w.self_is_aan:
             xs = np.stack([synth.aan_x(w, step, l)[seq_ids] for l in range(w.n_layers)])
             sb.x_aan.copy_(to_device(xs, w.dtype, dev))

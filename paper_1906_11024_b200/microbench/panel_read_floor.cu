@@ -5,6 +5,7 @@
 // launch and ramp included.
 //   nvcc -gencode arch=compute_100a,code=sm_100a -O3 -o panel_read_floor panel_read_floor.cu && ./panel_read_floor
 #include <cstdio>
+#include <cstdlib>
 #include <cstdint>
 #include <cuda_runtime.h>
 #include <vector>
@@ -20,15 +21,17 @@ __global__ void rd(const uint4* base, const int* lens, int n_panels, int planes,
     }
     if (acc == 0x12345678u) sink[0] = acc;
 }
-int main() {
-    const int seqs = 256, H = 8, cap = 66, planes = 9, R = 6;
+int main(int argc, char** argv) {
+    // optional arguments: rows a panel has room for (default 66), rows read of every panel (default 0: 6..33, as the workload)
+    const int cap = argc > 1 ? atoi(argv[1]) : 66, fixed = argc > 2 ? atoi(argv[2]) : 0;
+    const int seqs = 256, H = 8, planes = 9, R = 6;
     const int n_panels = seqs * H;
     const size_t plane_bytes = (size_t)n_panels * cap * 128;
     const size_t rep_bytes = plane_bytes * 16;      // a replica also holds other planes between
     char* buf; cudaMalloc(&buf, rep_bytes * R); cudaMemset(buf, 1, rep_bytes * R);
     std::vector<int> lens(seqs);
     size_t bytes = 0;
-    for (int s = 0; s < seqs; ++s) { lens[s] = 6 + ((s / 4) * 7919) % 28; bytes += (size_t)lens[s] * 128 * H * planes; }
+    for (int s = 0; s < seqs; ++s) { lens[s] = fixed > 0 ? fixed : 6 + ((s / 4) * 7919) % 28; bytes += (size_t)lens[s] * 128 * H * planes; }
     int* dl; cudaMalloc(&dl, seqs * 4); cudaMemcpy(dl, lens.data(), seqs * 4, cudaMemcpyHostToDevice);
     unsigned* sink; cudaMalloc(&sink, 4);
     cudaEvent_t e0, e1; cudaEventCreate(&e0); cudaEventCreate(&e1);

@@ -260,7 +260,8 @@ def test_one_launch_step_other_beam_sizes(beam, kernel):
 
 
 def test_automatic_kernel_choice():
-    """Rows long enough to be split over a team go to the team pipeline, sentence-sized rows to the per-warp kernel."""
+    """Rows long enough to be split over a team go to the team pipeline, sentence-sized rows to the per-warp kernel,
+    launches without self-attention to the short-rows kernel."""
     for name, want in (("base", 1), ("long", 2)):
         w = synth.scaled(synth.WORKLOADS[name], 2)
         dec = Decoder(w)
@@ -272,6 +273,18 @@ def test_automatic_kernel_choice():
         assert rc == 0 and which == want, (name, which, rpu)
         assert dec.device_status()[0] == 0
         dec.close()
+    # a beam wider than one query group: the launches after the first hold encoder-decoder attention alone
+    # and go to the short-rows kernel (the last launch is the one reported)
+    w = dataclasses.replace(synth.scaled(synth.WORKLOADS["base"], 2), beam=12, name="beam12")
+    dec = Decoder(w)
+    dec.load_encoder_memory()
+    sb = dec.new_step_buffers()
+    dec.fill_step_inputs(sb, 0, np.arange(w.n_seqs, dtype=np.int32), np.zeros(w.n_seqs, np.int32))
+    dec.step_fused(sb)
+    rc, which, rpu = B.san_step_kernel_used(dec.ctx)
+    assert rc == 0 and which == 3 and rpu[1] == 1, (which, rpu)
+    assert dec.device_status()[0] == 0
+    dec.close()
 
 
 def test_one_launch_step_writes_the_cache_like_append():
