@@ -43,7 +43,7 @@ FALLBACK_HBM_GBS = 6650.0
 # (the kernels and the host code that chooses kernel and cuts): once any of them changes the
 # counters no longer describe the kernel, and the line reports null until a new capture is
 # recorded here.
-KERNEL_SOURCES = ("san_fused.cuh", "san_step.cuh", "san_kernels.cuh", "san_api.cu")
+KERNEL_SOURCES = ("san_fused.cuh", "san_step.cuh", "san_rows.cuh", "san_kernels.cuh", "san_api.cu")
 NCU_TRAFFIC = {"digest": "f3da46ffebf5f3e3",
                "fused": {"long": 734.9e6, "base": 70.3e6, "big": 426.5e6, "aan": 25.4e6,
                          "long-unshared": 1256.5e6, "base-unshared": 105.2e6}}
@@ -558,13 +558,14 @@ def run_reference(args, w):
     print(json.dumps(line))
 
 
-KERNEL_NAMES = {0: "none", 1: "decode_step_kernel (per-warp pipeline)", 2: "decode_step_team_kernel (team pipeline)"}
+KERNEL_NAMES = {0: "none", 1: "decode_step_kernel (per-warp pipeline)", 2: "decode_step_team_kernel (team pipeline)",
+                3: "decode_step_rows_kernel (short rows)"}
 
 
 def kernel_used(dec):
     from paper_1906_11024_b200 import binding as B
     rc, which, rpu = B.san_step_kernel_used(dec.ctx)
-    return {"kernel": KERNEL_NAMES.get(which, "?"), "heads_per_unit": rpu if which == 2 else None}
+    return {"kernel": KERNEL_NAMES.get(which, "?"), "heads_per_unit": rpu if which >= 2 else None}
 
 
 def roofline_record(ab, secs_per_step, peak, peak_kind, name, traffic):

@@ -208,7 +208,8 @@ int32_t san_seq_reset(san_ctx* ctx, const int32_t* d_seq_ids, int32_t n, void* s
  * are host bounds on pos+1 / source lengths (0 = capacity).  Rows longer than the on-chip
  * score buffer are split into at most 32 spans; a bound that would need more returns
  * SAN_ERR_UNSUPPORTED (use the separate calls).  The kernel's waits on its own copies are
- * bounded: if one runs out the step reports SAN_ERR_TIMEOUT through san_device_status. */
+ * bounded: if one runs out the step reports SAN_ERR_TIMEOUT through san_device_status.  A beam
+ * wider than 8 takes one launch per group of 8 query rows. */
 typedef struct {
     const void* d_q_self; const void* d_k_new; const void* d_v_new;
     const int32_t* d_seq_ids; const int32_t* d_pos; int32_t n_seqs; int32_t max_len;
@@ -220,13 +221,19 @@ typedef struct {
 int32_t san_decode_step(san_ctx* ctx, const san_step_args* args, void* stream);
 
 /* Which kernel san_decode_step launches, and (for testing and tuning) how its rows are cut.
- * The library has two implementations of the one-launch step (same arithmetic, Eq. 1-5):
+ * The library has three implementations of the one-launch step (same arithmetic, Eq. 1-5):
  *   which = 1  per-warp pipeline: every warp streams the tiles of its own row (float32 and bf16);
  *   which = 2  team pipeline (bf16): four producer warps each stream bundles of two units to a team
  *              of two warps, a unit being up to four heads of one sequence or one of two spans of
  *              a long row; SAN_ERR_UNSUPPORTED from the step if a shape does not fit;
+ *   which = 3  short rows (bf16, max_len and max_src at most 96): a warp fetches whole planes of 1, 2
+ *              or 4 heads (heads_per_unit; fewer where they would not fit its ring) and keeps the
+ *              scores in registers; layers_per_unit as below; SAN_ERR_UNSUPPORTED from the step
+ *              if the bounds are larger;
  *   which = 0  automatic (the default): the team pipeline for steps whose rows are long enough to be
- *              split over the warps of a team (where it measured faster), else the per-warp one.
+ *              split over the warps of a team, the short-rows kernel for launches that hold
+ *              encoder-decoder attention alone (where each measured faster), else the per-warp one.
+ * A value may carry a second one for encoder-decoder attention in its bits 8 and up, as (v + 1) << 8.
  * spans_log2 >= 0 overrides the automatic cut of the team pipeline: every row is dealt to
  * 1 << spans_log2 warps (0..1); with one span up to heads_per_unit (1, 2 or 4) heads of one
  * sequence or sentence go to a warp where the head count allows (at most 2 where several
@@ -237,8 +244,8 @@ int32_t san_decode_step(san_ctx* ctx, const san_step_args* args, void* stream);
 int32_t san_step_kernel_select(san_ctx* ctx, int32_t which, int32_t spans_log2, int32_t heads_per_unit,
                                int32_t tile_pos, int32_t layers_per_unit, int32_t grab_mult);
 
-/* Which kernel the last san_decode_step of this context launched (1 or 2 as above, 0 before the
- * first step) and, for the team pipeline, how many heads of one sequence / sentence it gave
+/* Which kernel the last san_decode_step of this context launched (1, 2 or 3 as above, 0 before the
+ * first step) and, for the team pipeline and the short-rows kernel, how many heads of one sequence / sentence it gave
  * to one warp: rows_per_unit[0] for self-attention, [1] for encoder-decoder attention (may
  * be NULL).  For tests and benchmarks that must know what they measured. */
 int32_t san_step_kernel_used(const san_ctx* ctx, int32_t* which, int32_t* rows_per_unit);

@@ -80,7 +80,7 @@ struct RowWarp {
     uint32_t rec_base, rec_end;   // lane i < kRowsSlots: offset of the plane with sequence number i (mod kRowsSlots), head_v behind it
     unsigned long long fifo;      // items whose planes are (being) requested and whose arithmetic is still to do
     int fifo_n;
-    bool dead;                    // a wait ran out: leave
+    bool dead;                    // the ring's bookkeeping broke (reported as an error): leave
 
     __device__ RowWarp(const StepParams& pp) : p(pp) {}
 
