@@ -181,6 +181,25 @@ def test_step_refuses_rows_beyond_what_its_kernels_can_cut():
     dec.close()
 
 
+def test_kernel_select_refuses_cuts_it_cannot_launch():
+    """san_step_kernel_select checks every value (and the encoder-decoder value a field may carry in its
+    bits 8 and up) on the host: a tile that is no multiple of 16 positions, too many heads per unit or
+    spans per row never reach a kernel."""
+    w = _small()
+    dec = Decoder(w)
+    ok = B.SAN_OK
+    assert B.san_step_kernel_select(dec.ctx, 2, 1, 1, 64, 0, 1) == ok
+    assert B.san_step_kernel_select(dec.ctx, 2, 1, 1, 64 + ((128 + 1) << 8), 0, 1) == ok
+    for bad_tile in (63, 8, 0, 250, 64 + ((63 + 1) << 8), 64 + ((8 + 1) << 8), -16):
+        assert B.san_step_kernel_select(dec.ctx, 2, 1, 1, bad_tile, 0, 1) == B.SAN_ERR_RANGE, bad_tile
+    for bad_heads in (0, 5, 2 + ((7 + 1) << 8), -1):
+        assert B.san_step_kernel_select(dec.ctx, 2, 0, bad_heads, 64, 0, 1) == B.SAN_ERR_RANGE, bad_heads
+    assert B.san_step_kernel_select(dec.ctx, 2, 2, 1, 64, 0, 1) == B.SAN_ERR_RANGE          # at most two spans per row
+    assert B.san_step_kernel_select(dec.ctx, 4, -1, 1, 64, 0, 1) == B.SAN_ERR_RANGE         # no such kernel
+    assert B.san_step_kernel_select(dec.ctx, 0) == ok
+    dec.close()
+
+
 def test_policy_tables_and_runtime_change():
     """Integer tables are bit-exact; a policy with more blocks than key planes is refused."""
     w = _small(self_blocks=(2, 2), encdec_blocks=(4,))
