@@ -43,6 +43,7 @@ FALLBACK_HBM_GBS = 6650.0
 # (the kernels and the host code that chooses kernel and cuts): once any of them changes the
 # counters no longer describe the kernel, and the line reports null until a new capture is
 # recorded here.
+E2E_BATCHES = 4           # request batches in flight in the end-to-end leg
 KERNEL_SOURCES = ("san_fused.cuh", "san_step.cuh", "san_rows.cuh", "san_kernels.cuh", "san_api.cu")
 NCU_TRAFFIC = {"digest": "6076dc51fef45488",
                "fused": {"long": 735.5e6, "base": 70.7e6, "big": 426.9e6, "aan": 25.4e6,
@@ -285,12 +286,14 @@ def time_e2e(w, decs, sbs, steps, device, fused=True):
     """The same step with HOST buffers: every step copies its inputs from pinned host memory
     to the device, runs the library, and reads the outputs back.  On the one-launch path this
     is a single C-ABI call, san_decode_step_host, which issues the copies itself on the
-    caller's stream.  Two request batches (two contexts, each with its own stream and pinned
-    buffers) take turns, the way a server keeps PCIe busy in both directions: the copies of one
-    batch overlap the other's.  Returns (seconds for `steps` steps with two batches in flight,
-    seconds for `steps` steps of one batch alone, h2d bytes per step, d2h bytes per step)."""
+    caller's stream.  A step of one request batch is a chain (copy in, kernel, copy out) that the
+    next step of that batch has to wait for, so several batches (E2E_BATCHES contexts, each with its
+    own stream and pinned buffers) take turns, the way a server keeps the GPU and PCIe busy in both
+    directions: the copies of one batch overlap the kernels of the others.  Returns (seconds for
+    `steps` steps with all batches in flight, seconds for `steps` steps of one batch alone, h2d bytes
+    per step, d2h bytes per step, batches)."""
     import torch
-    n_ctx = 2 if len(decs) > 1 else 1
+    n_ctx = min(len(decs), E2E_BATCHES)
     hbs = [decs[i].host_buffers(sbs[i]) for i in range(n_ctx)]
     streams = [torch.cuda.Stream(device) for _ in range(n_ctx)]
     hb = hbs[0]
@@ -333,7 +336,7 @@ def time_e2e(w, decs, sbs, steps, device, fused=True):
 
     serial = timed(1)
     both = timed(n_ctx) if n_ctx > 1 else serial
-    return both, serial, h2d, d2h
+    return both, serial, h2d, d2h, n_ctx
 
 
 def time_beam_reorder(w, decs, sbs, pos, device, peak, reps=10):
@@ -681,7 +684,7 @@ def main():
     fused = args.path == "fused"
     pos = state_positions(w)
     ab = algorithmic_bytes(w, pos, fused)
-    n_rep = int(min(16, max(2, math.ceil(3 * L2_BYTES / max(ab["total"], 1)))))
+    n_rep = int(min(16, max(E2E_BATCHES, math.ceil(3 * L2_BYTES / max(ab["total"], 1)))))
     decs, sbs, pos = build_replicas(w, n_rep, device)
 
     phys = local_rank
@@ -709,7 +712,7 @@ def main():
                 "unit": "GB/s", "frac": dom_bytes / dom_s / 1e9 / peak, "peak_kind": peak_kind, "bytes_per_launch": dom_bytes,
                 "us_per_launch": dom_s * 1e6, "launches_per_step": dom_per_step, "traffic": None}
     e2e_steps = min(args.steps, 100)
-    e2e_s, e2e_serial_s, h2d, d2h = time_e2e(w, decs, sbs, e2e_steps, device, fused)
+    e2e_s, e2e_serial_s, h2d, d2h, e2e_batches = time_e2e(w, decs, sbs, e2e_steps, device, fused)
     next_rows = {}
     if rank == 0 and not args.only:
         next_rows["beam_reorder"] = time_beam_reorder(w, decs, sbs, pos, device, peak)
@@ -810,8 +813,10 @@ def main():
         "e2e": {"value": w.n_seqs * e2e_steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": e2e_s / e2e_steps * 1e3,
                 "one_batch_alone_ms_per_step": e2e_serial_s / e2e_steps * 1e3,
-                "how": "san_decode_step_host, one C-ABI call per step with pinned host buffers; two request batches "
-                       "(two contexts, two streams) take turns so that uploads and downloads overlap"},
+                "batches_in_flight": e2e_batches,
+                "how": "san_decode_step_host, one C-ABI call per step with pinned host buffers; a batch's step is a chain "
+                       "(copy in, kernel, copy out), so several request batches (one context, stream and set of pinned "
+                       "buffers each) take turns and the copies of one overlap the kernels of the others"},
         "clocks": clocks,
     }
     if workloads:

@@ -63,6 +63,7 @@ class Decoder:
         self.w = w
         self.device = torch.device(device)
         self.shared_ctx = bool(encdec_shared_context)
+        self._host_step_args = {}
         self.tdtype = torch.bfloat16 if w.dtype == synth.BF16 else torch.float32
         self.cfg = B.san_config(
             n_layers=w.n_layers, n_heads=w.n_heads, d_head=w.d_head, max_sent=w.n_sent, beam=w.beam,
@@ -91,6 +92,7 @@ class Decoder:
         if getattr(self, "ctx", None):
             B.san_destroy(self.ctx)
             self.ctx = None
+        self._host_step_args = {}
 
     def __del__(self):
         try:
@@ -238,9 +240,16 @@ class Decoder:
     def step_fused_host(self, sb: StepBuffers, hb: dict, stream=None) -> int:
         """The decode step through san_decode_step_host: inputs come from and outputs go to the
         pinned host tensors of ``hb``; the library issues the copies around its one launch."""
-        host = B.step_args(**{k: hb[k] for k in hb["_in"] + hb["_out"]})
-        dev = B.step_args(**self._dev_step_args(sb))
-        B.check(B.san_decode_step_host(self.ctx, host, dev, stream), "san_decode_step_host")
+        # the two argument structs hold raw pointers and bounds: built once per pair of buffer sets and
+        # rebuilt when the step's bounds change (a serving loop calls this every step)
+        key = (id(sb), id(hb))
+        cached = self._host_step_args.get(key)
+        if cached is None or cached[2] != (sb.max_len, sb.max_src):
+            host = B.step_args(**{k: hb[k] for k in hb["_in"] + hb["_out"]})
+            dev = B.step_args(**self._dev_step_args(sb))
+            cached = (host, dev, (sb.max_len, sb.max_src), sb, hb)      # keeps the buffers alive with their pointers
+            self._host_step_args[key] = cached
+        B.check(B.san_decode_step_host(self.ctx, cached[0], cached[1], stream), "san_decode_step_host")
         return 1
 
     def device_status(self, stream=None):
