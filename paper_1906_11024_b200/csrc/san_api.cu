@@ -893,7 +893,7 @@ static int32_t decode_step_launch(san_ctx* ctx, const san_step_args* a, int max_
             if (cudaFuncSetAttribute(rfn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rsmem) != cudaSuccess) return SAN_ERR_CUDA;
             ctx->rows_attr_set = true;
         }
-        long long rctas = std::min<long long>(ctx->sm_count, (p.n_items + kRowsWarps - 1) / kRowsWarps);
+        long long rctas = std::min<long long>(ctx->sm_count, p.n_items);      // few items: spread them over the SMs rather than fill the warps of fewer
         if (p.x_aan) rctas = ctx->sm_count;
         if (rctas < 1) rctas = 1;
         cudaLaunchAttribute rattr;
