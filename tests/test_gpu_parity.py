@@ -60,7 +60,8 @@ def _run(w, check_steps=None, max_steps=None, shared_context=False, jumps=None, 
     segments for long runs: the caches are re-prefilled to start_pos before each segment."""
     dec = Decoder(w, encdec_shared_context=shared_context)
     if STEP_KERNEL[0]:
-        B.check(B.san_step_kernel_select(dec.ctx, STEP_KERNEL[0]), "san_step_kernel_select")
+        sel = STEP_KERNEL[0] if isinstance(STEP_KERNEL[0], tuple) else (STEP_KERNEL[0],)
+        B.check(B.san_step_kernel_select(dec.ctx, *sel), "san_step_kernel_select")
     orc = OracleRun(w, shared_context)
     dec.load_encoder_memory()
     T = np.repeat(w.tgt_lens(), w.beam)
@@ -83,7 +84,8 @@ def _run(w, check_steps=None, max_steps=None, shared_context=False, jumps=None, 
             host = dec.fill_step_inputs(sb, step_id, active, pos[active], sent)
             (dec.step_fused if fused else dec.step)(sb)
             if fused and STEP_KERNEL[0]:
-                assert B.san_step_kernel_used(dec.ctx)[1] == STEP_KERNEL[0]      # the forced kernel is the one that ran
+                want = STEP_KERNEL[0][0] if isinstance(STEP_KERNEL[0], tuple) else STEP_KERNEL[0]
+                assert B.san_step_kernel_used(dec.ctx)[1] == want                # the forced kernel is the one that ran
             do_check = check_steps is None or g in check_steps
             ref = orc.step(host, active, pos[active], want_S=do_check)
             if do_check:
@@ -246,6 +248,33 @@ def test_short_rows_kernel_every_length_up_to_its_limit():
         _run(w, fused=True)
     finally:
         STEP_KERNEL[0] = 0
+
+
+def _rows_kernel_args(heads):
+    """san_step_kernel_select arguments: short-rows kernel, heads per item for (self, encoder-decoder) attention."""
+    return (3, -1, heads[0] + ((heads[1] + 1) << 8), 64, 0, 1)
+
+
+@pytest.mark.parametrize("heads", [(1, 1), (2, 1), (2, 2), (4, 1), (4, 2)])
+def test_short_rows_kernel_heads_per_item(heads):
+    """Items of 1, 2 or 4 heads for self-attention and 1 or 2 for encoder-decoder attention, on rows short
+    enough for four heads of a plane to fit a warp's ring (the kernel takes fewer where they would not)."""
+    w = dataclasses.replace(synth.WORKLOADS["base"], name=f"rows-heads-{heads[0]}-{heads[1]}", n_sent=6, src_lo=5, src_hi=30,
+                            tgt_rule="fixed", tgt_fixed=34, self_blocks=(3, 1, 2), encdec_blocks=(2, 4))
+    STEP_KERNEL[0] = _rows_kernel_args(heads)
+    try:
+        _run(w, fused=True)
+    finally:
+        STEP_KERNEL[0] = 0
+    dec = Decoder(w)
+    B.check(B.san_step_kernel_select(dec.ctx, *_rows_kernel_args(heads)), "san_step_kernel_select")
+    dec.load_encoder_memory()
+    sb = dec.new_step_buffers()
+    dec.fill_step_inputs(sb, 0, np.arange(w.n_seqs, dtype=np.int32), np.zeros(w.n_seqs, np.int32))
+    dec.step_fused(sb)
+    rc, which, rpu = B.san_step_kernel_used(dec.ctx)
+    assert rc == 0 and which == 3 and rpu == [heads[0], heads[1]], (which, rpu)      # the first step's rows are one position long
+    dec.close()
 
 
 @pytest.mark.parametrize("kernel", [0, 2, 3])
